@@ -1,0 +1,140 @@
+"""ctypes front end of the CPU oracle (`gsd_oracle.c`).
+
+TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the benchmark's CPU-baseline
+leg may import this; the product package never does.  It shares nothing with the CUDA
+path.  See the header of `gsd_oracle.c` for what is computed and which passages of the
+paper it follows (Sec. 3 deterministic verification, Sec. 4.1 tree attention and
+longest-path selection, Sec. 5.3 merged token graph).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gsd_oracle.c")
+_LIB = os.path.join(_HERE, "_gsd_oracle.so")
+_lib: Optional[ctypes.CDLL] = None
+
+
+class _Dims(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("N", ctypes.c_int32), ("Hq", ctypes.c_int32),
+                ("Hkv", ctypes.c_int32), ("D", ctypes.c_int32), ("Lmax", ctypes.c_int32),
+                ("scale", ctypes.c_double)]
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP over independent output rows) if it is stale."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + f".tmp{os.getpid()}"
+    cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-Wall", "-Wextra",
+           "-o", tmp, _SRC, "-lm"]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.gsd_oracle_threads.restype = ctypes.c_int
+        _lib.gsd_oracle_argmax_row.restype = ctypes.c_int32
+        for name in ("gsd_oracle_attn", "gsd_oracle_attn_rows", "gsd_oracle_accept"):
+            getattr(_lib, name).restype = ctypes.c_int
+        _lib.gsd_oracle_argmax.restype = None
+    return _lib
+
+
+def threads() -> int:
+    return int(_load().gsd_oracle_threads())
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype) -> np.ndarray:
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def _attn_args(q, k_cache, v_cache, draft_k, draft_v, ancestor_mask, seq_lens, scale):
+    q = _c(q, np.uint16); k_cache = _c(k_cache, np.uint16); v_cache = _c(v_cache, np.uint16)
+    draft_k = _c(draft_k, np.uint16); draft_v = _c(draft_v, np.uint16)
+    ancestor_mask = _c(ancestor_mask, np.uint32); seq_lens = _c(seq_lens, np.int32)
+    B, N, Hq, D = q.shape
+    _, Lmax, Hkv, _ = k_cache.shape
+    assert v_cache.shape == k_cache.shape
+    assert draft_k.shape == (B, N, Hkv, D) and draft_v.shape == (B, N, Hkv, D)
+    assert ancestor_mask.shape == (B, N, (N + 31) // 32)
+    assert seq_lens.shape == (B,) and (seq_lens >= 0).all() and (seq_lens <= Lmax).all()
+    assert Hq % Hkv == 0
+    dims = _Dims(B, N, Hq, Hkv, D, Lmax, float(scale) if scale else 0.0)
+    keep = (q, k_cache, v_cache, draft_k, draft_v, ancestor_mask, seq_lens)
+    return dims, keep
+
+
+def attn(q, k_cache, v_cache, draft_k, draft_v, ancestor_mask, seq_lens, scale: float = 0.0
+         ) -> np.ndarray:
+    """fp64 DAG-masked attention; bf16 inputs as uint16 bit patterns. Returns [B,N,Hq,D] f64."""
+    dims, keep = _attn_args(q, k_cache, v_cache, draft_k, draft_v, ancestor_mask, seq_lens, scale)
+    out = np.zeros(keep[0].shape, dtype=np.float64)
+    rc = _load().gsd_oracle_attn(ctypes.byref(dims), *[_p(a) for a in keep], _p(out))
+    if rc != 0:
+        raise RuntimeError("oracle attention failed")
+    return out
+
+
+def attn_rows(q, k_cache, v_cache, draft_k, draft_v, ancestor_mask, seq_lens,
+              rows: Sequence[Sequence[int]], scale: float = 0.0) -> np.ndarray:
+    """Same as `attn` for the listed (b, n, h) rows only. Returns [len(rows), D] f64."""
+    dims, keep = _attn_args(q, k_cache, v_cache, draft_k, draft_v, ancestor_mask, seq_lens, scale)
+    rows = _c(rows, np.int32).reshape(-1, 3)
+    out = np.zeros((rows.shape[0], dims.D), dtype=np.float64)
+    rc = _load().gsd_oracle_attn_rows(ctypes.byref(dims), *[_p(a) for a in keep], _p(rows),
+                                      ctypes.c_long(rows.shape[0]), _p(out))
+    if rc != 0:
+        raise RuntimeError("oracle attention failed")
+    return out
+
+
+def argmax(logits) -> np.ndarray:
+    """Row-wise argmax over the last axis, ties to the lowest index, NaN never wins."""
+    logits = _c(logits, np.float32)
+    V = logits.shape[-1]
+    rows = logits.size // V if V else 0
+    out = np.zeros(logits.shape[:-1], dtype=np.int32)
+    _load().gsd_oracle_argmax(_p(logits), ctypes.c_long(rows), ctypes.c_int32(V), _p(out))
+    return out
+
+
+def accept(logits, draft_tokens, parent_ptr, parent_idx, Tcap: int = 0, visit_cap: int = 0):
+    """Brute-force longest accepted path.
+
+    Returns (accepted_tokens [B,Tcap] padded with -1, accepted_len [B],
+    accepted_nodes [B,Tcap] padded with -1, paths_visited [B]; a negative count means the
+    walk stopped extending rejected paths after `visit_cap` paths)."""
+    logits = _c(logits, np.float32); draft_tokens = _c(draft_tokens, np.int32)
+    parent_ptr = _c(parent_ptr, np.int32); parent_idx = _c(parent_idx, np.int32)
+    B, N, V = logits.shape
+    assert draft_tokens.shape == (B, N) and parent_ptr.shape == (B, N + 1)
+    Ecap = parent_idx.shape[1]
+    Tcap = Tcap or N
+    toks = np.zeros((B, Tcap), dtype=np.int32)
+    lens = np.zeros((B,), dtype=np.int32)
+    nodes = np.zeros((B, Tcap), dtype=np.int32)
+    visited = np.zeros((B,), dtype=np.int64)
+    rc = _load().gsd_oracle_accept(_p(logits), _p(draft_tokens), _p(parent_ptr), _p(parent_idx),
+                                   ctypes.c_int32(B), ctypes.c_int32(N), ctypes.c_int32(V),
+                                   ctypes.c_int32(Ecap), ctypes.c_int32(Tcap), _p(toks), _p(lens),
+                                   _p(nodes), _p(visited), ctypes.c_int64(visit_cap))
+    if rc != 0:
+        raise ValueError("oracle accept: malformed DAG or Tcap too small")
+    return toks, lens, nodes, visited

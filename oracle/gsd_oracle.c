@@ -1,0 +1,322 @@
+/*
+ * CPU oracle for the verification step of Graph-structured Speculative Decoding.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition that the CUDA
+ * library is checked against; it shares no code with the CUDA path, and nothing in the
+ * product may call it.  Only the tests, the smoke check and the benchmark's CPU-baseline
+ * leg use it.
+ *
+ * What it computes
+ *  - Attention (tree attention, Sec. 4.1: a flattened draft token attends only to its
+ *    ancestors; the committed context sits in the KV cache, Sec. 4.2; all hypotheses are
+ *    scored in one pass, Sec. 3 and Sec. 4.1).  For every sequence b, draft node n and
+ *    query head h the visible keys are the first seq_lens[b] rows of the cache plus the
+ *    draft nodes whose bit is set in ancestor_mask[b][n]; the output row is the
+ *    max-subtracted softmax of scale * <q, k_j> over those keys applied to the matching
+ *    value rows.  Everything is evaluated in double precision from the exact values of
+ *    the bf16 inputs.  An empty key set gives a row of zeros.
+ *  - Acceptance (deterministic verification, Sec. 3: a drafted token is kept only if the
+ *    target model would emit it; a rejection discards the rest of that hypothesis and
+ *    the target model supplies the next token; the longest hypothesis from the root is
+ *    adopted, Sec. 4.1 and Sec. 1).  a[n] is the lowest index holding the row maximum
+ *    of logits[b][n][:].  Every root-to-node path of the DAG is enumerated by a
+ *    depth-first walk over child lists (no dynamic programming, no memo); a path
+ *    v0=0,v1..vm is accepted iff tok[v_i] == a[v_{i-1}] on each of its edges.  The
+ *    longest accepted path wins; among equally long ones the path whose node sequence,
+ *    read from its last node backwards, is lexicographically smallest.  Output:
+ *    tok[v1..vm] followed by a[vm], so accepted_len = m + 1.
+ *
+ * Readings where the paper is silent are listed in the repository's design notes
+ * (scale default 1/sqrt(D), q-head h uses kv-head h / G, mask bits honoured literally,
+ * node 0 is the root whose token is not re-emitted, NaN logits never win the argmax).
+ *
+ * Every function here is pinned by tests that do not re-use it: closed forms (uniform
+ * softmax, two-key sigmoid), library attention on chain / tree / full-mask special
+ * cases, numpy argmax, hand-built DAGs with hand-derived answers, and invariants.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef struct {
+    int32_t B, N, Hq, Hkv, D, Lmax;
+    double scale; /* <= 0 means 1/sqrt(D) */
+} gsd_oracle_attn_dims;
+
+static double bf16_to_double(uint16_t bits)
+{
+    uint32_t u = ((uint32_t)bits) << 16; /* bf16 is the top half of an IEEE float */
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+int gsd_oracle_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* One output row out_row[0..D) for (b, n, h).  scratch holds Lmax + N doubles. */
+void gsd_oracle_attn_row(const gsd_oracle_attn_dims *dm, const uint16_t *q,
+                         const uint16_t *k_cache, const uint16_t *v_cache,
+                         const uint16_t *draft_k, const uint16_t *draft_v,
+                         const uint32_t *ancestor_mask, const int32_t *seq_lens,
+                         int b, int n, int h, double *out_row, double *scratch)
+{
+    const int N = dm->N, Hq = dm->Hq, Hkv = dm->Hkv, D = dm->D, Lmax = dm->Lmax;
+    const int G = Hq / Hkv;
+    const int c = h / G; /* kv head serving query head h */
+    const int W = (N + 31) / 32;
+    const double scale = dm->scale > 0 ? dm->scale : 1.0 / sqrt((double)D);
+    const int L = seq_lens[b];
+    const uint16_t *qrow = q + (((size_t)b * N + n) * Hq + h) * D;
+    const uint32_t *mrow = ancestor_mask + ((size_t)b * N + n) * W;
+    double *s = scratch;
+    int nk = 0;
+    double smax = -INFINITY;
+
+    /* scores of the visible keys, prefix first then draft nodes */
+    for (int j = 0; j < L; ++j) {
+        const uint16_t *krow = k_cache + (((size_t)b * Lmax + j) * Hkv + c) * D;
+        double dot = 0.0;
+        for (int d = 0; d < D; ++d) dot += bf16_to_double(qrow[d]) * bf16_to_double(krow[d]);
+        s[nk] = scale * dot;
+        if (s[nk] > smax) smax = s[nk];
+        ++nk;
+    }
+    for (int j = 0; j < N; ++j) {
+        if (!((mrow[j / 32] >> (j % 32)) & 1u)) continue;
+        const uint16_t *krow = draft_k + (((size_t)b * N + j) * Hkv + c) * D;
+        double dot = 0.0;
+        for (int d = 0; d < D; ++d) dot += bf16_to_double(qrow[d]) * bf16_to_double(krow[d]);
+        s[nk] = scale * dot;
+        if (s[nk] > smax) smax = s[nk];
+        ++nk;
+    }
+    for (int d = 0; d < D; ++d) out_row[d] = 0.0;
+    if (nk == 0) return;
+
+    double denom = 0.0;
+    for (int i = 0; i < nk; ++i) {
+        s[i] = exp(s[i] - smax);
+        denom += s[i];
+    }
+    int i = 0;
+    for (int j = 0; j < L; ++j, ++i) {
+        const uint16_t *vrow = v_cache + (((size_t)b * Lmax + j) * Hkv + c) * D;
+        const double p = s[i] / denom;
+        for (int d = 0; d < D; ++d) out_row[d] += p * bf16_to_double(vrow[d]);
+    }
+    for (int j = 0; j < N; ++j) {
+        if (!((mrow[j / 32] >> (j % 32)) & 1u)) continue;
+        const uint16_t *vrow = draft_v + (((size_t)b * N + j) * Hkv + c) * D;
+        const double p = s[i] / denom;
+        for (int d = 0; d < D; ++d) out_row[d] += p * bf16_to_double(vrow[d]);
+        ++i;
+    }
+}
+
+/* All rows: out[B,N,Hq,D] in double.  Rows are independent; they are handed to the host
+ * threads as they are, nothing else is reorganised. */
+int gsd_oracle_attn(const gsd_oracle_attn_dims *dm, const uint16_t *q, const uint16_t *k_cache,
+                    const uint16_t *v_cache, const uint16_t *draft_k, const uint16_t *draft_v,
+                    const uint32_t *ancestor_mask, const int32_t *seq_lens, double *out)
+{
+    const long rows = (long)dm->B * dm->N * dm->Hq;
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *scratch = (double *)malloc(sizeof(double) * (size_t)(dm->Lmax + dm->N + 1));
+        if (!scratch) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp for schedule(dynamic, 16)
+        for (long r = 0; r < rows; ++r) {
+            if (!scratch) continue;
+            const int h = (int)(r % dm->Hq);
+            const int n = (int)((r / dm->Hq) % dm->N);
+            const int b = (int)(r / ((long)dm->Hq * dm->N));
+            gsd_oracle_attn_row(dm, q, k_cache, v_cache, draft_k, draft_v, ancestor_mask,
+                                seq_lens, b, n, h, out + (size_t)r * dm->D, scratch);
+        }
+        free(scratch);
+    }
+    return failed ? -1 : 0;
+}
+
+/* A listed subset of rows: rows[3*i..3*i+2] = (b, n, h); out[i*D..]. */
+int gsd_oracle_attn_rows(const gsd_oracle_attn_dims *dm, const uint16_t *q,
+                         const uint16_t *k_cache, const uint16_t *v_cache,
+                         const uint16_t *draft_k, const uint16_t *draft_v,
+                         const uint32_t *ancestor_mask, const int32_t *seq_lens,
+                         const int32_t *rows, long nrows, double *out)
+{
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *scratch = (double *)malloc(sizeof(double) * (size_t)(dm->Lmax + dm->N + 1));
+        if (!scratch) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp for schedule(dynamic, 4)
+        for (long i = 0; i < nrows; ++i) {
+            if (!scratch) continue;
+            gsd_oracle_attn_row(dm, q, k_cache, v_cache, draft_k, draft_v, ancestor_mask,
+                                seq_lens, rows[3 * i], rows[3 * i + 1], rows[3 * i + 2],
+                                out + (size_t)i * dm->D, scratch);
+        }
+        free(scratch);
+    }
+    return failed ? -1 : 0;
+}
+
+/* Lowest index holding the largest non-NaN value; 0 when every entry is NaN.
+ * A later entry replaces the current best only when strictly greater. */
+int32_t gsd_oracle_argmax_row(const float *row, int32_t V)
+{
+    int32_t best = -1;
+    for (int32_t i = 0; i < V; ++i) {
+        if (row[i] != row[i]) continue; /* NaN never wins */
+        if (best < 0 || row[i] > row[best]) best = i;
+    }
+    return best < 0 ? 0 : best;
+}
+
+void gsd_oracle_argmax(const float *logits, long rows, int32_t V, int32_t *out)
+{
+#pragma omp parallel for schedule(static)
+    for (long r = 0; r < rows; ++r) out[r] = gsd_oracle_argmax_row(logits + (size_t)r * V, V);
+}
+
+/* ---- brute-force path enumeration for one sequence ---- */
+typedef struct {
+    int N;
+    const int32_t *tok;   /* [N] */
+    const int32_t *amax;  /* [N] */
+    const int *child_ptr; /* [N+1] */
+    const int *child_idx;
+    int *stack;           /* current path, stack[0] = 0 */
+    int *best;            /* best accepted path so far */
+    int best_edges;       /* its edge count, -1 if none yet */
+    long visited;         /* number of root-to-node paths enumerated */
+    long visit_cap;       /* > 0: beyond this many paths, stop extending rejected paths */
+    int pruned;           /* set when the cap changed the walk */
+} walk_t;
+
+static int path_is_accepted(const walk_t *w, int len)
+{
+    for (int i = 1; i < len; ++i)
+        if (w->tok[w->stack[i]] != w->amax[w->stack[i - 1]]) return 0;
+    return 1;
+}
+
+/* 1 if the candidate (w->stack, same length as w->best) comes first when both are read
+ * from the last node backwards */
+static int reversed_less(const walk_t *w, int len)
+{
+    for (int i = len - 1; i >= 0; --i) {
+        if (w->stack[i] < w->best[i]) return 1;
+        if (w->stack[i] > w->best[i]) return 0;
+    }
+    return 0;
+}
+
+static void walk(walk_t *w, int len)
+{
+    const int v = w->stack[len - 1];
+    const int ok = path_is_accepted(w, len);
+    w->visited++;
+    if (ok) {
+        const int edges = len - 1;
+        if (edges > w->best_edges || (edges == w->best_edges && reversed_less(w, len))) {
+            memcpy(w->best, w->stack, sizeof(int) * (size_t)len);
+            w->best_edges = edges;
+        }
+    } else if (w->visit_cap > 0 && w->visited > w->visit_cap) {
+        /* an extension of a rejected path is rejected too: once over the cap, skip them */
+        w->pruned = 1;
+        return;
+    }
+    for (int e = w->child_ptr[v]; e < w->child_ptr[v + 1]; ++e) {
+        w->stack[len] = w->child_idx[e];
+        walk(w, len + 1);
+    }
+}
+
+/*
+ * logits [B,N,V] f32; draft_tokens [B,N]; parent_ptr [B,N+1]; parent_idx [B,Ecap];
+ * accepted_tokens [B,Tcap] (padded with -1); accepted_len [B]; accepted_nodes [B,Tcap]
+ * (may be NULL; the chosen path's node ids v0..vm, padded with -1); paths_visited [B] (may be
+ * NULL).  visit_cap <= 0 enumerates everything.  Returns 0, or -1 on malformed input
+ * (a parent index not below its child, Tcap too small) or allocation failure.
+ */
+int gsd_oracle_accept(const float *logits, const int32_t *draft_tokens, const int32_t *parent_ptr,
+                      const int32_t *parent_idx, int32_t B, int32_t N, int32_t V, int32_t Ecap,
+                      int32_t Tcap, int32_t *accepted_tokens, int32_t *accepted_len,
+                      int32_t *accepted_nodes, int64_t *paths_visited, int64_t visit_cap)
+{
+    int rc = 0;
+    for (int b = 0; b < B; ++b) {
+        const int32_t *tok = draft_tokens + (size_t)b * N;
+        const int32_t *pp = parent_ptr + (size_t)b * (N + 1);
+        const int32_t *pi = parent_idx + (size_t)b * Ecap;
+        int32_t *amax = (int32_t *)malloc(sizeof(int32_t) * (size_t)N);
+        int *cptr = (int *)calloc((size_t)N + 2, sizeof(int));
+        int *cidx = (int *)malloc(sizeof(int) * (size_t)(pp[N] > 0 ? pp[N] : 1));
+        int *fill = (int *)calloc((size_t)N + 1, sizeof(int));
+        int *stack = (int *)malloc(sizeof(int) * (size_t)(N + 1));
+        int *best = (int *)malloc(sizeof(int) * (size_t)(N + 1));
+        if (!amax || !cptr || !cidx || !fill || !stack || !best) rc = -1;
+
+        if (rc == 0) {
+            gsd_oracle_argmax(logits + (size_t)b * N * V, N, V, amax);
+            /* child lists (children ascending) from the parent lists */
+            for (int v = 0; v < N && rc == 0; ++v)
+                for (int e = pp[v]; e < pp[v + 1]; ++e) {
+                    if (pi[e] < 0 || pi[e] >= v) { rc = -1; break; }
+                    cptr[pi[e] + 1]++;
+                }
+        }
+        if (rc == 0) {
+            for (int v = 0; v < N; ++v) cptr[v + 1] += cptr[v];
+            for (int v = 0; v < N; ++v)
+                for (int e = pp[v]; e < pp[v + 1]; ++e) {
+                    const int p = pi[e];
+                    cidx[cptr[p] + fill[p]++] = v;
+                }
+            walk_t w;
+            w.N = N; w.tok = tok; w.amax = amax; w.child_ptr = cptr; w.child_idx = cidx;
+            w.stack = stack; w.best = best; w.best_edges = -1; w.visited = 0;
+            w.visit_cap = visit_cap; w.pruned = 0;
+            stack[0] = 0;
+            walk(&w, 1); /* the one-node path (root alone) is always accepted */
+            const int m = w.best_edges;
+            if (m + 1 > Tcap) rc = -1;
+            if (rc == 0) {
+                for (int i = 0; i < Tcap; ++i) {
+                    accepted_tokens[(size_t)b * Tcap + i] = -1;
+                    if (accepted_nodes) accepted_nodes[(size_t)b * Tcap + i] = -1;
+                }
+                for (int i = 1; i <= m; ++i) accepted_tokens[(size_t)b * Tcap + i - 1] = tok[best[i]];
+                accepted_tokens[(size_t)b * Tcap + m] = amax[best[m]];
+                accepted_len[b] = m + 1;
+                if (accepted_nodes)
+                    for (int i = 0; i <= m; ++i) accepted_nodes[(size_t)b * Tcap + i] = best[i];
+                if (paths_visited) paths_visited[b] = w.pruned ? -w.visited : w.visited;
+            }
+        }
+        free(amax); free(cptr); free(cidx); free(fill); free(stack); free(best);
+        if (rc != 0) return rc;
+    }
+    return 0;
+}
