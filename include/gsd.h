@@ -1,0 +1,199 @@
+/*
+ * gsd.h - C ABI of the B200 (sm_100a) verification kernels for Graph-structured
+ * Speculative Decoding (GSD).
+ *
+ * The verification stage scores every drafted token of a token graph in ONE pass of the
+ * target model and adopts the longest hypothesis the model agrees with (Sec. 1; Sec. 3,
+ * single-pass verification; Sec. 4.1, tree attention and longest-path selection;
+ * Sec. 5.3-5.4, the merged token graph).  This library provides the two data-parallel
+ * parts of that stage for one attention layer / one LM-head output:
+ *
+ *   gsd_verify_attn  attention of all draft nodes over the committed prefix (KV cache,
+ *                    Sec. 4.2) plus exactly the draft nodes named by a per-node ancestor
+ *                    bitmask (a flattened token may attend only to its ancestors, Sec. 4.1)
+ *   gsd_accept       greedy (deterministic) verification, Sec. 3: per-node vocabulary
+ *                    argmax, then the longest accepted root path through the DAG
+ *
+ * Conventions
+ *  - All tensors are dense, row-major, innermost dimension last.  "device" pointers are
+ *    CUDA global memory of the current device; "host" pointers are ordinary host memory.
+ *  - bf16 tensors are passed as const void* / void* (2-byte elements, IEEE bfloat16).
+ *  - Nothing is allocated, freed or synchronised by the device-pointer calls: every
+ *    buffer including the workspace is owned by the caller, all work is enqueued on
+ *    `stream`, outputs are valid once the stream reaches that point.
+ *  - Return value: GSD_OK (0) or a negative gsd_status.  When a host-side check fails
+ *    nothing is launched.  Problems only the device can see (malformed CSR, token out of
+ *    range, output capacity exceeded, a bounded wait that expired) never trap: the kernel
+ *    ORs a GSD_DEV_* bit into *status (if given) and finishes cleanly.
+ *  - `stream` is a cudaStream_t passed as void* so that this header needs no CUDA header.
+ */
+#ifndef GSD_H_
+#define GSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GSD_VERSION 100
+
+typedef enum gsd_status {
+    GSD_OK = 0,
+    GSD_ERR_NULL_POINTER = -1,   /* a required pointer is NULL */
+    GSD_ERR_BAD_SHAPE = -2,      /* unsupported or inconsistent sizes */
+    GSD_ERR_MISALIGNED = -3,     /* a tensor base is not sufficiently aligned */
+    GSD_ERR_WORKSPACE = -4,      /* workspace missing or too small */
+    GSD_ERR_CUDA = -5,           /* a CUDA runtime/driver call failed (see gsd_last_cuda_error) */
+    GSD_ERR_UNSUPPORTED = -6     /* requested kernel variant cannot run this shape */
+} gsd_status;
+
+/* bits OR-ed into the device status word */
+#define GSD_DEV_BAD_CSR      0x1u  /* a parent index outside [0, child) or a bad row pointer; the edge is ignored */
+#define GSD_DEV_BAD_TOKEN    0x2u  /* a draft token outside [0, V) (still compared as is) */
+#define GSD_DEV_TCAP         0x4u  /* accepted_len exceeded Tcap; the token list was truncated */
+#define GSD_DEV_WAIT_EXPIRED 0x8u  /* a bounded in-kernel wait gave up; the output is not valid */
+#define GSD_DEV_BAD_SEQ_LEN  0x10u /* seq_lens[b] outside [0, Lmax]; it was clamped */
+
+#define GSD_MAX_NODES 512          /* largest supported N (draft nodes per sequence) */
+
+/* kernel selection for gsd_verify_attn */
+#define GSD_ATTN_AUTO 0
+#define GSD_ATTN_MMA  1            /* warp-level mma.sync kernel: D in {64,128}, any N */
+#define GSD_ATTN_TCGEN05 2         /* tcgen05/TMEM/TMA kernel: D == 128 */
+
+typedef struct gsd_attn_params {
+    int32_t B;            /* sequences */
+    int32_t N;            /* draft nodes per sequence, 1..GSD_MAX_NODES; node 0 is the root */
+    int32_t Hq;           /* query heads */
+    int32_t Hkv;          /* key/value heads; Hq % Hkv == 0; q-head h uses kv-head h / (Hq/Hkv) */
+    int32_t D;            /* head dimension: 64 or 128 */
+    int32_t Lmax;         /* padded cache length (rows per sequence in k_cache/v_cache), >= 1 */
+    float softmax_scale;  /* <= 0 selects 1/sqrt(D) */
+    int32_t num_splits;   /* key-range splits per (sequence, kv head, row tile); 0 = choose */
+    int32_t kernel;       /* GSD_ATTN_AUTO / _MMA / _TCGEN05 */
+} gsd_attn_params;
+
+typedef struct gsd_accept_params {
+    int32_t B;     /* sequences */
+    int32_t N;     /* draft nodes per sequence, 1..GSD_MAX_NODES */
+    int32_t V;     /* vocabulary size, >= 1 */
+    int32_t Ecap;  /* row length of parent_idx, >= 1 */
+    int32_t Tcap;  /* row length of accepted_tokens / accepted_nodes, >= 1 (N always suffices) */
+} gsd_accept_params;
+
+int gsd_version(void);
+const char* gsd_status_string(int status);
+/* Text of the last CUDA error this library saw on the calling thread ("" if none). */
+const char* gsd_last_cuda_error(void);
+
+/*
+ * gsd_verify_attn - DAG-masked attention of the draft nodes (Sec. 4.1 tree attention over
+ * the flattened token graph, Sec. 4.2 KV cache).
+ *
+ * For every sequence b, node n and query head h (kv head c = h / (Hq/Hkv)):
+ *   keys   = cache rows j < seq_lens[b]  plus  draft rows j with bit j of ancestor_mask[b][n] set
+ *   out[b,n,h,:] = sum_j softmax_j(scale * <q[b,n,h,:], K_j[c,:]>) * V_j[c,:]
+ * bf16 inputs, fp32 accumulation, bf16 output (round to nearest even).  Mask bits are
+ * honoured literally (no implicit diagonal, no triangularity assumed); bits >= N are
+ * ignored.  Cache rows at positions >= seq_lens[b] never reach the result, whatever
+ * they contain.  A row with no visible key yields zeros.
+ *
+ *   q              [B, N, Hq, D]      bf16  device  in
+ *   k_cache        [B, Lmax, Hkv, D]  bf16  device  in
+ *   v_cache        [B, Lmax, Hkv, D]  bf16  device  in
+ *   draft_k        [B, N, Hkv, D]     bf16  device  in
+ *   draft_v        [B, N, Hkv, D]     bf16  device  in
+ *   ancestor_mask  [B, N, W] uint32, W = ceil(N/32), device, in; bit j of a row is
+ *                  word j / 32, bit j % 32
+ *   seq_lens       [B] int32 device in; 0 <= seq_lens[b] <= Lmax (clamped and flagged otherwise)
+ *   out            [B, N, Hq, D]      bf16  device  out
+ *   p              host
+ *   workspace      device scratch of at least gsd_verify_attn_workspace_bytes(p) bytes,
+ *                  256-byte aligned; may be NULL when that size is 0.  Contents are
+ *                  undefined before and after the call.
+ *   status         device int32 word or NULL; GSD_DEV_* bits are OR-ed in (never cleared)
+ *   stream         cudaStream_t
+ *
+ * All tensor bases must be 16-byte aligned.  Calls that share a workspace must not
+ * overlap on the device.  Errors: see gsd_status; nothing is launched on a host error.
+ */
+int gsd_verify_attn(const void* q, const void* k_cache, const void* v_cache,
+                    const void* draft_k, const void* draft_v, const uint32_t* ancestor_mask,
+                    const int32_t* seq_lens, void* out, const gsd_attn_params* p,
+                    void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+
+/* Bytes of workspace gsd_verify_attn needs for *p on the current device (0 on invalid
+ * parameters or when none is needed). */
+size_t gsd_verify_attn_workspace_bytes(const gsd_attn_params* p);
+
+/* The number of key-range splits gsd_verify_attn would use for *p on the current device
+ * (p->num_splits if non-zero, else the automatic choice); <= 0 on invalid parameters. */
+int gsd_verify_attn_num_splits(const gsd_attn_params* p);
+
+/*
+ * gsd_accept - deterministic verification and longest-path selection (Sec. 3: a drafted
+ * token is accepted only if the target model would generate the same token; after a
+ * rejection the rest of the hypothesis is dropped and the target model supplies the next
+ * token.  Sec. 4.1 / Sec. 1: the longest hypothesis from the root is adopted).
+ *
+ *   a[b,n] = lowest index i with logits[b,n,i] equal to the row maximum over non-NaN
+ *            entries (0 if the row is all NaN)
+ *   edge p->v is accepted iff draft_tokens[b,v] == a[b,p]
+ *   the chosen path v0=0,v1..vm is the longest root path of accepted edges; among equally
+ *   long ones the lowest end node, then step by step the lowest predecessor that carries
+ *   length-1
+ *   accepted_tokens[b,:] = tok[v1..vm], a[b,vm], then -1 padding;  accepted_len[b] = m+1
+ *
+ *   logits          [B, N, V] fp32 device in
+ *   draft_tokens    [B, N] int32 device in; node 0 is the root (its token is not emitted)
+ *   parent_ptr      [B, N+1] int32 device in; CSR row pointers, local to sequence b
+ *   parent_idx      [B, Ecap] int32 device in; parents of v are idx[ptr[v] .. ptr[v+1]);
+ *                   every parent index must be < v (topological numbering)
+ *   accepted_tokens [B, Tcap] int32 device out
+ *   accepted_len    [B] int32 device out
+ *   accepted_nodes  [B, Tcap] int32 device out or NULL: v0..vm then -1 padding
+ *   p               host
+ *   workspace       device scratch >= gsd_accept_workspace_bytes(p), 8-byte aligned
+ *   status          device int32 word or NULL
+ *   stream          cudaStream_t
+ *
+ * logits must be 4-byte aligned; 16-byte alignment with V % 4 == 0 enables vector loads.
+ */
+int gsd_accept(const float* logits, const int32_t* draft_tokens, const int32_t* parent_ptr,
+               const int32_t* parent_idx, int32_t* accepted_tokens, int32_t* accepted_len,
+               int32_t* accepted_nodes, const gsd_accept_params* p, void* workspace,
+               size_t workspace_bytes, int32_t* status, void* stream);
+
+size_t gsd_accept_workspace_bytes(const gsd_accept_params* p);
+
+/*
+ * gsd_verify_step_host - one whole verification step from HOST buffers: copies every
+ * input to the device arena, runs gsd_verify_attn and gsd_accept, copies `out`,
+ * accepted_tokens, accepted_len (and accepted_nodes if non-NULL) back and waits for the
+ * stream.  Same operations and passages as the two calls above; this entry point exists
+ * for callers that keep their tensors in host memory and to measure the step end to end.
+ *
+ * All tensor pointers are host pointers with the layouts given above (pinned memory makes
+ * the copies asynchronous and faster, pageable memory works too).  `arena` is a device
+ * buffer of at least gsd_verify_step_host_arena_bytes(ap, cp) bytes, 256-byte aligned,
+ * owned by the caller.  `device_status_out` (host, may be NULL) receives the device
+ * status word of this step.  ap->B == cp->B and ap->N == cp->N are required.
+ */
+int gsd_verify_step_host(const void* q, const void* k_cache, const void* v_cache,
+                         const void* draft_k, const void* draft_v,
+                         const uint32_t* ancestor_mask, const int32_t* seq_lens, void* out,
+                         const gsd_attn_params* ap, const float* logits,
+                         const int32_t* draft_tokens, const int32_t* parent_ptr,
+                         const int32_t* parent_idx, int32_t* accepted_tokens,
+                         int32_t* accepted_len, int32_t* accepted_nodes,
+                         const gsd_accept_params* cp, void* arena, size_t arena_bytes,
+                         int32_t* device_status_out, void* stream);
+
+size_t gsd_verify_step_host_arena_bytes(const gsd_attn_params* ap, const gsd_accept_params* cp);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GSD_H_ */
