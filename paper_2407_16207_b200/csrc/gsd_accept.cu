@@ -1,0 +1,330 @@
+// gsd_accept: greedy verification (vocabulary argmax per draft node) and the longest
+// accepted root path through the draft DAG (Sec. 3 deterministic verification and the
+// rejection cascade; Sec. 4.1 longest-path selection).
+//
+// One launch.  Grid (splits, B*N): each CTA streams one slice of one logits row with
+// 16-byte loads and reduces (value, index) pairs; slices of a row meet in a packed 64-bit
+// atomicMax.  The CTA that finishes last for a sequence runs the path pass for it:
+// level-synchronous relaxation of best[v] = 1 + max over accepted parents, selection of
+// the end node, backtracking, emission.
+#include "gsd_internal.cuh"
+#include <math_constants.h>
+
+namespace gsd {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kNone = 0x7FFFFFFF;
+constexpr int kNodeSlots = (GSD_MAX_NODES + kThreads - 1) / kThreads;
+
+struct Best {
+    float v;
+    int i;
+};
+
+__device__ __forceinline__ void take(Best& b, float v, int i) {
+    if (v > b.v) {  // false for NaN; strict: an equal later value never replaces
+        b.v = v;
+        b.i = i;
+    }
+}
+
+__device__ __forceinline__ Best better(Best a, Best b) {
+    return (b.v > a.v || (b.v == a.v && b.i < a.i)) ? b : a;
+}
+
+// monotone map of non-NaN floats to unsigned (with -0 folded onto +0)
+__device__ __forceinline__ unsigned ordered_bits(float v) {
+    if (v == 0.0f) v = 0.0f;
+    unsigned u = __float_as_uint(v);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ unsigned long long pack_key(float v, int i) {
+    return ((unsigned long long)ordered_bits(v) << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned)i);
+}
+
+__device__ __forceinline__ int key_index(unsigned long long key) {
+    return key == 0ull ? 0 : (int)(0xFFFFFFFFu - (unsigned)(key & 0xFFFFFFFFull));
+}
+
+__device__ Best block_best(Best b, Best* sh) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Best t;
+        t.v = __shfl_xor_sync(0xFFFFFFFFu, b.v, o);
+        t.i = __shfl_xor_sync(0xFFFFFFFFu, b.i, o);
+        b = better(b, t);
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) sh[warp] = b;
+    __syncthreads();
+    if (warp == 0) {
+        b = lane < (kThreads / 32) ? sh[lane] : Best{-CUDART_INF_F, kNone};
+#pragma unroll
+        for (int o = 4; o > 0; o >>= 1) {
+            Best t;
+            t.v = __shfl_xor_sync(0xFFFFFFFFu, b.v, o);
+            t.i = __shfl_xor_sync(0xFFFFFFFFu, b.i, o);
+            b = better(b, t);
+        }
+        if (lane == 0) sh[0] = b;
+    }
+    __syncthreads();
+    b = sh[0];
+    __syncthreads();
+    return b;
+}
+
+struct AcceptArgs {
+    const float* logits;
+    const int32_t* tok;
+    const int32_t* pptr;
+    const int32_t* pidx;
+    int32_t* out_tok;
+    int32_t* out_len;
+    int32_t* out_nodes;
+    unsigned long long* keys;  // [B*N], zeroed before the launch
+    unsigned* done;            // [B], zeroed before the launch
+    int32_t* status;
+    int B, N, V, Ecap, Tcap, splits;
+};
+
+__device__ void path_pass(const AcceptArgs& a, int b) {
+    __shared__ int s_best[GSD_MAX_NODES];
+    __shared__ int s_amax[GSD_MAX_NODES];
+    __shared__ int s_tok[GSD_MAX_NODES];
+    __shared__ int s_ptr[GSD_MAX_NODES + 1];
+    __shared__ int s_red[kThreads / 32];
+    __shared__ unsigned s_flags;
+    __shared__ int s_m;
+    const int N = a.N, tid = threadIdx.x;
+    const int32_t* tok = a.tok + (size_t)b * N;
+    const int32_t* pptr = a.pptr + (size_t)b * (N + 1);
+    const int32_t* pidx = a.pidx + (size_t)b * a.Ecap;
+    unsigned flags = 0;
+    if (tid == 0) s_flags = 0;
+    for (int v = tid; v < N; v += kThreads) {
+        // the keys were written by other CTAs: read them past L1
+        s_amax[v] = key_index(__ldcg(a.keys + (size_t)b * N + v));
+        const int t = tok[v];
+        s_tok[v] = t;
+        if (t < 0 || t >= a.V) flags |= GSD_DEV_BAD_TOKEN;
+        s_best[v] = v == 0 ? 0 : -1;
+    }
+    for (int v = tid; v <= N; v += kThreads) {
+        int e = pptr[v];
+        if (e < 0 || e > a.Ecap) {
+            flags |= GSD_DEV_BAD_CSR;
+            e = e < 0 ? 0 : a.Ecap;
+        }
+        s_ptr[v] = e;
+    }
+    __syncthreads();
+
+    // level-synchronous relaxation: after round r every node whose longest accepted root
+    // path has <= r edges is final; values only grow, so it stops when nothing changed
+    for (int round = 0; round < N; ++round) {
+        int nb[kNodeSlots];
+        int changed = 0;
+#pragma unroll
+        for (int k = 0; k < kNodeSlots; ++k) {
+            const int v = tid + k * kThreads;
+            nb[k] = -1;
+            if (v > 0 && v < N) {
+                int cur = s_best[v];
+                const int t = s_tok[v];
+                for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
+                    const int p = pidx[e];
+                    if (p < 0 || p >= v) {
+                        flags |= GSD_DEV_BAD_CSR;
+                        continue;
+                    }
+                    const int bp = s_best[p];
+                    if (bp >= 0 && t == s_amax[p] && bp + 1 > cur) cur = bp + 1;
+                }
+                nb[k] = cur;
+                changed |= (cur != s_best[v]);
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < kNodeSlots; ++k) {
+            const int v = tid + k * kThreads;
+            if (v > 0 && v < N) s_best[v] = nb[k];
+        }
+        if (!__syncthreads_or(changed)) break;
+    }
+
+    // end node: longest, then lowest index
+    int key = -1;
+    for (int v = tid; v < N; v += kThreads)
+        if (s_best[v] >= 0) key = max(key, (s_best[v] << 10) | (1023 - v));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xFFFFFFFFu, key, o));
+    if ((tid & 31) == 0) s_red[tid >> 5] = key;
+    if (flags) atomicOr(&s_flags, flags);
+    __syncthreads();
+
+    int32_t* out_tok = a.out_tok + (size_t)b * a.Tcap;
+    int32_t* out_nodes = a.out_nodes ? a.out_nodes + (size_t)b * a.Tcap : nullptr;
+    if (tid == 0) {
+        for (int w = 1; w < kThreads / 32; ++w) key = max(key, s_red[w]);
+        const int m = key >> 10;
+        int v = 1023 - (key & 1023);
+        unsigned fl = s_flags;
+        if (m + 1 > a.Tcap) fl |= GSD_DEV_TCAP;
+        if (m < a.Tcap) out_tok[m] = s_amax[v];  // the target model's own next token
+        // walk back: the lowest predecessor that is accepted and carries length - 1
+        for (int len = m; len >= 0; --len) {
+            if (out_nodes && len < a.Tcap) out_nodes[len] = v;
+            if (len == 0) break;
+            if (len - 1 < a.Tcap) out_tok[len - 1] = s_tok[v];
+            int pred = kNone;
+            for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
+                const int p = pidx[e];
+                if (p < 0 || p >= v) continue;
+                if (s_best[p] == len - 1 && s_tok[v] == s_amax[p] && p < pred) pred = p;
+            }
+            if (pred == kNone) break;  // cannot happen for a consistent best[]
+            v = pred;
+        }
+        a.out_len[b] = m + 1;
+        s_m = m;
+        if (fl && a.status) atomicOr((unsigned*)a.status, fl);
+    }
+    __syncthreads();
+    for (int i = s_m + 1 + tid; i < a.Tcap; i += kThreads) {
+        out_tok[i] = -1;
+        if (out_nodes) out_nodes[i] = -1;
+    }
+}
+
+template <bool kVec>
+__global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a) {
+    __shared__ Best sh[kThreads / 32];
+    __shared__ int s_last;
+    const int row = blockIdx.y;  // b * N + n
+    const int split = blockIdx.x;
+    const float* x = a.logits + (size_t)row * a.V;
+    Best best{-CUDART_INF_F, kNone};
+    int lo, hi;  // element range of this slice
+    if (kVec) {
+        const int nvec = a.V >> 2;
+        const int per = (nvec + a.splits - 1) / a.splits;
+        const int v0 = min(split * per, nvec), v1 = min(v0 + per, nvec);
+        lo = v0 * 4;
+        hi = v1 * 4;
+        const float4* x4 = reinterpret_cast<const float4*>(x);
+        int i = v0 + threadIdx.x;
+        // four independent 16-byte loads in flight per thread
+        for (; i + 3 * kThreads < v1; i += 4 * kThreads) {
+            float4 r0 = __ldcs(x4 + i), r1 = __ldcs(x4 + i + kThreads);
+            float4 r2 = __ldcs(x4 + i + 2 * kThreads), r3 = __ldcs(x4 + i + 3 * kThreads);
+            int e = i * 4;
+            take(best, r0.x, e); take(best, r0.y, e + 1); take(best, r0.z, e + 2); take(best, r0.w, e + 3);
+            e += 4 * kThreads;
+            take(best, r1.x, e); take(best, r1.y, e + 1); take(best, r1.z, e + 2); take(best, r1.w, e + 3);
+            e += 4 * kThreads;
+            take(best, r2.x, e); take(best, r2.y, e + 1); take(best, r2.z, e + 2); take(best, r2.w, e + 3);
+            e += 4 * kThreads;
+            take(best, r3.x, e); take(best, r3.y, e + 1); take(best, r3.z, e + 2); take(best, r3.w, e + 3);
+        }
+        for (; i < v1; i += kThreads) {
+            float4 r = __ldcs(x4 + i);
+            const int e = i * 4;
+            take(best, r.x, e); take(best, r.y, e + 1); take(best, r.z, e + 2); take(best, r.w, e + 3);
+        }
+    } else {
+        const int per = (a.V + a.splits - 1) / a.splits;
+        lo = min(split * per, a.V);
+        hi = min(lo + per, a.V);
+        for (int i = lo + threadIdx.x; i < hi; i += kThreads) take(best, __ldcs(x + i), i);
+    }
+    best = block_best(best, sh);
+    if (best.i == kNone) {
+        // nothing above -inf in this slice: the lowest non-NaN entry (a -inf), if any, stands
+        int first = kNone;
+        for (int i = lo + threadIdx.x; i < hi; i += kThreads)
+            if (x[i] == x[i]) { first = i; break; }
+        Best f{first == kNone ? -CUDART_INF_F : 0.0f, first};  // the value only orders this reduction
+        f = block_best(f, sh);
+        best.i = f.i;
+        best.v = -CUDART_INF_F;
+    }
+    if (threadIdx.x == 0) {
+        if (best.i != kNone) atomicMax(a.keys + row, pack_key(best.v, best.i));
+        __threadfence();
+        const int b = row / a.N;
+        const unsigned prev = atomicAdd(a.done + b, 1u);
+        s_last = (prev == (unsigned)(a.N * a.splits) - 1u);
+    }
+    __syncthreads();
+    if (s_last) {
+        __threadfence();
+        path_pass(a, row / a.N);
+    }
+}
+
+}  // namespace
+}  // namespace gsd
+
+extern "C" size_t gsd_accept_workspace_bytes(const gsd_accept_params* p) {
+    if (!p || p->B < 1 || p->N < 1 || p->N > GSD_MAX_NODES) return 0;
+    return gsd::align_up((size_t)p->B * p->N * 8 + (size_t)p->B * 4, 256);
+}
+
+extern "C" int gsd_accept(const float* logits, const int32_t* draft_tokens,
+                          const int32_t* parent_ptr, const int32_t* parent_idx,
+                          int32_t* accepted_tokens, int32_t* accepted_len, int32_t* accepted_nodes,
+                          const gsd_accept_params* p, void* workspace, size_t workspace_bytes,
+                          int32_t* status, void* stream) {
+    using namespace gsd;
+    if (!p || !logits || !draft_tokens || !parent_ptr || !parent_idx || !accepted_tokens ||
+        !accepted_len)
+        return GSD_ERR_NULL_POINTER;
+    if (p->B < 1 || p->N < 1 || p->N > GSD_MAX_NODES || p->V < 1 || p->Ecap < 1 || p->Tcap < 1)
+        return GSD_ERR_BAD_SHAPE;
+    if ((long long)p->B * p->N > (1ll << 30)) return GSD_ERR_BAD_SHAPE;
+    if (((uintptr_t)logits & 3u) != 0) return GSD_ERR_MISALIGNED;
+    const size_t need = gsd_accept_workspace_bytes(p);
+    if (!workspace || workspace_bytes < need) return GSD_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 7u) != 0) return GSD_ERR_MISALIGNED;
+    DeviceInfo di;
+    if (device_info(&di) != 0) return GSD_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    AcceptArgs a;
+    a.logits = logits; a.tok = draft_tokens; a.pptr = parent_ptr; a.pidx = parent_idx;
+    a.out_tok = accepted_tokens; a.out_len = accepted_len; a.out_nodes = accepted_nodes;
+    a.keys = (unsigned long long*)workspace;
+    a.done = (unsigned*)((char*)workspace + (size_t)p->B * p->N * 8);
+    a.status = status;
+    a.B = p->B; a.N = p->N; a.V = p->V; a.Ecap = p->Ecap; a.Tcap = p->Tcap;
+    const bool vec = (p->V % 4 == 0) && (((uintptr_t)logits & 15u) == 0);
+    // enough CTAs to cover the machine a few times over, slices of at least 4096 floats
+    const long rows = (long)p->B * p->N;
+    int splits = 1;
+    const long want = (long)di.sm_count * 8;
+    while (rows * splits < want && (p->V / (splits * 2)) >= 4096) splits *= 2;
+    a.splits = splits;
+
+    GSD_CUDA_TRY(cudaMemsetAsync(workspace, 0, (size_t)p->B * p->N * 8 + (size_t)p->B * 4, st));
+    // grid.y holds at most 65535 rows: larger problems go out in blocks of whole sequences
+    // so that the per-sequence completion counter still works
+    const int seq_per = 65535 / p->N;
+    for (int b0 = 0; b0 < p->B; b0 += seq_per) {
+        const int nb = (p->B - b0 < seq_per) ? p->B - b0 : seq_per;
+        AcceptArgs s = a;
+        s.logits += (size_t)b0 * p->N * p->V; s.tok += (size_t)b0 * p->N;
+        s.pptr += (size_t)b0 * (p->N + 1); s.pidx += (size_t)b0 * p->Ecap;
+        s.out_tok += (size_t)b0 * p->Tcap; s.out_len += b0;
+        if (s.out_nodes) s.out_nodes += (size_t)b0 * p->Tcap;
+        s.keys += (size_t)b0 * p->N; s.done += b0; s.B = nb;
+        dim3 grid(splits, (unsigned)(nb * p->N));
+        if (vec) accept_kernel<true><<<grid, kThreads, 0, st>>>(s);
+        else accept_kernel<false><<<grid, kThreads, 0, st>>>(s);
+    }
+    GSD_CUDA_TRY(cudaGetLastError());
+    return GSD_OK;
+}
