@@ -1,0 +1,249 @@
+// C ABI entry points of libgsd: argument validation, kernel selection, split planning,
+// workspace layout, and the host-buffer step.  The arithmetic lives in the kernel files.
+#include "gsd_internal.cuh"
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+namespace gsd {
+
+static thread_local char g_err[256] = "";
+
+void set_cuda_error(cudaError_t e, const char* where) {
+    snprintf(g_err, sizeof g_err, "%s: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e), where);
+    (void)cudaGetLastError();  // clear a non-sticky error so that the caller's next check is clean
+}
+void set_error_text(const char* text) { snprintf(g_err, sizeof g_err, "%s", text); }
+
+int device_info(DeviceInfo* out) {
+    static DeviceInfo cache[64];
+    static bool have[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { set_cuda_error(e, "cudaGetDevice"); return -1; }
+    if (dev >= 0 && dev < 64 && have[dev]) { *out = cache[dev]; return 0; }
+    DeviceInfo di;
+    e = cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&di.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) { set_cuda_error(e, "cudaDeviceGetAttribute"); return -1; }
+    if (dev >= 0 && dev < 64) { cache[dev] = di; have[dev] = true; }
+    *out = di;
+    return 0;
+}
+
+static int attn_params_ok(const gsd_attn_params* p) {
+    if (!p) return GSD_ERR_NULL_POINTER;
+    if (p->B < 1 || p->N < 1 || p->N > GSD_MAX_NODES || p->Hq < 1 || p->Hkv < 1 ||
+        p->Hq % p->Hkv != 0 || (p->D != 64 && p->D != 128) || p->Lmax < 1 || p->num_splits < 0 ||
+        p->num_splits > 64)
+        return GSD_ERR_BAD_SHAPE;
+    if ((long long)p->B * p->Hkv > 65535) return GSD_ERR_BAD_SHAPE;
+    if ((long long)p->N * (p->Hq / p->Hkv) > (1 << 20)) return GSD_ERR_BAD_SHAPE;
+    if (p->kernel != GSD_ATTN_AUTO && p->kernel != GSD_ATTN_MMA && p->kernel != GSD_ATTN_TCGEN05)
+        return GSD_ERR_BAD_SHAPE;
+    if (p->kernel == GSD_ATTN_TCGEN05 && p->D != 128) return GSD_ERR_UNSUPPORTED;
+    return GSD_OK;
+}
+
+int attn_pick_kernel(const gsd_attn_params* p) {
+    if (p->kernel != GSD_ATTN_AUTO) return p->kernel;
+    return GSD_ATTN_MMA;
+}
+
+int attn_auto_splits(const gsd_attn_params* p, int kernel, int sm_count) {
+    if (p->num_splits > 0) return p->num_splits;
+    const int G = p->Hq / p->Hkv;
+    const int R = p->N * G;
+    const int bm = kernel == GSD_ATTN_TCGEN05 ? 128 : 64;
+    const int bn = kernel == GSD_ATTN_TCGEN05 ? 128 : 64;
+    const long ctas = (long)((R + bm - 1) / bm) * p->B * p->Hkv;
+    const int tiles = (p->Lmax + bn - 1) / bn + (p->N + bn - 1) / bn;
+    const long target = (long)sm_count * (kernel == GSD_ATTN_TCGEN05 ? 1 : 3);
+    long s = (target + ctas - 1) / ctas;
+    const int min_tiles = 4;                       // keep at least this many key tiles per split
+    if (s > tiles / min_tiles) s = tiles / min_tiles;
+    if (s > 32) s = 32;
+    if (s < 1) s = 1;
+    return (int)s;
+}
+
+size_t attn_partial_bytes(const gsd_attn_params* p, int splits) {
+    if (splits <= 1) return 0;
+    const size_t R = (size_t)p->N * (p->Hq / p->Hkv);
+    const size_t po = (size_t)p->B * p->Hkv * splits * R * p->D * sizeof(float);
+    const size_t pml = (size_t)p->B * p->Hkv * splits * R * 2 * sizeof(float);
+    return align_up(po, 256) + align_up(pml, 256);
+}
+
+}  // namespace gsd
+
+using namespace gsd;
+
+extern "C" int gsd_version(void) { return GSD_VERSION; }
+
+extern "C" const char* gsd_status_string(int s) {
+    switch (s) {
+        case GSD_OK: return "ok";
+        case GSD_ERR_NULL_POINTER: return "a required pointer is NULL";
+        case GSD_ERR_BAD_SHAPE: return "unsupported or inconsistent sizes";
+        case GSD_ERR_MISALIGNED: return "a tensor base is misaligned";
+        case GSD_ERR_WORKSPACE: return "workspace missing or too small";
+        case GSD_ERR_CUDA: return "a CUDA call failed";
+        case GSD_ERR_UNSUPPORTED: return "the requested kernel cannot run this shape";
+        default: return "unknown status";
+    }
+}
+
+extern "C" const char* gsd_last_cuda_error(void) { return g_err; }
+
+extern "C" int gsd_verify_attn_num_splits(const gsd_attn_params* p) {
+    if (attn_params_ok(p) != GSD_OK) return 0;
+    DeviceInfo di;
+    if (device_info(&di) != 0) return 0;
+    return attn_auto_splits(p, attn_pick_kernel(p), di.sm_count);
+}
+
+extern "C" size_t gsd_verify_attn_workspace_bytes(const gsd_attn_params* p) {
+    const int s = gsd_verify_attn_num_splits(p);
+    if (s <= 0) return 0;
+    return attn_partial_bytes(p, s);
+}
+
+extern "C" int gsd_verify_attn(const void* q, const void* k_cache, const void* v_cache,
+                               const void* draft_k, const void* draft_v,
+                               const uint32_t* ancestor_mask, const int32_t* seq_lens, void* out,
+                               const gsd_attn_params* p, void* workspace, size_t workspace_bytes,
+                               int32_t* status, void* stream) {
+    if (!p || !q || !k_cache || !v_cache || !draft_k || !draft_v || !ancestor_mask || !seq_lens || !out)
+        return GSD_ERR_NULL_POINTER;
+    const int ok = attn_params_ok(p);
+    if (ok != GSD_OK) return ok;
+    const void* ptrs[] = {q, k_cache, v_cache, draft_k, draft_v, out};
+    for (const void* ptr : ptrs)
+        if (((uintptr_t)ptr & 15u) != 0) return GSD_ERR_MISALIGNED;
+    if (((uintptr_t)ancestor_mask & 3u) != 0 || ((uintptr_t)seq_lens & 3u) != 0) return GSD_ERR_MISALIGNED;
+    DeviceInfo di;
+    if (device_info(&di) != 0) return GSD_ERR_CUDA;
+    const int kernel = attn_pick_kernel(p);
+    const int splits = attn_auto_splits(p, kernel, di.sm_count);
+    const size_t need = attn_partial_bytes(p, splits);
+    if (need > 0) {
+        if (!workspace || workspace_bytes < need) return GSD_ERR_WORKSPACE;
+        if (((uintptr_t)workspace & 255u) != 0) return GSD_ERR_MISALIGNED;
+    }
+    AttnArgs a;
+    a.q = q; a.k_cache = k_cache; a.v_cache = v_cache; a.draft_k = draft_k; a.draft_v = draft_v;
+    a.mask = ancestor_mask; a.seq_lens = seq_lens; a.out = out;
+    a.B = p->B; a.N = p->N; a.Hq = p->Hq; a.Hkv = p->Hkv; a.D = p->D; a.Lmax = p->Lmax;
+    a.G = p->Hq / p->Hkv; a.W = (p->N + 31) / 32;
+    const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->D);
+    a.scale_log2 = scale * 1.4426950408889634f;
+    a.num_splits = splits; a.workspace = workspace; a.status = status;
+    a.stream = (cudaStream_t)stream;
+    int rc = kernel == GSD_ATTN_TCGEN05 ? launch_attn_tcgen05(a) : launch_attn_mma(a);
+    if (rc != GSD_OK) return rc;
+    if (splits > 1) rc = launch_attn_merge(a);
+    return rc;
+}
+
+// ---------------------------------------------------------------- host-buffer step
+namespace {
+struct ArenaLayout {
+    size_t q, kc, vc, dk, dv, mask, sl, out, logits, tok, pptr, pidx, atok, alen, anodes, status,
+        ws_attn, ws_acc, total;
+    size_t b_q, b_kv, b_d, b_mask, b_sl, b_logits, b_tok, b_pptr, b_pidx, b_acc, b_len;
+};
+
+bool arena_layout(const gsd_attn_params* ap, const gsd_accept_params* cp, ArenaLayout* L) {
+    if (!ap || !cp || ap->B != cp->B || ap->N != cp->N) return false;
+    const size_t B = ap->B, N = ap->N;
+    L->b_q = B * N * ap->Hq * ap->D * 2;
+    L->b_kv = B * (size_t)ap->Lmax * ap->Hkv * ap->D * 2;
+    L->b_d = B * N * ap->Hkv * ap->D * 2;
+    L->b_mask = B * N * ((N + 31) / 32) * 4;
+    L->b_sl = B * 4;
+    L->b_logits = B * N * (size_t)cp->V * 4;
+    L->b_tok = B * N * 4;
+    L->b_pptr = B * (N + 1) * 4;
+    L->b_pidx = B * (size_t)cp->Ecap * 4;
+    L->b_acc = B * (size_t)cp->Tcap * 4;
+    L->b_len = B * 4;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L->q = take(L->b_q); L->kc = take(L->b_kv); L->vc = take(L->b_kv); L->dk = take(L->b_d);
+    L->dv = take(L->b_d); L->mask = take(L->b_mask); L->sl = take(L->b_sl); L->out = take(L->b_q);
+    L->logits = take(L->b_logits); L->tok = take(L->b_tok); L->pptr = take(L->b_pptr);
+    L->pidx = take(L->b_pidx); L->atok = take(L->b_acc); L->alen = take(L->b_len);
+    L->anodes = take(L->b_acc); L->status = take(4);
+    L->ws_attn = take(gsd_verify_attn_workspace_bytes(ap));
+    L->ws_acc = take(gsd_accept_workspace_bytes(cp));
+    L->total = off;
+    return true;
+}
+}  // namespace
+
+extern "C" size_t gsd_verify_step_host_arena_bytes(const gsd_attn_params* ap, const gsd_accept_params* cp) {
+    ArenaLayout L;
+    if (attn_params_ok(ap) != GSD_OK || !cp || cp->V < 1 || cp->Ecap < 1 || cp->Tcap < 1) return 0;
+    if (!arena_layout(ap, cp, &L)) return 0;
+    return L.total;
+}
+
+extern "C" int gsd_verify_step_host(const void* q, const void* k_cache, const void* v_cache,
+                                    const void* draft_k, const void* draft_v,
+                                    const uint32_t* ancestor_mask, const int32_t* seq_lens, void* out,
+                                    const gsd_attn_params* ap, const float* logits,
+                                    const int32_t* draft_tokens, const int32_t* parent_ptr,
+                                    const int32_t* parent_idx, int32_t* accepted_tokens,
+                                    int32_t* accepted_len, int32_t* accepted_nodes,
+                                    const gsd_accept_params* cp, void* arena, size_t arena_bytes,
+                                    int32_t* device_status_out, void* stream) {
+    if (!ap || !cp || !q || !k_cache || !v_cache || !draft_k || !draft_v || !ancestor_mask ||
+        !seq_lens || !out || !logits || !draft_tokens || !parent_ptr || !parent_idx ||
+        !accepted_tokens || !accepted_len || !arena)
+        return GSD_ERR_NULL_POINTER;
+    const int ok = attn_params_ok(ap);
+    if (ok != GSD_OK) return ok;
+    ArenaLayout L;
+    if (!arena_layout(ap, cp, &L)) return GSD_ERR_BAD_SHAPE;
+    if (arena_bytes < L.total) return GSD_ERR_WORKSPACE;
+    if (((uintptr_t)arena & 255u) != 0) return GSD_ERR_MISALIGNED;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* base = (char*)arena;
+    auto h2d = [&](size_t off, const void* src, size_t bytes) {
+        return cudaMemcpyAsync(base + off, src, bytes, cudaMemcpyHostToDevice, st);
+    };
+    GSD_CUDA_TRY(h2d(L.q, q, L.b_q));
+    GSD_CUDA_TRY(h2d(L.kc, k_cache, L.b_kv));
+    GSD_CUDA_TRY(h2d(L.vc, v_cache, L.b_kv));
+    GSD_CUDA_TRY(h2d(L.dk, draft_k, L.b_d));
+    GSD_CUDA_TRY(h2d(L.dv, draft_v, L.b_d));
+    GSD_CUDA_TRY(h2d(L.mask, ancestor_mask, L.b_mask));
+    GSD_CUDA_TRY(h2d(L.sl, seq_lens, L.b_sl));
+    GSD_CUDA_TRY(h2d(L.logits, logits, L.b_logits));
+    GSD_CUDA_TRY(h2d(L.tok, draft_tokens, L.b_tok));
+    GSD_CUDA_TRY(h2d(L.pptr, parent_ptr, L.b_pptr));
+    GSD_CUDA_TRY(h2d(L.pidx, parent_idx, L.b_pidx));
+    GSD_CUDA_TRY(cudaMemsetAsync(base + L.status, 0, 4, st));
+    int rc = gsd_verify_attn(base + L.q, base + L.kc, base + L.vc, base + L.dk, base + L.dv,
+                             (const uint32_t*)(base + L.mask), (const int32_t*)(base + L.sl),
+                             base + L.out, ap, base + L.ws_attn,
+                             gsd_verify_attn_workspace_bytes(ap), (int32_t*)(base + L.status), stream);
+    if (rc != GSD_OK) return rc;
+    rc = gsd_accept((const float*)(base + L.logits), (const int32_t*)(base + L.tok),
+                    (const int32_t*)(base + L.pptr), (const int32_t*)(base + L.pidx),
+                    (int32_t*)(base + L.atok), (int32_t*)(base + L.alen),
+                    (int32_t*)(base + L.anodes), cp, base + L.ws_acc,
+                    gsd_accept_workspace_bytes(cp), (int32_t*)(base + L.status), stream);
+    if (rc != GSD_OK) return rc;
+    GSD_CUDA_TRY(cudaMemcpyAsync(out, base + L.out, L.b_q, cudaMemcpyDeviceToHost, st));
+    GSD_CUDA_TRY(cudaMemcpyAsync(accepted_tokens, base + L.atok, L.b_acc, cudaMemcpyDeviceToHost, st));
+    GSD_CUDA_TRY(cudaMemcpyAsync(accepted_len, base + L.alen, L.b_len, cudaMemcpyDeviceToHost, st));
+    if (accepted_nodes)
+        GSD_CUDA_TRY(cudaMemcpyAsync(accepted_nodes, base + L.anodes, L.b_acc, cudaMemcpyDeviceToHost, st));
+    int32_t dev_status = 0;
+    GSD_CUDA_TRY(cudaMemcpyAsync(&dev_status, base + L.status, 4, cudaMemcpyDeviceToHost, st));
+    GSD_CUDA_TRY(cudaStreamSynchronize(st));
+    if (device_status_out) *device_status_out = dev_status;
+    return GSD_OK;
+}
