@@ -1,0 +1,257 @@
+"""ctypes binding of libgsd.so with the same names as the C ABI (include/gsd.h).
+
+The functions take torch tensors (CUDA tensors for the device calls, CPU tensors for the
+host-buffer step), check dtype / shape / contiguity, and pass raw pointers, sizes and the
+current CUDA stream.  PyTorch is used for memory and streams only.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+GSD_ATTN_AUTO, GSD_ATTN_MMA, GSD_ATTN_TCGEN05 = 0, 1, 2
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libgsd.so")
+_lib: Optional[ctypes.CDLL] = None
+
+
+class GsdError(RuntimeError):
+    """A negative gsd_status returned by the library."""
+
+    def __init__(self, code: int, what: str):
+        super().__init__(what)
+        self.code = code
+
+
+class AttnParams(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("N", ctypes.c_int32), ("Hq", ctypes.c_int32),
+                ("Hkv", ctypes.c_int32), ("D", ctypes.c_int32), ("Lmax", ctypes.c_int32),
+                ("softmax_scale", ctypes.c_float), ("num_splits", ctypes.c_int32),
+                ("kernel", ctypes.c_int32)]
+
+
+class AcceptParams(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("N", ctypes.c_int32), ("V", ctypes.c_int32),
+                ("Ecap", ctypes.c_int32), ("Tcap", ctypes.c_int32)]
+
+
+EXPORTS = ["gsd_version", "gsd_status_string", "gsd_last_cuda_error", "gsd_verify_attn",
+           "gsd_verify_attn_workspace_bytes", "gsd_verify_attn_num_splits", "gsd_accept",
+           "gsd_accept_workspace_bytes", "gsd_verify_step_host",
+           "gsd_verify_step_host_arena_bytes"]
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def lib() -> ctypes.CDLL:
+    """Load libgsd.so (built in-tree by paper_2407_16207_b200/build.py). No fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise GsdError(-100, f"{_LIB_PATH} is missing: run `python -m paper_2407_16207_b200.build` "
+                                 "(there is no CPU fallback)")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, sz, i32 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+        L.gsd_version.restype = i32
+        L.gsd_status_string.restype = ctypes.c_char_p
+        L.gsd_status_string.argtypes = [i32]
+        L.gsd_last_cuda_error.restype = ctypes.c_char_p
+        L.gsd_verify_attn.restype = i32
+        L.gsd_verify_attn.argtypes = [vp] * 8 + [ctypes.POINTER(AttnParams), vp, sz, vp, vp]
+        L.gsd_verify_attn_workspace_bytes.restype = sz
+        L.gsd_verify_attn_workspace_bytes.argtypes = [ctypes.POINTER(AttnParams)]
+        L.gsd_verify_attn_num_splits.restype = i32
+        L.gsd_verify_attn_num_splits.argtypes = [ctypes.POINTER(AttnParams)]
+        L.gsd_accept.restype = i32
+        L.gsd_accept.argtypes = [vp] * 7 + [ctypes.POINTER(AcceptParams), vp, sz, vp, vp]
+        L.gsd_accept_workspace_bytes.restype = sz
+        L.gsd_accept_workspace_bytes.argtypes = [ctypes.POINTER(AcceptParams)]
+        L.gsd_verify_step_host.restype = i32
+        L.gsd_verify_step_host.argtypes = ([vp] * 8 + [ctypes.POINTER(AttnParams)] + [vp] * 7
+                                           + [ctypes.POINTER(AcceptParams), vp, sz, vp, vp])
+        L.gsd_verify_step_host_arena_bytes.restype = sz
+        L.gsd_verify_step_host_arena_bytes.argtypes = [ctypes.POINTER(AttnParams),
+                                                       ctypes.POINTER(AcceptParams)]
+        _lib = L
+    return _lib
+
+
+def _check(rc: int) -> None:
+    if rc != 0:
+        L = lib()
+        msg = L.gsd_status_string(rc).decode()
+        if rc == -5:
+            msg += ": " + L.gsd_last_cuda_error().decode()
+        raise GsdError(rc, f"gsd error {rc}: {msg}")
+
+
+def gsd_version() -> int:
+    return int(lib().gsd_version())
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _want(t: torch.Tensor, dtype, shape, name: str, cuda: bool) -> None:
+    if t.dtype != dtype or tuple(t.shape) != tuple(shape) or not t.is_contiguous():
+        raise ValueError(f"{name}: expected contiguous {dtype} {tuple(shape)}, got {t.dtype} "
+                         f"{tuple(t.shape)}")
+    if t.is_cuda != cuda:
+        raise ValueError(f"{name}: expected a {'CUDA' if cuda else 'CPU'} tensor")
+
+
+def _stream(t: torch.Tensor) -> int:
+    return torch.cuda.current_stream(t.device).cuda_stream
+
+
+def _attn_params(q, k_cache, draft_k, softmax_scale, num_splits, kernel) -> AttnParams:
+    B, N, Hq, D = q.shape
+    Lmax, Hkv = k_cache.shape[1], k_cache.shape[2]
+    return AttnParams(B, N, Hq, Hkv, D, Lmax, float(softmax_scale), int(num_splits), int(kernel))
+
+
+def _check_attn_tensors(q, k_cache, v_cache, draft_k, draft_v, ancestor_mask, seq_lens, cuda):
+    bf = torch.bfloat16
+    if q.dim() != 4 or k_cache.dim() != 4:
+        raise ValueError("q must be [B,N,Hq,D] and k_cache [B,Lmax,Hkv,D]")
+    B, N, Hq, D = q.shape
+    Lmax, Hkv = k_cache.shape[1], k_cache.shape[2]
+    _want(q, bf, (B, N, Hq, D), "q", cuda)
+    _want(k_cache, bf, (B, Lmax, Hkv, D), "k_cache", cuda)
+    _want(v_cache, bf, (B, Lmax, Hkv, D), "v_cache", cuda)
+    _want(draft_k, bf, (B, N, Hkv, D), "draft_k", cuda)
+    _want(draft_v, bf, (B, N, Hkv, D), "draft_v", cuda)
+    if ancestor_mask.dtype not in (torch.int32, torch.uint32):
+        raise ValueError("ancestor_mask must hold 32-bit words (int32 or uint32)")
+    _want(ancestor_mask, ancestor_mask.dtype, (B, N, (N + 31) // 32), "ancestor_mask", cuda)
+    _want(seq_lens, torch.int32, (B,), "seq_lens", cuda)
+
+
+def gsd_verify_attn_num_splits(B, N, Hq, Hkv, D, Lmax, num_splits=0, kernel=GSD_ATTN_AUTO) -> int:
+    p = AttnParams(B, N, Hq, Hkv, D, Lmax, 0.0, num_splits, kernel)
+    return int(lib().gsd_verify_attn_num_splits(ctypes.byref(p)))
+
+
+def gsd_verify_attn_workspace_bytes(B, N, Hq, Hkv, D, Lmax, num_splits=0,
+                                    kernel=GSD_ATTN_AUTO) -> int:
+    p = AttnParams(B, N, Hq, Hkv, D, Lmax, 0.0, num_splits, kernel)
+    return int(lib().gsd_verify_attn_workspace_bytes(ctypes.byref(p)))
+
+
+def gsd_verify_attn(q, k_cache, v_cache, draft_k, draft_v, ancestor_mask, seq_lens,
+                    out: Optional[torch.Tensor] = None, *, softmax_scale: float = 0.0,
+                    num_splits: int = 0, kernel: int = GSD_ATTN_AUTO,
+                    workspace: Optional[torch.Tensor] = None,
+                    status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """DAG-masked attention of the draft nodes; see gsd_verify_attn in include/gsd.h.
+    Enqueued on the current stream; returns `out` [B,N,Hq,D] bf16."""
+    _check_attn_tensors(q, k_cache, v_cache, draft_k, draft_v, ancestor_mask, seq_lens, True)
+    if out is None:
+        out = torch.empty_like(q)
+    _want(out, torch.bfloat16, q.shape, "out", True)
+    p = _attn_params(q, k_cache, draft_k, softmax_scale, num_splits, kernel)
+    L = lib()
+    with torch.cuda.device(q.device):
+        need = int(L.gsd_verify_attn_workspace_bytes(ctypes.byref(p)))
+        if workspace is None and need:
+            workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+        ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        _check(L.gsd_verify_attn(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(),
+                                 draft_k.data_ptr(), draft_v.data_ptr(), ancestor_mask.data_ptr(),
+                                 seq_lens.data_ptr(), out.data_ptr(), ctypes.byref(p),
+                                 _ptr(workspace), ws_bytes, _ptr(status), _stream(q)))
+    return out
+
+
+def gsd_accept_workspace_bytes(B, N, V=1, Ecap=1, Tcap=1) -> int:
+    p = AcceptParams(B, N, V, Ecap, Tcap)
+    return int(lib().gsd_accept_workspace_bytes(ctypes.byref(p)))
+
+
+def gsd_accept(logits, draft_tokens, parent_ptr, parent_idx, *, Tcap: int = 0,
+               want_nodes: bool = True, workspace: Optional[torch.Tensor] = None,
+               status: Optional[torch.Tensor] = None,
+               out: Optional[Tuple[torch.Tensor, torch.Tensor, Optional[torch.Tensor]]] = None
+               ) -> Tuple[torch.Tensor, torch.Tensor, Optional[torch.Tensor]]:
+    """Greedy verification + longest accepted path; see gsd_accept in include/gsd.h.
+    Returns (accepted_tokens [B,Tcap], accepted_len [B], accepted_nodes [B,Tcap] or None)."""
+    if logits.dim() != 3:
+        raise ValueError("logits must be [B,N,V]")
+    B, N, V = logits.shape
+    _want(logits, torch.float32, (B, N, V), "logits", True)
+    _want(draft_tokens, torch.int32, (B, N), "draft_tokens", True)
+    _want(parent_ptr, torch.int32, (B, N + 1), "parent_ptr", True)
+    if parent_idx.dim() != 2:
+        raise ValueError("parent_idx must be [B,Ecap]")
+    Ecap = parent_idx.shape[1]
+    _want(parent_idx, torch.int32, (B, Ecap), "parent_idx", True)
+    Tcap = Tcap or N
+    if out is None:
+        toks = torch.empty((B, Tcap), dtype=torch.int32, device=logits.device)
+        lens = torch.empty((B,), dtype=torch.int32, device=logits.device)
+        nodes = torch.empty((B, Tcap), dtype=torch.int32, device=logits.device) if want_nodes else None
+    else:
+        toks, lens, nodes = out
+    p = AcceptParams(B, N, V, Ecap, Tcap)
+    L = lib()
+    with torch.cuda.device(logits.device):
+        need = int(L.gsd_accept_workspace_bytes(ctypes.byref(p)))
+        if workspace is None:
+            workspace = torch.empty(max(need, 8), dtype=torch.uint8, device=logits.device)
+        _check(L.gsd_accept(logits.data_ptr(), draft_tokens.data_ptr(), parent_ptr.data_ptr(),
+                            parent_idx.data_ptr(), toks.data_ptr(), lens.data_ptr(), _ptr(nodes),
+                            ctypes.byref(p), workspace.data_ptr(),
+                            workspace.numel() * workspace.element_size(), _ptr(status),
+                            _stream(logits)))
+    return toks, lens, nodes
+
+
+def gsd_verify_step_host_arena_bytes(B, N, Hq, Hkv, D, Lmax, V, Ecap, Tcap, num_splits=0,
+                                     kernel=GSD_ATTN_AUTO) -> int:
+    ap = AttnParams(B, N, Hq, Hkv, D, Lmax, 0.0, num_splits, kernel)
+    cp = AcceptParams(B, N, V, Ecap, Tcap)
+    return int(lib().gsd_verify_step_host_arena_bytes(ctypes.byref(ap), ctypes.byref(cp)))
+
+
+def gsd_verify_step_host(q, k_cache, v_cache, draft_k, draft_v, ancestor_mask, seq_lens, logits,
+                         draft_tokens, parent_ptr, parent_idx, arena: torch.Tensor, *,
+                         out=None, accepted=None, Tcap: int = 0, softmax_scale: float = 0.0,
+                         num_splits: int = 0, kernel: int = GSD_ATTN_AUTO):
+    """One whole verification step from HOST tensors through a caller-owned device arena;
+    see gsd_verify_step_host in include/gsd.h.  Synchronises the current stream.
+    Returns (out [B,N,Hq,D] bf16 CPU, accepted_tokens, accepted_len, accepted_nodes, status)."""
+    _check_attn_tensors(q, k_cache, v_cache, draft_k, draft_v, ancestor_mask, seq_lens, False)
+    B, N, V = logits.shape
+    Ecap = parent_idx.shape[1]
+    _want(logits, torch.float32, (B, N, V), "logits", False)
+    _want(draft_tokens, torch.int32, (B, N), "draft_tokens", False)
+    _want(parent_ptr, torch.int32, (B, N + 1), "parent_ptr", False)
+    _want(parent_idx, torch.int32, (B, Ecap), "parent_idx", False)
+    Tcap = Tcap or N
+    if out is None:
+        out = torch.empty_like(q)
+    if accepted is None:
+        accepted = (torch.empty((B, Tcap), dtype=torch.int32), torch.empty((B,), dtype=torch.int32),
+                    torch.empty((B, Tcap), dtype=torch.int32))
+    toks, lens, nodes = accepted
+    ap = _attn_params(q, k_cache, draft_k, softmax_scale, num_splits, kernel)
+    cp = AcceptParams(B, N, V, Ecap, Tcap)
+    dev_status = ctypes.c_int32(0)
+    if not arena.is_cuda:
+        raise ValueError("arena must be a CUDA tensor")
+    with torch.cuda.device(arena.device):
+        _check(lib().gsd_verify_step_host(
+            q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), draft_k.data_ptr(),
+            draft_v.data_ptr(), ancestor_mask.data_ptr(), seq_lens.data_ptr(), out.data_ptr(),
+            ctypes.byref(ap), logits.data_ptr(), draft_tokens.data_ptr(), parent_ptr.data_ptr(),
+            parent_idx.data_ptr(), toks.data_ptr(), lens.data_ptr(), _ptr(nodes), ctypes.byref(cp),
+            arena.data_ptr(), arena.numel() * arena.element_size(),
+            ctypes.addressof(dev_status), _stream(arena)))
+    return out, toks, lens, nodes, int(dev_status.value)

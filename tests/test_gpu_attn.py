@@ -1,0 +1,150 @@
+"""gsd_verify_attn on the GPU against the fp64 CPU oracle.
+
+Tolerance (bf16 output against fp64): max-abs <= 1e-2 and mean-abs <= 1e-3."""
+import numpy as np
+import pytest
+import torch
+
+import gsd_inputs as gi
+import oracle
+from gpu_util import attn_tensors, out_to_f64
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS = 1e-2, 1e-3
+KERNELS = [1, 2]        # GSD_ATTN_MMA, GSD_ATTN_TCGEN05
+
+
+def gpu_attn(inp, **kw):
+    import paper_2407_16207_b200 as gsd
+    t = attn_tensors(inp)
+    try:
+        out = gsd.gsd_verify_attn(t["q"], t["k_cache"], t["v_cache"], t["draft_k"], t["draft_v"],
+                                  t["ancestor_mask"], t["seq_lens"], **kw)
+    except gsd.GsdError as e:
+        if e.code == -6:
+            pytest.skip("kernel variant does not cover this shape")
+        raise
+    torch.cuda.synchronize()
+    return out
+
+
+def cpu_attn(inp, **kw):
+    return oracle.attn(inp["q"], inp["k_cache"], inp["v_cache"], inp["draft_k"], inp["draft_v"],
+                       inp["ancestor_mask"], inp["seq_lens"], **kw)
+
+
+def assert_close(got64, want):
+    assert np.isfinite(got64).all()
+    err = np.abs(got64 - want)
+    assert err.max() <= MAX_ABS, f"max-abs {err.max():.3e}"
+    assert err.mean() <= MEAN_ABS, f"mean-abs {err.mean():.3e}"
+
+
+def variant(cfg, **kw):
+    return gi.VerifyConfig(**{**cfg.__dict__, **kw})
+
+
+@pytest.mark.parametrize("kernel", [0] + KERNELS)
+@pytest.mark.parametrize("name", ["tiny", "llama7b", "llama13b"])
+def test_configs_full_compare(name, kernel):
+    cfg = gi.CONFIGS[name]
+    for trial in range(2 if name != "llama13b" else 1):
+        inp = gi.make_inputs(cfg, gi.seed_for(cfg, trial), accept=False)
+        assert_close(out_to_f64(gpu_attn(inp, kernel=kernel)), cpu_attn(inp))
+
+
+@pytest.mark.parametrize("kernel", [0] + KERNELS)
+def test_llama70b_sampled_rows_and_one_full_unit(kernel):
+    # full-size configuration: the oracle recomputes one whole (sequence, kv head) unit and
+    # 1024 random rows one by one
+    cfg = gi.CONFIGS["llama70b"]
+    inp = gi.make_inputs(cfg, accept=False)
+    got = out_to_f64(gpu_attn(inp, kernel=kernel))
+    rng = np.random.default_rng(4)
+    rows = [(3, n, 5 * cfg.G + g) for n in range(cfg.N) for g in range(cfg.G)]
+    rows += [(int(rng.integers(cfg.B)), int(rng.integers(cfg.N)), int(rng.integers(cfg.Hq)))
+             for _ in range(1024)]
+    want = oracle.attn_rows(inp["q"], inp["k_cache"], inp["v_cache"], inp["draft_k"],
+                            inp["draft_v"], inp["ancestor_mask"], inp["seq_lens"], rows)
+    g = np.stack([got[b, n, h] for b, n, h in rows])
+    assert_close(g, want)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("shape", [
+    dict(B=2, Hq=8, Hkv=2, D=64, L=(1, 300), N=37, depth=8),          # GQA, D=64, ragged, odd N
+    dict(B=3, Hq=6, Hkv=2, D=128, L=(100, 700), N=130, depth=12, kmax=4, pmax=3),
+    dict(B=2, Hq=8, Hkv=1, D=128, L=(0, 65), N=200, depth=14, kmax=4, pmax=3),   # MQA, short prefixes
+    dict(B=1, Hq=16, Hkv=2, D=128, L=129, N=512, depth=18, kmax=4, pmax=3),      # maximum N
+    dict(B=1, Hq=2, Hkv=2, D=64, L=5, N=1, depth=0),                   # a single node
+])
+def test_ragged_shapes_nan_padding(shape, kernel):
+    base = dict(name="t", config_id=7, kmax=3, pmax=2, V=8, vtok=8, p_agree=0.5)
+    cfg = gi.VerifyConfig(**{**base, **shape})
+    inp = gi.make_inputs(cfg, 77, accept=False, pad_fill="nan")
+    assert_close(out_to_f64(gpu_attn(inp, kernel=kernel)), cpu_attn(inp))
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_arbitrary_mask_bits_and_empty_rows(kernel):
+    # random bit patterns (not triangular, padding bits set), some rows with no key at all
+    cfg = gi.VerifyConfig("t", 7, 2, 8, 4, 128, (0, 40), 70, 8, 3, 2, 8, 8, 0.5)
+    inp = gi.make_inputs(cfg, 5, accept=False, pad_fill="nan")
+    rng = np.random.default_rng(9)
+    inp["ancestor_mask"] = rng.integers(0, 2 ** 32, size=inp["ancestor_mask"].shape, dtype=np.uint32)
+    inp["ancestor_mask"][0, 3] = 0
+    inp["ancestor_mask"][1, :, :] &= np.uint32(0x00010001)
+    inp["seq_lens"][0] = 0
+    got = out_to_f64(gpu_attn(inp, kernel=kernel))
+    want = cpu_attn(inp)
+    assert_close(got, want)
+    assert np.all(got[0, 3] == 0)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_split_count_invariance_and_determinism(kernel):
+    cfg = gi.CONFIGS["llama7b"]
+    inp = gi.make_inputs(cfg, accept=False)
+    want = cpu_attn(inp)
+    outs = {}
+    for s in (1, 2, 3, 7):
+        outs[s] = gpu_attn(inp, kernel=kernel, num_splits=s)
+        assert_close(out_to_f64(outs[s]), want)
+        again = gpu_attn(inp, kernel=kernel, num_splits=s)
+        assert torch.equal(outs[s], again)                     # bit-identical run to run
+    for s in (2, 3, 7):
+        assert (outs[s].float() - outs[1].float()).abs().max().item() <= 4e-3
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_softmax_scale_override(kernel):
+    cfg = gi.CONFIGS["tiny"] if kernel == 1 else variant(gi.CONFIGS["tiny"], D=128)
+    inp = gi.make_inputs(cfg, accept=False)
+    assert_close(out_to_f64(gpu_attn(inp, kernel=kernel, softmax_scale=0.3)), cpu_attn(inp, scale=0.3))
+
+
+def test_canary_padding_is_untouched():
+    import paper_2407_16207_b200 as gsd
+    cfg = gi.CONFIGS["tiny"]
+    inp = gi.make_inputs(cfg, accept=False)
+    t = attn_tensors(inp)
+    n = t["q"].numel()
+    buf = torch.full((n + 512,), 7.0, dtype=torch.bfloat16, device="cuda")
+    out = buf[256:256 + n].view_as(t["q"])
+    gsd.gsd_verify_attn(t["q"], t["k_cache"], t["v_cache"], t["draft_k"], t["draft_v"],
+                        t["ancestor_mask"], t["seq_lens"], out=out)
+    torch.cuda.synchronize()
+    assert (buf[:256] == 7.0).all() and (buf[256 + n:] == 7.0).all()
+
+
+def test_bad_seq_len_is_clamped_and_flagged():
+    cfg = gi.CONFIGS["tiny"]
+    inp = gi.make_inputs(cfg, accept=False)
+    want = cpu_attn(inp)
+    inp2 = dict(inp)
+    inp2["seq_lens"] = np.array([10_000], dtype=np.int32)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got = out_to_f64(gpu_attn(inp2, status=status))
+    assert int(status.item()) == 0x10
+    assert_close(got, want)          # clamped to Lmax == the true length here
