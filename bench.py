@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Benchmark of the GSD verification step (gsd_verify_attn + gsd_accept) on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama70b] [--impl ours|reference]
+
+A step is one pass of the whole hot path over one batch of synthetic LLaMA-2-shaped input:
+DAG-masked attention of all draft nodes, then vocabulary argmax and longest accepted path.
+Prints ONE JSON line (rank 0).  With N > 1 every rank runs an independent replica of the
+workload (the path has no cross-GPU exchange), timed as the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+sys.path.insert(0, os.path.join(ROOT, "tests"))
+
+import gsd_inputs as gi  # noqa: E402
+
+METRIC = "draft_tokens_verified_per_s_per_attn_layer"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+def algorithmic_work(cfg, inp):
+    """Algorithmic flops and bytes of one gsd_verify_attn call and bytes of one gsd_accept call.
+
+    flops: 4 * Hq * D per (node, visible key): prefix keys seq_lens[b] plus the set mask bits.
+    bytes: K and V of the visible prefix and of the draft block once per kv head, Q in and
+    out once, the mask once; accept reads the logits once."""
+    B, N, Hq, Hkv, D = cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.D
+    L = inp["seq_lens"].astype(np.int64)
+    bits = np.unpackbits(inp["ancestor_mask"].view(np.uint8), axis=-1).reshape(B, N, -1).sum(-1)
+    visible = (L[:, None] + bits).sum()
+    flops = 4.0 * Hq * D * float(visible)
+    kv_bytes = 2 * 2 * D * Hkv * float((L + N).sum())
+    qo_bytes = 2 * 2 * D * Hq * B * N
+    mask_bytes = inp["ancestor_mask"].nbytes
+    accept_bytes = 4.0 * B * N * cfg.V
+    return flops, kv_bytes + qo_bytes + mask_bytes, accept_bytes
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            uuid = torch.cuda.get_device_properties(index).uuid
+            sel = f"GPU-{uuid}"
+        except Exception:
+            sel = str(index)
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", sel], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+def dist_setup(n_gpus: int):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        return rank, world, local, dist
+    torch.cuda.set_device(local)
+    return rank, world, local, None
+
+
+def cpu_oracle_sample(cfg, inp, budget_rows: int):
+    """Times the CPU oracle (as it stands) on a bounded sample of the workload: `budget_rows`
+    random attention rows plus the full acceptance step.  Returns (tokens/s extrapolated to
+    the whole step, threads, description)."""
+    import oracle
+    rng = np.random.default_rng(0)
+    total_rows = cfg.B * cfg.N * cfg.Hq
+    n = min(budget_rows, total_rows)
+    rows = np.stack([rng.integers(cfg.B, size=n), rng.integers(cfg.N, size=n),
+                     rng.integers(cfg.Hq, size=n)], axis=1).astype(np.int32)
+    t0 = time.perf_counter()
+    oracle.attn_rows(inp["q"], inp["k_cache"], inp["v_cache"], inp["draft_k"], inp["draft_v"],
+                     inp["ancestor_mask"], inp["seq_lens"], rows)
+    t_attn = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    oracle.accept(inp["logits"], inp["draft_tokens"], inp["parent_ptr"], inp["parent_idx"])
+    t_acc = time.perf_counter() - t0
+    t_step = t_attn * (total_rows / n) + t_acc
+    desc = (f"{n} of {total_rows} attention rows (random (b,n,h), {t_attn:.2f} s, scaled to all rows) "
+            f"+ full acceptance ({t_acc:.2f} s)")
+    return cfg.B * cfg.N / t_step, oracle.threads(), desc
+
+
+def run_reference(args, cfg):
+    """The reference arm: the CPU oracle, timed on the host cores, each step a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    inp = gi.make_inputs(cfg)
+    total_rows = cfg.B * cfg.N * cfg.Hq
+    rows_per_step = min(total_rows, max(256, 8192 // max(1, (args.steps + args.warmup) // 4)))
+    vals = []
+    desc = ""
+    for i in range(args.warmup + args.steps):
+        v, threads, desc = cpu_oracle_sample(cfg, inp, rows_per_step)
+        if i >= args.warmup:
+            vals.append(v)
+    value = cfg.B * cfg.N * len(vals) / sum(cfg.B * cfg.N / v for v in vals)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * cfg.B * cfg.N / value, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "B": cfg.B, "N": cfg.N, "Hq": cfg.Hq, "Hkv": cfg.Hkv,
+                       "D": cfg.D, "L": cfg.L, "V": cfg.V},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": "per step: " + desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="llama70b", choices=sorted(gi.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 mma.sync, 2 tcgen05")
+    ap.add_argument("--num-splits", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--cpu-rows", type=int, default=16384,
+                    help="attention rows in the CPU-oracle sample (0 = skip the CPU baseline)")
+    args = ap.parse_args()
+    cfg = gi.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import paper_2407_16207_b200 as gsd
+    from gpu_util import accept_tensors, attn_tensors
+    gsd.lib()  # fail loudly if the CUDA library is missing
+    rank, world, local, dist = dist_setup(args.gpus)
+    dev = torch.device("cuda", local)
+
+    # inputs: two independent sets, rotated, so that every step reads ~0.5 GB it has not just
+    # touched (more than the 126 MB L2)
+    NSETS = 2
+    host_sets = [gi.make_inputs(cfg, gi.seed_for(cfg, 10 * rank + s)) for s in range(NSETS)]
+    sets = []
+    for inp in host_sets:
+        t = {**attn_tensors(inp, dev), **accept_tensors(inp, dev)}
+        t["out"] = torch.empty_like(t["q"])
+        sets.append(t)
+    Lmax = host_sets[0]["Lmax"]
+    ws_bytes = gsd.gsd_verify_attn_workspace_bytes(cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.D,
+                                                   max(h["Lmax"] for h in host_sets),
+                                                   args.num_splits, args.kernel)
+    ws_attn = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=dev)
+    ws_acc = torch.empty(gsd.gsd_accept_workspace_bytes(cfg.B, cfg.N), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    acc_out = (torch.empty((cfg.B, cfg.N), dtype=torch.int32, device=dev),
+               torch.empty((cfg.B,), dtype=torch.int32, device=dev),
+               torch.empty((cfg.B, cfg.N), dtype=torch.int32, device=dev))
+    splits = gsd.gsd_verify_attn_num_splits(cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.D, Lmax,
+                                            args.num_splits, args.kernel)
+
+    def step(i, ev=None):
+        t = sets[i % NSETS]
+        if ev:
+            ev[0].record()
+        gsd.gsd_verify_attn(t["q"], t["k_cache"], t["v_cache"], t["draft_k"], t["draft_v"],
+                            t["ancestor_mask"], t["seq_lens"], out=t["out"], kernel=args.kernel,
+                            num_splits=args.num_splits, workspace=ws_attn, status=status)
+        if ev:
+            ev[1].record()
+        gsd.gsd_accept(t["logits"], t["draft_tokens"], t["parent_ptr"], t["parent_idx"],
+                       workspace=ws_acc, status=status, out=acc_out)
+        if ev:
+            ev[2].record()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    e_begin.record()
+    for i in range(args.steps):
+        step(i, events[i])
+    e_end.record()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    total_ms = e_begin.elapsed_time(e_end)
+    attn_ms = [ev[0].elapsed_time(ev[1]) for ev in events]
+    acc_ms = [ev[1].elapsed_time(ev[2]) for ev in events]
+    if int(status.item()) != 0:
+        raise RuntimeError(f"device status {int(status.item()):#x}")
+    if dist is not None:
+        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    tokens = cfg.B * cfg.N
+    value = world * tokens / (ms_per_step * 1e-3)
+
+    # ---- end to end through the host-buffer C-ABI call (pinned host tensors)
+    e2e = None
+    if args.e2e_steps > 0:
+        h = {**attn_tensors(host_sets[0], "cpu"), **accept_tensors(host_sets[0], "cpu")}
+        h = {k: v.pin_memory() for k, v in h.items()}
+        Ecap = h["parent_idx"].shape[1]
+        nbytes = gsd.gsd_verify_step_host_arena_bytes(cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.D, Lmax,
+                                                      cfg.V, Ecap, cfg.N, args.num_splits, args.kernel)
+        arena = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        h_out = torch.empty_like(h["q"]).pin_memory()
+        h_acc = (torch.empty((cfg.B, cfg.N), dtype=torch.int32).pin_memory(),
+                 torch.empty((cfg.B,), dtype=torch.int32).pin_memory(),
+                 torch.empty((cfg.B, cfg.N), dtype=torch.int32).pin_memory())
+
+        def host_step():
+            return gsd.gsd_verify_step_host(
+                h["q"], h["k_cache"], h["v_cache"], h["draft_k"], h["draft_v"], h["ancestor_mask"],
+                h["seq_lens"], h["logits"], h["draft_tokens"], h["parent_ptr"], h["parent_idx"], arena,
+                out=h_out, accepted=h_acc, kernel=args.kernel, num_splits=args.num_splits)
+
+        for _ in range(2):
+            host_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            host_step()
+        torch.cuda.synchronize()
+        t_e2e = (time.perf_counter() - t0) / args.e2e_steps
+        if dist is not None:
+            tt = torch.tensor([t_e2e], dtype=torch.float64, device=dev)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            t_e2e = float(tt.item())
+        h2d = sum(h[k].numel() * h[k].element_size() for k in h)
+        d2h = h_out.numel() * 2 + sum(x.numel() * 4 for x in h_acc) + 4
+        e2e = {"value": world * tokens / t_e2e, "unit": UNIT, "ms_per_step": t_e2e * 1e3,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        del arena
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_src = load_peaks()
+    flops, attn_bytes, accept_bytes = algorithmic_work(cfg, host_sets[0])
+    attn_med = statistics.median(attn_ms) * 1e-3
+    attn_mean = sum(attn_ms) / len(attn_ms) * 1e-3
+    acc_mean = sum(acc_ms) / len(acc_ms) * 1e-3
+    t_tc = flops / (peaks["bf16_tflops_sustained"] * 1e12)
+    t_hbm = attn_bytes / (peaks["hbm_gbs"] * 1e9)
+    sustained = total_ms >= 2000.0
+    if t_tc >= t_hbm:
+        peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+        achieved = flops / attn_mean / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "traffic": None,
+                "peak_kind": f"{'sustained' if sustained else 'burst'} bf16, of {peak_src}",
+                "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+                "frac_of_burst": achieved / peaks["bf16_tflops"],
+                "frac_of_nominal_2250": achieved / 2250.0}
+    else:
+        peak = peaks["hbm_gbs"]
+        achieved = attn_bytes / attn_mean / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": None, "peak_kind": f"copy bandwidth, of {peak_src}",
+                "frac_of_nominal_8000": achieved / 8000.0}
+    roof["kernel"] = "gsd_verify_attn" + (" (split pass + merge pass)" if splits > 1 else "")
+    roof["algorithmic_flops"] = flops
+    roof["algorithmic_bytes"] = attn_bytes
+    roof["launch_us_mean"] = attn_mean * 1e6
+    roof["launch_us_median"] = attn_med * 1e6
+
+    cpu = None
+    if args.cpu_rows > 0 and world == 1:
+        v, threads, desc = cpu_oracle_sample(cfg, host_sets[0], args.cpu_rows)
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "N": cfg.N, "Hq": cfg.Hq, "Hkv": cfg.Hkv,
+                   "D": cfg.D, "L": cfg.L, "V": cfg.V, "depth": cfg.depth,
+                   "l2": "two input sets rotated; each step reads more than the L2 size",
+                   "replicas": world, "attn_kernel": args.kernel, "num_splits": splits},
+        "attn_us": attn_mean * 1e6, "accept_us": acc_mean * 1e6,
+        "attn_tokens_per_s": tokens / attn_mean,
+        "accept_gbs": accept_bytes / acc_mean / 1e9,
+        "accept_frac_of_hbm": accept_bytes / acc_mean / 1e9 / peaks["hbm_gbs"],
+        "roofline": roof, "cpu_baseline": cpu, "e2e": e2e,
+        "gpu_launches": args.steps * ((2 if splits > 1 else 1) + 1),
+        "clocks": clocks,
+    }
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
