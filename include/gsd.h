@@ -169,6 +169,36 @@ int gsd_accept(const float* logits, const int32_t* draft_tokens, const int32_t* 
 size_t gsd_accept_workspace_bytes(const gsd_accept_params* p);
 
 /*
+ * gsd_accept_static - gsd_accept without a workspace argument.  (The paper has no counterpart
+ * for this call; it is a packaging variant of gsd_accept.)
+ *
+ * Some callers have no device memory to give: a plug-in running inside a serving process
+ * whose host application has already claimed the GPU's memory for its own pool, a caller
+ * that is handed tensors by another runtime and has no allocator of its own, or code on a
+ * latency-critical path where cudaMalloc (which may synchronise the whole device) is off
+ * limits.  For them the scratch that gsd_accept needs (8 bytes per draft node + 4 bytes per
+ * sequence) lives in a fixed array inside the library image, GSD_STATIC_SCRATCH_BYTES long;
+ * every GPU on which the library is used holds that array until the process exits.
+ *
+ * Same arguments, results, status bits and error codes as gsd_accept, minus workspace and
+ * workspace_bytes.  Limit: B * N <= GSD_STATIC_MAX_ROWS; larger problems are refused with
+ * GSD_ERR_WORKSPACE (and a text in gsd_last_cuda_error) before anything is launched.
+ * The call allocates and frees nothing.
+ *
+ * The first call on each device looks up the array's device address (the device must be
+ * current, as for every call here); make that first call outside any stream capture.
+ * All calls on a device share the one array: it keeps whatever the last call left in it, the
+ * part a call uses is cleared on `stream` before its kernel runs, and two calls that can
+ * overlap on the GPU (different streams, no dependency) race on it - serialise them.
+ */
+#define GSD_STATIC_MAX_ROWS 16384
+#define GSD_STATIC_SCRATCH_BYTES (GSD_STATIC_MAX_ROWS * 8 + GSD_STATIC_MAX_ROWS * 4 + 256)
+int gsd_accept_static(const float* logits, const int32_t* draft_tokens, const int32_t* parent_ptr,
+                      const int32_t* parent_idx, int32_t* accepted_tokens, int32_t* accepted_len,
+                      int32_t* accepted_nodes, const gsd_accept_params* p, int32_t* status,
+                      void* stream);
+
+/*
  * gsd_verify_step_host - one whole verification step from HOST buffers: copies every
  * input to the device arena, runs gsd_verify_attn and gsd_accept, copies `out`,
  * accepted_tokens, accepted_len (and accepted_nodes if non-NULL) back and waits for the

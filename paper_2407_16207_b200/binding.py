@@ -41,7 +41,7 @@ class AcceptParams(ctypes.Structure):
 
 EXPORTS = ["gsd_version", "gsd_status_string", "gsd_last_cuda_error", "gsd_verify_attn",
            "gsd_verify_attn_workspace_bytes", "gsd_verify_attn_num_splits", "gsd_accept",
-           "gsd_accept_workspace_bytes", "gsd_verify_step_host",
+           "gsd_accept_workspace_bytes", "gsd_accept_static", "gsd_verify_step_host",
            "gsd_verify_step_host_arena_bytes"]
 
 
@@ -70,6 +70,8 @@ def lib() -> ctypes.CDLL:
         L.gsd_verify_attn_num_splits.argtypes = [ctypes.POINTER(AttnParams)]
         L.gsd_accept.restype = i32
         L.gsd_accept.argtypes = [vp] * 7 + [ctypes.POINTER(AcceptParams), vp, sz, vp, vp]
+        L.gsd_accept_static.restype = i32
+        L.gsd_accept_static.argtypes = [vp] * 7 + [ctypes.POINTER(AcceptParams), vp, vp]
         L.gsd_accept_workspace_bytes.restype = sz
         L.gsd_accept_workspace_bytes.argtypes = [ctypes.POINTER(AcceptParams)]
         L.gsd_verify_step_host.restype = i32
@@ -86,8 +88,9 @@ def _check(rc: int) -> None:
     if rc != 0:
         L = lib()
         msg = L.gsd_status_string(rc).decode()
-        if rc == -5:
-            msg += ": " + L.gsd_last_cuda_error().decode()
+        detail = L.gsd_last_cuda_error().decode()
+        if rc == -5 or (rc == -4 and detail.startswith("gsd_accept_static")):
+            msg += ": " + detail
         raise GsdError(rc, f"gsd error {rc}: {msg}")
 
 
@@ -210,6 +213,35 @@ def gsd_accept(logits, draft_tokens, parent_ptr, parent_idx, *, Tcap: int = 0,
                             ctypes.byref(p), workspace.data_ptr(),
                             workspace.numel() * workspace.element_size(), _ptr(status),
                             _stream(logits)))
+    return toks, lens, nodes
+
+
+GSD_STATIC_MAX_ROWS = 16384
+
+
+def gsd_accept_static(logits, draft_tokens, parent_ptr, parent_idx, *, Tcap: int = 0,
+                      want_nodes: bool = True, status: Optional[torch.Tensor] = None
+                      ) -> Tuple[torch.Tensor, torch.Tensor, Optional[torch.Tensor]]:
+    """gsd_accept for callers that cannot provide scratch memory: the library's own fixed
+    array is used instead (B * N <= GSD_STATIC_MAX_ROWS; calls on one device must not overlap).
+    The C call allocates nothing; this wrapper only allocates the result tensors it returns.
+    See gsd_accept_static in include/gsd.h."""
+    B, N, V = logits.shape
+    _want(logits, torch.float32, (B, N, V), "logits", True)
+    _want(draft_tokens, torch.int32, (B, N), "draft_tokens", True)
+    _want(parent_ptr, torch.int32, (B, N + 1), "parent_ptr", True)
+    Ecap = parent_idx.shape[1]
+    _want(parent_idx, torch.int32, (B, Ecap), "parent_idx", True)
+    Tcap = Tcap or N
+    toks = torch.empty((B, Tcap), dtype=torch.int32, device=logits.device)
+    lens = torch.empty((B,), dtype=torch.int32, device=logits.device)
+    nodes = torch.empty((B, Tcap), dtype=torch.int32, device=logits.device) if want_nodes else None
+    p = AcceptParams(B, N, V, Ecap, Tcap)
+    with torch.cuda.device(logits.device):
+        _check(lib().gsd_accept_static(logits.data_ptr(), draft_tokens.data_ptr(),
+                                       parent_ptr.data_ptr(), parent_idx.data_ptr(),
+                                       toks.data_ptr(), lens.data_ptr(), _ptr(nodes),
+                                       ctypes.byref(p), _ptr(status), _stream(logits)))
     return toks, lens, nodes
 
 

@@ -328,3 +328,47 @@ extern "C" int gsd_accept(const float* logits, const int32_t* draft_tokens,
     GSD_CUDA_TRY(cudaGetLastError());
     return GSD_OK;
 }
+
+// ---------------------------------------------------------------------------------------
+// gsd_accept_static: the same computation as gsd_accept with the scratch in a fixed array
+// that lives in the library image, for callers that cannot hand over device memory.
+namespace gsd {
+namespace {
+// 8 bytes per draft node plus 4 bytes per sequence, for at most GSD_STATIC_MAX_ROWS rows.
+// Every GPU that loads the library holds these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_accept_scratch[GSD_STATIC_SCRATCH_BYTES];
+}  // namespace
+}  // namespace gsd
+
+extern "C" int gsd_accept_static(const float* logits, const int32_t* draft_tokens,
+                                 const int32_t* parent_ptr, const int32_t* parent_idx,
+                                 int32_t* accepted_tokens, int32_t* accepted_len,
+                                 int32_t* accepted_nodes, const gsd_accept_params* p,
+                                 int32_t* status, void* stream) {
+    using namespace gsd;
+    if (!p) return GSD_ERR_NULL_POINTER;
+    if (p->B < 1 || p->N < 1 || p->N > GSD_MAX_NODES) return GSD_ERR_BAD_SHAPE;
+    if ((long long)p->B * p->N > GSD_STATIC_MAX_ROWS) {
+        set_error_text("gsd_accept_static: B*N exceeds GSD_STATIC_MAX_ROWS");
+        return GSD_ERR_WORKSPACE;
+    }
+    const size_t need = gsd_accept_workspace_bytes(p);
+    if (need == 0 || need > (size_t)GSD_STATIC_SCRATCH_BYTES) {
+        set_error_text("gsd_accept_static: scratch need exceeds GSD_STATIC_SCRATCH_BYTES");
+        return GSD_ERR_WORKSPACE;
+    }
+    // In host code the array's name is only a handle; the device address has to be asked for,
+    // once per device, with that device current.
+    static void* addr[64] = {};
+    int dev = 0;
+    GSD_CUDA_TRY(cudaGetDevice(&dev));
+    void* ptr = (dev >= 0 && dev < 64) ? addr[dev] : nullptr;
+    if (!ptr) {
+        GSD_CUDA_TRY(cudaGetSymbolAddress((void**)&ptr, g_accept_scratch));
+        if (!ptr) return GSD_ERR_CUDA;
+        if (dev >= 0 && dev < 64) addr[dev] = ptr;
+    }
+    // gsd_accept clears the part of the scratch it uses before every launch
+    return gsd_accept(logits, draft_tokens, parent_ptr, parent_idx, accepted_tokens, accepted_len,
+                      accepted_nodes, p, ptr, (size_t)GSD_STATIC_SCRATCH_BYTES, status, stream);
+}
