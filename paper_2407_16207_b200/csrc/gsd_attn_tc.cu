@@ -1,8 +1,679 @@
-// gsd_verify_attn, tcgen05 back end (placeholder until the TMEM kernel lands).
+// gsd_verify_attn, tcgen05 back end for D = 128 (sm_100a): TMA-fed, TMEM-resident
+// flash-attention over the stacked (draft node x GQA head) rows.
+//
+// Tree attention over the flattened token graph (Sec. 4.1) with the committed prefix in the
+// KV cache (Sec. 4.2): row r = (node r / G, head r % G) of kv head c attends to cache rows
+// j < seq_lens[b] and to the draft rows whose bit is set in the node's ancestor mask.
+//
+// One CTA owns up to two row tiles of 128 stacked rows of one (sequence, kv head) and a
+// contiguous range of 128-key tiles (prefix tiles, then the draft tiles that hold a visible
+// key for any of its rows).  Warp roles:
+//   warps 0-3   softmax of row tile 0 (thread = row = TMEM lane)
+//   warps 4-7   softmax of row tile 1
+//   warp  8     TMA producer (one thread): Q once, then K and V tiles into two smem rings
+//   warp  9     MMA issuer (one thread): S_i = Q_i K^T into TMEM, O_i += P_i V with P read
+//               from TMEM (P overwrites the first half of S_i as bf16)
+//   warp 10     TMEM allocation / release
+// The issue order QK0(j) PV1(j-1) QK1(j) PV0(j) lets the softmax of one row tile run under
+// the MMAs of the other.  The running maximum is only raised when a tile exceeds it by more
+// than 2^8 (the accumulator rescale is then done in place in TMEM by the row's own thread),
+// so P <= 256 and the rescale is rare.  Every mbarrier wait is bounded: on expiry the kernel
+// raises GSD_DEV_WAIT_EXPIRED, all roles leave their loops, TMEM is released.
 #include "gsd_internal.cuh"
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <math_constants.h>
+#include <stdio.h>
+
 namespace gsd {
-int launch_attn_tcgen05(const AttnArgs&) {
-    set_error_text("tcgen05 back end not built");
-    return GSD_ERR_UNSUPPORTED;
+namespace {
+
+constexpr int BM = 128;            // rows per row tile
+constexpr int BN = 128;            // keys per tile
+constexpr int HD = 128;            // head dimension
+constexpr int KST = 2;             // K ring stages
+constexpr int VST = 2;             // V ring stages
+constexpr uint32_t HALF_BYTES = 128 * 64 * 2;     // one [128 rows][64 bf16] swizzled block
+constexpr uint32_t TILE_BYTES = 2 * HALF_BYTES;   // a 128 x 128 bf16 tile (two column halves)
+constexpr int kThreads = 384;
+constexpr uint32_t kSmemBytes = (2 + KST + VST) * TILE_BYTES + 1024;  // + alignment slack
+constexpr float kRescaleThreshold = 8.0f;         // log2 units
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+// TMEM columns (fp32 words): S0, S1, O0, O1; P_i lives in the first 64 columns of S_i
+constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O0 = 256, COL_O1 = 384;
+
+enum Bar {
+    BAR_Q_FULL = 0,
+    BAR_K_FULL = 1,                   // KST
+    BAR_K_EMPTY = BAR_K_FULL + KST,   // KST
+    BAR_V_FULL = BAR_K_EMPTY + KST,   // VST
+    BAR_V_EMPTY = BAR_V_FULL + VST,   // VST
+    BAR_S_FULL = BAR_V_EMPTY + VST,   // 2
+    BAR_P_READY = BAR_S_FULL + 2,     // 2
+    BAR_O_DONE = BAR_P_READY + 2,     // 2
+    BAR_COUNT = BAR_O_DONE + 2
+};
+
+struct TcParams {
+    const uint32_t* mask;
+    const int32_t* seq_lens;
+    __nv_bfloat16* out;
+    float* part_o;
+    float* part_ml;
+    int32_t* status;
+    int B, N, Hq, Hkv, Lmax, G, W, R, splits;
+    float scale_log2;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait.  Returns false when the wait gave up (time limit, or another role raised the
+// abort flag); the caller then leaves its loop.  `ignore_abort` is for the final drain.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                            int32_t* status, bool ignore_abort) {
+    const unsigned long long t0 = global_ns();
+    for (unsigned it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u) {
+            if (!ignore_abort && *abort_flag) return false;
+            if (global_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                if (status) atomicOr((unsigned*)status, GSD_DEV_WAIT_EXPIRED);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, status, false);
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
+}
+
+// 32 lanes x 32 consecutive fp32 columns: thread t of the warp gets lane (base + t)
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t* r = reinterpret_cast<uint32_t*>(v);
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const float (&v)[32]) {
+    const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+// ---- shared-memory matrix descriptors (128-byte swizzle, 8-row groups 1024 bytes apart)
+constexpr uint64_t kDescBase = (1ull << 46) | (2ull << 61);   // descriptor version 1, SWIZZLE_128B
+// K-major operand (rows x 64 bf16 per block): leading offset unused (1), stride = 1024 B
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
+    return kDescBase | (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32);
+}
+// MN-major operand (V: [key][64 d] blocks): leading offset = distance between the two
+// 64-column blocks, stride = 1024 B between 8-key groups
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
+    return kDescBase | (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(HALF_BYTES >> 4) << 16) |
+           ((uint64_t)(1024 >> 4) << 32);
+}
+// instruction descriptors: bf16 x bf16 -> fp32, M = 128, N = 128
+constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);   // B (= V) is MN-major
+
+struct TileInfo {
+    int kind;     // 0 full prefix tile, 1 ragged prefix tile, 2 draft tile
+    int key0;     // first key (prefix position or draft node) of the tile
+    int nvalid;   // prefix: visible keys in the tile
+};
+
+__device__ __forceinline__ TileInfo tile_info(int t, int nPT, int L, unsigned live) {
+    TileInfo ti;
+    if (t < nPT) {
+        ti.key0 = t * BN;
+        ti.nvalid = min(BN, L - ti.key0);
+        ti.kind = ti.nvalid == BN ? 0 : 1;
+    } else {
+        int k = t - nPT, d = 0;
+        for (;; ++d) {   // the k-th set bit of `live`
+            if ((live >> d) & 1u) {
+                if (k == 0) break;
+                --k;
+            }
+        }
+        ti.key0 = d * BN;
+        ti.nvalid = BN;
+        ti.kind = 2;
+    }
+    return ti;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+               const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_dk,
+               const __grid_constant__ CUtensorMap tm_dv, const TcParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ __align__(8) unsigned long long s_bars[BAR_COUNT];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+    __shared__ unsigned s_live;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int row0 = blockIdx.x * (2 * BM);
+    const int unit = blockIdx.y;
+    const int b = unit / p.Hkv, c = unit % p.Hkv;
+    const int split = blockIdx.z;
+    const int N = p.N, G = p.G, R = p.R;
+    const bool two = row0 + BM < R;          // does the second row tile exist
+    const int ntile_rows = two ? 2 : 1;
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ = smem_base;                                   // 2 tiles
+    const uint32_t sK = smem_base + 2 * TILE_BYTES;                  // KST tiles
+    const uint32_t sV = sK + KST * TILE_BYTES;                       // VST tiles
+    const uint32_t bar0 = smem_u32(s_bars);
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    volatile int* abort_flag = &s_abort;
+
+    int L = p.seq_lens[b];
+    if (L < 0 || L > p.Lmax) {
+        if (tid == 0 && p.status) atomicOr((unsigned*)p.status, GSD_DEV_BAD_SEQ_LEN);
+        L = L < 0 ? 0 : p.Lmax;
+    }
+
+    if (tid == 0) {
+        s_abort = 0;
+        s_live = 0;
+        mbar_init(bar(BAR_Q_FULL), 1);
+        for (int s = 0; s < KST; ++s) { mbar_init(bar(BAR_K_FULL + s), 1); mbar_init(bar(BAR_K_EMPTY + s), 1); }
+        for (int s = 0; s < VST; ++s) { mbar_init(bar(BAR_V_FULL + s), 1); mbar_init(bar(BAR_V_EMPTY + s), 1); }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar(BAR_S_FULL + i), 1);
+            mbar_init(bar(BAR_P_READY + i), 128);
+            mbar_init(bar(BAR_O_DONE + i), 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 10) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&s_tmem_base)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    __syncthreads();
+
+    // draft tiles (128 nodes each) that hold a visible key for any row of this CTA
+    if (tid < 2 * BM) {
+        const int r = row0 + tid;
+        unsigned live = 0;
+        if (r < R) {
+            const uint32_t* mrow = p.mask + ((size_t)b * N + r / G) * p.W;
+            for (int w = 0; w < p.W; ++w) {
+                uint32_t word = mrow[w];
+                if (w == p.W - 1 && (N & 31)) word &= (1u << (N & 31)) - 1u;
+                if (word) live |= 1u << (w >> 2);
+            }
+        }
+        live = __reduce_or_sync(0xFFFFFFFFu, live);
+        if (lane == 0 && live) atomicOr(&s_live, live);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem_base;
+    const unsigned live = s_live;
+
+    const int nPT = (L + BN - 1) / BN;
+    const int T = nPT + __popc(live);
+    const int per = (T + p.splits - 1) / p.splits;
+    const int t_begin = min(split * per, T), t_end = min(t_begin + per, T);
+    const int ntiles = t_end - t_begin;
+
+    if (warp == 8) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0 && ntiles > 0) {
+            mbar_expect_tx(bar(BAR_Q_FULL), (uint32_t)ntile_rows * TILE_BYTES);
+            for (int i = 0; i < ntile_rows; ++i)
+                for (int h = 0; h < 2; ++h)
+                    tma_load_4d(sQ + i * TILE_BYTES + h * HALF_BYTES, &tm_q, bar(BAR_Q_FULL), h * 64, c * G,
+                                (row0 + i * BM) / G, b);
+            int issued_k = 0, issued_v = 0;
+            bool ok = true;
+            for (int idx = 0; idx < ntiles && ok; ++idx) {
+                const TileInfo ti = tile_info(t_begin + idx, nPT, L, live);
+                const CUtensorMap* mk = ti.kind == 2 ? &tm_dk : &tm_k;
+                const CUtensorMap* mv = ti.kind == 2 ? &tm_dv : &tm_v;
+                {
+                    const int s = idx % KST;
+                    ok = mbar_wait(bar(BAR_K_EMPTY + s), ((idx / KST) & 1) ^ 1, abort_flag, p.status);
+                    if (!ok) break;
+                    mbar_expect_tx(bar(BAR_K_FULL + s), TILE_BYTES);
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_4d(sK + s * TILE_BYTES + h * HALF_BYTES, mk, bar(BAR_K_FULL + s), h * 64, c, ti.key0, b);
+                    issued_k = idx + 1;
+                }
+                {
+                    const int s = idx % VST;
+                    ok = mbar_wait(bar(BAR_V_EMPTY + s), ((idx / VST) & 1) ^ 1, abort_flag, p.status);
+                    if (!ok) break;
+                    mbar_expect_tx(bar(BAR_V_FULL + s), TILE_BYTES);
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_4d(sV + s * TILE_BYTES + h * HALF_BYTES, mv, bar(BAR_V_FULL + s), h * 64, c, ti.key0, b);
+                    issued_v = idx + 1;
+                }
+            }
+            if (!ok) {
+                // gave up: let the copies already in flight land before the CTA retires
+                mbar_wait_slow(bar(BAR_Q_FULL), 0, abort_flag, nullptr, true);
+                for (int idx = max(0, issued_k - KST); idx < issued_k; ++idx)
+                    mbar_wait_slow(bar(BAR_K_FULL + idx % KST), (idx / KST) & 1, abort_flag, nullptr, true);
+                for (int idx = max(0, issued_v - VST); idx < issued_v; ++idx)
+                    mbar_wait_slow(bar(BAR_V_FULL + idx % VST), (idx / VST) & 1, abort_flag, nullptr, true);
+            }
+        }
+    } else if (warp == 9) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0 && ntiles > 0) {
+            bool ok = mbar_wait(bar(BAR_Q_FULL), 0, abort_flag, p.status);
+            tc_fence_after();
+            auto issue_qk = [&](int i, int ks_stage) {
+                // S_i = Q_i K^T : 8 k-steps of 16 over the head dimension
+                const uint32_t qa = sQ + i * TILE_BYTES, ka = sK + ks_stage * TILE_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < HD / 16; ++ks) {
+                    const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+                    tc_mma_ss(tmem + (i ? COL_S1 : COL_S0), desc_kmajor(qa + off), desc_kmajor(ka + off), kIdescQK, ks > 0);
+                }
+            };
+            auto issue_pv = [&](int i, int vs_stage, bool accumulate) {
+                // O_i += P_i V : 8 k-steps of 16 keys; P (bf16 pairs) sits in S_i's first 64 columns
+                const uint32_t va = sV + vs_stage * TILE_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < BN / 16; ++ks)
+                    tc_mma_ts(tmem + (i ? COL_O1 : COL_O0), tmem + (i ? COL_S1 : COL_S0) + ks * 8,
+                              desc_mnmajor(va + ks * 2048), kIdescPV, (accumulate || ks > 0) ? 1u : 0u);
+            };
+            for (int idx = 0; idx < ntiles && ok; ++idx) {
+                const int ks_stage = idx % KST, vs_stage = idx % VST;
+                ok = mbar_wait(bar(BAR_K_FULL + ks_stage), (idx / KST) & 1, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                issue_qk(0, ks_stage);
+                tc_commit(bar(BAR_S_FULL + 0));
+                if (two) {
+                    if (idx > 0) {
+                        ok = mbar_wait(bar(BAR_P_READY + 1), (idx - 1) & 1, abort_flag, p.status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(1, (idx - 1) % VST, idx - 1 > 0);
+                        tc_commit(bar(BAR_V_EMPTY + (idx - 1) % VST));
+                    }
+                    issue_qk(1, ks_stage);
+                    tc_commit(bar(BAR_S_FULL + 1));
+                }
+                tc_commit(bar(BAR_K_EMPTY + ks_stage));
+                ok = mbar_wait(bar(BAR_V_FULL + vs_stage), (idx / VST) & 1, abort_flag, p.status);
+                if (!ok) break;
+                ok = mbar_wait(bar(BAR_P_READY + 0), idx & 1, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                issue_pv(0, vs_stage, idx > 0);
+                if (!two) tc_commit(bar(BAR_V_EMPTY + vs_stage));
+                if (idx == ntiles - 1) tc_commit(bar(BAR_O_DONE + 0));
+            }
+            if (ok && two) {
+                const int idx = ntiles - 1;
+                ok = mbar_wait(bar(BAR_P_READY + 1), idx & 1, abort_flag, p.status);
+                if (ok) {
+                    tc_fence_after();
+                    issue_pv(1, idx % VST, idx > 0);
+                    tc_commit(bar(BAR_V_EMPTY + idx % VST));
+                    tc_commit(bar(BAR_O_DONE + 1));
+                }
+            }
+        }
+    } else if (warp < 8) {
+        // ------------------------------------------------------------ softmax + epilogue
+        const int i = warp >> 2;                         // row tile of this warpgroup
+        const int rloc = (warp & 3) * 32 + lane;         // row inside the tile = TMEM lane
+        const int row = row0 + i * BM + rloc;
+        const bool rvalid = row < R;
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + lane_addr + (i ? COL_S1 : COL_S0);
+        const uint32_t tO = tmem + lane_addr + (i ? COL_O1 : COL_O0);
+        float m_ref = -CUDART_INF_F, l_run = 0.f;
+        bool ok = true;
+        if (i == 0 || two) {
+            const uint32_t* mrow = p.mask + ((size_t)b * N + (rvalid ? row / G : 0)) * p.W;
+            for (int idx = 0; idx < ntiles; ++idx) {
+                const TileInfo ti = tile_info(t_begin + idx, nPT, L, live);
+                // visibility words of this row for the 128 keys of the tile
+                uint32_t mw[4];
+                if (ti.kind == 0) {
+                    mw[0] = mw[1] = mw[2] = mw[3] = 0xFFFFFFFFu;
+                } else if (ti.kind == 1) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int rem = ti.nvalid - 32 * k;
+                        mw[k] = rem >= 32 ? 0xFFFFFFFFu : (rem <= 0 ? 0u : ((1u << rem) - 1u));
+                    }
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int wi = (ti.key0 >> 5) + k;
+                        uint32_t word = (rvalid && wi < p.W) ? mrow[wi] : 0u;
+                        const int rem = N - 32 * wi;
+                        if (rem < 32) word &= rem <= 0 ? 0u : ((1u << rem) - 1u);
+                        mw[k] = word;
+                    }
+                }
+                ok = mbar_wait(bar(BAR_S_FULL + i), idx & 1, abort_flag, p.status);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after();
+
+                // pass 1: row maximum over the visible keys
+                float mx = -CUDART_INF_F;
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    float v[32];
+                    tc_ld32(tS + ch * 32, v);
+                    tc_wait_ld();
+                    if (ti.kind == 0) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, v[e]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, ((mw[ch] >> e) & 1u) ? v[e] : -CUDART_INF_F);
+                    }
+                }
+                const float m_tile = mx * p.scale_log2;     // scale > 0 keeps the order
+                float m_new = m_ref, alpha = 1.f;
+                bool need = false;
+                if (m_ref == -CUDART_INF_F) {
+                    m_new = m_tile;                         // nothing accumulated for this row yet
+                } else if (m_tile > m_ref + kRescaleThreshold) {
+                    m_new = m_tile;
+                    alpha = fast_exp2(m_ref - m_new);
+                    need = true;
+                }
+                if (__any_sync(0xFFFFFFFFu, need)) {
+                    // the accumulator of this row is final for all earlier tiles (MMAs complete in
+                    // order and S of this tile is complete): rescale it in place
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        float v[32];
+                        tc_ld32(tO + ch * 32, v);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) v[e] *= alpha;
+                        tc_st32(tO + ch * 32, v);
+                    }
+                    l_run *= alpha;
+                }
+                m_ref = m_new;
+                const float m_use = m_ref == -CUDART_INF_F ? 0.f : m_ref;
+
+                // pass 2: P = 2^(s*scale - m) as bf16 pairs into the first 64 columns of S
+                float sum = 0.f;
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    float v[32];
+                    uint32_t pk[16];
+                    tc_ld32(tS + ch * 32, v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        float pe = fast_exp2(fmaf(v[e], p.scale_log2, -m_use));
+                        if (ti.kind != 0) pe = ((mw[ch] >> e) & 1u) ? pe : 0.f;
+                        v[e] = pe;
+                        sum += pe;
+                    }
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) pk[e] = pack_bf16(v[2 * e], v[2 * e + 1]);
+                    tc_st16(tS + ch * 16, pk);
+                }
+                l_run += sum;
+
+                if (ti.kind == 1 && i == 0) {
+                    // cache rows past the sequence end may hold anything: clear them in the V tile
+                    // so that 0 * junk cannot reach the accumulator
+                    const int vs_stage = idx % VST;
+                    ok = mbar_wait(bar(BAR_V_FULL + vs_stage), (idx / VST) & 1, abort_flag, p.status);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    if (rloc >= ti.nvalid) {
+                        unsigned char* vrow = smem_raw + (sV - smem_u32(smem_raw)) + vs_stage * TILE_BYTES + rloc * 128;
+#pragma unroll
+                        for (int h = 0; h < 2; ++h)
+#pragma unroll
+                            for (int k = 0; k < 8; ++k)
+                                *reinterpret_cast<uint4*>(vrow + h * HALF_BYTES + k * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                }
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar(BAR_P_READY + i));
+            }
+
+            // ---- epilogue
+            if (ok && ntiles > 0) {
+                ok = mbar_wait(bar(BAR_O_DONE + i), 0, abort_flag, p.status);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                tc_fence_after();
+            }
+            if (ok) {
+                const int n = rvalid ? row / G : 0, g = rvalid ? row % G : 0;
+                if (p.splits == 1) {
+                    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+                    __nv_bfloat16* dst = p.out + (((size_t)b * N + n) * p.Hq + c * G + g) * HD;
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        float v[32];
+                        if (ntiles > 0) {
+                            tc_ld32(tO + ch * 32, v);
+                            tc_wait_ld();
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) v[e] = 0.f;
+                        }
+                        if (rvalid) {
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                uint4 u;
+                                u.x = pack_bf16(v[8 * k + 0] * inv, v[8 * k + 1] * inv);
+                                u.y = pack_bf16(v[8 * k + 2] * inv, v[8 * k + 3] * inv);
+                                u.z = pack_bf16(v[8 * k + 4] * inv, v[8 * k + 5] * inv);
+                                u.w = pack_bf16(v[8 * k + 6] * inv, v[8 * k + 7] * inv);
+                                *reinterpret_cast<uint4*>(dst + ch * 32 + k * 8) = u;
+                            }
+                        }
+                    }
+                } else {
+                    const size_t prow = ((size_t)unit * p.splits + split) * R + (rvalid ? row : 0);
+                    float* dst = p.part_o + prow * HD;
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        float v[32];
+                        if (ntiles > 0) {
+                            tc_ld32(tO + ch * 32, v);
+                            tc_wait_ld();
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) v[e] = 0.f;
+                        }
+                        if (rvalid) {
+#pragma unroll
+                            for (int k = 0; k < 8; ++k)
+                                *reinterpret_cast<float4*>(dst + ch * 32 + k * 4) =
+                                    make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+                        }
+                    }
+                    if (rvalid) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(m_ref, l_run);
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 10) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !ptr) {
+            if (e != cudaSuccess) set_cuda_error(e, "cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)");
+            else set_error_text("cuTensorMapEncodeTiled is not available in this driver");
+            return nullptr;
+        }
+        fn = (EncodeTiledFn)ptr;
+    }
+    return fn;
+}
+
+// [d3][d2][d1][D] bf16 tensor; box = 64 columns x box1 x box2 x 1, 128-byte swizzle, zero fill
+int make_map(CUtensorMap* m, const void* base, uint64_t d1, uint64_t d2, uint64_t d3, uint32_t box1, uint32_t box2) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return GSD_ERR_CUDA;
+    const cuuint64_t dims[4] = {(cuuint64_t)HD, d1, d2, d3};
+    const cuuint64_t strides[3] = {(cuuint64_t)HD * 2, (cuuint64_t)HD * 2 * d1, (cuuint64_t)HD * 2 * d1 * d2};
+    const cuuint32_t box[4] = {64, box1, box2, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        char msg[96];
+        snprintf(msg, sizeof msg, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        set_error_text(msg);
+        return GSD_ERR_CUDA;
+    }
+    return GSD_OK;
+}
+
+}  // namespace
+
+bool attn_tcgen05_supports(int D, int G) { return D == HD && G >= 1 && G <= BM && BM % G == 0; }
+
+int launch_attn_tcgen05(const AttnArgs& a) {
+    if (!attn_tcgen05_supports(a.D, a.G)) {
+        set_error_text("tcgen05 back end needs D == 128 and a group size that divides 128");
+        return GSD_ERR_UNSUPPORTED;
+    }
+    CUtensorMap tq, tk, tv, tdk, tdv;
+    int rc;
+    if ((rc = make_map(&tq, a.q, a.Hq, a.N, a.B, a.G, BM / a.G)) != GSD_OK) return rc;
+    if ((rc = make_map(&tk, a.k_cache, a.Hkv, a.Lmax, a.B, 1, BN)) != GSD_OK) return rc;
+    if ((rc = make_map(&tv, a.v_cache, a.Hkv, a.Lmax, a.B, 1, BN)) != GSD_OK) return rc;
+    if ((rc = make_map(&tdk, a.draft_k, a.Hkv, a.N, a.B, 1, BN)) != GSD_OK) return rc;
+    if ((rc = make_map(&tdv, a.draft_v, a.Hkv, a.N, a.B, 1, BN)) != GSD_OK) return rc;
+    TcParams p;
+    p.mask = a.mask; p.seq_lens = a.seq_lens; p.out = (__nv_bfloat16*)a.out; p.status = a.status;
+    p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv; p.Lmax = a.Lmax; p.G = a.G; p.W = a.W;
+    p.R = a.N * a.G; p.splits = a.num_splits; p.scale_log2 = a.scale_log2;
+    const size_t po = (size_t)a.B * a.Hkv * a.num_splits * p.R * a.D * sizeof(float);
+    p.part_o = (float*)a.workspace;
+    p.part_ml = (float*)((char*)a.workspace + align_up(po, 256));
+    GSD_CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    dim3 grid((p.R + 2 * BM - 1) / (2 * BM), a.B * a.Hkv, a.num_splits);
+    attn_tc_kernel<<<grid, kThreads, kSmemBytes, a.stream>>>(tq, tk, tv, tdk, tdv, p);
+    GSD_CUDA_TRY(cudaGetLastError());
+    return GSD_OK;
+}
+
 }  // namespace gsd

@@ -49,6 +49,7 @@ size_t attn_partial_bytes(const gsd_attn_params* p, int splits);
 
 int launch_attn_mma(const AttnArgs& a);
 int launch_attn_tcgen05(const AttnArgs& a);
+bool attn_tcgen05_supports(int D, int G);
 int launch_attn_merge(const AttnArgs& a);
 
 }  // namespace gsd
