@@ -93,7 +93,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
 
 // Bounded wait.  Returns false when the wait gave up (time limit, or another role raised the
 // abort flag); the caller then leaves its loop.  `ignore_abort` is for the final drain.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                             int32_t* status, bool ignore_abort) {
     const unsigned long long t0 = global_ns();
     for (unsigned it = 0;; ++it) {
@@ -174,6 +174,39 @@ __device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16])
         ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
           "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
         : "memory");
+}
+
+// pointer form: v[0..31] must be register-resident (constant indices after unrolling)
+__device__ __forceinline__ void tc_ld32p(uint32_t taddr, float* v) {
+    uint32_t* r = reinterpret_cast<uint32_t*>(v);
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// packed fp32 pairs (one instruction for two lanes of arithmetic)
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d)
+        : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)),
+          "l"(*reinterpret_cast<unsigned long long*>(&c)));
+    return *reinterpret_cast<float2*>(&d);
+}
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d)
+        : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)));
+    return *reinterpret_cast<float2*>(&d);
 }
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -309,6 +342,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const int t_begin = min(split * per, T), t_end = min(t_begin + per, T);
     const int ntiles = t_end - t_begin;
 
+    if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
     if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0 && ntiles > 0) {
@@ -412,7 +447,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 }
             }
         }
-    } else if (warp < 8) {
+    }
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         // ------------------------------------------------------------ softmax + epilogue
         const int i = warp >> 2;                         // row tile of this warpgroup
         const int rloc = (warp & 3) * 32 + lane;         // row inside the tile = TMEM lane
@@ -452,21 +489,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (!ok) break;
                 tc_fence_after();
 
-                // pass 1: row maximum over the visible keys
-                float mx = -CUDART_INF_F;
+                // the whole score row of this thread: 128 fp32 registers
+                float sc[BN];
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    float v[32];
-                    tc_ld32(tS + ch * 32, v);
-                    tc_wait_ld();
-                    if (ti.kind == 0) {
+                for (int ch = 0; ch < 4; ++ch) tc_ld32p(tS + ch * 32, sc + ch * 32);
+                tc_wait_ld();
+                if (ti.kind != 0) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, v[e]);
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, ((mw[ch] >> e) & 1u) ? v[e] : -CUDART_INF_F);
-                    }
+                    for (int e = 0; e < BN; ++e) sc[e] = ((mw[e >> 5] >> (e & 31)) & 1u) ? sc[e] : -CUDART_INF_F;
                 }
+                float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+#pragma unroll
+                for (int e = 0; e < BN; e += 8) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) mx4[k] = max3(mx4[k], sc[e + 2 * k], sc[e + 2 * k + 1]);
+                }
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 const float m_tile = mx * p.scale_log2;     // scale > 0 keeps the order
                 float m_new = m_ref, alpha = 1.f;
                 bool need = false;
@@ -480,7 +518,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (__any_sync(0xFFFFFFFFu, need)) {
                     // the accumulator of this row is final for all earlier tiles (MMAs complete in
                     // order and S of this tile is complete): rescale it in place
-#pragma unroll
+#pragma unroll 1
                     for (int ch = 0; ch < 4; ++ch) {
                         float v[32];
                         tc_ld32(tO + ch * 32, v);
@@ -494,26 +532,24 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 m_ref = m_new;
                 const float m_use = m_ref == -CUDART_INF_F ? 0.f : m_ref;
 
-                // pass 2: P = 2^(s*scale - m) as bf16 pairs into the first 64 columns of S
-                float sum = 0.f;
+                // P = 2^(s*scale - m) as bf16 pairs into the first 64 columns of S; a masked
+                // score is -inf and comes out as exactly 0
+                const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
+                const float2 negm2 = make_float2(-m_use, -m_use);
+                float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) {
-                    float v[32];
                     uint32_t pk[16];
-                    tc_ld32(tS + ch * 32, v);
-                    tc_wait_ld();
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        float pe = fast_exp2(fmaf(v[e], p.scale_log2, -m_use));
-                        if (ti.kind != 0) pe = ((mw[ch] >> e) & 1u) ? pe : 0.f;
-                        v[e] = pe;
-                        sum += pe;
+                    for (int e = 0; e < 16; ++e) {
+                        const float2 t = ffma2(make_float2(sc[ch * 32 + 2 * e], sc[ch * 32 + 2 * e + 1]), scale2, negm2);
+                        const float2 pe = make_float2(fast_exp2(t.x), fast_exp2(t.y));
+                        sum2[e & 1] = fadd2(sum2[e & 1], pe);
+                        pk[e] = pack_bf16(pe.x, pe.y);
                     }
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) pk[e] = pack_bf16(v[2 * e], v[2 * e + 1]);
                     tc_st16(tS + ch * 16, pk);
                 }
-                l_run += sum;
+                l_run += (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
 
                 if (ti.kind == 1 && i == 0) {
                     // cache rows past the sequence end may hold anything: clear them in the V tile
