@@ -53,29 +53,48 @@ int attn_pick_kernel(const gsd_attn_params* p) {
     return GSD_ATTN_MMA;
 }
 
-int attn_auto_splits(const gsd_attn_params* p, int kernel, int sm_count) {
-    if (p->num_splits > 0) return p->num_splits;
+AttnPlan attn_make_plan(const gsd_attn_params* p, int sm_count) {
+    AttnPlan pl;
+    pl.kernel = attn_pick_kernel(p);
+    const bool tc = pl.kernel == GSD_ATTN_TCGEN05;
     const int G = p->Hq / p->Hkv;
     const int R = p->N * G;
-    const int bm = kernel == GSD_ATTN_TCGEN05 ? 128 : 64;
-    const int bn = kernel == GSD_ATTN_TCGEN05 ? 128 : 64;
-    const long ctas = (long)((R + bm - 1) / bm) * p->B * p->Hkv;
+    const int bn = tc ? 128 : 64;
+    pl.rows_per_item = tc ? 256 : 64;
+    pl.dev.tiles_per_unit = (R + pl.rows_per_item - 1) / pl.rows_per_item;
+    pl.items = pl.dev.tiles_per_unit * p->B * p->Hkv;
     const int tiles = (p->Lmax + bn - 1) / bn + (p->N + bn - 1) / bn;
-    const long target = (long)sm_count * (kernel == GSD_ATTN_TCGEN05 ? 1 : 3);
-    long s = (target + ctas - 1) / ctas;
-    const int min_tiles = 4;                       // keep at least this many key tiles per split
-    if (s > tiles / min_tiles) s = tiles / min_tiles;
-    if (s > 32) s = 32;
-    if (s < 1) s = 1;
-    return (int)s;
-}
-
-size_t attn_partial_bytes(const gsd_attn_params* p, int splits) {
-    if (splits <= 1) return 0;
-    const size_t R = (size_t)p->N * (p->Hq / p->Hkv);
-    const size_t po = (size_t)p->B * p->Hkv * splits * R * p->D * sizeof(float);
-    const size_t pml = (size_t)p->B * p->Hkv * splits * R * 2 * sizeof(float);
-    return align_up(po, 256) + align_up(pml, 256);
+    int max_split = tiles / 4;                     // keep at least four key tiles per split
+    if (max_split > 32) max_split = 32;
+    if (max_split < 1) max_split = 1;
+    const int resident = sm_count * (tc ? 1 : 3);  // CTAs the device holds at once
+    pl.dev.items_a = pl.items;
+    pl.dev.splits_a = 1;
+    pl.dev.splits_b = 1;
+    if (p->num_splits > 0) {
+        pl.dev.splits_a = p->num_splits;
+    } else if (pl.items < resident) {
+        int s = resident / pl.items;
+        pl.dev.splits_a = s < max_split ? s : max_split;
+    } else if (tc) {
+        // whole items fill complete waves; the items of the last, partial wave are cut so that
+        // they cover the machine once more instead of leaving most of it idle
+        const int r = pl.items % resident;
+        if (r > 0) {
+            int s = resident / r;
+            if (s > max_split) s = max_split;
+            if (s > 1) {
+                pl.dev.items_a = pl.items - r;
+                pl.dev.splits_b = s;
+            }
+        }
+    }
+    const int items_b = pl.items - pl.dev.items_a;
+    pl.ctas = pl.dev.items_a * pl.dev.splits_a + items_b * pl.dev.splits_b;
+    pl.slots = (pl.dev.splits_a > 1 ? pl.dev.items_a * pl.dev.splits_a : 0) +
+               (pl.dev.splits_b > 1 ? items_b * pl.dev.splits_b : 0);
+    pl.ws_bytes = pl.slots ? plan_part_o_bytes(pl, p->D) + plan_part_ml_bytes(pl) : 0;
+    return pl;
 }
 
 }  // namespace gsd
@@ -103,13 +122,15 @@ extern "C" int gsd_verify_attn_num_splits(const gsd_attn_params* p) {
     if (attn_params_ok(p) != GSD_OK) return 0;
     DeviceInfo di;
     if (device_info(&di) != 0) return 0;
-    return attn_auto_splits(p, attn_pick_kernel(p), di.sm_count);
+    const AttnPlan pl = attn_make_plan(p, di.sm_count);
+    return pl.dev.splits_a > pl.dev.splits_b ? pl.dev.splits_a : pl.dev.splits_b;
 }
 
 extern "C" size_t gsd_verify_attn_workspace_bytes(const gsd_attn_params* p) {
-    const int s = gsd_verify_attn_num_splits(p);
-    if (s <= 0) return 0;
-    return attn_partial_bytes(p, s);
+    if (attn_params_ok(p) != GSD_OK) return 0;
+    DeviceInfo di;
+    if (device_info(&di) != 0) return 0;
+    return attn_make_plan(p, di.sm_count).ws_bytes;
 }
 
 extern "C" int gsd_verify_attn(const void* q, const void* k_cache, const void* v_cache,
@@ -127,9 +148,8 @@ extern "C" int gsd_verify_attn(const void* q, const void* k_cache, const void* v
     if (((uintptr_t)ancestor_mask & 3u) != 0 || ((uintptr_t)seq_lens & 3u) != 0) return GSD_ERR_MISALIGNED;
     DeviceInfo di;
     if (device_info(&di) != 0) return GSD_ERR_CUDA;
-    const int kernel = attn_pick_kernel(p);
-    const int splits = attn_auto_splits(p, kernel, di.sm_count);
-    const size_t need = attn_partial_bytes(p, splits);
+    const AttnPlan plan = attn_make_plan(p, di.sm_count);
+    const size_t need = plan.ws_bytes;
     if (need > 0) {
         if (!workspace || workspace_bytes < need) return GSD_ERR_WORKSPACE;
         if (((uintptr_t)workspace & 255u) != 0) return GSD_ERR_MISALIGNED;
@@ -141,11 +161,11 @@ extern "C" int gsd_verify_attn(const void* q, const void* k_cache, const void* v
     a.G = p->Hq / p->Hkv; a.W = (p->N + 31) / 32;
     const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->D);
     a.scale_log2 = scale * 1.4426950408889634f;
-    a.num_splits = splits; a.workspace = workspace; a.status = status;
+    a.plan = plan; a.workspace = workspace; a.status = status;
     a.stream = (cudaStream_t)stream;
-    int rc = kernel == GSD_ATTN_TCGEN05 ? launch_attn_tcgen05(a) : launch_attn_mma(a);
+    int rc = plan.kernel == GSD_ATTN_TCGEN05 ? launch_attn_tcgen05(a) : launch_attn_mma(a);
     if (rc != GSD_OK) return rc;
-    if (splits > 1) rc = launch_attn_merge(a);
+    if (plan.slots > 0) rc = launch_attn_merge(a);
     return rc;
 }
 

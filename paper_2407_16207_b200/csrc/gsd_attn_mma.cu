@@ -7,8 +7,8 @@
 // are stacked into R = N*G rows (row r = node r / G, head r % G) so that K and V are read
 // once per row tile.
 //
-// Grid: (row tiles, B*Hkv, splits).  A CTA of 4 warps owns 64 stacked rows and walks its
-// share of the key tiles (64 keys each; prefix tiles first, then draft tiles) with a
+// Grid: one CTA per (work item, key-range split) of the call's plan.  A CTA of 4 warps owns
+// 64 stacked rows and walks its share of the key tiles (64 keys each; prefix tiles first, then draft tiles) with a
 // two-stage cp.async pipeline.  Rows of the cache at positions >= seq_lens[b] and draft
 // rows >= N are zero-filled by the copy itself, so junk (even NaN patterns) never reaches
 // the arithmetic.  Draft tiles whose mask words are all zero for the CTA's rows are
@@ -69,10 +69,11 @@ struct MmaParams {
     const uint32_t* mask;
     const int32_t* seq_lens;
     __nv_bfloat16* out;
-    float* part_o;   // [B*Hkv][S][R][D]
-    float* part_ml;  // [B*Hkv][S][R][2]
+    float* part_o;   // [slot][64][D]
+    float* part_ml;  // [slot][64][2]
+    PlanDev plan;
     int32_t* status;
-    int B, N, Hq, Hkv, Lmax, G, W, R, splits;
+    int B, N, Hq, Hkv, Lmax, G, W, R;
     float scale_log2;
 };
 
@@ -89,10 +90,11 @@ __global__ void __launch_bounds__(kThreads) attn_mma_kernel(MmaParams p) {
     __shared__ unsigned s_live;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int row0 = blockIdx.x * BM;
-    const int unit = blockIdx.y;           // b * Hkv + c
+    int item, split, nsplit, slot;
+    plan_decode(p.plan, blockIdx.x, item, split, nsplit, slot);
+    const int unit = item / p.plan.tiles_per_unit;   // b * Hkv + c
+    const int row0 = (item % p.plan.tiles_per_unit) * BM;
     const int b = unit / p.Hkv, c = unit % p.Hkv;
-    const int split = blockIdx.z;
     const int N = p.N, G = p.G, R = p.R;
 
     int L = p.seq_lens[b];
@@ -102,7 +104,7 @@ __global__ void __launch_bounds__(kThreads) attn_mma_kernel(MmaParams p) {
     }
     const int nPT = (L + BN - 1) / BN, nDT = (N + BN - 1) / BN;
     const int T = nPT + nDT;
-    const int per = (T + p.splits - 1) / p.splits;
+    const int per = (T + nsplit - 1) / nsplit;
     const int t_begin = min(split * per, T), t_end = min(t_begin + per, T);
 
     // which draft tiles hold at least one visible key for this CTA's rows
@@ -308,7 +310,7 @@ __global__ void __launch_bounds__(kThreads) attn_mma_kernel(MmaParams p) {
         l_run[h] += __shfl_xor_sync(0xFFFFFFFFu, l_run[h], 1);
         l_run[h] += __shfl_xor_sync(0xFFFFFFFFu, l_run[h], 2);
     }
-    if (p.splits == 1) {
+    if (nsplit == 1) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             if (!rvalid[h]) continue;
@@ -325,8 +327,7 @@ __global__ void __launch_bounds__(kThreads) attn_mma_kernel(MmaParams p) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             if (!rvalid[h]) continue;
-            const int row = row0 + rloc[h];
-            const size_t prow = ((size_t)unit * p.splits + split) * R + row;
+            const size_t prow = (size_t)slot * BM + rloc[h];
             float* dst = p.part_o + prow * D;
 #pragma unroll
             for (int dt = 0; dt < DT; ++dt) {
@@ -338,41 +339,54 @@ __global__ void __launch_bounds__(kThreads) attn_mma_kernel(MmaParams p) {
     }
 }
 
-// Merge of split-KV partial results: one warp per output row.
+// Merge of split-KV partial results: one warp per (split item, row of the item).
 //   m = max_s m_s;  out = sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s
 struct MergeParams {
     const float* part_o;
     const float* part_ml;
     __nv_bfloat16* out;
-    int N, Hq, Hkv, G, R, D, splits;
-    long rows_total;  // B*Hkv*R
+    PlanDev plan;
+    int N, Hq, Hkv, G, R, D, rows_per_item, items;
+    long warps_total;  // split items * rows_per_item
 };
 
 __global__ void __launch_bounds__(256) attn_merge_kernel(MergeParams p) {
-    const long wrow = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (wrow >= p.rows_total) return;
+    const long w = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (w >= p.warps_total) return;
     const int lane = threadIdx.x & 31;
-    const int unit = (int)(wrow / p.R), row = (int)(wrow % p.R);
+    const int k = (int)(w / p.rows_per_item), rloc = (int)(w % p.rows_per_item);
+    // the k-th item that owns slots: group a comes first when it is split at all
+    int item, nsplit, slot0;
+    const int split_a = p.plan.splits_a > 1 ? p.plan.items_a : 0;
+    if (k < split_a) {
+        item = k; nsplit = p.plan.splits_a; slot0 = k * p.plan.splits_a;
+    } else {
+        item = p.plan.items_a + (k - split_a); nsplit = p.plan.splits_b;
+        slot0 = split_a * p.plan.splits_a + (k - split_a) * p.plan.splits_b;
+    }
+    const int unit = item / p.plan.tiles_per_unit;
+    const int row = (item % p.plan.tiles_per_unit) * p.rows_per_item + rloc;
+    if (row >= p.R) return;
     const int b = unit / p.Hkv, c = unit % p.Hkv;
     float m = -CUDART_INF_F;
-    for (int s = 0; s < p.splits; ++s)
-        m = fmaxf(m, p.part_ml[(((size_t)unit * p.splits + s) * p.R + row) * 2]);
+    for (int s = 0; s < nsplit; ++s)
+        m = fmaxf(m, p.part_ml[((size_t)(slot0 + s) * p.rows_per_item + rloc) * 2]);
     const float m_use = m == -CUDART_INF_F ? 0.f : m;
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     float l = 0.f;
     const int per_lane = p.D / 32;  // 2 or 4 consecutive floats per lane
-    for (int s = 0; s < p.splits; ++s) {
-        const size_t prow = ((size_t)unit * p.splits + s) * p.R + row;
+    for (int s = 0; s < nsplit; ++s) {
+        const size_t prow = (size_t)(slot0 + s) * p.rows_per_item + rloc;
         const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + prow * 2);
-        const float w = exp2f(ml.x - m_use);
-        l += w * ml.y;
+        const float wgt = exp2f(ml.x - m_use);
+        l += wgt * ml.y;
         const float* src = p.part_o + prow * p.D + lane * per_lane;
         if (per_lane == 4) {
             const float4 v = *reinterpret_cast<const float4*>(src);
-            acc[0] += w * v.x; acc[1] += w * v.y; acc[2] += w * v.z; acc[3] += w * v.w;
+            acc[0] += wgt * v.x; acc[1] += wgt * v.y; acc[2] += wgt * v.z; acc[3] += wgt * v.w;
         } else {
             const float2 v = *reinterpret_cast<const float2*>(src);
-            acc[0] += w * v.x; acc[1] += w * v.y;
+            acc[0] += wgt * v.x; acc[1] += wgt * v.y;
         }
     }
     const float inv = l > 0.f ? 1.f / l : 0.f;
@@ -395,13 +409,12 @@ int launch_mma_t(const AttnArgs& a) {
     p.draft_v = (const __nv_bfloat16*)a.draft_v; p.mask = a.mask; p.seq_lens = a.seq_lens;
     p.out = (__nv_bfloat16*)a.out; p.status = a.status;
     p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv; p.Lmax = a.Lmax; p.G = a.G; p.W = a.W;
-    p.R = a.N * a.G; p.splits = a.num_splits; p.scale_log2 = a.scale_log2;
-    const size_t po = (size_t)a.B * a.Hkv * a.num_splits * p.R * a.D * sizeof(float);
+    p.R = a.N * a.G; p.scale_log2 = a.scale_log2; p.plan = a.plan.dev;
     p.part_o = (float*)a.workspace;
-    p.part_ml = (float*)((char*)a.workspace + align_up(po, 256));
+    p.part_ml = (float*)((char*)a.workspace + plan_part_o_bytes(a.plan, a.D));
     const int smem = 4 * BN * D * 2;
     GSD_CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    dim3 grid((p.R + BM - 1) / BM, a.B * a.Hkv, a.num_splits);
+    dim3 grid(a.plan.ctas);
     attn_mma_kernel<D><<<grid, kThreads, smem, a.stream>>>(p);
     GSD_CUDA_TRY(cudaGetLastError());
     return GSD_OK;
@@ -417,15 +430,18 @@ int launch_attn_mma(const AttnArgs& a) {
 
 int launch_attn_merge(const AttnArgs& a) {
     MergeParams p;
-    const int R = a.N * a.G;
-    const size_t po = (size_t)a.B * a.Hkv * a.num_splits * R * a.D * sizeof(float);
     p.part_o = (const float*)a.workspace;
-    p.part_ml = (const float*)((const char*)a.workspace + align_up(po, 256));
+    p.part_ml = (const float*)((const char*)a.workspace + plan_part_o_bytes(a.plan, a.D));
     p.out = (__nv_bfloat16*)a.out;
-    p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv; p.G = a.G; p.R = R; p.D = a.D; p.splits = a.num_splits;
-    p.rows_total = (long)a.B * a.Hkv * R;
+    p.plan = a.plan.dev;
+    p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv; p.G = a.G; p.R = a.N * a.G; p.D = a.D;
+    p.rows_per_item = a.plan.rows_per_item; p.items = a.plan.items;
+    const int split_items = (a.plan.dev.splits_a > 1 ? a.plan.dev.items_a : 0) +
+                            (a.plan.dev.splits_b > 1 ? a.plan.items - a.plan.dev.items_a : 0);
+    p.warps_total = (long)split_items * a.plan.rows_per_item;
+    if (p.warps_total == 0) return GSD_OK;
     const int warps = 8;
-    const long blocks = (p.rows_total + warps - 1) / warps;
+    const long blocks = (p.warps_total + warps - 1) / warps;
     attn_merge_kernel<<<(unsigned)blocks, warps * 32, 0, a.stream>>>(p);
     GSD_CUDA_TRY(cudaGetLastError());
     return GSD_OK;

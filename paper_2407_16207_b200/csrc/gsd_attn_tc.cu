@@ -62,8 +62,9 @@ struct TcParams {
     float* part_o;
     float* part_ml;
     int32_t* status;
-    int B, N, Hq, Hkv, Lmax, G, W, R, splits;
+    int B, N, Hq, Hkv, Lmax, G, W, R;
     float scale_log2;
+    PlanDev plan;
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -274,10 +275,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     __shared__ unsigned s_live;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int row0 = blockIdx.x * (2 * BM);
-    const int unit = blockIdx.y;
+    int item, split, nsplit, slot;
+    plan_decode(p.plan, blockIdx.x, item, split, nsplit, slot);
+    const int unit = item / p.plan.tiles_per_unit;
+    const int row0 = (item % p.plan.tiles_per_unit) * (2 * BM);
     const int b = unit / p.Hkv, c = unit % p.Hkv;
-    const int split = blockIdx.z;
     const int N = p.N, G = p.G, R = p.R;
     const bool two = row0 + BM < R;          // does the second row tile exist
     const int ntile_rows = two ? 2 : 1;
@@ -338,7 +340,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
     const int nPT = (L + BN - 1) / BN;
     const int T = nPT + __popc(live);
-    const int per = (T + p.splits - 1) / p.splits;
+    const int per = (T + nsplit - 1) / nsplit;
     const int t_begin = min(split * per, T), t_end = min(t_begin + per, T);
     const int ntiles = t_end - t_begin;
 
@@ -581,7 +583,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
             if (ok) {
                 const int n = rvalid ? row / G : 0, g = rvalid ? row % G : 0;
-                if (p.splits == 1) {
+                if (nsplit == 1) {
                     const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
                     __nv_bfloat16* dst = p.out + (((size_t)b * N + n) * p.Hq + c * G + g) * HD;
 #pragma unroll
@@ -607,7 +609,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         }
                     }
                 } else {
-                    const size_t prow = ((size_t)unit * p.splits + split) * R + (rvalid ? row : 0);
+                    const size_t prow = (size_t)slot * (2 * BM) + i * BM + rloc;
                     float* dst = p.part_o + prow * HD;
 #pragma unroll
                     for (int ch = 0; ch < 4; ++ch) {
@@ -701,12 +703,11 @@ int launch_attn_tcgen05(const AttnArgs& a) {
     TcParams p;
     p.mask = a.mask; p.seq_lens = a.seq_lens; p.out = (__nv_bfloat16*)a.out; p.status = a.status;
     p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv; p.Lmax = a.Lmax; p.G = a.G; p.W = a.W;
-    p.R = a.N * a.G; p.splits = a.num_splits; p.scale_log2 = a.scale_log2;
-    const size_t po = (size_t)a.B * a.Hkv * a.num_splits * p.R * a.D * sizeof(float);
+    p.R = a.N * a.G; p.scale_log2 = a.scale_log2; p.plan = a.plan.dev;
     p.part_o = (float*)a.workspace;
-    p.part_ml = (float*)((char*)a.workspace + align_up(po, 256));
+    p.part_ml = (float*)((char*)a.workspace + plan_part_o_bytes(a.plan, a.D));
     GSD_CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
-    dim3 grid((p.R + 2 * BM - 1) / (2 * BM), a.B * a.Hkv, a.num_splits);
+    dim3 grid(a.plan.ctas);
     attn_tc_kernel<<<grid, kThreads, kSmemBytes, a.stream>>>(tq, tk, tv, tdk, tdv, p);
     GSD_CUDA_TRY(cudaGetLastError());
     return GSD_OK;

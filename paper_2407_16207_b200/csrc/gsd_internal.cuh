@@ -28,6 +28,41 @@ struct DeviceInfo {
 // Properties of the current device (cached per device ordinal).
 int device_info(DeviceInfo* out);
 
+// ---- work plan of one gsd_verify_attn call ----
+// A work item is one row tile (rows_per_item stacked rows) of one (sequence, kv head); item
+// index = unit * tiles_per_unit + row tile.  The first items_a items are cut into splits_a
+// key ranges, the remaining ones into splits_b; CTAs are numbered group a first.  Only items
+// with more than one split own partial-result slots (one per split, numbered in CTA order).
+struct PlanDev {
+    int items_a, splits_a, splits_b, tiles_per_unit;
+};
+struct AttnPlan {
+    int kernel;         // GSD_ATTN_MMA or GSD_ATTN_TCGEN05
+    int rows_per_item;  // 64 (mma.sync back end) or 256 (tcgen05 back end)
+    int items;
+    int ctas;
+    int slots;          // partial-result slots; 0 when nothing is split
+    PlanDev dev;
+    size_t ws_bytes;
+};
+__host__ __device__ inline void plan_decode(const PlanDev& pl, int cta, int& item, int& split, int& nsplit, int& slot) {
+    const int ctas_a = pl.items_a * pl.splits_a;
+    if (cta < ctas_a) {
+        item = cta / pl.splits_a;
+        split = cta - item * pl.splits_a;
+        nsplit = pl.splits_a;
+        slot = cta;
+    } else {
+        const int rem = cta - ctas_a;
+        const int k = rem / pl.splits_b;
+        item = pl.items_a + k;
+        split = rem - k * pl.splits_b;
+        nsplit = pl.splits_b;
+        slot = (pl.splits_a > 1 ? ctas_a : 0) + rem;
+    }
+}
+AttnPlan attn_make_plan(const gsd_attn_params* p, int sm_count);
+
 // ---- verify-attention back ends (they validate nothing: the API layer did) ----
 struct AttnArgs {
     const void *q, *k_cache, *v_cache, *draft_k, *draft_v;
@@ -36,16 +71,16 @@ struct AttnArgs {
     void* out;
     int B, N, Hq, Hkv, D, Lmax, G, W;
     float scale_log2;   // softmax_scale * log2(e)
-    int num_splits;
+    AttnPlan plan;
     void* workspace;
     int32_t* status;
     cudaStream_t stream;
 };
 
-// split planning shared by the back ends and the workspace query
 int attn_pick_kernel(const gsd_attn_params* p);                 // GSD_ATTN_MMA or GSD_ATTN_TCGEN05
-int attn_auto_splits(const gsd_attn_params* p, int kernel, int sm_count);
-size_t attn_partial_bytes(const gsd_attn_params* p, int splits);
+// partial results: fp32 accumulators [slot][rows_per_item][D], then (max, sum) [slot][rows_per_item][2]
+inline size_t plan_part_o_bytes(const AttnPlan& pl, int D) { return align_up((size_t)pl.slots * pl.rows_per_item * D * sizeof(float), 256); }
+inline size_t plan_part_ml_bytes(const AttnPlan& pl) { return align_up((size_t)pl.slots * pl.rows_per_item * 2 * sizeof(float), 256); }
 
 int launch_attn_mma(const AttnArgs& a);
 int launch_attn_tcgen05(const AttnArgs& a);
