@@ -50,8 +50,9 @@ enum Bar {
     BAR_V_FULL = BAR_K_EMPTY + KST,   // VST
     BAR_V_EMPTY = BAR_V_FULL + VST,   // VST
     BAR_S_FULL = BAR_V_EMPTY + VST,   // 2
-    BAR_P_READY = BAR_S_FULL + 2,     // 2
-    BAR_O_DONE = BAR_P_READY + 2,     // 2
+    BAR_P_READY = BAR_S_FULL + 2,     // 2: keys 0..63 of P are in TMEM
+    BAR_P_READY2 = BAR_P_READY + 2,   // 2: keys 64..127 of P are in TMEM
+    BAR_O_DONE = BAR_P_READY2 + 2,    // 2
     BAR_COUNT = BAR_O_DONE + 2
 };
 
@@ -307,6 +308,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(BAR_S_FULL + i), 1);
             mbar_init(bar(BAR_P_READY + i), 128);
+            mbar_init(bar(BAR_P_READY2 + i), 128);
             mbar_init(bar(BAR_O_DONE + i), 1);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -402,13 +404,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     tc_mma_ss(tmem + (i ? COL_S1 : COL_S0), desc_kmajor(qa + off), desc_kmajor(ka + off), kIdescQK, ks > 0);
                 }
             };
-            auto issue_pv = [&](int i, int vs_stage, bool accumulate) {
-                // O_i += P_i V : 8 k-steps of 16 keys; P (bf16 pairs) sits in S_i's first 64 columns
+            // O_i += P_i V : 8 k-steps of 16 keys; P (bf16 pairs) sits in S_i's first 64 columns.
+            // The softmax hands P over in two halves of 64 keys, so the first four k-steps run
+            // while the second half of the exponentials is still being computed.
+            auto issue_pv_half = [&](int i, int vs_stage, int half, bool accumulate) {
                 const uint32_t va = sV + vs_stage * TILE_BYTES;
 #pragma unroll
-                for (int ks = 0; ks < BN / 16; ++ks)
+                for (int k4 = 0; k4 < BN / 32; ++k4) {
+                    const int ks = half * (BN / 32) + k4;
                     tc_mma_ts(tmem + (i ? COL_O1 : COL_O0), tmem + (i ? COL_S1 : COL_S0) + ks * 8,
                               desc_mnmajor(va + ks * 2048), kIdescPV, (accumulate || ks > 0) ? 1u : 0u);
+                }
+            };
+            auto issue_pv = [&](int i, int vs_stage, int idx, bool accumulate) -> bool {
+                if (!mbar_wait(bar(BAR_P_READY + i), idx & 1, abort_flag, p.status)) return false;
+                tc_fence_after();
+                issue_pv_half(i, vs_stage, 0, accumulate);
+                if (!mbar_wait(bar(BAR_P_READY2 + i), idx & 1, abort_flag, p.status)) return false;
+                tc_fence_after();
+                issue_pv_half(i, vs_stage, 1, accumulate);
+                return true;
             };
             for (int idx = 0; idx < ntiles && ok; ++idx) {
                 const int ks_stage = idx % KST, vs_stage = idx % VST;
@@ -419,10 +434,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 tc_commit(bar(BAR_S_FULL + 0));
                 if (two) {
                     if (idx > 0) {
-                        ok = mbar_wait(bar(BAR_P_READY + 1), (idx - 1) & 1, abort_flag, p.status);
+                        ok = issue_pv(1, (idx - 1) % VST, idx - 1, idx - 1 > 0);
                         if (!ok) break;
-                        tc_fence_after();
-                        issue_pv(1, (idx - 1) % VST, idx - 1 > 0);
                         tc_commit(bar(BAR_V_EMPTY + (idx - 1) % VST));
                     }
                     issue_qk(1, ks_stage);
@@ -431,19 +444,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 tc_commit(bar(BAR_K_EMPTY + ks_stage));
                 ok = mbar_wait(bar(BAR_V_FULL + vs_stage), (idx / VST) & 1, abort_flag, p.status);
                 if (!ok) break;
-                ok = mbar_wait(bar(BAR_P_READY + 0), idx & 1, abort_flag, p.status);
+                ok = issue_pv(0, vs_stage, idx, idx > 0);
                 if (!ok) break;
-                tc_fence_after();
-                issue_pv(0, vs_stage, idx > 0);
                 if (!two) tc_commit(bar(BAR_V_EMPTY + vs_stage));
                 if (idx == ntiles - 1) tc_commit(bar(BAR_O_DONE + 0));
             }
             if (ok && two) {
                 const int idx = ntiles - 1;
-                ok = mbar_wait(bar(BAR_P_READY + 1), idx & 1, abort_flag, p.status);
+                ok = issue_pv(1, idx % VST, idx, idx > 0);
                 if (ok) {
-                    tc_fence_after();
-                    issue_pv(1, idx % VST, idx > 0);
                     tc_commit(bar(BAR_V_EMPTY + idx % VST));
                     tc_commit(bar(BAR_O_DONE + 1));
                 }
@@ -534,25 +543,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 m_ref = m_new;
                 const float m_use = m_ref == -CUDART_INF_F ? 0.f : m_ref;
 
-                // P = 2^(s*scale - m) as bf16 pairs into the first 64 columns of S; a masked
-                // score is -inf and comes out as exactly 0
-                const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
-                const float2 negm2 = make_float2(-m_use, -m_use);
-                float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const float2 t = ffma2(make_float2(sc[ch * 32 + 2 * e], sc[ch * 32 + 2 * e + 1]), scale2, negm2);
-                        const float2 pe = make_float2(fast_exp2(t.x), fast_exp2(t.y));
-                        sum2[e & 1] = fadd2(sum2[e & 1], pe);
-                        pk[e] = pack_bf16(pe.x, pe.y);
-                    }
-                    tc_st16(tS + ch * 16, pk);
-                }
-                l_run += (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
-
                 if (ti.kind == 1 && i == 0) {
                     // cache rows past the sequence end may hold anything: clear them in the V tile
                     // so that 0 * junk cannot reach the accumulator
@@ -570,9 +560,33 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
+                // P = 2^(s*scale - m) as bf16 pairs into the first 64 columns of S; a masked
+                // score is -inf and comes out as exactly 0
+                const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
+                const float2 negm2 = make_float2(-m_use, -m_use);
+                float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const float2 t = ffma2(make_float2(sc[ch * 32 + 2 * e], sc[ch * 32 + 2 * e + 1]), scale2, negm2);
+                        const float2 pe = make_float2(fast_exp2(t.x), fast_exp2(t.y));
+                        sum2[e & 1] = fadd2(sum2[e & 1], pe);
+                        pk[e] = pack_bf16(pe.x, pe.y);
+                    }
+                    tc_st16(tS + ch * 16, pk);
+                    if (ch == 1) {            // keys 0..63 are in place (and any rescale of O is done)
+                        tc_wait_st();
+                        tc_fence_before();
+                        mbar_arrive(bar(BAR_P_READY + i));
+                    }
+                }
+                l_run += (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
+
                 tc_wait_st();
                 tc_fence_before();
-                mbar_arrive(bar(BAR_P_READY + i));
+                mbar_arrive(bar(BAR_P_READY2 + i));
             }
 
             // ---- epilogue
