@@ -338,6 +338,10 @@ def main():
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": None, "peak_kind": f"copy bandwidth, of {peak_src}",
                 "frac_of_nominal_8000": achieved / 8000.0}
+    # DRAM bytes of one launch of the dominant kernel from the committed ncu capture
+    # (profiles/attn_tcgen05_llama70b.md); only valid for that kernel on that workload
+    if cfg.name == "llama70b" and args.kernel in (0, 2) and args.num_splits == 0:
+        roof["traffic"] = 198.2e6
     roof["kernel"] = "gsd_verify_attn" + (" (split pass + merge pass)" if splits > 1 else "")
     roof["algorithmic_flops"] = flops
     roof["algorithmic_bytes"] = attn_bytes
