@@ -5,7 +5,7 @@
 // KV cache (Sec. 4.2): row r = (node r / G, head r % G) of kv head c attends to cache rows
 // j < seq_lens[b] and to the draft rows whose bit is set in the node's ancestor mask.
 //
-// One CTA owns up to two row tiles of 128 stacked rows of one (sequence, kv head) and a
+// A unit of work is up to two row tiles of 128 stacked rows of one (sequence, kv head) and a
 // contiguous range of 128-key tiles (prefix tiles, then the draft tiles that hold a visible
 // key for any of its rows).  Warp roles:
 //   warps 0-3   softmax of row tile 0 (thread = row = TMEM lane)
@@ -52,8 +52,10 @@ enum Bar {
     BAR_S_FULL = BAR_V_EMPTY + VST,   // 2
     BAR_P_READY = BAR_S_FULL + 2,     // 2: keys 0..63 of P are in TMEM
     BAR_P_READY2 = BAR_P_READY + 2,   // 2: keys 64..127 of P are in TMEM
-    BAR_O_DONE = BAR_P_READY2 + 2,    // 2
-    BAR_COUNT = BAR_O_DONE + 2
+    BAR_O_DONE = BAR_P_READY2 + 2,    // 2: every PV of the unit has completed
+    BAR_O_FREE = BAR_O_DONE + 2,      // 2: the accumulator rows of the unit have been read out
+    BAR_Q_EMPTY = BAR_O_FREE + 2,     // 1: every QK^T of the unit has completed
+    BAR_COUNT = BAR_Q_EMPTY + 1
 };
 
 struct TcParams {
@@ -66,6 +68,7 @@ struct TcParams {
     int B, N, Hq, Hkv, Lmax, G, W, R;
     float scale_log2;
     PlanDev plan;
+    int total_work;   // CTAs of the plan = units of work
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -265,6 +268,53 @@ __device__ __forceinline__ TileInfo tile_info(int t, int nPT, int L, unsigned li
     return ti;
 }
 
+// What a role needs to know about one unit of work (a row pair of one (sequence, kv head) and
+// a key range).  Every warp derives it on its own from the work index, so the roles never
+// have to meet at a CTA-wide barrier between units.
+struct UnitInfo {
+    int b, c, row0, split, nsplit, slot;
+    int L, nPT, t_begin, ntiles;
+    unsigned live;   // draft tiles (128 nodes each) holding a visible key for any row of the unit
+    bool two;        // the second row tile exists
+};
+
+__device__ __forceinline__ UnitInfo unit_info(const TcParams& p, int w, int lane) {
+    UnitInfo u;
+    int item;
+    plan_decode(p.plan, w, item, u.split, u.nsplit, u.slot);
+    const int unit = item / p.plan.tiles_per_unit;
+    u.row0 = (item % p.plan.tiles_per_unit) * (2 * BM);
+    u.b = unit / p.Hkv;
+    u.c = unit % p.Hkv;
+    u.two = u.row0 + BM < p.R;
+    int L = p.seq_lens[u.b];
+    L = L < 0 ? 0 : (L > p.Lmax ? p.Lmax : L);
+    u.L = L;
+    // OR the mask rows of the unit's nodes, one node per lane
+    const int n_lo = u.row0 / p.G;
+    const int n_hi = (min(u.row0 + 2 * BM, p.R) - 1) / p.G + 1;
+    unsigned live = 0;
+    for (int n = n_lo + lane; n < n_hi; n += 32) {
+        const uint32_t* mrow = p.mask + ((size_t)u.b * p.N + n) * p.W;
+        for (int wi = 0; wi < p.W; ++wi) {
+            uint32_t word = mrow[wi];
+            if (wi == p.W - 1 && (p.N & 31)) word &= (1u << (p.N & 31)) - 1u;
+            if (word) live |= 1u << (wi >> 2);
+        }
+    }
+    u.live = __reduce_or_sync(0xFFFFFFFFu, live);
+    u.nPT = (L + BN - 1) / BN;
+    const int T = u.nPT + __popc(u.live);
+    const int per = (T + u.nsplit - 1) / u.nsplit;
+    u.t_begin = min(u.split * per, T);
+    u.ntiles = min(u.t_begin + per, T) - u.t_begin;
+    return u;
+}
+
+// Persistent kernel: CTA k walks the work indices k, k + gridDim.x, ...  Barrier phases are
+// counted across units, so the producer and the MMA issuer run ahead into the next unit
+// (Q, the first K/V tiles and the first QK^T) while the softmax warps still drain the
+// accumulators of the previous one.
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_dk,
@@ -273,17 +323,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     __shared__ __align__(8) unsigned long long s_bars[BAR_COUNT];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
-    __shared__ unsigned s_live;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    int item, split, nsplit, slot;
-    plan_decode(p.plan, blockIdx.x, item, split, nsplit, slot);
-    const int unit = item / p.plan.tiles_per_unit;
-    const int row0 = (item % p.plan.tiles_per_unit) * (2 * BM);
-    const int b = unit / p.Hkv, c = unit % p.Hkv;
     const int N = p.N, G = p.G, R = p.R;
-    const bool two = row0 + BM < R;          // does the second row tile exist
-    const int ntile_rows = two ? 2 : 1;
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = smem_base;                                   // 2 tiles
@@ -293,16 +335,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     volatile int* abort_flag = &s_abort;
 
-    int L = p.seq_lens[b];
-    if (L < 0 || L > p.Lmax) {
-        if (tid == 0 && p.status) atomicOr((unsigned*)p.status, GSD_DEV_BAD_SEQ_LEN);
-        L = L < 0 ? 0 : p.Lmax;
-    }
-
     if (tid == 0) {
         s_abort = 0;
-        s_live = 0;
         mbar_init(bar(BAR_Q_FULL), 1);
+        mbar_init(bar(BAR_Q_EMPTY), 1);
         for (int s = 0; s < KST; ++s) { mbar_init(bar(BAR_K_FULL + s), 1); mbar_init(bar(BAR_K_EMPTY + s), 1); }
         for (int s = 0; s < VST; ++s) { mbar_init(bar(BAR_V_FULL + s), 1); mbar_init(bar(BAR_V_EMPTY + s), 1); }
         for (int i = 0; i < 2; ++i) {
@@ -310,6 +346,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             mbar_init(bar(BAR_P_READY + i), 128);
             mbar_init(bar(BAR_P_READY2 + i), 128);
             mbar_init(bar(BAR_O_DONE + i), 1);
+            mbar_init(bar(BAR_O_FREE + i), 128);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -317,146 +354,157 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&s_tmem_base)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    __syncthreads();
-
-    // draft tiles (128 nodes each) that hold a visible key for any row of this CTA
-    if (tid < 2 * BM) {
-        const int r = row0 + tid;
-        unsigned live = 0;
-        if (r < R) {
-            const uint32_t* mrow = p.mask + ((size_t)b * N + r / G) * p.W;
-            for (int w = 0; w < p.W; ++w) {
-                uint32_t word = mrow[w];
-                if (w == p.W - 1 && (N & 31)) word &= (1u << (N & 31)) - 1u;
-                if (word) live |= 1u << (w >> 2);
-            }
-        }
-        live = __reduce_or_sync(0xFFFFFFFFu, live);
-        if (lane == 0 && live) atomicOr(&s_live, live);
-    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem_base;
-    const unsigned live = s_live;
-
-    const int nPT = (L + BN - 1) / BN;
-    const int T = nPT + __popc(live);
-    const int per = (T + nsplit - 1) / nsplit;
-    const int t_begin = min(split * per, T), t_end = min(t_begin + per, T);
-    const int ntiles = t_end - t_begin;
+    const int total_work = p.total_work;
 
     if (warp >= 8) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
     if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
-        if (lane == 0 && ntiles > 0) {
-            mbar_expect_tx(bar(BAR_Q_FULL), (uint32_t)ntile_rows * TILE_BYTES);
-            for (int i = 0; i < ntile_rows; ++i)
-                for (int h = 0; h < 2; ++h)
-                    tma_load_4d(sQ + i * TILE_BYTES + h * HALF_BYTES, &tm_q, bar(BAR_Q_FULL), h * 64, c * G,
-                                (row0 + i * BM) / G, b);
-            int issued_k = 0, issued_v = 0;
-            bool ok = true;
-            for (int idx = 0; idx < ntiles && ok; ++idx) {
-                const TileInfo ti = tile_info(t_begin + idx, nPT, L, live);
-                const CUtensorMap* mk = ti.kind == 2 ? &tm_dk : &tm_k;
-                const CUtensorMap* mv = ti.kind == 2 ? &tm_dv : &tm_v;
-                {
-                    const int s = idx % KST;
-                    ok = mbar_wait(bar(BAR_K_EMPTY + s), ((idx / KST) & 1) ^ 1, abort_flag, p.status);
+        int kvc = 0;          // key tiles loaded so far (ring position)
+        int au = 0;           // non-empty units so far
+        bool ok = true, q_pending = false;
+        for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+            const UnitInfo u = unit_info(p, w, lane);
+            if (u.ntiles == 0) continue;
+            if (lane == 0) {
+                // Q of the previous unit is free once its last QK^T has completed
+                ok = mbar_wait(bar(BAR_Q_EMPTY), (au & 1) ^ 1, abort_flag, p.status);
+                if (ok) {
+                    const int ntile_rows = u.two ? 2 : 1;
+                    mbar_expect_tx(bar(BAR_Q_FULL), (uint32_t)ntile_rows * TILE_BYTES);
+                    for (int i = 0; i < ntile_rows; ++i)
+                        for (int h = 0; h < 2; ++h)
+                            tma_load_4d(sQ + i * TILE_BYTES + h * HALF_BYTES, &tm_q, bar(BAR_Q_FULL), h * 64, u.c * G,
+                                        (u.row0 + i * BM) / G, u.b);
+                    q_pending = true;
+                }
+                for (int idx = 0; idx < u.ntiles && ok; ++idx) {
+                    const TileInfo ti = tile_info(u.t_begin + idx, u.nPT, u.L, u.live);
+                    const CUtensorMap* mk = ti.kind == 2 ? &tm_dk : &tm_k;
+                    const CUtensorMap* mv = ti.kind == 2 ? &tm_dv : &tm_v;
+                    const int s = kvc % KST;
+                    const uint32_t par = (uint32_t)((kvc / KST) & 1) ^ 1u;
+                    ok = mbar_wait(bar(BAR_K_EMPTY + s), par, abort_flag, p.status);
                     if (!ok) break;
                     mbar_expect_tx(bar(BAR_K_FULL + s), TILE_BYTES);
                     for (int h = 0; h < 2; ++h)
-                        tma_load_4d(sK + s * TILE_BYTES + h * HALF_BYTES, mk, bar(BAR_K_FULL + s), h * 64, c, ti.key0, b);
-                    issued_k = idx + 1;
-                }
-                {
-                    const int s = idx % VST;
-                    ok = mbar_wait(bar(BAR_V_EMPTY + s), ((idx / VST) & 1) ^ 1, abort_flag, p.status);
-                    if (!ok) break;
+                        tma_load_4d(sK + s * TILE_BYTES + h * HALF_BYTES, mk, bar(BAR_K_FULL + s), h * 64, u.c, ti.key0, u.b);
+                    ok = mbar_wait(bar(BAR_V_EMPTY + s), par, abort_flag, p.status);
+                    if (!ok) {
+                        // the K copy just issued is still in flight: let it land
+                        mbar_wait_slow(bar(BAR_K_FULL + s), (kvc / KST) & 1, abort_flag, nullptr, true);
+                        break;
+                    }
                     mbar_expect_tx(bar(BAR_V_FULL + s), TILE_BYTES);
                     for (int h = 0; h < 2; ++h)
-                        tma_load_4d(sV + s * TILE_BYTES + h * HALF_BYTES, mv, bar(BAR_V_FULL + s), h * 64, c, ti.key0, b);
-                    issued_v = idx + 1;
+                        tma_load_4d(sV + s * TILE_BYTES + h * HALF_BYTES, mv, bar(BAR_V_FULL + s), h * 64, u.c, ti.key0, u.b);
+                    ++kvc;
+                }
+                if (!ok) {
+                    // gave up: let the copies already in flight land before the CTA retires
+                    if (q_pending) mbar_wait_slow(bar(BAR_Q_FULL), au & 1, abort_flag, nullptr, true);
+                    for (int t = max(0, kvc - KST); t < kvc; ++t) {
+                        mbar_wait_slow(bar(BAR_K_FULL + t % KST), (t / KST) & 1, abort_flag, nullptr, true);
+                        mbar_wait_slow(bar(BAR_V_FULL + t % VST), (t / VST) & 1, abort_flag, nullptr, true);
+                    }
                 }
             }
-            if (!ok) {
-                // gave up: let the copies already in flight land before the CTA retires
-                mbar_wait_slow(bar(BAR_Q_FULL), 0, abort_flag, nullptr, true);
-                for (int idx = max(0, issued_k - KST); idx < issued_k; ++idx)
-                    mbar_wait_slow(bar(BAR_K_FULL + idx % KST), (idx / KST) & 1, abort_flag, nullptr, true);
-                for (int idx = max(0, issued_v - VST); idx < issued_v; ++idx)
-                    mbar_wait_slow(bar(BAR_V_FULL + idx % VST), (idx / VST) & 1, abort_flag, nullptr, true);
-            }
+            ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+            kvc = __shfl_sync(0xFFFFFFFFu, kvc, 0);
+            ++au;
         }
     } else if (warp == 9) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0 && ntiles > 0) {
-            bool ok = mbar_wait(bar(BAR_Q_FULL), 0, abort_flag, p.status);
+        int kvc = 0;              // key tiles consumed so far (ring position)
+        int au = 0, au1 = 0;      // non-empty units so far; those of them with a second row tile
+        int tc0 = 0, tc1 = 0;     // key tiles handed to the softmax of row tile 0 / 1 so far
+        bool ok = true;
+        auto issue_qk = [&](int i, int stage) {
+            // S_i = Q_i K^T : 8 k-steps of 16 over the head dimension
+            const uint32_t qa = sQ + i * TILE_BYTES, ka = sK + stage * TILE_BYTES;
+#pragma unroll
+            for (int ks = 0; ks < HD / 16; ++ks) {
+                const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+                tc_mma_ss(tmem + (i ? COL_S1 : COL_S0), desc_kmajor(qa + off), desc_kmajor(ka + off), kIdescQK, ks > 0);
+            }
+        };
+        // O_i += P_i V : 8 k-steps of 16 keys; P (bf16 pairs) sits in S_i's first 64 columns.
+        // The softmax hands P over in two halves of 64 keys, so the first four k-steps run
+        // while the second half of the exponentials is still being computed.
+        auto issue_pv_half = [&](int i, int stage, int half, bool accumulate) {
+            const uint32_t va = sV + stage * TILE_BYTES;
+#pragma unroll
+            for (int k4 = 0; k4 < BN / 32; ++k4) {
+                const int ks = half * (BN / 32) + k4;
+                tc_mma_ts(tmem + (i ? COL_O1 : COL_O0), tmem + (i ? COL_S1 : COL_S0) + ks * 8,
+                          desc_mnmajor(va + ks * 2048), kIdescPV, (accumulate || ks > 0) ? 1u : 0u);
+            }
+        };
+        // tile = running tile number of row tile i (barrier phase); first = first tile of the unit
+        auto issue_pv = [&](int i, int stage, int tile, bool first, int units_before) -> bool {
+            if (!mbar_wait(bar(BAR_P_READY + i), tile & 1, abort_flag, p.status)) return false;
+            if (first && units_before > 0) {
+                // the accumulator still belongs to the previous unit until its rows were read out
+                if (!mbar_wait(bar(BAR_O_FREE + i), (units_before - 1) & 1, abort_flag, p.status)) return false;
+            }
             tc_fence_after();
-            auto issue_qk = [&](int i, int ks_stage) {
-                // S_i = Q_i K^T : 8 k-steps of 16 over the head dimension
-                const uint32_t qa = sQ + i * TILE_BYTES, ka = sK + ks_stage * TILE_BYTES;
-#pragma unroll
-                for (int ks = 0; ks < HD / 16; ++ks) {
-                    const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
-                    tc_mma_ss(tmem + (i ? COL_S1 : COL_S0), desc_kmajor(qa + off), desc_kmajor(ka + off), kIdescQK, ks > 0);
-                }
-            };
-            // O_i += P_i V : 8 k-steps of 16 keys; P (bf16 pairs) sits in S_i's first 64 columns.
-            // The softmax hands P over in two halves of 64 keys, so the first four k-steps run
-            // while the second half of the exponentials is still being computed.
-            auto issue_pv_half = [&](int i, int vs_stage, int half, bool accumulate) {
-                const uint32_t va = sV + vs_stage * TILE_BYTES;
-#pragma unroll
-                for (int k4 = 0; k4 < BN / 32; ++k4) {
-                    const int ks = half * (BN / 32) + k4;
-                    tc_mma_ts(tmem + (i ? COL_O1 : COL_O0), tmem + (i ? COL_S1 : COL_S0) + ks * 8,
-                              desc_mnmajor(va + ks * 2048), kIdescPV, (accumulate || ks > 0) ? 1u : 0u);
-                }
-            };
-            auto issue_pv = [&](int i, int vs_stage, int idx, bool accumulate) -> bool {
-                if (!mbar_wait(bar(BAR_P_READY + i), idx & 1, abort_flag, p.status)) return false;
+            issue_pv_half(i, stage, 0, !first);
+            if (!mbar_wait(bar(BAR_P_READY2 + i), tile & 1, abort_flag, p.status)) return false;
+            tc_fence_after();
+            issue_pv_half(i, stage, 1, !first);
+            return true;
+        };
+        for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+            const UnitInfo u = unit_info(p, w, lane);
+            if (u.ntiles == 0) continue;
+            if (lane == 0) {
+                const bool two = u.two;
+                const int ntiles = u.ntiles;
+                ok = mbar_wait(bar(BAR_Q_FULL), au & 1, abort_flag, p.status);
                 tc_fence_after();
-                issue_pv_half(i, vs_stage, 0, accumulate);
-                if (!mbar_wait(bar(BAR_P_READY2 + i), idx & 1, abort_flag, p.status)) return false;
-                tc_fence_after();
-                issue_pv_half(i, vs_stage, 1, accumulate);
-                return true;
-            };
-            for (int idx = 0; idx < ntiles && ok; ++idx) {
-                const int ks_stage = idx % KST, vs_stage = idx % VST;
-                ok = mbar_wait(bar(BAR_K_FULL + ks_stage), (idx / KST) & 1, abort_flag, p.status);
-                if (!ok) break;
-                tc_fence_after();
-                issue_qk(0, ks_stage);
-                tc_commit(bar(BAR_S_FULL + 0));
-                if (two) {
-                    if (idx > 0) {
-                        ok = issue_pv(1, (idx - 1) % VST, idx - 1, idx - 1 > 0);
-                        if (!ok) break;
-                        tc_commit(bar(BAR_V_EMPTY + (idx - 1) % VST));
+                for (int idx = 0; idx < ntiles && ok; ++idx) {
+                    const int st = kvc % KST;
+                    ok = mbar_wait(bar(BAR_K_FULL + st), (kvc / KST) & 1, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(0, st);
+                    tc_commit(bar(BAR_S_FULL + 0));
+                    if (two) {
+                        if (idx > 0) {
+                            ok = issue_pv(1, (kvc - 1) % VST, tc1 + idx - 1, idx == 1, au1);
+                            if (!ok) break;
+                            tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
+                        }
+                        issue_qk(1, st);
+                        tc_commit(bar(BAR_S_FULL + 1));
                     }
-                    issue_qk(1, ks_stage);
-                    tc_commit(bar(BAR_S_FULL + 1));
+                    tc_commit(bar(BAR_K_EMPTY + st));
+                    if (idx == ntiles - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
+                    ok = mbar_wait(bar(BAR_V_FULL + st), (kvc / VST) & 1, abort_flag, p.status);
+                    if (!ok) break;
+                    ok = issue_pv(0, st, tc0 + idx, idx == 0, au);
+                    if (!ok) break;
+                    if (!two) tc_commit(bar(BAR_V_EMPTY + st));
+                    if (idx == ntiles - 1) tc_commit(bar(BAR_O_DONE + 0));
+                    ++kvc;
                 }
-                tc_commit(bar(BAR_K_EMPTY + ks_stage));
-                ok = mbar_wait(bar(BAR_V_FULL + vs_stage), (idx / VST) & 1, abort_flag, p.status);
-                if (!ok) break;
-                ok = issue_pv(0, vs_stage, idx, idx > 0);
-                if (!ok) break;
-                if (!two) tc_commit(bar(BAR_V_EMPTY + vs_stage));
-                if (idx == ntiles - 1) tc_commit(bar(BAR_O_DONE + 0));
-            }
-            if (ok && two) {
-                const int idx = ntiles - 1;
-                ok = issue_pv(1, idx % VST, idx, idx > 0);
-                if (ok) {
-                    tc_commit(bar(BAR_V_EMPTY + idx % VST));
-                    tc_commit(bar(BAR_O_DONE + 1));
+                if (ok && two) {
+                    ok = issue_pv(1, (kvc - 1) % VST, tc1 + ntiles - 1, ntiles == 1, au1);
+                    if (ok) {
+                        tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
+                        tc_commit(bar(BAR_O_DONE + 1));
+                    }
                 }
             }
+            ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+            kvc = __shfl_sync(0xFFFFFFFFu, kvc, 0);
+            tc0 += u.ntiles;
+            ++au;
+            if (u.two) { tc1 += u.ntiles; ++au1; }
         }
     }
     } else {
@@ -464,17 +512,31 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         // ------------------------------------------------------------ softmax + epilogue
         const int i = warp >> 2;                         // row tile of this warpgroup
         const int rloc = (warp & 3) * 32 + lane;         // row inside the tile = TMEM lane
-        const int row = row0 + i * BM + rloc;
-        const bool rvalid = row < R;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + lane_addr + (i ? COL_S1 : COL_S0);
         const uint32_t tO = tmem + lane_addr + (i ? COL_O1 : COL_O0);
-        float m_ref = -CUDART_INF_F, l_run = 0.f;
+        int kvc = 0;      // key tiles of all non-empty units so far (ring position of the V tiles)
+        int tcnt = 0;     // key tiles this row tile has processed so far (barrier phase)
+        int auc = 0;      // units this row tile has finished so far
         bool ok = true;
-        if (i == 0 || two) {
+        for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+            const UnitInfo u = unit_info(p, w, lane);
+            if (i == 1 && !u.two) {
+                kvc += u.ntiles;
+                continue;
+            }
+            const int ntiles = u.ntiles;
+            const int b = u.b, c = u.c;
+            const int row = u.row0 + i * BM + rloc;
+            const bool rvalid = row < R;
+            if (warp == 0 && lane == 0) {
+                const int Lraw = p.seq_lens[b];
+                if ((Lraw < 0 || Lraw > p.Lmax) && p.status) atomicOr((unsigned*)p.status, GSD_DEV_BAD_SEQ_LEN);
+            }
+            float m_ref = -CUDART_INF_F, l_run = 0.f;
             const uint32_t* mrow = p.mask + ((size_t)b * N + (rvalid ? row / G : 0)) * p.W;
             for (int idx = 0; idx < ntiles; ++idx) {
-                const TileInfo ti = tile_info(t_begin + idx, nPT, L, live);
+                const TileInfo ti = tile_info(u.t_begin + idx, u.nPT, u.L, u.live);
                 // visibility words of this row for the 128 keys of the tile
                 uint32_t mw[4];
                 if (ti.kind == 0) {
@@ -495,7 +557,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         mw[k] = word;
                     }
                 }
-                ok = mbar_wait(bar(BAR_S_FULL + i), idx & 1, abort_flag, p.status);
+                const uint32_t par = (uint32_t)((tcnt + idx) & 1);
+                ok = mbar_wait(bar(BAR_S_FULL + i), par, abort_flag, p.status);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
@@ -546,8 +609,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (ti.kind == 1 && i == 0) {
                     // cache rows past the sequence end may hold anything: clear them in the V tile
                     // so that 0 * junk cannot reach the accumulator
-                    const int vs_stage = idx % VST;
-                    ok = mbar_wait(bar(BAR_V_FULL + vs_stage), (idx / VST) & 1, abort_flag, p.status);
+                    const int vs_stage = (kvc + idx) % VST;
+                    ok = mbar_wait(bar(BAR_V_FULL + vs_stage), (uint32_t)(((kvc + idx) / VST) & 1), abort_flag, p.status);
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     if (rloc >= ti.nvalid) {
@@ -583,68 +646,54 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     }
                 }
                 l_run += (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
-
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(BAR_P_READY2 + i));
             }
+            if (!ok) break;
 
-            // ---- epilogue
-            if (ok && ntiles > 0) {
-                ok = mbar_wait(bar(BAR_O_DONE + i), 0, abort_flag, p.status);
+            // ---- epilogue: pull the accumulator row into registers, give TMEM back, then store
+            float acc[HD];
+            if (ntiles > 0) {
+                ok = mbar_wait(bar(BAR_O_DONE + i), (uint32_t)(auc & 1), abort_flag, p.status);
                 ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
                 tc_fence_after();
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) tc_ld32p(tO + ch * 32, acc + ch * 32);
+                tc_wait_ld();
+                tc_fence_before();
+                mbar_arrive(bar(BAR_O_FREE + i));
+            } else {
+#pragma unroll
+                for (int e = 0; e < HD; ++e) acc[e] = 0.f;
             }
-            if (ok) {
-                const int n = rvalid ? row / G : 0, g = rvalid ? row % G : 0;
-                if (nsplit == 1) {
+            if (rvalid) {
+                if (u.nsplit == 1) {
                     const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-                    __nv_bfloat16* dst = p.out + (((size_t)b * N + n) * p.Hq + c * G + g) * HD;
+                    __nv_bfloat16* dst = p.out + (((size_t)b * N + row / G) * p.Hq + c * G + row % G) * HD;
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        float v[32];
-                        if (ntiles > 0) {
-                            tc_ld32(tO + ch * 32, v);
-                            tc_wait_ld();
-                        } else {
-#pragma unroll
-                            for (int e = 0; e < 32; ++e) v[e] = 0.f;
-                        }
-                        if (rvalid) {
-#pragma unroll
-                            for (int k = 0; k < 4; ++k) {
-                                uint4 u;
-                                u.x = pack_bf16(v[8 * k + 0] * inv, v[8 * k + 1] * inv);
-                                u.y = pack_bf16(v[8 * k + 2] * inv, v[8 * k + 3] * inv);
-                                u.z = pack_bf16(v[8 * k + 4] * inv, v[8 * k + 5] * inv);
-                                u.w = pack_bf16(v[8 * k + 6] * inv, v[8 * k + 7] * inv);
-                                *reinterpret_cast<uint4*>(dst + ch * 32 + k * 8) = u;
-                            }
-                        }
+                    for (int k = 0; k < HD / 8; ++k) {
+                        uint4 v;
+                        v.x = pack_bf16(acc[8 * k + 0] * inv, acc[8 * k + 1] * inv);
+                        v.y = pack_bf16(acc[8 * k + 2] * inv, acc[8 * k + 3] * inv);
+                        v.z = pack_bf16(acc[8 * k + 4] * inv, acc[8 * k + 5] * inv);
+                        v.w = pack_bf16(acc[8 * k + 6] * inv, acc[8 * k + 7] * inv);
+                        *reinterpret_cast<uint4*>(dst + k * 8) = v;
                     }
                 } else {
-                    const size_t prow = (size_t)slot * (2 * BM) + i * BM + rloc;
+                    const size_t prow = (size_t)u.slot * (2 * BM) + i * BM + rloc;
                     float* dst = p.part_o + prow * HD;
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        float v[32];
-                        if (ntiles > 0) {
-                            tc_ld32(tO + ch * 32, v);
-                            tc_wait_ld();
-                        } else {
-#pragma unroll
-                            for (int e = 0; e < 32; ++e) v[e] = 0.f;
-                        }
-                        if (rvalid) {
-#pragma unroll
-                            for (int k = 0; k < 8; ++k)
-                                *reinterpret_cast<float4*>(dst + ch * 32 + k * 4) =
-                                    make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
-                        }
-                    }
-                    if (rvalid) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(m_ref, l_run);
+                    for (int k = 0; k < HD / 4; ++k)
+                        *reinterpret_cast<float4*>(dst + k * 4) =
+                            make_float4(acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]);
+                    *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(m_ref, l_run);
                 }
             }
+            kvc += ntiles;
+            tcnt += ntiles;
+            if (ntiles > 0) ++auc;
         }
     }
 
@@ -721,7 +770,10 @@ int launch_attn_tcgen05(const AttnArgs& a) {
     p.part_o = (float*)a.workspace;
     p.part_ml = (float*)((char*)a.workspace + plan_part_o_bytes(a.plan, a.D));
     GSD_CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
-    dim3 grid(a.plan.ctas);
+    p.total_work = a.plan.ctas;
+    DeviceInfo di;
+    if (device_info(&di) != 0) return GSD_ERR_CUDA;
+    dim3 grid(a.plan.ctas < di.sm_count ? a.plan.ctas : di.sm_count);
     attn_tc_kernel<<<grid, kThreads, kSmemBytes, a.stream>>>(tq, tk, tv, tdk, tdv, p);
     GSD_CUDA_TRY(cudaGetLastError());
     return GSD_OK;
