@@ -361,7 +361,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const int total_work = p.total_work;
 
     if (warp >= 8) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 96;");
     if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
         int kvc = 0;          // key tiles loaded so far (ring position)
@@ -508,7 +508,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
     }
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
         // ------------------------------------------------------------ softmax + epilogue
         const int i = warp >> 2;                         // row tile of this warpgroup
         const int rloc = (warp & 3) * 32 + lane;         // row inside the tile = TMEM lane
