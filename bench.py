@@ -128,6 +128,15 @@ def dist_setup(n_gpus: int):
     return rank, world, local, None
 
 
+def aggregate_over_ranks(ms_per_step, tokens_per_step, world, dist, device):
+    """Step time = the maximum over ranks; value = the tokens of all replicas over that time."""
+    if dist is not None and world > 1:
+        tt = torch.tensor([ms_per_step], dtype=torch.float64, device=device)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_per_step = float(tt.item())
+    return {"ms_per_step": ms_per_step, "value": world * tokens_per_step / (ms_per_step * 1e-3)}
+
+
 def cpu_oracle_sample(cfg, inp, budget_rows: int):
     """Times the CPU oracle (as it stands) on a bounded sample of the workload: `budget_rows`
     random attention rows plus the full acceptance step.  Returns (tokens/s extrapolated to
@@ -182,8 +191,8 @@ def run_reference(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=6000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default="llama70b", choices=sorted(gi.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 mma.sync, 2 tcgen05")
@@ -264,13 +273,10 @@ def main():
     acc_ms = [ev[1].elapsed_time(ev[2]) for ev in events]
     if int(status.item()) != 0:
         raise RuntimeError(f"device status {int(status.item()):#x}")
-    if dist is not None:
-        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
-    ms_per_step = total_ms / args.steps
     tokens = cfg.B * cfg.N
-    value = world * tokens / (ms_per_step * 1e-3)
+    agg = aggregate_over_ranks(total_ms / args.steps, tokens, world, dist, dev)
+    ms_per_step, value = agg["ms_per_step"], agg["value"]
+    total_ms = ms_per_step * args.steps
 
     # ---- end to end through the host-buffer C-ABI call (pinned host tensors)
     e2e = None
@@ -300,10 +306,7 @@ def main():
             host_step()
         torch.cuda.synchronize()
         t_e2e = (time.perf_counter() - t0) / args.e2e_steps
-        if dist is not None:
-            tt = torch.tensor([t_e2e], dtype=torch.float64, device=dev)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            t_e2e = float(tt.item())
+        t_e2e = aggregate_over_ranks(t_e2e * 1e3, tokens, world, dist, dev)["ms_per_step"] * 1e-3
         h2d = sum(h[k].numel() * h[k].element_size() for k in h)
         d2h = h_out.numel() * 2 + sum(x.numel() * 4 for x in h_acc) + 4
         e2e = {"value": world * tokens / t_e2e, "unit": UNIT, "ms_per_step": t_e2e * 1e3,

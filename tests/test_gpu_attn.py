@@ -148,3 +148,40 @@ def test_bad_seq_len_is_clamped_and_flagged():
     got = out_to_f64(gpu_attn(inp2, status=status))
     assert int(status.item()) == 0x10
     assert_close(got, want)          # clamped to Lmax == the true length here
+
+
+@pytest.mark.parametrize("point", [(1, 512, 32), (8, 2048, 128), (1, 8192, 512)])
+def test_sweep_points_sampled_rows(point):
+    # 70B-shaped sweep (64 q heads over 8 kv heads, D 128): one whole (sequence, kv head) unit
+    # of stacked rows plus 256 random rows, each recomputed one by one by the oracle
+    B, L, N = point
+    cfg = gi.sweep_config(B, L, N)
+    inp = gi.make_inputs(cfg, accept=False)
+    got = out_to_f64(gpu_attn(inp))
+    rng = np.random.default_rng(B * 1000 + N)
+    b0, c0 = int(rng.integers(cfg.B)), int(rng.integers(cfg.Hkv))
+    rows = [(b0, n, c0 * cfg.G + g) for n in range(0, cfg.N, max(1, cfg.N // 64)) for g in range(cfg.G)]
+    rows += [(int(rng.integers(cfg.B)), int(rng.integers(cfg.N)), int(rng.integers(cfg.Hq)))
+             for _ in range(256)]
+    want = oracle.attn_rows(inp["q"], inp["k_cache"], inp["v_cache"], inp["draft_k"],
+                            inp["draft_v"], inp["ancestor_mask"], inp["seq_lens"], rows)
+    assert_close(np.stack([got[b, n, h] for b, n, h in rows]), want)
+
+
+def test_dominant_key_and_large_score_jumps():
+    # one cache key scores 2^k times above the rest from some tile on: the running maximum has
+    # to be raised (accumulator rescale path) and nothing may overflow
+    cfg = gi.VerifyConfig("t", 7, 1, 8, 1, 128, 700, 130, 10, 4, 3, 8, 8, 0.5)
+    inp = gi.make_inputs(cfg, 3, accept=False)
+    k = gi.bf16_bits_to_f32(inp["k_cache"])
+    q = gi.bf16_bits_to_f32(inp["q"])
+    q[0, :, :, 5] = 24.0
+    k[0, :, 0, 5] = 0.0
+    k[0, 300, 0, 5] = 6.0          # +144/sqrt(128) = +12.7 in score units at key 300
+    k[0, 650, 0, 5] = 24.0         # +50.9 at key 650 (a later tile)
+    inp["q"], inp["k_cache"] = gi.f32_to_bf16_bits(q), gi.f32_to_bf16_bits(k)
+    dk = gi.bf16_bits_to_f32(inp["draft_k"]); dk[0, :, 0, 5] = 0.0
+    inp["draft_k"] = gi.f32_to_bf16_bits(dk)
+    want = cpu_attn(inp)
+    for kernel in KERNELS:
+        assert_close(out_to_f64(gpu_attn(inp, kernel=kernel)), want)
