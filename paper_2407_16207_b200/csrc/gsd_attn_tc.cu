@@ -294,12 +294,28 @@ __device__ __forceinline__ UnitInfo unit_info(const TcParams& p, int w, int lane
     const int n_lo = u.row0 / p.G;
     const int n_hi = (min(u.row0 + 2 * BM, p.R) - 1) / p.G + 1;
     unsigned live = 0;
-    for (int n = n_lo + lane; n < n_hi; n += 32) {
-        const uint32_t* mrow = p.mask + ((size_t)u.b * p.N + n) * p.W;
-        for (int wi = 0; wi < p.W; ++wi) {
-            uint32_t word = mrow[wi];
-            if (wi == p.W - 1 && (p.N & 31)) word &= (1u << (p.N & 31)) - 1u;
-            if (word) live |= 1u << (wi >> 2);
+    const uint32_t tail = (p.N & 31) ? (1u << (p.N & 31)) - 1u : 0xFFFFFFFFu;   // valid bits of the last word
+    if ((p.W & 3) == 0 && (reinterpret_cast<uintptr_t>(p.mask) & 15u) == 0) {
+        // four words = one draft tile per 16-byte load; all loads of a row are issued before any is used
+        for (int n = n_lo + lane; n < n_hi; n += 32) {
+            const uint4* mrow = reinterpret_cast<const uint4*>(p.mask + ((size_t)u.b * p.N + n) * p.W);
+            uint4 q[GSD_MAX_NODES / 128];
+#pragma unroll
+            for (int t = 0; t < GSD_MAX_NODES / 128; ++t) q[t] = t < (p.W >> 2) ? mrow[t] : make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int t = 0; t < GSD_MAX_NODES / 128; ++t) {
+                if (t == (p.W >> 2) - 1) q[t].w &= tail;
+                if (q[t].x | q[t].y | q[t].z | q[t].w) live |= 1u << t;
+            }
+        }
+    } else {
+        for (int n = n_lo + lane; n < n_hi; n += 32) {
+            const uint32_t* mrow = p.mask + ((size_t)u.b * p.N + n) * p.W;
+            for (int wi = 0; wi < p.W; ++wi) {
+                uint32_t word = mrow[wi];
+                if (wi == p.W - 1) word &= tail;
+                if (word) live |= 1u << (wi >> 2);
+            }
         }
     }
     u.live = __reduce_or_sync(0xFFFFFFFFu, live);
