@@ -359,10 +359,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         for (int s = 0; s < VST; ++s) { mbar_init(bar(BAR_V_FULL + s), 1); mbar_init(bar(BAR_V_EMPTY + s), 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(BAR_S_FULL + i), 1);
-            mbar_init(bar(BAR_P_READY + i), 128);
-            mbar_init(bar(BAR_P_READY2 + i), 128);
+            mbar_init(bar(BAR_P_READY + i), 4);    // one arrival per softmax warp
+            mbar_init(bar(BAR_P_READY2 + i), 4);
             mbar_init(bar(BAR_O_DONE + i), 1);
-            mbar_init(bar(BAR_O_FREE + i), 128);
+            mbar_init(bar(BAR_O_FREE + i), 4);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -644,27 +644,33 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
                 const float2 negm2 = make_float2(-m_use, -m_use);
                 float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t pk[16];
+                uint32_t pk[4][16];
+                auto exp_chunk = [&](int ch) {
 #pragma unroll
                     for (int e = 0; e < 16; ++e) {
                         const float2 t = ffma2(make_float2(sc[ch * 32 + 2 * e], sc[ch * 32 + 2 * e + 1]), scale2, negm2);
                         const float2 pe = make_float2(fast_exp2(t.x), fast_exp2(t.y));
                         sum2[e & 1] = fadd2(sum2[e & 1], pe);
-                        pk[e] = pack_bf16(pe.x, pe.y);
+                        pk[ch][e] = pack_bf16(pe.x, pe.y);
                     }
-                    tc_st16(tS + ch * 16, pk);
-                    if (ch == 1) {            // keys 0..63 are in place (and any rescale of O is done)
-                        tc_wait_st();
-                        tc_fence_before();
-                        mbar_arrive(bar(BAR_P_READY + i));
-                    }
-                }
+                };
+                // The TMEM stores of one half are in flight while the next chunk's exponentials are
+                // computed; the hand-off of a half follows once its stores have landed.
+                exp_chunk(0);
+                exp_chunk(1);
+                tc_st16(tS + 0, pk[0]);
+                tc_st16(tS + 16, pk[1]);
+                exp_chunk(2);
+                tc_wait_st();              // keys 0..63 are in place (and any rescale of O is done)
+                tc_fence_before();
+                if (lane == 0) mbar_arrive(bar(BAR_P_READY + i));
+                exp_chunk(3);
+                tc_st16(tS + 32, pk[2]);
+                tc_st16(tS + 48, pk[3]);
                 l_run += (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
                 tc_wait_st();
                 tc_fence_before();
-                mbar_arrive(bar(BAR_P_READY2 + i));
+                if (lane == 0) mbar_arrive(bar(BAR_P_READY2 + i));
             }
             if (!ok) break;
 
@@ -679,7 +685,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 for (int ch = 0; ch < 4; ++ch) tc_ld32p(tO + ch * 32, acc + ch * 32);
                 tc_wait_ld();
                 tc_fence_before();
-                mbar_arrive(bar(BAR_O_FREE + i));
+                if (lane == 0) mbar_arrive(bar(BAR_O_FREE + i));
             } else {
 #pragma unroll
                 for (int e = 0; e < HD; ++e) acc[e] = 0.f;
