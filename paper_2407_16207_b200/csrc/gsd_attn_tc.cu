@@ -11,9 +11,9 @@
 //   warps 0-3   softmax of row tile 0 (thread = row = TMEM lane)
 //   warps 4-7   softmax of row tile 1
 //   warp  8     TMA producer (one thread): Q once, then K and V tiles into two smem rings
-//   warps 9,10  MMA issuers (one thread each, one per row tile): S_i = Q_i K^T into TMEM,
-//               O_i += P_i V with P read from TMEM (P overwrites the first half of S_i as bf16)
-//   warp 11     TMEM allocation / release
+//   warp  9     MMA issuer (one thread): S_i = Q_i K^T into TMEM, O_i += P_i V with P read
+//               from TMEM (P overwrites the first half of S_i as bf16)
+//   warp 10     TMEM allocation / release
 // The issue order QK0(j) PV1(j-1) QK1(j) PV0(j) lets the softmax of one row tile run under
 // the MMAs of the other.  The running maximum is only raised when a tile exceeds it by more
 // than 2^8 (the accumulator rescale is then done in place in TMEM by the row's own thread),
@@ -354,9 +354,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     if (tid == 0) {
         s_abort = 0;
         mbar_init(bar(BAR_Q_FULL), 1);
-        mbar_init(bar(BAR_Q_EMPTY), 2);       // released by both MMA streams
-        for (int s = 0; s < KST; ++s) { mbar_init(bar(BAR_K_FULL + s), 1); mbar_init(bar(BAR_K_EMPTY + s), 2); }
-        for (int s = 0; s < VST; ++s) { mbar_init(bar(BAR_V_FULL + s), 1); mbar_init(bar(BAR_V_EMPTY + s), 2); }
+        mbar_init(bar(BAR_Q_EMPTY), 1);
+        for (int s = 0; s < KST; ++s) { mbar_init(bar(BAR_K_FULL + s), 1); mbar_init(bar(BAR_K_EMPTY + s), 1); }
+        for (int s = 0; s < VST; ++s) { mbar_init(bar(BAR_V_FULL + s), 1); mbar_init(bar(BAR_V_EMPTY + s), 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(BAR_S_FULL + i), 1);
             mbar_init(bar(BAR_P_READY + i), 4);    // one arrival per softmax warp
@@ -366,7 +366,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 11) {
+    if (warp == 10) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&s_tmem_base)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -433,84 +433,94 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             kvc = __shfl_sync(0xFFFFFFFFu, kvc, 0);
             ++au;
         }
-    } else if (warp == 9 || warp == 10) {
-        // ------------------------------------------------------------ MMA issuers
-        // One issuing thread per row tile: warp 9 feeds row tile 0, warp 10 row tile 1.  Each
-        // keeps the order QK(j) PV(j) QK(j+1) of its own row tile (P aliases S); between the
-        // two streams there is no data dependence, so the tensor pipe always has the other
-        // row tile's MMAs to run while one stream waits for its softmax.  The K/V stages and
-        // Q are released by both streams (barrier count 2).
-        const int i = warp - 9;
-        int kvc = 0;          // key tiles consumed so far (ring position)
-        int au = 0;           // non-empty units so far (all of them, for the Q barrier phase)
-        int auc = 0;          // non-empty units this row tile took part in
-        int tcnt = 0;         // key tiles handed to this row tile's softmax so far
+    } else if (warp == 9) {
+        // ------------------------------------------------------------ MMA issuer
+        int kvc = 0;              // key tiles consumed so far (ring position)
+        int au = 0, au1 = 0;      // non-empty units so far; those of them with a second row tile
+        int tc0 = 0, tc1 = 0;     // key tiles handed to the softmax of row tile 0 / 1 so far
         bool ok = true;
-        const uint32_t tSi = tmem + (i ? COL_S1 : COL_S0), tOi = tmem + (i ? COL_O1 : COL_O0);
+        auto issue_qk = [&](int i, int stage) {
+            // S_i = Q_i K^T : 8 k-steps of 16 over the head dimension
+            const uint32_t qa = sQ + i * TILE_BYTES, ka = sK + stage * TILE_BYTES;
+#pragma unroll
+            for (int ks = 0; ks < HD / 16; ++ks) {
+                const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+                tc_mma_ss(tmem + (i ? COL_S1 : COL_S0), desc_kmajor(qa + off), desc_kmajor(ka + off), kIdescQK, ks > 0);
+            }
+        };
+        // O_i += P_i V : 8 k-steps of 16 keys; P (bf16 pairs) sits in S_i's first 64 columns.
+        // The softmax hands P over in two halves of 64 keys, so the first four k-steps run
+        // while the second half of the exponentials is still being computed.
+        auto issue_pv_half = [&](int i, int stage, int half, bool accumulate) {
+            const uint32_t va = sV + stage * TILE_BYTES;
+#pragma unroll
+            for (int k4 = 0; k4 < BN / 32; ++k4) {
+                const int ks = half * (BN / 32) + k4;
+                tc_mma_ts(tmem + (i ? COL_O1 : COL_O0), tmem + (i ? COL_S1 : COL_S0) + ks * 8,
+                          desc_mnmajor(va + ks * 2048), kIdescPV, (accumulate || ks > 0) ? 1u : 0u);
+            }
+        };
+        // tile = running tile number of row tile i (barrier phase); first = first tile of the unit
+        auto issue_pv = [&](int i, int stage, int tile, bool first, int units_before) -> bool {
+            if (!mbar_wait(bar(BAR_P_READY + i), tile & 1, abort_flag, p.status)) return false;
+            if (first && units_before > 0) {
+                // the accumulator still belongs to the previous unit until its rows were read out
+                if (!mbar_wait(bar(BAR_O_FREE + i), (units_before - 1) & 1, abort_flag, p.status)) return false;
+            }
+            tc_fence_after();
+            issue_pv_half(i, stage, 0, !first);
+            if (!mbar_wait(bar(BAR_P_READY2 + i), tile & 1, abort_flag, p.status)) return false;
+            tc_fence_after();
+            issue_pv_half(i, stage, 1, !first);
+            return true;
+        };
         for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
             const UnitInfo u = unit_info(p, w, lane);
             if (u.ntiles == 0) continue;
-            const bool active = i == 0 || u.two;
             if (lane == 0) {
-                if (active) {
-                    ok = mbar_wait(bar(BAR_Q_FULL), au & 1, abort_flag, p.status);
-                    tc_fence_after();
-                }
-                for (int idx = 0; idx < u.ntiles && ok; ++idx, ++kvc) {
+                const bool two = u.two;
+                const int ntiles = u.ntiles;
+                ok = mbar_wait(bar(BAR_Q_FULL), au & 1, abort_flag, p.status);
+                tc_fence_after();
+                for (int idx = 0; idx < ntiles && ok; ++idx) {
                     const int st = kvc % KST;
-                    if (!active) continue;
                     ok = mbar_wait(bar(BAR_K_FULL + st), (kvc / KST) & 1, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
-                    {
-                        // S_i = Q_i K^T : 8 k-steps of 16 over the head dimension
-                        const uint32_t qa = sQ + i * TILE_BYTES, ka = sK + st * TILE_BYTES;
-#pragma unroll
-                        for (int ks = 0; ks < HD / 16; ++ks) {
-                            const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
-                            tc_mma_ss(tSi, desc_kmajor(qa + off), desc_kmajor(ka + off), kIdescQK, ks > 0);
+                    issue_qk(0, st);
+                    tc_commit(bar(BAR_S_FULL + 0));
+                    if (two) {
+                        if (idx > 0) {
+                            ok = issue_pv(1, (kvc - 1) % VST, tc1 + idx - 1, idx == 1, au1);
+                            if (!ok) break;
+                            tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
                         }
+                        issue_qk(1, st);
+                        tc_commit(bar(BAR_S_FULL + 1));
                     }
-                    tc_commit(bar(BAR_S_FULL + i));
                     tc_commit(bar(BAR_K_EMPTY + st));
-                    if (!u.two) tc_commit(bar(BAR_K_EMPTY + st));       // stands in for the absent row tile
-                    if (idx == u.ntiles - 1) {                           // every QK^T of the unit is issued
-                        tc_commit(bar(BAR_Q_EMPTY));
-                        if (!u.two) tc_commit(bar(BAR_Q_EMPTY));
-                    }
+                    if (idx == ntiles - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
                     ok = mbar_wait(bar(BAR_V_FULL + st), (kvc / VST) & 1, abort_flag, p.status);
                     if (!ok) break;
-                    // O_i += P_i V : 8 k-steps of 16 keys; P (bf16 pairs) sits in S_i's first 64
-                    // columns and arrives in two halves of 64 keys, so the first four k-steps run
-                    // while the second half of the exponentials is still being computed
-                    const uint32_t par = (uint32_t)((tcnt + idx) & 1);
-                    const uint32_t va = sV + st * TILE_BYTES;
-                    ok = mbar_wait(bar(BAR_P_READY + i), par, abort_flag, p.status);
+                    ok = issue_pv(0, st, tc0 + idx, idx == 0, au);
                     if (!ok) break;
-                    if (idx == 0 && auc > 0) {
-                        // the accumulator belongs to the previous unit until its rows were read out
-                        ok = mbar_wait(bar(BAR_O_FREE + i), (auc - 1) & 1, abort_flag, p.status);
-                        if (!ok) break;
+                    if (!two) tc_commit(bar(BAR_V_EMPTY + st));
+                    if (idx == ntiles - 1) tc_commit(bar(BAR_O_DONE + 0));
+                    ++kvc;
+                }
+                if (ok && two) {
+                    ok = issue_pv(1, (kvc - 1) % VST, tc1 + ntiles - 1, ntiles == 1, au1);
+                    if (ok) {
+                        tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
+                        tc_commit(bar(BAR_O_DONE + 1));
                     }
-                    tc_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < BN / 32; ++ks)
-                        tc_mma_ts(tOi, tSi + ks * 8, desc_mnmajor(va + ks * 2048), kIdescPV, (idx > 0 || ks > 0) ? 1u : 0u);
-                    ok = mbar_wait(bar(BAR_P_READY2 + i), par, abort_flag, p.status);
-                    if (!ok) break;
-                    tc_fence_after();
-#pragma unroll
-                    for (int ks = BN / 32; ks < BN / 16; ++ks)
-                        tc_mma_ts(tOi, tSi + ks * 8, desc_mnmajor(va + ks * 2048), kIdescPV, 1u);
-                    tc_commit(bar(BAR_V_EMPTY + st));
-                    if (!u.two) tc_commit(bar(BAR_V_EMPTY + st));
-                    if (idx == u.ntiles - 1) tc_commit(bar(BAR_O_DONE + i));
                 }
             }
             ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
             kvc = __shfl_sync(0xFFFFFFFFu, kvc, 0);
+            tc0 += u.ntiles;
             ++au;
-            if (active) { tcnt += u.ntiles; ++auc; }
+            if (u.two) { tc1 += u.ntiles; ++au1; }
         }
     }
     } else {
@@ -712,7 +722,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     // ---------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
-    if (warp == 11) {
+    if (warp == 10) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
     }
