@@ -16,6 +16,7 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kNone = 0x7FFFFFFF;
 constexpr int kNodeSlots = (GSD_MAX_NODES + kThreads - 1) / kThreads;
+constexpr int kEdgeCache = 3 * GSD_MAX_NODES;   // parent edges of one sequence kept in shared memory
 
 struct Best {
     float v;
@@ -98,6 +99,7 @@ __device__ void path_pass(const AcceptArgs& a, int b) {
     __shared__ int s_red[kThreads / 32];
     __shared__ unsigned s_flags;
     __shared__ int s_m;
+    __shared__ int s_edge[kEdgeCache];
     const int N = a.N, tid = threadIdx.x;
     const int32_t* tok = a.tok + (size_t)b * N;
     const int32_t* pptr = a.pptr + (size_t)b * (N + 1);
@@ -121,6 +123,13 @@ __device__ void path_pass(const AcceptArgs& a, int b) {
         s_ptr[v] = e;
     }
     __syncthreads();
+    // the relaxation rounds walk the parent lists again and again: keep them on chip
+    const int n_edges = s_ptr[N];
+    const bool cached = n_edges <= kEdgeCache;
+    if (cached) {
+        for (int e = tid; e < n_edges; e += kThreads) s_edge[e] = pidx[e];
+        __syncthreads();
+    }
 
     // level-synchronous relaxation: after round r every node whose longest accepted root
     // path has <= r edges is final; values only grow, so it stops when nothing changed
@@ -135,7 +144,7 @@ __device__ void path_pass(const AcceptArgs& a, int b) {
                 int cur = s_best[v];
                 const int t = s_tok[v];
                 for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
-                    const int p = pidx[e];
+                    const int p = cached ? s_edge[e] : pidx[e];
                     if (p < 0 || p >= v) {
                         flags |= GSD_DEV_BAD_CSR;
                         continue;
@@ -182,7 +191,7 @@ __device__ void path_pass(const AcceptArgs& a, int b) {
             if (len - 1 < a.Tcap) out_tok[len - 1] = s_tok[v];
             int pred = kNone;
             for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
-                const int p = pidx[e];
+                const int p = cached ? s_edge[e] : pidx[e];
                 if (p < 0 || p >= v) continue;
                 if (s_best[p] == len - 1 && s_tok[v] == s_amax[p] && p < pred) pred = p;
             }
