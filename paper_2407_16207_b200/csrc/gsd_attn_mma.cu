@@ -368,25 +368,42 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(MergeParams p) {
     const int row = (item % p.plan.tiles_per_unit) * p.rows_per_item + rloc;
     if (row >= p.R) return;
     const int b = unit / p.Hkv, c = unit % p.Hkv;
+    // Loads are issued in groups of four before any of them is used, so that a row costs a few
+    // memory round trips instead of two per split.
+    const float* ml_base = p.part_ml + ((size_t)slot0 * p.rows_per_item + rloc) * 2;
+    const size_t ml_stride = (size_t)p.rows_per_item * 2;
     float m = -CUDART_INF_F;
-    for (int s = 0; s < nsplit; ++s)
-        m = fmaxf(m, p.part_ml[((size_t)(slot0 + s) * p.rows_per_item + rloc) * 2]);
+    for (int s0 = 0; s0 < nsplit; s0 += 4) {
+        float mv[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) mv[j] = s0 + j < nsplit ? ml_base[(size_t)(s0 + j) * ml_stride] : -CUDART_INF_F;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) m = fmaxf(m, mv[j]);
+    }
     const float m_use = m == -CUDART_INF_F ? 0.f : m;
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     float l = 0.f;
     const int per_lane = p.D / 32;  // 2 or 4 consecutive floats per lane
-    for (int s = 0; s < nsplit; ++s) {
-        const size_t prow = (size_t)(slot0 + s) * p.rows_per_item + rloc;
-        const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + prow * 2);
-        const float wgt = exp2f(ml.x - m_use);
-        l += wgt * ml.y;
-        const float* src = p.part_o + prow * p.D + lane * per_lane;
-        if (per_lane == 4) {
-            const float4 v = *reinterpret_cast<const float4*>(src);
-            acc[0] += wgt * v.x; acc[1] += wgt * v.y; acc[2] += wgt * v.z; acc[3] += wgt * v.w;
-        } else {
-            const float2 v = *reinterpret_cast<const float2*>(src);
-            acc[0] += wgt * v.x; acc[1] += wgt * v.y;
+    const float* o_base = p.part_o + ((size_t)slot0 * p.rows_per_item + rloc) * p.D + lane * per_lane;
+    const size_t o_stride = (size_t)p.rows_per_item * p.D;
+    for (int s0 = 0; s0 < nsplit; s0 += 4) {
+        float2 ml[4];
+        float4 v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const bool in = s0 + j < nsplit;
+            ml[j] = in ? *reinterpret_cast<const float2*>(ml_base + (size_t)(s0 + j) * ml_stride)
+                       : make_float2(-CUDART_INF_F, 0.f);
+            const float* src = o_base + (size_t)(s0 + j) * o_stride;
+            if (!in) v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            else if (per_lane == 4) v[j] = *reinterpret_cast<const float4*>(src);
+            else { const float2 t = *reinterpret_cast<const float2*>(src); v[j] = make_float4(t.x, t.y, 0.f, 0.f); }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float wgt = exp2f(ml[j].x - m_use);     // 0 for an absent or empty split
+            l += wgt * ml[j].y;
+            acc[0] += wgt * v[j].x; acc[1] += wgt * v[j].y; acc[2] += wgt * v[j].z; acc[3] += wgt * v[j].w;
         }
     }
     const float inv = l > 0.f ? 1.f / l : 0.f;
