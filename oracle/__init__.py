@@ -46,7 +46,8 @@ def _load() -> ctypes.CDLL:
         _lib = ctypes.CDLL(build())
         _lib.gsd_oracle_threads.restype = ctypes.c_int
         _lib.gsd_oracle_argmax_row.restype = ctypes.c_int32
-        for name in ("gsd_oracle_attn", "gsd_oracle_attn_rows", "gsd_oracle_accept"):
+        for name in ("gsd_oracle_attn", "gsd_oracle_attn_rows", "gsd_oracle_accept",
+                     "gsd_oracle_commit_kv"):
             getattr(_lib, name).restype = ctypes.c_int
         _lib.gsd_oracle_argmax.restype = None
     return _lib
@@ -138,3 +139,21 @@ def accept(logits, draft_tokens, parent_ptr, parent_idx, Tcap: int = 0, visit_ca
     if rc != 0:
         raise ValueError("oracle accept: malformed DAG or Tcap too small")
     return toks, lens, nodes, visited
+
+
+def commit_kv(k_cache, v_cache, draft_k, draft_v, accepted_nodes, accepted_len, seq_lens):
+    """Append the draft K/V rows of the accepted path to the cache (copies of the inputs are
+    modified and returned).  Returns (k_cache, v_cache, seq_lens, number of sequences that hit Lmax)."""
+    k_cache = _c(k_cache, np.uint16).copy(); v_cache = _c(v_cache, np.uint16).copy()
+    draft_k = _c(draft_k, np.uint16); draft_v = _c(draft_v, np.uint16)
+    accepted_nodes = _c(accepted_nodes, np.int32); accepted_len = _c(accepted_len, np.int32)
+    seq_lens = _c(seq_lens, np.int32).copy()
+    B, Lmax, Hkv, D = k_cache.shape
+    N = draft_k.shape[1]
+    Tcap = accepted_nodes.shape[1]
+    assert draft_k.shape == (B, N, Hkv, D) and v_cache.shape == k_cache.shape
+    rc = _load().gsd_oracle_commit_kv(_p(k_cache), _p(v_cache), _p(draft_k), _p(draft_v),
+                                      _p(accepted_nodes), _p(accepted_len), _p(seq_lens),
+                                      ctypes.c_int32(B), ctypes.c_int32(N), ctypes.c_int32(Hkv),
+                                      ctypes.c_int32(D), ctypes.c_int32(Lmax), ctypes.c_int32(Tcap))
+    return k_cache, v_cache, seq_lens, int(rc)

@@ -320,3 +320,38 @@ int gsd_oracle_accept(const float *logits, const int32_t *draft_tokens, const in
     }
     return 0;
 }
+
+/*
+ * KV-cache commit of the accepted path (the cache update that follows verification; the paper
+ * counts it under "Others" in its time breakdown, Sec. 7.1 / Table 3, and names KV caching in
+ * Sec. 4.2).  The accepted path v0=0, v1..vm of sequence b (accepted_nodes[b][0..len), len =
+ * accepted_len[b] = m + 1) becomes part of the committed context: the draft K/V rows of those
+ * nodes are appended to the cache at positions seq_lens[b] .. seq_lens[b] + len - 1 and
+ * seq_lens[b] grows by len.  Rows that would fall past Lmax are dropped and the length is
+ * clamped (returns the number of sequences that overflowed).  Everything else is untouched.
+ *
+ * k_cache/v_cache [B,Lmax,Hkv,D] (in/out), draft_k/draft_v [B,N,Hkv,D], accepted_nodes [B,Tcap],
+ * accepted_len [B], seq_lens [B] (in/out); elements are 2-byte bf16 patterns, copied as they are.
+ */
+int gsd_oracle_commit_kv(uint16_t *k_cache, uint16_t *v_cache, const uint16_t *draft_k,
+                         const uint16_t *draft_v, const int32_t *accepted_nodes,
+                         const int32_t *accepted_len, int32_t *seq_lens, int32_t B, int32_t N,
+                         int32_t Hkv, int32_t D, int32_t Lmax, int32_t Tcap)
+{
+    int overflowed = 0;
+    const size_t row = (size_t)Hkv * D;
+    for (int b = 0; b < B; ++b) {
+        const int len = accepted_len[b];
+        int pos = seq_lens[b];
+        for (int i = 0; i < len && i < Tcap; ++i) {
+            const int node = accepted_nodes[(size_t)b * Tcap + i];
+            if (node < 0 || node >= N) continue;
+            if (pos >= Lmax) { overflowed++; break; }
+            memcpy(k_cache + ((size_t)b * Lmax + pos) * row, draft_k + ((size_t)b * N + node) * row, row * 2);
+            memcpy(v_cache + ((size_t)b * Lmax + pos) * row, draft_v + ((size_t)b * N + node) * row, row * 2);
+            ++pos;
+        }
+        seq_lens[b] = pos;
+    }
+    return overflowed;
+}
