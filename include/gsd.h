@@ -55,6 +55,7 @@ typedef enum gsd_status {
 #define GSD_DEV_TCAP         0x4u  /* accepted_len exceeded Tcap; the token list was truncated */
 #define GSD_DEV_WAIT_EXPIRED 0x8u  /* a bounded in-kernel wait gave up; the output is not valid */
 #define GSD_DEV_BAD_SEQ_LEN  0x10u /* seq_lens[b] outside [0, Lmax]; it was clamped */
+#define GSD_DEV_CACHE_FULL   0x20u /* gsd_commit_kv: the accepted rows did not all fit below Lmax; the rest was dropped */
 
 #define GSD_MAX_NODES 512          /* largest supported N (draft nodes per sequence) */
 
@@ -197,6 +198,40 @@ int gsd_accept_static(const float* logits, const int32_t* draft_tokens, const in
                       const int32_t* parent_idx, int32_t* accepted_tokens, int32_t* accepted_len,
                       int32_t* accepted_nodes, const gsd_accept_params* p, int32_t* status,
                       void* stream);
+
+typedef struct gsd_commit_params {
+    int32_t B;     /* sequences */
+    int32_t N;     /* draft nodes per sequence */
+    int32_t Hkv;   /* key/value heads */
+    int32_t D;     /* head dimension, a multiple of 8 */
+    int32_t Lmax;  /* rows per sequence in k_cache / v_cache */
+    int32_t Tcap;  /* row length of accepted_nodes */
+} gsd_commit_params;
+
+/*
+ * gsd_commit_kv - make the accepted path part of the committed context: the KV-cache update
+ * that follows verification (the paper counts the cache update under "Others" in its time
+ * breakdown, Sec. 7.1 / Table 3; KV caching, Sec. 4.2).
+ *
+ * For every sequence b, with len = min(accepted_len[b], Tcap) and the path nodes
+ * accepted_nodes[b][0..len) (node 0, the root whose K/V were not yet cached, then the accepted
+ * draft nodes), the draft_k / draft_v rows of those nodes are copied to cache positions
+ * seq_lens[b], seq_lens[b]+1, ... and seq_lens[b] is advanced by the number of rows written.
+ * Rows that would land at or past Lmax are dropped (GSD_DEV_CACHE_FULL); node ids outside
+ * [0, N) are skipped (GSD_DEV_BAD_CSR).  Nothing else in the cache is touched.
+ *
+ *   k_cache, v_cache  [B, Lmax, Hkv, D] bf16 device in/out
+ *   draft_k, draft_v  [B, N, Hkv, D]    bf16 device in
+ *   accepted_nodes    [B, Tcap] int32 device in   (as written by gsd_accept)
+ *   accepted_len      [B]       int32 device in
+ *   seq_lens          [B]       int32 device in/out
+ *   status            device int32 word or NULL;  stream: cudaStream_t
+ *
+ * Tensor bases 16-byte aligned.  No workspace, no allocation, asynchronous on `stream`.
+ */
+int gsd_commit_kv(void* k_cache, void* v_cache, const void* draft_k, const void* draft_v,
+                  const int32_t* accepted_nodes, const int32_t* accepted_len, int32_t* seq_lens,
+                  const gsd_commit_params* p, int32_t* status, void* stream);
 
 /*
  * gsd_verify_step_host - one whole verification step from HOST buffers: copies every

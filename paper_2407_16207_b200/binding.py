@@ -34,6 +34,11 @@ class AttnParams(ctypes.Structure):
                 ("kernel", ctypes.c_int32)]
 
 
+class CommitParams(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("N", ctypes.c_int32), ("Hkv", ctypes.c_int32),
+                ("D", ctypes.c_int32), ("Lmax", ctypes.c_int32), ("Tcap", ctypes.c_int32)]
+
+
 class AcceptParams(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("N", ctypes.c_int32), ("V", ctypes.c_int32),
                 ("Ecap", ctypes.c_int32), ("Tcap", ctypes.c_int32)]
@@ -41,7 +46,7 @@ class AcceptParams(ctypes.Structure):
 
 EXPORTS = ["gsd_version", "gsd_status_string", "gsd_last_cuda_error", "gsd_verify_attn",
            "gsd_verify_attn_workspace_bytes", "gsd_verify_attn_num_splits", "gsd_accept",
-           "gsd_accept_workspace_bytes", "gsd_accept_static", "gsd_verify_step_host",
+           "gsd_accept_workspace_bytes", "gsd_accept_static", "gsd_commit_kv", "gsd_verify_step_host",
            "gsd_verify_step_host_arena_bytes"]
 
 
@@ -72,6 +77,8 @@ def lib() -> ctypes.CDLL:
         L.gsd_accept.argtypes = [vp] * 7 + [ctypes.POINTER(AcceptParams), vp, sz, vp, vp]
         L.gsd_accept_static.restype = i32
         L.gsd_accept_static.argtypes = [vp] * 7 + [ctypes.POINTER(AcceptParams), vp, vp]
+        L.gsd_commit_kv.restype = i32
+        L.gsd_commit_kv.argtypes = [vp] * 7 + [ctypes.POINTER(CommitParams), vp, vp]
         L.gsd_accept_workspace_bytes.restype = sz
         L.gsd_accept_workspace_bytes.argtypes = [ctypes.POINTER(AcceptParams)]
         L.gsd_verify_step_host.restype = i32
@@ -214,6 +221,29 @@ def gsd_accept(logits, draft_tokens, parent_ptr, parent_idx, *, Tcap: int = 0,
                             workspace.numel() * workspace.element_size(), _ptr(status),
                             _stream(logits)))
     return toks, lens, nodes
+
+
+def gsd_commit_kv(k_cache, v_cache, draft_k, draft_v, accepted_nodes, accepted_len, seq_lens, *,
+                  status: Optional[torch.Tensor] = None) -> None:
+    """Append the draft K/V rows of the accepted path to the cache in place and advance
+    seq_lens; see gsd_commit_kv in include/gsd.h.  Enqueued on the current stream."""
+    B, Lmax, Hkv, D = k_cache.shape
+    N = draft_k.shape[1]
+    Tcap = accepted_nodes.shape[1]
+    bf = torch.bfloat16
+    _want(k_cache, bf, (B, Lmax, Hkv, D), "k_cache", True)
+    _want(v_cache, bf, (B, Lmax, Hkv, D), "v_cache", True)
+    _want(draft_k, bf, (B, N, Hkv, D), "draft_k", True)
+    _want(draft_v, bf, (B, N, Hkv, D), "draft_v", True)
+    _want(accepted_nodes, torch.int32, (B, Tcap), "accepted_nodes", True)
+    _want(accepted_len, torch.int32, (B,), "accepted_len", True)
+    _want(seq_lens, torch.int32, (B,), "seq_lens", True)
+    p = CommitParams(B, N, Hkv, D, Lmax, Tcap)
+    with torch.cuda.device(k_cache.device):
+        _check(lib().gsd_commit_kv(k_cache.data_ptr(), v_cache.data_ptr(), draft_k.data_ptr(),
+                                   draft_v.data_ptr(), accepted_nodes.data_ptr(),
+                                   accepted_len.data_ptr(), seq_lens.data_ptr(), ctypes.byref(p),
+                                   _ptr(status), _stream(k_cache)))
 
 
 GSD_STATIC_MAX_ROWS = 16384
