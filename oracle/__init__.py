@@ -47,7 +47,7 @@ def _load() -> ctypes.CDLL:
         _lib.gsd_oracle_threads.restype = ctypes.c_int
         _lib.gsd_oracle_argmax_row.restype = ctypes.c_int32
         for name in ("gsd_oracle_attn", "gsd_oracle_attn_rows", "gsd_oracle_accept",
-                     "gsd_oracle_commit_kv"):
+                     "gsd_oracle_commit_kv", "gsd_oracle_build_mask"):
             getattr(_lib, name).restype = ctypes.c_int
         _lib.gsd_oracle_argmax.restype = None
     return _lib
@@ -157,3 +157,16 @@ def commit_kv(k_cache, v_cache, draft_k, draft_v, accepted_nodes, accepted_len, 
                                       ctypes.c_int32(B), ctypes.c_int32(N), ctypes.c_int32(Hkv),
                                       ctypes.c_int32(D), ctypes.c_int32(Lmax), ctypes.c_int32(Tcap))
     return k_cache, v_cache, seq_lens, int(rc)
+
+
+def build_mask(parent_ptr, parent_idx) -> np.ndarray:
+    """Ancestor bitmask [B,N,ceil(N/32)] uint32 (self bit included) from the parent CSR."""
+    parent_ptr = _c(parent_ptr, np.int32); parent_idx = _c(parent_idx, np.int32)
+    B, N1 = parent_ptr.shape
+    N = N1 - 1
+    mask = np.zeros((B, N, (N + 31) // 32), dtype=np.uint32)
+    rc = _load().gsd_oracle_build_mask(_p(parent_ptr), _p(parent_idx), ctypes.c_int32(B),
+                                       ctypes.c_int32(N), ctypes.c_int32(parent_idx.shape[1]), _p(mask))
+    if rc != 0:
+        raise RuntimeError("oracle build_mask failed")
+    return mask

@@ -355,3 +355,46 @@ int gsd_oracle_commit_kv(uint16_t *k_cache, uint16_t *v_cache, const uint16_t *d
     }
     return overflowed;
 }
+
+/*
+ * Ancestor bitmask of a draft DAG from its parent lists (what "each token may only attend to
+ * its ancestor nodes" of tree attention, Sec. 4.1, means for the merged token graph of
+ * Sec. 5.3: a node sees itself and every node from which it can be reached).  For each node
+ * the ancestors are collected by an explicit upward search over the parent lists with a
+ * visited array (no reuse of other rows).  mask [B,N,W] uint32, W = ceil(N/32); bit j of row n
+ * (word j / 32, bit j % 32) set iff j == n or j is an ancestor of n.  Parent indices outside
+ * [0, n) are ignored.  Returns -1 on allocation failure.
+ */
+int gsd_oracle_build_mask(const int32_t *parent_ptr, const int32_t *parent_idx, int32_t B, int32_t N,
+                          int32_t Ecap, uint32_t *mask)
+{
+    const int W = (N + 31) / 32;
+    unsigned char *seen = (unsigned char *)malloc((size_t)N);
+    int *todo = (int *)malloc(sizeof(int) * (size_t)N);
+    if (!seen || !todo) { free(seen); free(todo); return -1; }
+    for (int b = 0; b < B; ++b) {
+        const int32_t *pp = parent_ptr + (size_t)b * (N + 1);
+        const int32_t *pi = parent_idx + (size_t)b * Ecap;
+        for (int n = 0; n < N; ++n) {
+            uint32_t *row = mask + ((size_t)b * N + n) * W;
+            memset(row, 0, sizeof(uint32_t) * (size_t)W);
+            memset(seen, 0, (size_t)N);
+            int top = 0;
+            seen[n] = 1;
+            todo[top++] = n;
+            while (top > 0) {
+                const int v = todo[--top];
+                row[v / 32] |= 1u << (v % 32);
+                for (int e = pp[v]; e < pp[v + 1]; ++e) {
+                    const int p = pi[e];
+                    if (p < 0 || p >= v || seen[p]) continue;
+                    seen[p] = 1;
+                    todo[top++] = p;
+                }
+            }
+        }
+    }
+    free(seen);
+    free(todo);
+    return 0;
+}
