@@ -199,6 +199,26 @@ int gsd_accept_static(const float* logits, const int32_t* draft_tokens, const in
                       int32_t* accepted_nodes, const gsd_accept_params* p, int32_t* status,
                       void* stream);
 
+/*
+ * gsd_build_mask - the ancestor bitmask that gsd_verify_attn takes, built on the device from
+ * the parent lists (tree attention lets a token attend only to its ancestors, Sec. 4.1; in
+ * the merged token graph of Sec. 5.3 a node has several parents and sees the union of their
+ * ancestors).
+ *
+ *   ancestor_mask[b][n] has bit j (word j / 32, bit j % 32) set iff j == n or node n can be
+ *   reached from node j along parent edges; bits >= N are zero.
+ *
+ *   parent_ptr     [B, N+1] int32 device in   (CSR row pointers, local to the sequence)
+ *   parent_idx     [B, Ecap] int32 device in  (every parent index must be < its child)
+ *   ancestor_mask  [B, N, ceil(N/32)] uint32 device out
+ *   status         device int32 word or NULL (GSD_DEV_BAD_CSR: an edge or row pointer was ignored)
+ *   stream         cudaStream_t
+ *
+ * N <= GSD_MAX_NODES.  No workspace, no allocation, asynchronous on `stream`.
+ */
+int gsd_build_mask(const int32_t* parent_ptr, const int32_t* parent_idx, uint32_t* ancestor_mask,
+                   int32_t B, int32_t N, int32_t Ecap, int32_t* status, void* stream);
+
 typedef struct gsd_commit_params {
     int32_t B;     /* sequences */
     int32_t N;     /* draft nodes per sequence */

@@ -46,7 +46,7 @@ class AcceptParams(ctypes.Structure):
 
 EXPORTS = ["gsd_version", "gsd_status_string", "gsd_last_cuda_error", "gsd_verify_attn",
            "gsd_verify_attn_workspace_bytes", "gsd_verify_attn_num_splits", "gsd_accept",
-           "gsd_accept_workspace_bytes", "gsd_accept_static", "gsd_commit_kv", "gsd_verify_step_host",
+           "gsd_accept_workspace_bytes", "gsd_accept_static", "gsd_commit_kv", "gsd_build_mask", "gsd_verify_step_host",
            "gsd_verify_step_host_arena_bytes"]
 
 
@@ -77,6 +77,8 @@ def lib() -> ctypes.CDLL:
         L.gsd_accept.argtypes = [vp] * 7 + [ctypes.POINTER(AcceptParams), vp, sz, vp, vp]
         L.gsd_accept_static.restype = i32
         L.gsd_accept_static.argtypes = [vp] * 7 + [ctypes.POINTER(AcceptParams), vp, vp]
+        L.gsd_build_mask.restype = i32
+        L.gsd_build_mask.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp]
         L.gsd_commit_kv.restype = i32
         L.gsd_commit_kv.argtypes = [vp] * 7 + [ctypes.POINTER(CommitParams), vp, vp]
         L.gsd_accept_workspace_bytes.restype = sz
@@ -221,6 +223,24 @@ def gsd_accept(logits, draft_tokens, parent_ptr, parent_idx, *, Tcap: int = 0,
                             workspace.numel() * workspace.element_size(), _ptr(status),
                             _stream(logits)))
     return toks, lens, nodes
+
+
+def gsd_build_mask(parent_ptr, parent_idx, out: Optional[torch.Tensor] = None, *,
+                   status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Ancestor bitmask [B,N,ceil(N/32)] (int32 words) from the parent CSR; see gsd_build_mask in
+    include/gsd.h.  Enqueued on the current stream."""
+    B, N1 = parent_ptr.shape
+    N = N1 - 1
+    Ecap = parent_idx.shape[1]
+    _want(parent_ptr, torch.int32, (B, N + 1), "parent_ptr", True)
+    _want(parent_idx, torch.int32, (B, Ecap), "parent_idx", True)
+    if out is None:
+        out = torch.empty((B, N, (N + 31) // 32), dtype=torch.int32, device=parent_ptr.device)
+    _want(out, out.dtype, (B, N, (N + 31) // 32), "ancestor_mask", True)
+    with torch.cuda.device(parent_ptr.device):
+        _check(lib().gsd_build_mask(parent_ptr.data_ptr(), parent_idx.data_ptr(), out.data_ptr(),
+                                    B, N, Ecap, _ptr(status), _stream(parent_ptr)))
+    return out
 
 
 def gsd_commit_kv(k_cache, v_cache, draft_k, draft_v, accepted_nodes, accepted_len, seq_lens, *,
