@@ -439,55 +439,39 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         int au = 0, au1 = 0;      // non-empty units so far; those of them with a second row tile
         int tc0 = 0, tc1 = 0;     // key tiles handed to the softmax of row tile 0 / 1 so far
         bool ok = true;
-        // O_i += P_i V : 8 k-steps of 16 keys; P (bf16 pairs) sits in S_i's first 64 columns and
-        // arrives in two halves of 64 keys, so the first four k-steps can run while the second half
-        // of the exponentials is still being computed.
-        auto pv_instr = [&](int i, int stage, int ks, bool accumulate) {
-            tc_mma_ts(tmem + (i ? COL_O1 : COL_O0), tmem + (i ? COL_S1 : COL_S0) + ks * 8,
-                      desc_mnmajor(sV + stage * TILE_BYTES + ks * 2048), kIdescPV, (accumulate || ks > 0) ? 1u : 0u);
-        };
-        // QK^T of row tile i and, as far as P of the other row tile j has already arrived, the
-        // PV of j interleaved with it instruction by instruction: the two groups write different
-        // accumulators, and alternating independent MMAs hides part of the latency of the
-        // dependent accumulate steps.  Returns the number of PV instructions that went out.
-        auto issue_qk_with_pv = [&](int i, int stage, int j, int vstage, int tile, bool first, bool allow) -> int {
+        auto issue_qk = [&](int i, int stage) {
+            // S_i = Q_i K^T : 8 k-steps of 16 over the head dimension
             const uint32_t qa = sQ + i * TILE_BYTES, ka = sK + stage * TILE_BYTES;
-            int done = 0;
-            bool p1 = false, p2 = false;
 #pragma unroll
             for (int ks = 0; ks < HD / 16; ++ks) {
                 const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
                 tc_mma_ss(tmem + (i ? COL_S1 : COL_S0), desc_kmajor(qa + off), desc_kmajor(ka + off), kIdescQK, ks > 0);
-                if (allow) {
-                    if (done < BN / 32) {
-                        if (!p1 && mbar_try_wait(bar(BAR_P_READY + j), tile & 1)) { p1 = true; tc_fence_after(); }
-                        if (p1) pv_instr(j, vstage, done++, !first);
-                    } else if (done < BN / 16) {
-                        if (!p2 && mbar_try_wait(bar(BAR_P_READY2 + j), tile & 1)) { p2 = true; tc_fence_after(); }
-                        if (p2) pv_instr(j, vstage, done++, !first);
-                    }
-                }
             }
-            return done;
         };
-        // the rest of PV_i from instruction `from` on, waiting for the halves of P as needed.
+        // O_i += P_i V : 8 k-steps of 16 keys; P (bf16 pairs) sits in S_i's first 64 columns.
+        // The softmax hands P over in two halves of 64 keys, so the first four k-steps run
+        // while the second half of the exponentials is still being computed.
+        auto issue_pv_half = [&](int i, int stage, int half, bool accumulate) {
+            const uint32_t va = sV + stage * TILE_BYTES;
+#pragma unroll
+            for (int k4 = 0; k4 < BN / 32; ++k4) {
+                const int ks = half * (BN / 32) + k4;
+                tc_mma_ts(tmem + (i ? COL_O1 : COL_O0), tmem + (i ? COL_S1 : COL_S0) + ks * 8,
+                          desc_mnmajor(va + ks * 2048), kIdescPV, (accumulate || ks > 0) ? 1u : 0u);
+            }
+        };
         // tile = running tile number of row tile i (barrier phase); first = first tile of the unit
-        auto issue_pv = [&](int i, int stage, int tile, bool first, int units_before, int from) -> bool {
-            if (from < BN / 32) {
-                if (!mbar_wait(bar(BAR_P_READY + i), tile & 1, abort_flag, p.status)) return false;
-                if (first && units_before > 0) {
-                    // the accumulator still belongs to the previous unit until its rows were read out
-                    if (!mbar_wait(bar(BAR_O_FREE + i), (units_before - 1) & 1, abort_flag, p.status)) return false;
-                }
-                tc_fence_after();
-                for (int ks = from; ks < BN / 32; ++ks) pv_instr(i, stage, ks, !first);
-                from = BN / 32;
+        auto issue_pv = [&](int i, int stage, int tile, bool first, int units_before) -> bool {
+            if (!mbar_wait(bar(BAR_P_READY + i), tile & 1, abort_flag, p.status)) return false;
+            if (first && units_before > 0) {
+                // the accumulator still belongs to the previous unit until its rows were read out
+                if (!mbar_wait(bar(BAR_O_FREE + i), (units_before - 1) & 1, abort_flag, p.status)) return false;
             }
-            if (from < BN / 16) {
-                if (!mbar_wait(bar(BAR_P_READY2 + i), tile & 1, abort_flag, p.status)) return false;
-                tc_fence_after();
-                for (int ks = from; ks < BN / 16; ++ks) pv_instr(i, stage, ks, !first);
-            }
+            tc_fence_after();
+            issue_pv_half(i, stage, 0, !first);
+            if (!mbar_wait(bar(BAR_P_READY2 + i), tile & 1, abort_flag, p.status)) return false;
+            tc_fence_after();
+            issue_pv_half(i, stage, 1, !first);
             return true;
         };
         for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
@@ -498,44 +482,34 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const int ntiles = u.ntiles;
                 ok = mbar_wait(bar(BAR_Q_FULL), au & 1, abort_flag, p.status);
                 tc_fence_after();
-                int pv0_done = 0;   // PV0 instructions of the current tile already interleaved
                 for (int idx = 0; idx < ntiles && ok; ++idx) {
                     const int st = kvc % KST;
                     ok = mbar_wait(bar(BAR_K_FULL + st), (kvc / KST) & 1, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
-                    // QK0(idx), with PV1(idx-1) woven in as far as its P is there
-                    const bool have_pv1 = two && idx > 0;
-                    const bool first1 = idx == 1;
-                    const int pv1_done = issue_qk_with_pv(0, st, 1, (kvc - 1) % VST, tc1 + idx - 1, first1,
-                                                          have_pv1 && !(first1 && au1 > 0));
+                    issue_qk(0, st);
                     tc_commit(bar(BAR_S_FULL + 0));
                     if (two) {
                         if (idx > 0) {
-                            ok = issue_pv(1, (kvc - 1) % VST, tc1 + idx - 1, first1, au1, pv1_done);
+                            ok = issue_pv(1, (kvc - 1) % VST, tc1 + idx - 1, idx == 1, au1);
                             if (!ok) break;
                             tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
                         }
-                        // QK1(idx), with PV0(idx) woven in (needs this tile's V)
-                        const bool first0 = idx == 0;
-                        const bool v_ready = mbar_try_wait(bar(BAR_V_FULL + st), (kvc / VST) & 1);
-                        pv0_done = issue_qk_with_pv(1, st, 0, st, tc0 + idx, first0, v_ready && !(first0 && au > 0));
+                        issue_qk(1, st);
                         tc_commit(bar(BAR_S_FULL + 1));
-                    } else {
-                        pv0_done = 0;
                     }
                     tc_commit(bar(BAR_K_EMPTY + st));
                     if (idx == ntiles - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
                     ok = mbar_wait(bar(BAR_V_FULL + st), (kvc / VST) & 1, abort_flag, p.status);
                     if (!ok) break;
-                    ok = issue_pv(0, st, tc0 + idx, idx == 0, au, pv0_done);
+                    ok = issue_pv(0, st, tc0 + idx, idx == 0, au);
                     if (!ok) break;
                     if (!two) tc_commit(bar(BAR_V_EMPTY + st));
                     if (idx == ntiles - 1) tc_commit(bar(BAR_O_DONE + 0));
                     ++kvc;
                 }
                 if (ok && two) {
-                    ok = issue_pv(1, (kvc - 1) % VST, tc1 + ntiles - 1, ntiles == 1, au1, 0);
+                    ok = issue_pv(1, (kvc - 1) % VST, tc1 + ntiles - 1, ntiles == 1, au1);
                     if (ok) {
                         tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
                         tc_commit(bar(BAR_O_DONE + 1));
