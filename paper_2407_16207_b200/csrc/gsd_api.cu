@@ -49,7 +49,7 @@ int attn_pick_kernel(const gsd_attn_params* p) {
     if (p->kernel != GSD_ATTN_AUTO) return p->kernel;
     // the TMEM kernel pays off once the stacked rows fill its 128-row tiles
     const int G = p->Hq / p->Hkv;
-    if (attn_tcgen05_supports(p->D, G) && p->N * G >= 128) return GSD_ATTN_TCGEN05;
+    if (attn_tcgen05_supports(p->D, G) && p->N * G >= 64) return GSD_ATTN_TCGEN05;
     return GSD_ATTN_MMA;
 }
 

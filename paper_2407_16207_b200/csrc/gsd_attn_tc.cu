@@ -55,7 +55,8 @@ enum Bar {
     BAR_O_DONE = BAR_P_READY2 + 2,    // 2: every PV of the unit has completed
     BAR_O_FREE = BAR_O_DONE + 2,      // 2: the accumulator rows of the unit have been read out
     BAR_Q_EMPTY = BAR_O_FREE + 2,     // 1: every QK^T of the unit has completed
-    BAR_COUNT = BAR_Q_EMPTY + 1
+    BAR_ML_READY = BAR_Q_EMPTY + 1,   // 1: (max, sum) of the odd-tile stream are in shared memory
+    BAR_COUNT = BAR_ML_READY + 1
 };
 
 struct TcParams {
@@ -339,6 +340,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     __shared__ __align__(8) unsigned long long s_bars[BAR_COUNT];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
+    __shared__ float2 s_ml1[BM];      // (max, sum) of the odd-tile stream, one per row
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int N = p.N, G = p.G, R = p.R;
@@ -355,6 +357,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         s_abort = 0;
         mbar_init(bar(BAR_Q_FULL), 1);
         mbar_init(bar(BAR_Q_EMPTY), 1);
+        mbar_init(bar(BAR_ML_READY), 4);
         for (int s = 0; s < KST; ++s) { mbar_init(bar(BAR_K_FULL + s), 1); mbar_init(bar(BAR_K_EMPTY + s), 1); }
         for (int s = 0; s < VST; ++s) { mbar_init(bar(BAR_V_FULL + s), 1); mbar_init(bar(BAR_V_EMPTY + s), 1); }
         for (int i = 0; i < 2; ++i) {
@@ -436,12 +439,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     } else if (warp == 9) {
         // ------------------------------------------------------------ MMA issuer
         int kvc = 0;              // key tiles consumed so far (ring position)
-        int au = 0, au1 = 0;      // non-empty units so far; those of them with a second row tile
-        int tc0 = 0, tc1 = 0;     // key tiles handed to the softmax of row tile 0 / 1 so far
+        int au = 0, au1 = 0;      // non-empty units so far; those of them in which stream 1 had tiles
+        int tc0 = 0, tc1 = 0;     // key tiles handed to the softmax of stream 0 / 1 so far
         bool ok = true;
-        auto issue_qk = [&](int i, int stage) {
-            // S_i = Q_i K^T : 8 k-steps of 16 over the head dimension
-            const uint32_t qa = sQ + i * TILE_BYTES, ka = sK + stage * TILE_BYTES;
+        auto issue_qk = [&](int i, int qtile, int stage) {
+            // S_i = Q_qtile K^T : 8 k-steps of 16 over the head dimension
+            const uint32_t qa = sQ + qtile * TILE_BYTES, ka = sK + stage * TILE_BYTES;
 #pragma unroll
             for (int ks = 0; ks < HD / 16; ++ks) {
                 const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
@@ -477,50 +480,101 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
             const UnitInfo u = unit_info(p, w, lane);
             if (u.ntiles == 0) continue;
+            const int n0 = u.two ? u.ntiles : (u.ntiles + 1) / 2;   // key tiles of stream 0 / stream 1
+            const int n1 = u.two ? u.ntiles : u.ntiles / 2;
             if (lane == 0) {
                 const bool two = u.two;
                 const int ntiles = u.ntiles;
                 ok = mbar_wait(bar(BAR_Q_FULL), au & 1, abort_flag, p.status);
                 tc_fence_after();
-                for (int idx = 0; idx < ntiles && ok; ++idx) {
-                    const int st = kvc % KST;
-                    ok = mbar_wait(bar(BAR_K_FULL + st), (kvc / KST) & 1, abort_flag, p.status);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_qk(0, st);
-                    tc_commit(bar(BAR_S_FULL + 0));
-                    if (two) {
-                        if (idx > 0) {
-                            ok = issue_pv(1, (kvc - 1) % VST, tc1 + idx - 1, idx == 1, au1);
-                            if (!ok) break;
-                            tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
+                if (two) {
+                    for (int idx = 0; idx < ntiles && ok; ++idx) {
+                        const int st = kvc % KST;
+                        ok = mbar_wait(bar(BAR_K_FULL + st), (kvc / KST) & 1, abort_flag, p.status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_qk(0, 0, st);
+                        tc_commit(bar(BAR_S_FULL + 0));
+                        if (two) {
+                            if (idx > 0) {
+                                ok = issue_pv(1, (kvc - 1) % VST, tc1 + idx - 1, idx == 1, au1);
+                                if (!ok) break;
+                                tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
+                            }
+                            issue_qk(1, 1, st);
+                            tc_commit(bar(BAR_S_FULL + 1));
                         }
-                        issue_qk(1, st);
-                        tc_commit(bar(BAR_S_FULL + 1));
+                        tc_commit(bar(BAR_K_EMPTY + st));
+                        if (idx == ntiles - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
+                        ok = mbar_wait(bar(BAR_V_FULL + st), (kvc / VST) & 1, abort_flag, p.status);
+                        if (!ok) break;
+                        ok = issue_pv(0, st, tc0 + idx, idx == 0, au);
+                        if (!ok) break;
+                        if (!two) tc_commit(bar(BAR_V_EMPTY + st));
+                        if (idx == ntiles - 1) tc_commit(bar(BAR_O_DONE + 0));
+                        ++kvc;
                     }
-                    tc_commit(bar(BAR_K_EMPTY + st));
-                    if (idx == ntiles - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
-                    ok = mbar_wait(bar(BAR_V_FULL + st), (kvc / VST) & 1, abort_flag, p.status);
-                    if (!ok) break;
-                    ok = issue_pv(0, st, tc0 + idx, idx == 0, au);
-                    if (!ok) break;
-                    if (!two) tc_commit(bar(BAR_V_EMPTY + st));
-                    if (idx == ntiles - 1) tc_commit(bar(BAR_O_DONE + 0));
-                    ++kvc;
-                }
-                if (ok && two) {
-                    ok = issue_pv(1, (kvc - 1) % VST, tc1 + ntiles - 1, ntiles == 1, au1);
-                    if (ok) {
-                        tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
-                        tc_commit(bar(BAR_O_DONE + 1));
+                    if (ok && two) {
+                        ok = issue_pv(1, (kvc - 1) % VST, tc1 + ntiles - 1, ntiles == 1, au1);
+                        if (ok) {
+                            tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
+                            tc_commit(bar(BAR_O_DONE + 1));
+                        }
                     }
+                } else {
+                    // One row tile only: the two accumulator pairs take the even and the odd key
+                    // tiles of the same rows (two independent partial attentions that the epilogue
+                    // merges), so the softmax of one tile still runs under the MMAs of the next.
+                    const int kv0 = kvc;
+                    int pv1_issued = 0;
+                    auto finish_pv1 = [&](int c1) -> bool {       // PV of stream 1's tile c1
+                        const int r = kv0 + 2 * c1 + 1;
+                        if (!mbar_wait(bar(BAR_V_FULL + r % VST), (r / VST) & 1, abort_flag, p.status)) return false;
+                        if (!issue_pv(1, r % VST, tc1 + c1, c1 == 0, au1)) return false;
+                        tc_commit(bar(BAR_V_EMPTY + r % VST));
+                        if (c1 == n1 - 1) tc_commit(bar(BAR_O_DONE + 1));
+                        return true;
+                    };
+                    for (int k = 0; k < n0 && ok; ++k) {
+                        const int r0 = kv0 + 2 * k, r1 = r0 + 1;
+                        const bool has1 = 2 * k + 1 < ntiles;
+                        ok = mbar_wait(bar(BAR_K_FULL + r0 % KST), (r0 / KST) & 1, abort_flag, p.status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_qk(0, 0, r0 % KST);
+                        tc_commit(bar(BAR_S_FULL + 0));
+                        tc_commit(bar(BAR_K_EMPTY + r0 % KST));
+                        if (k > 0) {
+                            ok = finish_pv1(k - 1);
+                            if (!ok) break;
+                            pv1_issued = k;
+                        }
+                        if (has1) {
+                            ok = mbar_wait(bar(BAR_K_FULL + r1 % KST), (r1 / KST) & 1, abort_flag, p.status);
+                            if (!ok) break;
+                            tc_fence_after();
+                            issue_qk(1, 0, r1 % KST);
+                            tc_commit(bar(BAR_S_FULL + 1));
+                            tc_commit(bar(BAR_K_EMPTY + r1 % KST));
+                        }
+                        if (k == n0 - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
+                        ok = mbar_wait(bar(BAR_V_FULL + r0 % VST), (r0 / VST) & 1, abort_flag, p.status);
+                        if (!ok) break;
+                        ok = issue_pv(0, r0 % VST, tc0 + k, k == 0, au);
+                        if (!ok) break;
+                        tc_commit(bar(BAR_V_EMPTY + r0 % VST));
+                        if (k == n0 - 1) tc_commit(bar(BAR_O_DONE + 0));
+                    }
+                    if (ok && pv1_issued < n1) ok = finish_pv1(n1 - 1);
+                    kvc = kv0 + ntiles;
                 }
             }
             ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
             kvc = __shfl_sync(0xFFFFFFFFu, kvc, 0);
-            tc0 += u.ntiles;
+            tc0 += n0;
+            tc1 += n1;
             ++au;
-            if (u.two) { tc1 += u.ntiles; ++au1; }
+            if (n1 > 0) ++au1;
         }
     }
     } else {
@@ -533,17 +587,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const uint32_t tO = tmem + lane_addr + (i ? COL_O1 : COL_O0);
         int kvc = 0;      // key tiles of all non-empty units so far (ring position of the V tiles)
         int tcnt = 0;     // key tiles this row tile has processed so far (barrier phase)
-        int auc = 0;      // units this row tile has finished so far
+        int auc = 0;      // non-empty units this stream has finished so far (barrier phase)
+        int auc1 = 0;     // units in which stream 1 had tiles (phase of its barriers as seen by warpgroup 0)
+        int mlc = 0;      // single-row-tile units whose odd-tile stream had tiles
         bool ok = true;
         for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
             const UnitInfo u = unit_info(p, w, lane);
-            if (i == 1 && !u.two) {
-                kvc += u.ntiles;
-                continue;
-            }
             const int ntiles = u.ntiles;
+            // with one row tile only, the two warpgroups take the even / odd key tiles of the
+            // same rows and warpgroup 0 merges the two partial results in the epilogue
+            const bool alt = !u.two;
+            const int my_n = alt ? (i == 0 ? (ntiles + 1) / 2 : ntiles / 2) : ntiles;
+            const int n1 = alt ? ntiles / 2 : ntiles;           // tiles of stream 1 in this unit
             const int b = u.b, c = u.c;
-            const int row = u.row0 + i * BM + rloc;
+            const int row = u.row0 + (alt ? 0 : i * BM) + rloc;
             const bool rvalid = row < R;
             if (warp == 0 && lane == 0) {
                 const int Lraw = p.seq_lens[b];
@@ -551,7 +608,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
             float m_ref = -CUDART_INF_F, l_run = 0.f;
             const uint32_t* mrow = p.mask + ((size_t)b * N + (rvalid ? row / G : 0)) * p.W;
-            for (int idx = 0; idx < ntiles; ++idx) {
+            for (int cnt = 0; cnt < my_n; ++cnt) {
+                const int idx = alt ? 2 * cnt + i : cnt;
                 const TileInfo ti = tile_info(u.t_begin + idx, u.nPT, u.L, u.live);
                 // visibility words of this row for the 128 keys of the tile
                 uint32_t mw[4];
@@ -573,7 +631,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         mw[k] = word;
                     }
                 }
-                const uint32_t par = (uint32_t)((tcnt + idx) & 1);
+                const uint32_t par = (uint32_t)((tcnt + cnt) & 1);
                 ok = mbar_wait(bar(BAR_S_FULL + i), par, abort_flag, p.status);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
@@ -622,7 +680,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 m_ref = m_new;
                 const float m_use = m_ref == -CUDART_INF_F ? 0.f : m_ref;
 
-                if (ti.kind == 1 && i == 0) {
+                if (ti.kind == 1 && (alt || i == 0)) {
                     // cache rows past the sequence end may hold anything: clear them in the V tile
                     // so that 0 * junk cannot reach the accumulator
                     const int vs_stage = (kvc + idx) % VST;
@@ -674,6 +732,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
             if (!ok) break;
 
+            if (alt && i == 1) {
+                // odd-tile stream: publish (max, sum); warpgroup 0 reads the accumulator itself
+                if (my_n > 0) {
+                    s_ml1[rloc] = make_float2(m_ref, l_run);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(BAR_ML_READY));
+                    ++mlc;
+                    ++auc;
+                }
+                kvc += ntiles;
+                tcnt += my_n;
+                continue;
+            }
             // ---- epilogue: pull the accumulator row into registers, give TMEM back, then store
             float acc[HD];
             if (ntiles > 0) {
@@ -684,6 +755,32 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) tc_ld32p(tO + ch * 32, acc + ch * 32);
                 tc_wait_ld();
+                if (alt && n1 > 0) {
+                    // merge the odd-tile stream: O = w0 O0 + w1 O1, l = w0 l0 + w1 l1 at the common maximum
+                    ok = mbar_wait(bar(BAR_O_DONE + 1), (uint32_t)(auc1 & 1), abort_flag, p.status);
+                    if (ok) ok = mbar_wait(bar(BAR_ML_READY), (uint32_t)(mlc & 1), abort_flag, p.status);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const float2 ml1 = s_ml1[rloc];
+                    const float m = fmaxf(m_ref, ml1.x);
+                    const float m_use = m == -CUDART_INF_F ? 0.f : m;
+                    const float w0 = fast_exp2(m_ref - m_use), w1 = fast_exp2(ml1.x - m_use);
+                    const uint32_t tO1 = tmem + lane_addr + COL_O1;
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        float v[32];
+                        tc_ld32(tO1 + ch * 32, v);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) acc[ch * 32 + e] = w0 * acc[ch * 32 + e] + w1 * v[e];
+                    }
+                    l_run = w0 * l_run + w1 * ml1.y;
+                    m_ref = m;
+                    tc_fence_before();
+                    if (lane == 0) mbar_arrive(bar(BAR_O_FREE + 1));
+                    ++mlc;
+                }
                 tc_fence_before();
                 if (lane == 0) mbar_arrive(bar(BAR_O_FREE + i));
             } else {
@@ -704,7 +801,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         *reinterpret_cast<uint4*>(dst + k * 8) = v;
                     }
                 } else {
-                    const size_t prow = (size_t)u.slot * (2 * BM) + i * BM + rloc;
+                    const size_t prow = (size_t)u.slot * (2 * BM) + (alt ? 0 : i * BM) + rloc;
                     float* dst = p.part_o + prow * HD;
 #pragma unroll
                     for (int k = 0; k < HD / 4; ++k)
@@ -714,8 +811,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 }
             }
             kvc += ntiles;
-            tcnt += ntiles;
+            tcnt += my_n;
             if (ntiles > 0) ++auc;
+            if (n1 > 0) ++auc1;
         }
     }
 
