@@ -36,7 +36,7 @@ constexpr int VST = 2;             // V ring stages
 constexpr uint32_t HALF_BYTES = 128 * 64 * 2;     // one [128 rows][64 bf16] swizzled block
 constexpr uint32_t TILE_BYTES = 2 * HALF_BYTES;   // a 128 x 128 bf16 tile (two column halves)
 constexpr int kThreads = 384;
-constexpr uint32_t kSmemBytes = (2 + KST + VST) * TILE_BYTES + 1024;  // + alignment slack
+constexpr uint32_t kSmemBytes = (2 + KST + VST) * TILE_BYTES + 2 * HALF_BYTES + 1024;  // tiles, output staging, alignment slack
 constexpr float kRescaleThreshold = 8.0f;         // log2 units
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
@@ -126,6 +126,17 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
+
+// shared -> global tile store; completion is tracked by bulk async-groups of the issuing thread
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+        ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void wg_barrier(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -335,7 +346,8 @@ __device__ __forceinline__ UnitInfo unit_info(const TcParams& p, int w, int lane
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_dk,
-               const __grid_constant__ CUtensorMap tm_dv, const TcParams p) {
+               const __grid_constant__ CUtensorMap tm_dv, const __grid_constant__ CUtensorMap tm_out,
+               const TcParams p) {
     extern __shared__ unsigned char smem_raw[];
     __shared__ __align__(8) unsigned long long s_bars[BAR_COUNT];
     __shared__ uint32_t s_tmem_base;
@@ -349,6 +361,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const uint32_t sQ = smem_base;                                   // 2 tiles
     const uint32_t sK = smem_base + 2 * TILE_BYTES;                  // KST tiles
     const uint32_t sV = sK + KST * TILE_BYTES;                       // VST tiles
+    const uint32_t sStage = sV + VST * TILE_BYTES;                   // one [128][64] bf16 block per softmax warpgroup
     const uint32_t bar0 = smem_u32(s_bars);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     volatile int* abort_flag = &s_abort;
@@ -787,20 +800,38 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
                 for (int e = 0; e < HD; ++e) acc[e] = 0.f;
             }
-            if (rvalid) {
-                if (u.nsplit == 1) {
-                    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-                    __nv_bfloat16* dst = p.out + (((size_t)b * N + row / G) * p.Hq + c * G + row % G) * HD;
+            if (u.nsplit == 1) {
+                // Normalise, round to bf16 and stage the rows in shared memory in the swizzled tile
+                // layout; one thread then writes each 64-column half with a TMA tile store (full
+                // 128-byte lines instead of 32 scattered 16-byte pieces per store instruction;
+                // rows of nodes >= N are clipped by the tensor map).
+                const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+                const uint32_t stage = sStage + (uint32_t)i * HALF_BYTES;
+                unsigned char* srow = smem_raw + (stage - smem_u32(smem_raw)) + rloc * 128;
+                const bool issuer = (warp & 3) == 0 && lane == 0;
 #pragma unroll
-                    for (int k = 0; k < HD / 8; ++k) {
+                for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const int e = h * 64 + k * 8;
                         uint4 v;
-                        v.x = pack_bf16(acc[8 * k + 0] * inv, acc[8 * k + 1] * inv);
-                        v.y = pack_bf16(acc[8 * k + 2] * inv, acc[8 * k + 3] * inv);
-                        v.z = pack_bf16(acc[8 * k + 4] * inv, acc[8 * k + 5] * inv);
-                        v.w = pack_bf16(acc[8 * k + 6] * inv, acc[8 * k + 7] * inv);
-                        *reinterpret_cast<uint4*>(dst + k * 8) = v;
+                        v.x = pack_bf16(acc[e + 0] * inv, acc[e + 1] * inv);
+                        v.y = pack_bf16(acc[e + 2] * inv, acc[e + 3] * inv);
+                        v.z = pack_bf16(acc[e + 4] * inv, acc[e + 5] * inv);
+                        v.w = pack_bf16(acc[e + 6] * inv, acc[e + 7] * inv);
+                        *reinterpret_cast<uint4*>(srow + ((k ^ (rloc & 7)) << 4)) = v;
                     }
-                } else {
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    wg_barrier(1 + i);
+                    if (issuer) {
+                        tma_store_4d(&tm_out, stage, h * 64, c * G, (u.row0 + (alt ? 0 : i * BM)) / G, b);
+                        bulk_commit();
+                        bulk_wait_read();          // the staging block may be overwritten again
+                    }
+                    wg_barrier(1 + i);
+                }
+            } else if (rvalid) {
+                {
                     const size_t prow = (size_t)u.slot * (2 * BM) + (alt ? 0 : i * BM) + rloc;
                     float* dst = p.part_o + prow * HD;
 #pragma unroll
@@ -815,6 +846,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             if (ntiles > 0) ++auc;
             if (n1 > 0) ++auc1;
         }
+        if ((warp & 3) == 0 && lane == 0) bulk_wait_all();   // the output stores have landed
     }
 
     // ---------------------------------------------------------------- teardown
@@ -876,13 +908,14 @@ int launch_attn_tcgen05(const AttnArgs& a) {
         set_error_text("tcgen05 back end needs D == 128 and a group size that divides 128");
         return GSD_ERR_UNSUPPORTED;
     }
-    CUtensorMap tq, tk, tv, tdk, tdv;
+    CUtensorMap tq, tk, tv, tdk, tdv, tout;
     int rc;
     if ((rc = make_map(&tq, a.q, a.Hq, a.N, a.B, a.G, BM / a.G)) != GSD_OK) return rc;
     if ((rc = make_map(&tk, a.k_cache, a.Hkv, a.Lmax, a.B, 1, BN)) != GSD_OK) return rc;
     if ((rc = make_map(&tv, a.v_cache, a.Hkv, a.Lmax, a.B, 1, BN)) != GSD_OK) return rc;
     if ((rc = make_map(&tdk, a.draft_k, a.Hkv, a.N, a.B, 1, BN)) != GSD_OK) return rc;
     if ((rc = make_map(&tdv, a.draft_v, a.Hkv, a.N, a.B, 1, BN)) != GSD_OK) return rc;
+    if ((rc = make_map(&tout, a.out, a.Hq, a.N, a.B, a.G, BM / a.G)) != GSD_OK) return rc;
     TcParams p;
     p.mask = a.mask; p.seq_lens = a.seq_lens; p.out = (__nv_bfloat16*)a.out; p.status = a.status;
     p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv; p.Lmax = a.Lmax; p.G = a.G; p.W = a.W;
@@ -894,7 +927,7 @@ int launch_attn_tcgen05(const AttnArgs& a) {
     DeviceInfo di;
     if (device_info(&di) != 0) return GSD_ERR_CUDA;
     dim3 grid(a.plan.ctas < di.sm_count ? a.plan.ctas : di.sm_count);
-    attn_tc_kernel<<<grid, kThreads, kSmemBytes, a.stream>>>(tq, tk, tv, tdk, tdv, p);
+    attn_tc_kernel<<<grid, kThreads, kSmemBytes, a.stream>>>(tq, tk, tv, tdk, tdv, tout, p);
     GSD_CUDA_TRY(cudaGetLastError());
     return GSD_OK;
 }
