@@ -367,9 +367,7 @@ def main():
     # (profiles/attn_tcgen05_llama70b.md); only valid for that kernel on that workload
     if cfg.name == "llama70b" and args.kernel in (0, 2) and args.num_splits == 0:
         roof["traffic"] = 197.9e6
-    # the tcgen05 kernel merges cut items itself; the mma.sync kernel needs the merge launch
-    uses_tc = args.kernel == 2 or (args.kernel == 0 and cfg.D == 128 and 128 % cfg.G == 0 and cfg.N * cfg.G >= 64)
-    roof["kernel"] = "gsd_verify_attn" + (" (split pass + merge pass)" if (splits > 1 and not uses_tc) else "")
+    roof["kernel"] = "gsd_verify_attn" + (" (split pass + merge pass)" if splits > 1 else "")
     roof["algorithmic_flops"] = flops
     roof["algorithmic_bytes"] = attn_bytes
     roof["launch_us_mean"] = attn_mean * 1e6
@@ -393,7 +391,7 @@ def main():
         "accept_gbs": accept_bytes / acc_mean / 1e9,
         "accept_frac_of_hbm": accept_bytes / acc_mean / 1e9 / peaks["hbm_gbs"],
         "roofline": roof, "cpu_baseline": cpu, "e2e": e2e,
-        "gpu_launches": args.steps * ((2 if (splits > 1 and not uses_tc) else 1) + 1),
+        "gpu_launches": args.steps * ((2 if splits > 1 else 1) + 1),
         "clocks": clocks,
     }
     print(json.dumps(line), flush=True)

@@ -93,7 +93,7 @@ AttnPlan attn_make_plan(const gsd_attn_params* p, int sm_count) {
     pl.ctas = pl.dev.items_a * pl.dev.splits_a + items_b * pl.dev.splits_b;
     pl.slots = (pl.dev.splits_a > 1 ? pl.dev.items_a * pl.dev.splits_a : 0) +
                (pl.dev.splits_b > 1 ? items_b * pl.dev.splits_b : 0);
-    pl.ws_bytes = pl.slots ? plan_part_o_bytes(pl, p->D) + plan_part_ml_bytes(pl) + (tc ? plan_counter_bytes(pl) : 0) : 0;
+    pl.ws_bytes = pl.slots ? plan_part_o_bytes(pl, p->D) + plan_part_ml_bytes(pl) : 0;
     return pl;
 }
 
@@ -165,9 +165,7 @@ extern "C" int gsd_verify_attn(const void* q, const void* k_cache, const void* v
     a.stream = (cudaStream_t)stream;
     int rc = plan.kernel == GSD_ATTN_TCGEN05 ? launch_attn_tcgen05(a) : launch_attn_mma(a);
     if (rc != GSD_OK) return rc;
-    // the tcgen05 kernel merges the pieces of a cut item itself (last arrival); the mma.sync
-    // kernel leaves them to the merge pass
-    if (plan.slots > 0 && plan.kernel != GSD_ATTN_TCGEN05) rc = launch_attn_merge(a);
+    if (plan.slots > 0) rc = launch_attn_merge(a);
     return rc;
 }
 

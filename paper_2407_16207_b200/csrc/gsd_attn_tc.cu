@@ -65,7 +65,6 @@ struct TcParams {
     __nv_bfloat16* out;
     float* part_o;
     float* part_ml;
-    int* counters;    // [slot][2] arrivals of the pieces of a cut item, zeroed before the launch
     int32_t* status;
     int B, N, Hq, Hkv, Lmax, G, W, R;
     float scale_log2;
@@ -353,7 +352,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     __shared__ __align__(8) unsigned long long s_bars[BAR_COUNT];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
-    __shared__ int s_last[2];         // did this warpgroup's piece arrive last (it merges the item then)
     __shared__ float2 s_ml1[BM];      // (max, sum) of the odd-tile stream, one per row
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -802,55 +800,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
                 for (int e = 0; e < HD; ++e) acc[e] = 0.f;
             }
-            bool store = u.nsplit == 1;
-            if (u.nsplit > 1) {
-                // A cut item: publish this piece (unnormalised fp32 accumulator, running maximum and
-                // sum); the piece that arrives last combines all of them and stores the rows.
-                const int ci = alt ? 0 : i;
-                const int slot0 = u.slot - u.split;
-                if (rvalid) {
-                    const size_t prow = (size_t)u.slot * (2 * BM) + ci * BM + rloc;
-                    float* dst = p.part_o + prow * HD;
-#pragma unroll
-                    for (int k = 0; k < HD / 4; ++k)
-                        *reinterpret_cast<float4*>(dst + k * 4) =
-                            make_float4(acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]);
-                    *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(m_ref, l_run);
-                }
-                __threadfence();
-                wg_barrier(1 + i);
-                if ((warp & 3) == 0 && lane == 0)
-                    s_last[i] = atomicAdd(p.counters + slot0 * 2 + ci, 1) == u.nsplit - 1;
-                wg_barrier(1 + i);
-                store = s_last[i] != 0;
-                if (store) {
-                    __threadfence();
-                    //   m = max_s m_s;  O = sum_s 2^(m_s - m) O_s;  l = sum_s 2^(m_s - m) l_s
-                    const size_t row0s = (size_t)slot0 * (2 * BM) + ci * BM + rloc;
-                    const size_t sstride = 2 * BM;
-                    float m = -CUDART_INF_F;
-                    for (int sp = 0; sp < u.nsplit; ++sp)
-                        m = fmaxf(m, __ldcg(p.part_ml + (row0s + sp * sstride) * 2));
-                    const float m_use = m == -CUDART_INF_F ? 0.f : m;
-#pragma unroll
-                    for (int e = 0; e < HD; ++e) acc[e] = 0.f;
-                    l_run = 0.f;
-                    for (int sp = 0; sp < u.nsplit; ++sp) {
-                        const size_t prow = row0s + sp * sstride;
-                        const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + prow * 2));
-                        const float wgt = fast_exp2(ml.x - m_use);
-                        l_run += wgt * ml.y;
-                        const float4* src = reinterpret_cast<const float4*>(p.part_o + prow * HD);
-#pragma unroll
-                        for (int k = 0; k < HD / 4; ++k) {
-                            const float4 v = __ldcg(src + k);
-                            acc[4 * k] += wgt * v.x; acc[4 * k + 1] += wgt * v.y;
-                            acc[4 * k + 2] += wgt * v.z; acc[4 * k + 3] += wgt * v.w;
-                        }
-                    }
-                }
-            }
-            if (store) {
+            if (u.nsplit == 1) {
                 // Normalise, round to bf16 and stage the rows in shared memory in the swizzled tile
                 // layout; one thread then writes each 64-column half with a TMA tile store (full
                 // 128-byte lines instead of 32 scattered 16-byte pieces per store instruction;
@@ -879,6 +829,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         bulk_wait_read();          // the staging block may be overwritten again
                     }
                     wg_barrier(1 + i);
+                }
+            } else if (rvalid) {
+                {
+                    const size_t prow = (size_t)u.slot * (2 * BM) + (alt ? 0 : i * BM) + rloc;
+                    float* dst = p.part_o + prow * HD;
+#pragma unroll
+                    for (int k = 0; k < HD / 4; ++k)
+                        *reinterpret_cast<float4*>(dst + k * 4) =
+                            make_float4(acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]);
+                    *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(m_ref, l_run);
                 }
             }
             kvc += ntiles;
@@ -962,8 +922,6 @@ int launch_attn_tcgen05(const AttnArgs& a) {
     p.R = a.N * a.G; p.scale_log2 = a.scale_log2; p.plan = a.plan.dev;
     p.part_o = (float*)a.workspace;
     p.part_ml = (float*)((char*)a.workspace + plan_part_o_bytes(a.plan, a.D));
-    p.counters = (int*)((char*)p.part_ml + plan_part_ml_bytes(a.plan));
-    if (a.plan.slots > 0) GSD_CUDA_TRY(cudaMemsetAsync(p.counters, 0, plan_counter_bytes(a.plan), a.stream));
     GSD_CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
     p.total_work = a.plan.ctas;
     DeviceInfo di;

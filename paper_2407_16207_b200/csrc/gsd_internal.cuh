@@ -81,8 +81,6 @@ int attn_pick_kernel(const gsd_attn_params* p);                 // GSD_ATTN_MMA 
 // partial results: fp32 accumulators [slot][rows_per_item][D], then (max, sum) [slot][rows_per_item][2]
 inline size_t plan_part_o_bytes(const AttnPlan& pl, int D) { return align_up((size_t)pl.slots * pl.rows_per_item * D * sizeof(float), 256); }
 inline size_t plan_part_ml_bytes(const AttnPlan& pl) { return align_up((size_t)pl.slots * pl.rows_per_item * 2 * sizeof(float), 256); }
-// tcgen05 back end: one arrival counter per (slot, row tile); the last piece of an item to arrive merges
-inline size_t plan_counter_bytes(const AttnPlan& pl) { return align_up((size_t)pl.slots * 2 * sizeof(int), 256); }
 
 int launch_attn_mma(const AttnArgs& a);
 int launch_attn_tcgen05(const AttnArgs& a);
