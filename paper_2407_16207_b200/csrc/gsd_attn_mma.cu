@@ -430,7 +430,15 @@ int launch_mma_t(const AttnArgs& a) {
     p.part_o = (float*)a.workspace;
     p.part_ml = (float*)((char*)a.workspace + plan_part_o_bytes(a.plan, a.D));
     const int smem = 4 * BN * D * 2;
-    GSD_CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    {
+        static bool done[64] = {};   // per template instance: the opt-in sticks per device
+        int dev = 0;
+        GSD_CUDA_TRY(cudaGetDevice(&dev));
+        if (dev < 0 || dev >= 64 || !done[dev]) {
+            GSD_CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            if (dev >= 0 && dev < 64) done[dev] = true;
+        }
+    }
     dim3 grid(a.plan.ctas);
     attn_mma_kernel<D><<<grid, kThreads, smem, a.stream>>>(p);
     GSD_CUDA_TRY(cudaGetLastError());

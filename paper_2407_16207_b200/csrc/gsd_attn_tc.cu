@@ -922,7 +922,16 @@ int launch_attn_tcgen05(const AttnArgs& a) {
     p.R = a.N * a.G; p.scale_log2 = a.scale_log2; p.plan = a.plan.dev;
     p.part_o = (float*)a.workspace;
     p.part_ml = (float*)((char*)a.workspace + plan_part_o_bytes(a.plan, a.D));
-    GSD_CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    {
+        // the opt-in for large dynamic shared memory is per device and sticks: do it once
+        static bool done[64] = {};
+        int dev = 0;
+        GSD_CUDA_TRY(cudaGetDevice(&dev));
+        if (dev < 0 || dev >= 64 || !done[dev]) {
+            GSD_CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+            if (dev >= 0 && dev < 64) done[dev] = true;
+        }
+    }
     p.total_work = a.plan.ctas;
     DeviceInfo di;
     if (device_info(&di) != 0) return GSD_ERR_CUDA;

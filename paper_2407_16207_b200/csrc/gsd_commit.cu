@@ -36,18 +36,41 @@ __global__ void __launch_bounds__(kThreads) commit_kernel(CommitArgs a) {
         flags |= GSD_DEV_BAD_SEQ_LEN;
         L = L < 0 ? 0 : a.Lmax;
     }
-    if (threadIdx.x == 0) {
-        // compact the valid node ids in path order (serial: at most Tcap <= a few hundred ints)
+    {
+        // compact the valid node ids in path order: every thread reads one entry, the positions
+        // come from warp ballots and a scan over the warp totals
+        __shared__ int s_warp_tot[kThreads / 32];
         int len = a.len[b];
         if (len > a.Tcap) len = a.Tcap;
-        int n = 0;
-        for (int i = 0; i < len; ++i) {
-            const int node = a.nodes[(size_t)b * a.Tcap + i];
-            if (node < 0 || node >= a.N) { flags |= GSD_DEV_BAD_CSR; continue; }
-            if (L + n >= a.Lmax) { flags |= GSD_DEV_CACHE_FULL; break; }
-            if (n < GSD_MAX_NODES) s_src[n++] = node;
+        if (len > GSD_MAX_NODES) len = GSD_MAX_NODES;
+        if (threadIdx.x == 0) s_count = 0;
+        int base = 0;
+        for (int i0 = 0; i0 < len; i0 += kThreads) {      // one pass unless Tcap > 256
+            const int i = i0 + threadIdx.x;
+            int node = -1;
+            bool valid = false;
+            if (i < len) {
+                node = a.nodes[(size_t)b * a.Tcap + i];
+                valid = node >= 0 && node < a.N;
+                if (!valid) flags |= GSD_DEV_BAD_CSR;
+            }
+            const unsigned vote = __ballot_sync(0xFFFFFFFFu, valid);
+            const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+            if (lane == 0) s_warp_tot[warp] = __popc(vote);
+            __syncthreads();
+            int before = base;
+            for (int w = 0; w < warp; ++w) before += s_warp_tot[w];
+            const int pos = before + __popc(vote & ((1u << lane) - 1u));
+            if (valid) {
+                if (L + pos < a.Lmax) s_src[pos] = node;
+                else flags |= GSD_DEV_CACHE_FULL;
+            }
+            int total = 0;
+            for (int w = 0; w < kThreads / 32; ++w) total += s_warp_tot[w];
+            base += total;
+            __syncthreads();
         }
-        s_count = n;
+        if (threadIdx.x == 0) s_count = min(base, a.Lmax - L);
         if (flags && a.status) atomicOr((unsigned*)a.status, flags);
     }
     __syncthreads();
