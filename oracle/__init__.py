@@ -16,8 +16,10 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = os.path.join(_HERE, "gsd_oracle.c")
-_LIB = os.path.join(_HERE, "_gsd_oracle.so")
+# GSD_ORACLE_SRC / GSD_ORACLE_LIB let the mutation tests point this loader at a deliberately
+# broken copy of the source (to show that the pins notice); nothing else uses them.
+_SRC = os.environ.get("GSD_ORACLE_SRC", os.path.join(_HERE, "gsd_oracle.c"))
+_LIB = os.environ.get("GSD_ORACLE_LIB", os.path.join(_HERE, "_gsd_oracle.so"))
 _lib: Optional[ctypes.CDLL] = None
 
 

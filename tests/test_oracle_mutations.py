@@ -1,0 +1,53 @@
+"""Are the oracle's pins sharp?  Each case plants ONE plausible mistake in a copy of the
+oracle's source (on the CPU; the real oracle is untouched), builds it, and runs the pin tests
+against the broken copy in a subprocess: they must fail.  A mistake that survives would mean a
+part of the oracle is not pinned."""
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SRC = os.path.join(ROOT, "oracle", "gsd_oracle.c")
+
+# (name, text to replace, replacement, pin files that must catch it)
+MUTATIONS = [
+    ("gqa_mapping", "const int c = h / G;", "const int c = h % Hkv;", "test_oracle_attn.py"),
+    ("mask_bit_order", "(mrow[j / 32] >> (j % 32))", "(mrow[j / 32] >> (31 - j % 32))", "test_oracle_attn.py"),
+    ("mask_word_order", "(mrow[j / 32] >> (j % 32))", "(mrow[W - 1 - j / 32] >> (j % 32))", "test_oracle_attn.py"),
+    ("softmax_scale", "1.0 / sqrt((double)D)", "1.0 / (double)D", "test_oracle_attn.py"),
+    ("prefix_length_off_by_one", "const int L = seq_lens[b];", "const int L = seq_lens[b] + (seq_lens[b] < Lmax);",
+     "test_oracle_attn.py"),
+    ("no_max_subtraction", "s[i] = exp(s[i] - smax);", "s[i] = exp(s[i]);", "test_oracle_attn.py"),
+    ("draft_value_index", "const uint16_t *vrow = draft_v + (((size_t)b * N + j)",
+     "const uint16_t *vrow = draft_v + (((size_t)b * N + (N - 1 - j))", "test_oracle_attn.py"),
+    ("tie_read_forwards", "for (int i = len - 1; i >= 0; --i) {", "for (int i = 0; i < len; ++i) {",
+     "test_oracle_accept.py"),
+    ("longest_ge", "edges > w->best_edges ||", "edges >= w->best_edges ||", "test_oracle_accept.py"),
+    ("argmax_last_of_ties", "row[i] > row[best]) best = i;", "row[i] >= row[best]) best = i;", "test_oracle_accept.py"),
+    ("bonus_token_node", "= amax[best[m]];", "= amax[best[m > 0 ? m - 1 : 0]];", "test_oracle_accept.py"),
+    ("edge_rule", "w->tok[w->stack[i]] != w->amax[w->stack[i - 1]]", "w->tok[w->stack[i]] != w->amax[w->stack[i]]",
+     "test_oracle_accept.py"),
+    ("commit_position", "k_cache + ((size_t)b * Lmax + pos) * row, draft_k",
+     "k_cache + ((size_t)b * Lmax + pos + 1 - (pos + 1 >= Lmax)) * row, draft_k", "test_oracle_commit.py"),
+    ("mask_without_self", "row[v / 32] |= 1u << (v % 32);", "if (v != n) row[v / 32] |= 1u << (v % 32);",
+     "test_oracle_mask.py"),
+    ("mask_parents_only", "seen[p] = 1;\n                    todo[top++] = p;", "seen[p] = 1;\n                    if (v == n) todo[top++] = p;",
+     "test_oracle_mask.py"),
+]
+
+
+@pytest.mark.parametrize("name,old,new,pins", MUTATIONS, ids=[m[0] for m in MUTATIONS])
+def test_planted_mistake_is_caught(tmp_path, name, old, new, pins):
+    text = open(SRC).read()
+    assert text.count(old) >= 1, f"mutation {name} no longer applies"
+    src = tmp_path / "gsd_oracle_mutated.c"
+    src.write_text(text.replace(old, new))
+    env = dict(os.environ, GSD_ORACLE_SRC=str(src), GSD_ORACLE_LIB=str(tmp_path / "mutated.so"))
+    # the quick pins only (the config-sized cross-checks are not needed to notice these)
+    cmd = [sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
+           os.path.join(ROOT, "tests", pins), "-k", "not configs and not matrix_closure"]
+    r = subprocess.run(cmd, env=env, capture_output=True, text=True, cwd=ROOT, timeout=300)
+    assert r.returncode != 0, f"the pins did not notice the planted mistake '{name}'"
+    assert "failed" in r.stdout or "error" in r.stdout.lower()
