@@ -137,10 +137,10 @@ def aggregate_over_ranks(ms_per_step, tokens_per_step, world, dist, device):
     return {"ms_per_step": ms_per_step, "value": world * tokens_per_step / (ms_per_step * 1e-3)}
 
 
-def cpu_oracle_sample(cfg, inp, budget_rows: int):
+def cpu_oracle_sample(cfg, inp, budget_rows: int, accept_seqs: int = 0):
     """Times the CPU oracle (as it stands) on a bounded sample of the workload: `budget_rows`
-    random attention rows plus the full acceptance step.  Returns (tokens/s extrapolated to
-    the whole step, threads, description)."""
+    random attention rows plus the acceptance step of `accept_seqs` sequences (0 = all).
+    Returns (tokens/s extrapolated to the whole step, threads, description)."""
     import oracle
     rng = np.random.default_rng(0)
     total_rows = cfg.B * cfg.N * cfg.Hq
@@ -151,27 +151,32 @@ def cpu_oracle_sample(cfg, inp, budget_rows: int):
     oracle.attn_rows(inp["q"], inp["k_cache"], inp["v_cache"], inp["draft_k"], inp["draft_v"],
                      inp["ancestor_mask"], inp["seq_lens"], rows)
     t_attn = time.perf_counter() - t0
+    nb = cfg.B if accept_seqs <= 0 else min(accept_seqs, cfg.B)
     t0 = time.perf_counter()
-    oracle.accept(inp["logits"], inp["draft_tokens"], inp["parent_ptr"], inp["parent_idx"])
-    t_acc = time.perf_counter() - t0
+    oracle.accept(inp["logits"][:nb], inp["draft_tokens"][:nb], inp["parent_ptr"][:nb], inp["parent_idx"][:nb])
+    t_acc = (time.perf_counter() - t0) * (cfg.B / nb)
     t_step = t_attn * (total_rows / n) + t_acc
-    desc = (f"{n} of {total_rows} attention rows (random (b,n,h), {t_attn:.2f} s, scaled to all rows) "
-            f"+ full acceptance ({t_acc:.2f} s)")
+    desc = (f"{n} of {total_rows} attention rows (random (b,n,h), {t_attn:.3f} s, scaled to all rows) "
+            f"+ acceptance of {nb} of {cfg.B} sequences ({t_acc:.3f} s scaled to all)")
     return cfg.B * cfg.N / t_step, oracle.threads(), desc
 
 
 def run_reference(args, cfg):
-    """The reference arm: the CPU oracle, timed on the host cores, each step a bounded sample."""
+    """The reference arm: the CPU oracle, timed on the host cores.  Each of the K steps is a
+    bounded sample of the workload, sized so that the whole run takes about a minute whatever K is."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     inp = gi.make_inputs(cfg)
     total_rows = cfg.B * cfg.N * cfg.Hq
-    rows_per_step = min(total_rows, max(256, 8192 // max(1, (args.steps + args.warmup) // 4)))
+    n_steps = args.warmup + args.steps
+    # ~2e5 rows/min on 16 threads at this size: spread ~40000 rows over the run, at least 16 per step
+    rows_per_step = int(min(total_rows, max(16, 40000 // max(1, n_steps))))
+    accept_seqs = 0 if n_steps <= 50 else 1
     vals = []
-    desc = ""
-    for i in range(args.warmup + args.steps):
-        v, threads, desc = cpu_oracle_sample(cfg, inp, rows_per_step)
+    desc, threads = "", 1
+    for i in range(n_steps):
+        v, threads, desc = cpu_oracle_sample(cfg, inp, rows_per_step, accept_seqs)
         if i >= args.warmup:
             vals.append(v)
     value = cfg.B * cfg.N * len(vals) / sum(cfg.B * cfg.N / v for v in vals)
