@@ -119,6 +119,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, abort_flag, status, false);
 }
+// the same, called by all lanes of a converged warp; the answer is made uniform
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               int32_t* status) {
+    return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag, status));
+}
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
                                             int c0, int c1, int c2, int c3) {
@@ -143,19 +148,27 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// The MMA warp runs its loops with all 32 lanes converged and elects one lane per tcgen05
+// instruction: addresses, descriptors and loop state are then warp-uniform, which costs the
+// warp far fewer issue slots than a single-lane branch would (the softmax warps on the same
+// scheduler are almost always ready to issue, so every extra instruction here waits its turn).
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile(
+        "{\n .reg .pred q;\n elect.sync _|q, 0xffffffff;\n"
+        " @q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}\n" ::"r"(bar) : "memory");
 }
 // D[tmem] (+)= A[smem desc] * B[smem desc]
 __device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
     asm volatile(
-        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+        "{\n .reg .pred p, q;\n elect.sync _|q, 0xffffffff;\n setp.ne.b32 p, %4, 0;\n"
+        " @q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem desc]
 __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
     asm volatile(
-        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
+        "{\n .reg .pred p, q;\n elect.sync _|q, 0xffffffff;\n setp.ne.b32 p, %4, 0;\n"
+        " @q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
         ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
 }
 
@@ -450,11 +463,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             ++au;
         }
     } else if (warp == 9) {
-        // ------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------ MMA issuer (all lanes converged)
         int kvc = 0;              // key tiles consumed so far (ring position)
         int au = 0, au1 = 0;      // non-empty units so far; those of them in which stream 1 had tiles
         int tc0 = 0, tc1 = 0;     // key tiles handed to the softmax of stream 0 / 1 so far
         bool ok = true;
+        auto wait = [&](int b, uint32_t par) -> bool { return mbar_wait_warp(bar(b), par, abort_flag, p.status); };
         auto issue_qk = [&](int i, int qtile, int stage) {
             // S_i = Q_qtile K^T : 8 k-steps of 16 over the head dimension
             const uint32_t qa = sQ + qtile * TILE_BYTES, ka = sK + stage * TILE_BYTES;
@@ -478,14 +492,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         };
         // tile = running tile number of row tile i (barrier phase); first = first tile of the unit
         auto issue_pv = [&](int i, int stage, int tile, bool first, int units_before) -> bool {
-            if (!mbar_wait(bar(BAR_P_READY + i), tile & 1, abort_flag, p.status)) return false;
+            if (!wait(BAR_P_READY + i, tile & 1)) return false;
             if (first && units_before > 0) {
                 // the accumulator still belongs to the previous unit until its rows were read out
-                if (!mbar_wait(bar(BAR_O_FREE + i), (units_before - 1) & 1, abort_flag, p.status)) return false;
+                if (!wait(BAR_O_FREE + i, (units_before - 1) & 1)) return false;
             }
             tc_fence_after();
             issue_pv_half(i, stage, 0, !first);
-            if (!mbar_wait(bar(BAR_P_READY2 + i), tile & 1, abort_flag, p.status)) return false;
+            if (!wait(BAR_P_READY2 + i, tile & 1)) return false;
             tc_fence_after();
             issue_pv_half(i, stage, 1, !first);
             return true;
@@ -495,95 +509,87 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             if (u.ntiles == 0) continue;
             const int n0 = u.two ? u.ntiles : (u.ntiles + 1) / 2;   // key tiles of stream 0 / stream 1
             const int n1 = u.two ? u.ntiles : u.ntiles / 2;
-            if (lane == 0) {
-                const bool two = u.two;
-                const int ntiles = u.ntiles;
-                ok = mbar_wait(bar(BAR_Q_FULL), au & 1, abort_flag, p.status);
-                tc_fence_after();
-                if (two) {
-                    for (int idx = 0; idx < ntiles && ok; ++idx) {
-                        const int st = kvc % KST;
-                        ok = mbar_wait(bar(BAR_K_FULL + st), (kvc / KST) & 1, abort_flag, p.status);
+            const int ntiles = u.ntiles;
+            ok = wait(BAR_Q_FULL, au & 1);
+            tc_fence_after();
+            if (u.two) {
+                for (int idx = 0; idx < ntiles && ok; ++idx) {
+                    const int st = kvc % KST;
+                    ok = wait(BAR_K_FULL + st, (kvc / KST) & 1);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(0, 0, st);
+                    tc_commit(bar(BAR_S_FULL + 0));
+                    if (idx > 0) {
+                        ok = issue_pv(1, (kvc - 1) % VST, tc1 + idx - 1, idx == 1, au1);
                         if (!ok) break;
-                        tc_fence_after();
-                        issue_qk(0, 0, st);
-                        tc_commit(bar(BAR_S_FULL + 0));
-                        if (two) {
-                            if (idx > 0) {
-                                ok = issue_pv(1, (kvc - 1) % VST, tc1 + idx - 1, idx == 1, au1);
-                                if (!ok) break;
-                                tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
-                            }
-                            issue_qk(1, 1, st);
-                            tc_commit(bar(BAR_S_FULL + 1));
-                        }
-                        tc_commit(bar(BAR_K_EMPTY + st));
-                        if (idx == ntiles - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
-                        ok = mbar_wait(bar(BAR_V_FULL + st), (kvc / VST) & 1, abort_flag, p.status);
-                        if (!ok) break;
-                        ok = issue_pv(0, st, tc0 + idx, idx == 0, au);
-                        if (!ok) break;
-                        if (!two) tc_commit(bar(BAR_V_EMPTY + st));
-                        if (idx == ntiles - 1) tc_commit(bar(BAR_O_DONE + 0));
-                        ++kvc;
+                        tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
                     }
-                    if (ok && two) {
-                        ok = issue_pv(1, (kvc - 1) % VST, tc1 + ntiles - 1, ntiles == 1, au1);
-                        if (ok) {
-                            tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
-                            tc_commit(bar(BAR_O_DONE + 1));
-                        }
-                    }
-                } else {
-                    // One row tile only: the two accumulator pairs take the even and the odd key
-                    // tiles of the same rows (two independent partial attentions that the epilogue
-                    // merges), so the softmax of one tile still runs under the MMAs of the next.
-                    const int kv0 = kvc;
-                    int pv1_issued = 0;
-                    auto finish_pv1 = [&](int c1) -> bool {       // PV of stream 1's tile c1
-                        const int r = kv0 + 2 * c1 + 1;
-                        if (!mbar_wait(bar(BAR_V_FULL + r % VST), (r / VST) & 1, abort_flag, p.status)) return false;
-                        if (!issue_pv(1, r % VST, tc1 + c1, c1 == 0, au1)) return false;
-                        tc_commit(bar(BAR_V_EMPTY + r % VST));
-                        if (c1 == n1 - 1) tc_commit(bar(BAR_O_DONE + 1));
-                        return true;
-                    };
-                    for (int k = 0; k < n0 && ok; ++k) {
-                        const int r0 = kv0 + 2 * k, r1 = r0 + 1;
-                        const bool has1 = 2 * k + 1 < ntiles;
-                        ok = mbar_wait(bar(BAR_K_FULL + r0 % KST), (r0 / KST) & 1, abort_flag, p.status);
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_qk(0, 0, r0 % KST);
-                        tc_commit(bar(BAR_S_FULL + 0));
-                        tc_commit(bar(BAR_K_EMPTY + r0 % KST));
-                        if (k > 0) {
-                            ok = finish_pv1(k - 1);
-                            if (!ok) break;
-                            pv1_issued = k;
-                        }
-                        if (has1) {
-                            ok = mbar_wait(bar(BAR_K_FULL + r1 % KST), (r1 / KST) & 1, abort_flag, p.status);
-                            if (!ok) break;
-                            tc_fence_after();
-                            issue_qk(1, 0, r1 % KST);
-                            tc_commit(bar(BAR_S_FULL + 1));
-                            tc_commit(bar(BAR_K_EMPTY + r1 % KST));
-                        }
-                        if (k == n0 - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
-                        ok = mbar_wait(bar(BAR_V_FULL + r0 % VST), (r0 / VST) & 1, abort_flag, p.status);
-                        if (!ok) break;
-                        ok = issue_pv(0, r0 % VST, tc0 + k, k == 0, au);
-                        if (!ok) break;
-                        tc_commit(bar(BAR_V_EMPTY + r0 % VST));
-                        if (k == n0 - 1) tc_commit(bar(BAR_O_DONE + 0));
-                    }
-                    if (ok && pv1_issued < n1) ok = finish_pv1(n1 - 1);
-                    kvc = kv0 + ntiles;
+                    issue_qk(1, 1, st);
+                    tc_commit(bar(BAR_S_FULL + 1));
+                    tc_commit(bar(BAR_K_EMPTY + st));
+                    if (idx == ntiles - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
+                    ok = wait(BAR_V_FULL + st, (kvc / VST) & 1);
+                    if (!ok) break;
+                    ok = issue_pv(0, st, tc0 + idx, idx == 0, au);
+                    if (!ok) break;
+                    if (idx == ntiles - 1) tc_commit(bar(BAR_O_DONE + 0));
+                    ++kvc;
                 }
+                if (ok) {
+                    ok = issue_pv(1, (kvc - 1) % VST, tc1 + ntiles - 1, ntiles == 1, au1);
+                    if (ok) {
+                        tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
+                        tc_commit(bar(BAR_O_DONE + 1));
+                    }
+                }
+            } else if (ok) {
+                // One row tile only: the two accumulator pairs take the even and the odd key
+                // tiles of the same rows (two independent partial attentions that the epilogue
+                // merges), so the softmax of one tile still runs under the MMAs of the next.
+                const int kv0 = kvc;
+                int pv1_issued = 0;
+                auto finish_pv1 = [&](int c1) -> bool {       // PV of stream 1's tile c1
+                    const int r = kv0 + 2 * c1 + 1;
+                    if (!wait(BAR_V_FULL + r % VST, (r / VST) & 1)) return false;
+                    if (!issue_pv(1, r % VST, tc1 + c1, c1 == 0, au1)) return false;
+                    tc_commit(bar(BAR_V_EMPTY + r % VST));
+                    if (c1 == n1 - 1) tc_commit(bar(BAR_O_DONE + 1));
+                    return true;
+                };
+                for (int k = 0; k < n0 && ok; ++k) {
+                    const int r0 = kv0 + 2 * k, r1 = r0 + 1;
+                    const bool has1 = 2 * k + 1 < ntiles;
+                    ok = wait(BAR_K_FULL + r0 % KST, (r0 / KST) & 1);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(0, 0, r0 % KST);
+                    tc_commit(bar(BAR_S_FULL + 0));
+                    tc_commit(bar(BAR_K_EMPTY + r0 % KST));
+                    if (k > 0) {
+                        ok = finish_pv1(k - 1);
+                        if (!ok) break;
+                        pv1_issued = k;
+                    }
+                    if (has1) {
+                        ok = wait(BAR_K_FULL + r1 % KST, (r1 / KST) & 1);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_qk(1, 0, r1 % KST);
+                        tc_commit(bar(BAR_S_FULL + 1));
+                        tc_commit(bar(BAR_K_EMPTY + r1 % KST));
+                    }
+                    if (k == n0 - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
+                    ok = wait(BAR_V_FULL + r0 % VST, (r0 / VST) & 1);
+                    if (!ok) break;
+                    ok = issue_pv(0, r0 % VST, tc0 + k, k == 0, au);
+                    if (!ok) break;
+                    tc_commit(bar(BAR_V_EMPTY + r0 % VST));
+                    if (k == n0 - 1) tc_commit(bar(BAR_O_DONE + 0));
+                }
+                if (ok && pv1_issued < n1) ok = finish_pv1(n1 - 1);
+                kvc = kv0 + ntiles;
             }
-            ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
-            kvc = __shfl_sync(0xFFFFFFFFu, kvc, 0);
             tc0 += n0;
             tc1 += n1;
             ++au;
