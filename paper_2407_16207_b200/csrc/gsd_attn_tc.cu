@@ -91,15 +91,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Non-blocking probe.  The MMA warp asks early and looks at the answer after it has issued
-// other work, so that the probe's latency is off its critical path.
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
 __device__ __forceinline__ unsigned long long global_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -522,59 +513,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             ok = wait(BAR_Q_FULL, au & 1);
             tc_fence_after();
             if (u.two) {
-                // Barriers whose completion is normally long past (K, V, the other row tile's P)
-                // are probed before the MMA group that precedes their use; the blocking wait is
-                // entered only if that early probe failed.
-                auto need = [&](bool pre, int b, uint32_t par) -> bool {
-                    return __all_sync(0xFFFFFFFFu, pre || mbar_wait(bar(b), par, abort_flag, p.status));
-                };
-                int st = kvc % KST;
-                uint32_t kpar = (uint32_t)(kvc / KST) & 1u;
-                bool kf = mbar_test(bar(BAR_K_FULL + st), kpar);
                 for (int idx = 0; idx < ntiles && ok; ++idx) {
-                    const int stp = st ^ 1;
-                    const uint32_t par1 = (uint32_t)(tc1 + idx - 1) & 1u, par0 = (uint32_t)(tc0 + idx) & 1u;
-                    const bool p1a = idx > 0 && mbar_test(bar(BAR_P_READY + 1), par1);
-                    if (!(ok = need(kf, BAR_K_FULL + st, kpar))) break;
+                    const int st = kvc % KST;
+                    ok = wait(BAR_K_FULL + st, (kvc / KST) & 1);
+                    if (!ok) break;
                     tc_fence_after();
                     issue_qk(0, 0, st);
                     tc_commit(bar(BAR_S_FULL + 0));
                     if (idx > 0) {
-                        const bool p1b = mbar_test(bar(BAR_P_READY2 + 1), par1);
-                        if (!(ok = need(p1a, BAR_P_READY + 1, par1))) break;
-                        if (idx == 1 && au1 > 0) {
-                            // the accumulator still belongs to the previous unit until its rows were read out
-                            if (!(ok = wait(BAR_O_FREE + 1, (au1 - 1) & 1))) break;
-                        }
-                        tc_fence_after();
-                        issue_pv_half(1, stp, 0, idx > 1);
-                        if (!(ok = need(p1b, BAR_P_READY2 + 1, par1))) break;
-                        tc_fence_after();
-                        issue_pv_half(1, stp, 1, idx > 1);
-                        tc_commit(bar(BAR_V_EMPTY + stp));
+                        ok = issue_pv(1, (kvc - 1) % VST, tc1 + idx - 1, idx == 1, au1);
+                        if (!ok) break;
+                        tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
                     }
-                    const bool vf = mbar_test(bar(BAR_V_FULL + st), kpar);
                     issue_qk(1, 1, st);
                     tc_commit(bar(BAR_S_FULL + 1));
                     tc_commit(bar(BAR_K_EMPTY + st));
                     if (idx == ntiles - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
-                    // the next tile's K: asked now, looked at after this tile's PV was issued
-                    const uint32_t kpar_next = kpar ^ (uint32_t)st;        // the parity flips when the ring wraps
-                    kf = mbar_test(bar(BAR_K_FULL + stp), kpar_next);
-                    if (!(ok = need(vf, BAR_V_FULL + st, kpar))) break;
-                    if (!(ok = wait(BAR_P_READY + 0, par0))) break;
-                    if (idx == 0 && au > 0) {
-                        if (!(ok = wait(BAR_O_FREE + 0, (au - 1) & 1))) break;
-                    }
-                    tc_fence_after();
-                    issue_pv_half(0, st, 0, idx > 0);
-                    if (!(ok = wait(BAR_P_READY2 + 0, par0))) break;
-                    tc_fence_after();
-                    issue_pv_half(0, st, 1, idx > 0);
+                    ok = wait(BAR_V_FULL + st, (kvc / VST) & 1);
+                    if (!ok) break;
+                    ok = issue_pv(0, st, tc0 + idx, idx == 0, au);
+                    if (!ok) break;
                     if (idx == ntiles - 1) tc_commit(bar(BAR_O_DONE + 0));
                     ++kvc;
-                    st = stp;
-                    kpar = kpar_next;
                 }
                 if (ok) {
                     ok = issue_pv(1, (kvc - 1) % VST, tc1 + ntiles - 1, ntiles == 1, au1);
