@@ -8,17 +8,23 @@
 // A unit of work is up to two row tiles of 128 stacked rows of one (sequence, kv head) and a
 // contiguous range of 128-key tiles (prefix tiles, then the draft tiles that hold a visible
 // key for any of its rows).  Warp roles:
-//   warps 0-3   softmax of row tile 0 (thread = row = TMEM lane)
-//   warps 4-7   softmax of row tile 1
+//   warps 0-3   softmax of stream 0 (thread = row = TMEM lane)
+//   warps 4-7   softmax of stream 1
 //   warp  8     TMA producer (one thread): Q once, then K and V tiles into two smem rings
-//   warp  9     MMA issuer (one thread): S_i = Q_i K^T into TMEM, O_i += P_i V with P read
-//               from TMEM (P overwrites the first half of S_i as bf16)
+//   warp  9     MMA issuer (converged, one elected lane per instruction)
 //   warp 10     TMEM allocation / release
-// The issue order QK0(j) PV1(j-1) QK1(j) PV0(j) lets the softmax of one row tile run under
-// the MMAs of the other.  The running maximum is only raised when a tile exceeds it by more
-// than 2^8 (the accumulator rescale is then done in place in TMEM by the row's own thread),
-// so P <= 256 and the rescale is rare.  Every mbarrier wait is bounded: on expiry the kernel
-// raises GSD_DEV_WAIT_EXPIRED, all roles leave their loops, TMEM is released.
+// A stream is a row tile (two row tiles: both streams see every key tile) or, for a unit with
+// one row tile, the even / odd key tiles of that row tile (merged in the epilogue).  A job is
+// one key tile of one stream; jobs alternate between the streams.
+// TMEM (512 columns): S (128) | P0 (64) | P1 (64) | O0 (128) | O1 (128).  There is one score
+// buffer: QK^T of job k+1 is issued as soon as the softmax of job k has pulled its score row
+// into registers, i.e. it runs under that softmax; P (bf16) has a buffer per stream and
+// O_i += P_i V follows when the softmax hands P over (in two halves of 64 keys).  So neither
+// softmax warpgroup ever waits for a QK^T that could not start, and the tensor pipe sees
+// QK(k+2), PV(k), QK(k+3), PV(k+1), ...  The running maximum is only raised when a tile
+// exceeds it by more than 2^8 (the accumulator rescale is then done in place in TMEM by the
+// row's own thread), so P <= 256 and the rescale is rare.  Every mbarrier wait is bounded: on
+// expiry the kernel raises GSD_DEV_WAIT_EXPIRED, all roles leave their loops, TMEM is released.
 #include "gsd_internal.cuh"
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -40,8 +46,8 @@ constexpr uint32_t kSmemBytes = (2 + KST + VST) * TILE_BYTES + 2 * HALF_BYTES + 
 constexpr float kRescaleThreshold = 8.0f;         // log2 units
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
-// TMEM columns (fp32 words): S0, S1, O0, O1; P_i lives in the first 64 columns of S_i
-constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O0 = 256, COL_O1 = 384;
+// TMEM columns (32-bit words): one score tile, a bf16 P tile per stream, an accumulator per stream
+constexpr uint32_t COL_S = 0, COL_P0 = 128, COL_P1 = 192, COL_O0 = 256, COL_O1 = 384;
 
 enum Bar {
     BAR_Q_FULL = 0,
@@ -49,10 +55,12 @@ enum Bar {
     BAR_K_EMPTY = BAR_K_FULL + KST,   // KST
     BAR_V_FULL = BAR_K_EMPTY + KST,   // VST
     BAR_V_EMPTY = BAR_V_FULL + VST,   // VST
-    BAR_S_FULL = BAR_V_EMPTY + VST,   // 2
-    BAR_P_READY = BAR_S_FULL + 2,     // 2: keys 0..63 of P are in TMEM
-    BAR_P_READY2 = BAR_P_READY + 2,   // 2: keys 64..127 of P are in TMEM
-    BAR_O_DONE = BAR_P_READY2 + 2,    // 2: every PV of the unit has completed
+    BAR_S_FULL = BAR_V_EMPTY + VST,   // 2: the scores of a job of stream i are in S
+    BAR_S_FREE = BAR_S_FULL + 2,      // 2: the softmax of stream i has read them out of S
+    BAR_P_READY = BAR_S_FREE + 2,     // 2: keys 0..63 of P_i are in TMEM
+    BAR_P_READY2 = BAR_P_READY + 2,   // 2: keys 64..127 of P_i are in TMEM
+    BAR_P_FREE = BAR_P_READY2 + 2,    // 2: the PV of a job of stream i (and all before it) has completed
+    BAR_O_DONE = BAR_P_FREE + 2,      // 2: every PV of the unit on stream i has completed
     BAR_O_FREE = BAR_O_DONE + 2,      // 2: the accumulator rows of the unit have been read out
     BAR_Q_EMPTY = BAR_O_FREE + 2,     // 1: every QK^T of the unit has completed
     BAR_ML_READY = BAR_Q_EMPTY + 1,   // 1: (max, sum) of the odd-tile stream are in shared memory
@@ -388,8 +396,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         for (int s = 0; s < VST; ++s) { mbar_init(bar(BAR_V_FULL + s), 1); mbar_init(bar(BAR_V_EMPTY + s), 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(BAR_S_FULL + i), 1);
-            mbar_init(bar(BAR_P_READY + i), 4);    // one arrival per softmax warp
+            mbar_init(bar(BAR_S_FREE + i), 4);     // one arrival per softmax warp
+            mbar_init(bar(BAR_P_READY + i), 4);
             mbar_init(bar(BAR_P_READY2 + i), 4);
+            mbar_init(bar(BAR_P_FREE + i), 1);
             mbar_init(bar(BAR_O_DONE + i), 1);
             mbar_init(bar(BAR_O_FREE + i), 4);
         }
@@ -464,134 +474,87 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
     } else if (warp == 9) {
         // ------------------------------------------------------------ MMA issuer (all lanes converged)
-        int kvc = 0;              // key tiles consumed so far (ring position)
-        int au = 0, au1 = 0;      // non-empty units so far; those of them in which stream 1 had tiles
-        int tc0 = 0, tc1 = 0;     // key tiles handed to the softmax of stream 0 / 1 so far
+        int kvc = 0;              // key tiles of earlier units (ring position of this unit's first tile)
+        int au = 0, au1 = 0;      // non-empty units so far; those of them in which stream 1 had jobs
+        int jq0 = 0, jq1 = 0;     // QK^T jobs issued per stream so far (phase of S_FULL / S_FREE)
+        int jp0 = 0, jp1 = 0;     // PV jobs issued per stream so far (phase of P_READY / P_FREE)
+        int s_owner = -1;         // stream whose scores were last written to S
         bool ok = true;
         auto wait = [&](int b, uint32_t par) -> bool { return mbar_wait_warp(bar(b), par, abort_flag, p.status); };
-        auto issue_qk = [&](int i, int qtile, int stage) {
-            // S_i = Q_qtile K^T : 8 k-steps of 16 over the head dimension
-            const uint32_t qa = sQ + qtile * TILE_BYTES, ka = sK + stage * TILE_BYTES;
-#pragma unroll
-            for (int ks = 0; ks < HD / 16; ++ks) {
-                const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
-                tc_mma_ss(tmem + (i ? COL_S1 : COL_S0), desc_kmajor(qa + off), desc_kmajor(ka + off), kIdescQK, ks > 0);
-            }
-        };
-        // O_i += P_i V : 8 k-steps of 16 keys; P (bf16 pairs) sits in S_i's first 64 columns.
-        // The softmax hands P over in two halves of 64 keys, so the first four k-steps run
-        // while the second half of the exponentials is still being computed.
-        auto issue_pv_half = [&](int i, int stage, int half, bool accumulate) {
-            const uint32_t va = sV + stage * TILE_BYTES;
-#pragma unroll
-            for (int k4 = 0; k4 < BN / 32; ++k4) {
-                const int ks = half * (BN / 32) + k4;
-                tc_mma_ts(tmem + (i ? COL_O1 : COL_O0), tmem + (i ? COL_S1 : COL_S0) + ks * 8,
-                          desc_mnmajor(va + ks * 2048), kIdescPV, (accumulate || ks > 0) ? 1u : 0u);
-            }
-        };
-        // tile = running tile number of row tile i (barrier phase); first = first tile of the unit
-        auto issue_pv = [&](int i, int stage, int tile, bool first, int units_before) -> bool {
-            if (!wait(BAR_P_READY + i, tile & 1)) return false;
-            if (first && units_before > 0) {
-                // the accumulator still belongs to the previous unit until its rows were read out
-                if (!wait(BAR_O_FREE + i, (units_before - 1) & 1)) return false;
-            }
-            tc_fence_after();
-            issue_pv_half(i, stage, 0, !first);
-            if (!wait(BAR_P_READY2 + i, tile & 1)) return false;
-            tc_fence_after();
-            issue_pv_half(i, stage, 1, !first);
-            return true;
-        };
         for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
             const UnitInfo u = unit_info(p, w, lane);
             if (u.ntiles == 0) continue;
-            const int n0 = u.two ? u.ntiles : (u.ntiles + 1) / 2;   // key tiles of stream 0 / stream 1
-            const int n1 = u.two ? u.ntiles : u.ntiles / 2;
+            const bool two = u.two;
             const int ntiles = u.ntiles;
+            const int njobs = two ? 2 * ntiles : ntiles;
+            const int n1 = two ? ntiles : ntiles / 2;          // jobs of stream 1
+            const int kv0 = kvc;
+            // S = Q K^T of job k: 8 k-steps of 16 over the head dimension
+            auto issue_qk = [&](int k) -> bool {
+                const int i = k & 1;
+                const int r = kv0 + (two ? (k >> 1) : k), st = r % KST;
+                if (!two || i == 0) {
+                    if (!wait(BAR_K_FULL + st, (r / KST) & 1)) return false;
+                }
+                if (s_owner >= 0) {
+                    // the previous job's scores must have left S
+                    if (!wait(BAR_S_FREE + s_owner, (uint32_t)((s_owner ? jq1 : jq0) - 1) & 1u)) return false;
+                }
+                tc_fence_after();
+                const uint32_t qa = sQ + (two ? i : 0) * TILE_BYTES, ka = sK + st * TILE_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < HD / 16; ++ks) {
+                    const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+                    tc_mma_ss(tmem + COL_S, desc_kmajor(qa + off), desc_kmajor(ka + off), kIdescQK, ks > 0);
+                }
+                tc_commit(bar(BAR_S_FULL + i));
+                if (!two || i == 1) tc_commit(bar(BAR_K_EMPTY + st));
+                if (k == njobs - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
+                s_owner = i;
+                if (i) ++jq1; else ++jq0;
+                return true;
+            };
+            // O_i += P_i V of job k: 8 k-steps of 16 keys, P (bf16 pairs) read from TMEM.  The
+            // softmax hands P over in two halves of 64 keys, so the first four k-steps run
+            // while the second half of the exponentials is still being computed.
+            auto issue_pv = [&](int k) -> bool {
+                const int i = k & 1;
+                const int r = kv0 + (two ? (k >> 1) : k), st = r % VST;
+                const bool first = k < 2;                          // first job of its stream in this unit
+                const uint32_t par = (uint32_t)(i ? jp1 : jp0) & 1u;
+                const uint32_t va = sV + st * TILE_BYTES;
+                const uint32_t tP = tmem + (i ? COL_P1 : COL_P0), tO = tmem + (i ? COL_O1 : COL_O0);
+                if (!two || i == 0) {
+                    if (!wait(BAR_V_FULL + st, (r / VST) & 1)) return false;
+                }
+                if (!wait(BAR_P_READY + i, par)) return false;
+                if (first && (i ? au1 : au) > 0) {
+                    // the accumulator still belongs to the previous unit until its rows were read out
+                    if (!wait(BAR_O_FREE + i, (uint32_t)((i ? au1 : au) - 1) & 1u)) return false;
+                }
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < BN / 32; ++ks)
+                    tc_mma_ts(tO, tP + ks * 8, desc_mnmajor(va + ks * 2048), kIdescPV, (!first || ks > 0) ? 1u : 0u);
+                if (!wait(BAR_P_READY2 + i, par)) return false;
+                tc_fence_after();
+#pragma unroll
+                for (int ks = BN / 32; ks < BN / 16; ++ks)
+                    tc_mma_ts(tO, tP + ks * 8, desc_mnmajor(va + ks * 2048), kIdescPV, 1u);
+                tc_commit(bar(BAR_P_FREE + i));
+                if (!two || i == 1) tc_commit(bar(BAR_V_EMPTY + st));
+                if (k + 2 >= njobs) tc_commit(bar(BAR_O_DONE + i));   // the stream's last job of the unit
+                if (i) ++jp1; else ++jp0;
+                return true;
+            };
             ok = wait(BAR_Q_FULL, au & 1);
-            tc_fence_after();
-            if (u.two) {
-                for (int idx = 0; idx < ntiles && ok; ++idx) {
-                    const int st = kvc % KST;
-                    ok = wait(BAR_K_FULL + st, (kvc / KST) & 1);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_qk(0, 0, st);
-                    tc_commit(bar(BAR_S_FULL + 0));
-                    if (idx > 0) {
-                        ok = issue_pv(1, (kvc - 1) % VST, tc1 + idx - 1, idx == 1, au1);
-                        if (!ok) break;
-                        tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
-                    }
-                    issue_qk(1, 1, st);
-                    tc_commit(bar(BAR_S_FULL + 1));
-                    tc_commit(bar(BAR_K_EMPTY + st));
-                    if (idx == ntiles - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
-                    ok = wait(BAR_V_FULL + st, (kvc / VST) & 1);
-                    if (!ok) break;
-                    ok = issue_pv(0, st, tc0 + idx, idx == 0, au);
-                    if (!ok) break;
-                    if (idx == ntiles - 1) tc_commit(bar(BAR_O_DONE + 0));
-                    ++kvc;
-                }
-                if (ok) {
-                    ok = issue_pv(1, (kvc - 1) % VST, tc1 + ntiles - 1, ntiles == 1, au1);
-                    if (ok) {
-                        tc_commit(bar(BAR_V_EMPTY + (kvc - 1) % VST));
-                        tc_commit(bar(BAR_O_DONE + 1));
-                    }
-                }
-            } else if (ok) {
-                // One row tile only: the two accumulator pairs take the even and the odd key
-                // tiles of the same rows (two independent partial attentions that the epilogue
-                // merges), so the softmax of one tile still runs under the MMAs of the next.
-                const int kv0 = kvc;
-                int pv1_issued = 0;
-                auto finish_pv1 = [&](int c1) -> bool {       // PV of stream 1's tile c1
-                    const int r = kv0 + 2 * c1 + 1;
-                    if (!wait(BAR_V_FULL + r % VST, (r / VST) & 1)) return false;
-                    if (!issue_pv(1, r % VST, tc1 + c1, c1 == 0, au1)) return false;
-                    tc_commit(bar(BAR_V_EMPTY + r % VST));
-                    if (c1 == n1 - 1) tc_commit(bar(BAR_O_DONE + 1));
-                    return true;
-                };
-                for (int k = 0; k < n0 && ok; ++k) {
-                    const int r0 = kv0 + 2 * k, r1 = r0 + 1;
-                    const bool has1 = 2 * k + 1 < ntiles;
-                    ok = wait(BAR_K_FULL + r0 % KST, (r0 / KST) & 1);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_qk(0, 0, r0 % KST);
-                    tc_commit(bar(BAR_S_FULL + 0));
-                    tc_commit(bar(BAR_K_EMPTY + r0 % KST));
-                    if (k > 0) {
-                        ok = finish_pv1(k - 1);
-                        if (!ok) break;
-                        pv1_issued = k;
-                    }
-                    if (has1) {
-                        ok = wait(BAR_K_FULL + r1 % KST, (r1 / KST) & 1);
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_qk(1, 0, r1 % KST);
-                        tc_commit(bar(BAR_S_FULL + 1));
-                        tc_commit(bar(BAR_K_EMPTY + r1 % KST));
-                    }
-                    if (k == n0 - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
-                    ok = wait(BAR_V_FULL + r0 % VST, (r0 / VST) & 1);
-                    if (!ok) break;
-                    ok = issue_pv(0, r0 % VST, tc0 + k, k == 0, au);
-                    if (!ok) break;
-                    tc_commit(bar(BAR_V_EMPTY + r0 % VST));
-                    if (k == n0 - 1) tc_commit(bar(BAR_O_DONE + 0));
-                }
-                if (ok && pv1_issued < n1) ok = finish_pv1(n1 - 1);
-                kvc = kv0 + ntiles;
+            if (ok) ok = issue_qk(0);
+            if (ok && njobs > 1) ok = issue_qk(1);
+            for (int k = 0; k < njobs && ok; ++k) {
+                if (k + 2 < njobs) ok = issue_qk(k + 2);
+                if (ok) ok = issue_pv(k);
             }
-            tc0 += n0;
-            tc1 += n1;
+            kvc = kv0 + ntiles;
             ++au;
             if (n1 > 0) ++au1;
         }
@@ -599,15 +562,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
         // ------------------------------------------------------------ softmax + epilogue
-        const int i = warp >> 2;                         // row tile of this warpgroup
+        const int i = warp >> 2;                         // stream of this warpgroup
         const int rloc = (warp & 3) * 32 + lane;         // row inside the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem + lane_addr + (i ? COL_S1 : COL_S0);
+        const uint32_t tS = tmem + lane_addr + COL_S;
+        const uint32_t tP = tmem + lane_addr + (i ? COL_P1 : COL_P0);
         const uint32_t tO = tmem + lane_addr + (i ? COL_O1 : COL_O0);
         int kvc = 0;      // key tiles of all non-empty units so far (ring position of the V tiles)
-        int tcnt = 0;     // key tiles this row tile has processed so far (barrier phase)
+        int tcnt = 0;     // jobs this stream has processed so far (barrier phase)
         int auc = 0;      // non-empty units this stream has finished so far (barrier phase)
-        int auc1 = 0;     // units in which stream 1 had tiles (phase of its barriers as seen by warpgroup 0)
+        int auc1 = 0;     // units in which stream 1 had jobs (phase of its barriers as seen by warpgroup 0)
         int mlc = 0;      // single-row-tile units whose odd-tile stream had tiles
         bool ok = true;
         for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
@@ -661,6 +625,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) tc_ld32p(tS + ch * 32, sc + ch * 32);
                 tc_wait_ld();
+                tc_fence_before();
+                if (lane == 0) mbar_arrive(bar(BAR_S_FREE + i));   // the next job's QK^T may overwrite S
                 if (ti.kind != 0) {
 #pragma unroll
                     for (int e = 0; e < BN; ++e) sc[e] = ((mw[e >> 5] >> (e & 31)) & 1u) ? sc[e] : -CUDART_INF_F;
@@ -683,8 +649,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     need = true;
                 }
                 if (__any_sync(0xFFFFFFFFu, need)) {
-                    // the accumulator of this row is final for all earlier tiles (MMAs complete in
-                    // order and S of this tile is complete): rescale it in place
+                    // once the PV of this stream's previous job has completed, the accumulator of
+                    // this row is final for all earlier tiles: rescale it in place
+                    ok = mbar_wait(bar(BAR_P_FREE + i), (uint32_t)((tcnt + cnt - 1) & 1), abort_flag, p.status);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
 #pragma unroll 1
                     for (int ch = 0; ch < 4; ++ch) {
                         float v[32];
@@ -716,8 +686,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
-                // P = 2^(s*scale - m) as bf16 pairs into the first 64 columns of S; a masked
-                // score is -inf and comes out as exactly 0
+                // P = 2^(s*scale - m) as bf16 pairs into the 64 columns of P_i; a masked score is
+                // -inf and comes out as exactly 0
                 const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
                 const float2 negm2 = make_float2(-m_use, -m_use);
                 float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
@@ -735,15 +705,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 // computed; the hand-off of a half follows once its stores have landed.
                 exp_chunk(0);
                 exp_chunk(1);
-                tc_st16(tS + 0, pk[0]);
-                tc_st16(tS + 16, pk[1]);
+                if (tcnt + cnt > 0) {
+                    // P_i is still being read until the PV of this stream's previous job has completed
+                    ok = mbar_wait(bar(BAR_P_FREE + i), (uint32_t)((tcnt + cnt - 1) & 1), abort_flag, p.status);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+                tc_st16(tP + 0, pk[0]);
+                tc_st16(tP + 16, pk[1]);
                 exp_chunk(2);
                 tc_wait_st();              // keys 0..63 are in place (and any rescale of O is done)
                 tc_fence_before();
                 if (lane == 0) mbar_arrive(bar(BAR_P_READY + i));
                 exp_chunk(3);
-                tc_st16(tS + 32, pk[2]);
-                tc_st16(tS + 48, pk[3]);
+                tc_st16(tP + 32, pk[2]);
+                tc_st16(tP + 48, pk[3]);
                 l_run += (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
                 tc_wait_st();
                 tc_fence_before();
