@@ -11,7 +11,7 @@
 //   warps 0-3   softmax of stream 0 (thread = row = TMEM lane)
 //   warps 4-7   softmax of stream 1
 //   warp  8     TMA producer (one thread): Q once, then K and V tiles into two smem rings
-//   warp  9     MMA issuer (converged, one elected lane per instruction)
+//   warp  9     QK^T issuer, warp 11 PV issuer (converged, one elected lane per instruction)
 //   warp 10     TMEM allocation / release
 // A stream is a row tile (two row tiles: both streams see every key tile) or, for a unit with
 // one row tile, the even / odd key tiles of that row tile (merged in the epilogue).  A job is
@@ -20,8 +20,10 @@
 // buffer: QK^T of job k+1 is issued as soon as the softmax of job k has pulled its score row
 // into registers, i.e. it runs under that softmax; P (bf16) has a buffer per stream and
 // O_i += P_i V follows when the softmax hands P over (in two halves of 64 keys).  So neither
-// softmax warpgroup ever waits for a QK^T that could not start, and the tensor pipe sees
-// QK(k+2), PV(k), QK(k+3), PV(k+1), ...  The running maximum is only raised when a tile
+// softmax warpgroup ever waits for a QK^T that could not start.  The two kinds of MMA are
+// issued by two warps on different schedulers, each paced only by its own barriers (the
+// softmax warps are almost always ready to issue, so one issuing warp gets too few slots
+// to feed the tensor pipe).  The running maximum is only raised when a tile
 // exceeds it by more than 2^8 (the accumulator rescale is then done in place in TMEM by the
 // row's own thread), so P <= 256 and the rescale is rare.  Every mbarrier wait is bounded: on
 // expiry the kernel raises GSD_DEV_WAIT_EXPIRED, all roles leave their loops, TMEM is released.
@@ -473,11 +475,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             ++au;
         }
     } else if (warp == 9) {
-        // ------------------------------------------------------------ MMA issuer (all lanes converged)
+        // ------------------------------------------------------------ QK^T issuer (all lanes converged)
+        // S = Q K^T job by job.  Nothing orders these MMAs against the PV MMAs of warp 11 in the
+        // tensor pipe, and nothing has to: they touch different TMEM columns, and every
+        // hand-over (S to the softmax, P to the PV, S back) goes through an mbarrier.
         int kvc = 0;              // key tiles of earlier units (ring position of this unit's first tile)
-        int au = 0, au1 = 0;      // non-empty units so far; those of them in which stream 1 had jobs
-        int jq0 = 0, jq1 = 0;     // QK^T jobs issued per stream so far (phase of S_FULL / S_FREE)
-        int jp0 = 0, jp1 = 0;     // PV jobs issued per stream so far (phase of P_READY / P_FREE)
+        int au = 0;               // non-empty units so far
+        int jq0 = 0, jq1 = 0;     // jobs issued per stream so far (phase of S_FULL / S_FREE)
         int s_owner = -1;         // stream whose scores were last written to S
         bool ok = true;
         auto wait = [&](int b, uint32_t par) -> bool { return mbar_wait_warp(bar(b), par, abort_flag, p.status); };
@@ -485,25 +489,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             const UnitInfo u = unit_info(p, w, lane);
             if (u.ntiles == 0) continue;
             const bool two = u.two;
-            const int ntiles = u.ntiles;
-            const int njobs = two ? 2 * ntiles : ntiles;
-            const int n1 = two ? ntiles : ntiles / 2;          // jobs of stream 1
-            const int kv0 = kvc;
-            // S = Q K^T of job k: 8 k-steps of 16 over the head dimension
-            auto issue_qk = [&](int k) -> bool {
+            const int njobs = two ? 2 * u.ntiles : u.ntiles;
+            ok = wait(BAR_Q_FULL, au & 1);
+            for (int k = 0; k < njobs && ok; ++k) {
                 const int i = k & 1;
-                const int r = kv0 + (two ? (k >> 1) : k), st = r % KST;
+                const int r = kvc + (two ? (k >> 1) : k), st = r % KST;
                 if (!two || i == 0) {
-                    if (!wait(BAR_K_FULL + st, (r / KST) & 1)) return false;
+                    if (!(ok = wait(BAR_K_FULL + st, (r / KST) & 1))) break;
                 }
                 if (s_owner >= 0) {
                     // the previous job's scores must have left S
-                    if (!wait(BAR_S_FREE + s_owner, (uint32_t)((s_owner ? jq1 : jq0) - 1) & 1u)) return false;
+                    if (!(ok = wait(BAR_S_FREE + s_owner, (uint32_t)((s_owner ? jq1 : jq0) - 1) & 1u))) break;
                 }
                 tc_fence_after();
                 const uint32_t qa = sQ + (two ? i : 0) * TILE_BYTES, ka = sK + st * TILE_BYTES;
 #pragma unroll
-                for (int ks = 0; ks < HD / 16; ++ks) {
+                for (int ks = 0; ks < HD / 16; ++ks) {     // 8 k-steps of 16 over the head dimension
                     const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
                     tc_mma_ss(tmem + COL_S, desc_kmajor(qa + off), desc_kmajor(ka + off), kIdescQK, ks > 0);
                 }
@@ -512,31 +513,46 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (k == njobs - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
                 s_owner = i;
                 if (i) ++jq1; else ++jq0;
-                return true;
-            };
-            // O_i += P_i V of job k: 8 k-steps of 16 keys, P (bf16 pairs) read from TMEM.  The
-            // softmax hands P over in two halves of 64 keys, so the first four k-steps run
-            // while the second half of the exponentials is still being computed.
-            auto issue_pv = [&](int k) -> bool {
+            }
+            kvc += u.ntiles;
+            ++au;
+        }
+    } else if (warp == 11) {
+        // ------------------------------------------------------------ PV issuer (all lanes converged)
+        // O_i += P_i V job by job: 8 k-steps of 16 keys, P (bf16 pairs) read from TMEM.  The
+        // softmax hands P over in two halves of 64 keys, so the first four k-steps run while
+        // the second half of the exponentials is still being computed.
+        int kvc = 0;
+        int au = 0, au1 = 0;      // non-empty units so far; those of them in which stream 1 had jobs
+        int jp0 = 0, jp1 = 0;     // jobs issued per stream so far (phase of P_READY / P_FREE)
+        bool ok = true;
+        auto wait = [&](int b, uint32_t par) -> bool { return mbar_wait_warp(bar(b), par, abort_flag, p.status); };
+        for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+            const UnitInfo u = unit_info(p, w, lane);
+            if (u.ntiles == 0) continue;
+            const bool two = u.two;
+            const int njobs = two ? 2 * u.ntiles : u.ntiles;
+            const int n1 = two ? u.ntiles : u.ntiles / 2;      // jobs of stream 1
+            for (int k = 0; k < njobs && ok; ++k) {
                 const int i = k & 1;
-                const int r = kv0 + (two ? (k >> 1) : k), st = r % VST;
-                const bool first = k < 2;                          // first job of its stream in this unit
+                const int r = kvc + (two ? (k >> 1) : k), st = r % VST;
+                const bool first = k < 2;                      // first job of its stream in this unit
                 const uint32_t par = (uint32_t)(i ? jp1 : jp0) & 1u;
                 const uint32_t va = sV + st * TILE_BYTES;
                 const uint32_t tP = tmem + (i ? COL_P1 : COL_P0), tO = tmem + (i ? COL_O1 : COL_O0);
                 if (!two || i == 0) {
-                    if (!wait(BAR_V_FULL + st, (r / VST) & 1)) return false;
+                    if (!(ok = wait(BAR_V_FULL + st, (r / VST) & 1))) break;
                 }
-                if (!wait(BAR_P_READY + i, par)) return false;
+                if (!(ok = wait(BAR_P_READY + i, par))) break;
                 if (first && (i ? au1 : au) > 0) {
                     // the accumulator still belongs to the previous unit until its rows were read out
-                    if (!wait(BAR_O_FREE + i, (uint32_t)((i ? au1 : au) - 1) & 1u)) return false;
+                    if (!(ok = wait(BAR_O_FREE + i, (uint32_t)((i ? au1 : au) - 1) & 1u))) break;
                 }
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < BN / 32; ++ks)
                     tc_mma_ts(tO, tP + ks * 8, desc_mnmajor(va + ks * 2048), kIdescPV, (!first || ks > 0) ? 1u : 0u);
-                if (!wait(BAR_P_READY2 + i, par)) return false;
+                if (!(ok = wait(BAR_P_READY2 + i, par))) break;
                 tc_fence_after();
 #pragma unroll
                 for (int ks = BN / 32; ks < BN / 16; ++ks)
@@ -545,16 +561,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (!two || i == 1) tc_commit(bar(BAR_V_EMPTY + st));
                 if (k + 2 >= njobs) tc_commit(bar(BAR_O_DONE + i));   // the stream's last job of the unit
                 if (i) ++jp1; else ++jp0;
-                return true;
-            };
-            ok = wait(BAR_Q_FULL, au & 1);
-            if (ok) ok = issue_qk(0);
-            if (ok && njobs > 1) ok = issue_qk(1);
-            for (int k = 0; k < njobs && ok; ++k) {
-                if (k + 2 < njobs) ok = issue_qk(k + 2);
-                if (ok) ok = issue_pv(k);
             }
-            kvc = kv0 + ntiles;
+            kvc += u.ntiles;
             ++au;
             if (n1 > 0) ++au1;
         }
