@@ -167,21 +167,6 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
         "{\n .reg .pred q;\n elect.sync _|q, 0xffffffff;\n"
         " @q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}\n" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem desc] * B[smem desc]
-__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
-    asm volatile(
-        "{\n .reg .pred p, q;\n elect.sync _|q, 0xffffffff;\n setp.ne.b32 p, %4, 0;\n"
-        " @q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem desc]
-__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
-    asm volatile(
-        "{\n .reg .pred p, q;\n elect.sync _|q, 0xffffffff;\n setp.ne.b32 p, %4, 0;\n"
-        " @q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
-}
-
 // 32 lanes x 32 consecutive fp32 columns: thread t of the warp gets lane (base + t)
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
     uint32_t* r = reinterpret_cast<uint32_t*>(v);
@@ -262,19 +247,53 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 // ---- shared-memory matrix descriptors (128-byte swizzle, 8-row groups 1024 bytes apart)
 constexpr uint64_t kDescBase = (1ull << 46) | (2ull << 61);   // descriptor version 1, SWIZZLE_128B
-// K-major operand (rows x 64 bf16 per block): leading offset unused (1), stride = 1024 B
-__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
-    return kDescBase | (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32);
-}
+// K-major operand (rows x 64 bf16 per block): leading offset unused (1), stride = 1024 B.
 // MN-major operand (V: [key][64 d] blocks): leading offset = distance between the two
-// 64-column blocks, stride = 1024 B between 8-key groups
-__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
-    return kDescBase | (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(HALF_BYTES >> 4) << 16) |
-           ((uint64_t)(1024 >> 4) << 32);
-}
+// 64-column blocks, stride = 1024 B between 8-key groups.
+// Descriptors are handled as (low word, high word): the high word is common to both kinds, and
+// a k-step only adds a small constant to the start-address field of the low word (the
+// tiles sit below 256 KB, so the sum stays inside the 14-bit field).
+constexpr uint32_t kDescHi = (uint32_t)((kDescBase | ((uint64_t)(1024 >> 4) << 32)) >> 32);
+__device__ __forceinline__ uint32_t desc_lo_kmajor(uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | (1u << 16); }
+__device__ __forceinline__ uint32_t desc_lo_mnmajor(uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | ((HALF_BYTES >> 4) << 16); }
 // instruction descriptors: bf16 x bf16 -> fp32, M = 128, N = 128
 constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);   // B (= V) is MN-major
+
+// S = A B^T over the head dimension (eight k-steps of 16) as one block issued by one elected
+// lane: per k-step one add per operand and the MMA, nothing else.  alo / blo are the low
+// descriptor words of two K-major [128][128] bf16 tiles (two swizzled 64-column blocks each).
+__device__ __forceinline__ void tc_qk8(uint32_t d_tmem, uint32_t alo, uint32_t blo) {
+#define GSD_QK_STEP(OFF, P)                                                         \
+    " add.u32 al, %1, " #OFF ";\n add.u32 bl, %2, " #OFF ";\n"                       \
+    " mov.b64 a, {al, %3};\n mov.b64 b, {bl, %3};\n"                                \
+    " @q tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %4, " #P ";\n"
+    asm volatile(
+        "{\n .reg .pred q, pt, pf;\n .reg .b64 a, b;\n .reg .b32 al, bl;\n"
+        " elect.sync _|q, 0xffffffff;\n"
+        " setp.eq.u32 pt, %4, %4;\n setp.ne.u32 pf, %4, %4;\n"
+        GSD_QK_STEP(0, pf) GSD_QK_STEP(2, pt) GSD_QK_STEP(4, pt) GSD_QK_STEP(6, pt)
+        GSD_QK_STEP(1024, pt) GSD_QK_STEP(1026, pt) GSD_QK_STEP(1028, pt) GSD_QK_STEP(1030, pt)
+        "}\n"
+        ::"r"(d_tmem), "r"(alo), "r"(blo), "r"(kDescHi), "r"(kIdescQK) : "memory");
+#undef GSD_QK_STEP
+}
+// O (+)= P V for four k-steps of 16 keys: A = 8 TMEM columns of bf16 pairs per step, B = the
+// MN-major V tile (2048 bytes per 16 keys).  `accum_first` = 0 makes the first step overwrite O.
+__device__ __forceinline__ void tc_pv4(uint32_t d_tmem, uint32_t a_tmem, uint32_t blo, uint32_t accum_first) {
+#define GSD_PV_STEP(ACOL, BOFF, P)                                                  \
+    " add.u32 at, %1, " #ACOL ";\n add.u32 bl, %2, " #BOFF ";\n mov.b64 b, {bl, %3};\n" \
+    " @q tcgen05.mma.cta_group::1.kind::f16 [%0], [at], b, %4, " #P ";\n"
+    asm volatile(
+        "{\n .reg .pred q, pt, p0;\n .reg .b64 b;\n .reg .b32 at, bl;\n"
+        " elect.sync _|q, 0xffffffff;\n"
+        " setp.eq.u32 pt, %4, %4;\n setp.ne.u32 p0, %5, 0;\n"
+        GSD_PV_STEP(0, 0, p0) GSD_PV_STEP(8, 128, pt) GSD_PV_STEP(16, 256, pt) GSD_PV_STEP(24, 384, pt)
+        "}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(blo), "r"(kDescHi), "r"(kIdescPV), "r"(accum_first) : "memory");
+#undef GSD_PV_STEP
+}
+
 
 struct TileInfo {
     int kind;     // 0 full prefix tile, 1 ragged prefix tile, 2 draft tile
@@ -485,6 +504,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         int s_owner = -1;         // stream whose scores were last written to S
         bool ok = true;
         auto wait = [&](int b, uint32_t par) -> bool { return mbar_wait_warp(bar(b), par, abort_flag, p.status); };
+        static_assert(KST == 2, "two K stages are selected by a flag");
+        const uint32_t qlo0 = desc_lo_kmajor(sQ), qlo1 = desc_lo_kmajor(sQ + TILE_BYTES);
+        const uint32_t klo0 = desc_lo_kmajor(sK), klo1 = desc_lo_kmajor(sK + TILE_BYTES);
         for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
             const UnitInfo u = unit_info(p, w, lane);
             if (u.ntiles == 0) continue;
@@ -502,12 +524,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     if (!(ok = wait(BAR_S_FREE + s_owner, (uint32_t)((s_owner ? jq1 : jq0) - 1) & 1u))) break;
                 }
                 tc_fence_after();
-                const uint32_t qa = sQ + (two ? i : 0) * TILE_BYTES, ka = sK + st * TILE_BYTES;
-#pragma unroll
-                for (int ks = 0; ks < HD / 16; ++ks) {     // 8 k-steps of 16 over the head dimension
-                    const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
-                    tc_mma_ss(tmem + COL_S, desc_kmajor(qa + off), desc_kmajor(ka + off), kIdescQK, ks > 0);
-                }
+                tc_qk8(tmem + COL_S, (two && i) ? qlo1 : qlo0, st ? klo1 : klo0);
                 tc_commit(bar(BAR_S_FULL + i));
                 if (!two || i == 1) tc_commit(bar(BAR_K_EMPTY + st));
                 if (k == njobs - 1) tc_commit(bar(BAR_Q_EMPTY));   // every QK^T of the unit is issued
@@ -527,6 +544,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         int jp0 = 0, jp1 = 0;     // jobs issued per stream so far (phase of P_READY / P_FREE)
         bool ok = true;
         auto wait = [&](int b, uint32_t par) -> bool { return mbar_wait_warp(bar(b), par, abort_flag, p.status); };
+        static_assert(VST == 2, "two V stages are selected by a flag");
+        const uint32_t vlo0 = desc_lo_mnmajor(sV), vlo1 = desc_lo_mnmajor(sV + TILE_BYTES);
         for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
             const UnitInfo u = unit_info(p, w, lane);
             if (u.ntiles == 0) continue;
@@ -538,7 +557,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const int r = kvc + (two ? (k >> 1) : k), st = r % VST;
                 const bool first = k < 2;                      // first job of its stream in this unit
                 const uint32_t par = (uint32_t)(i ? jp1 : jp0) & 1u;
-                const uint32_t va = sV + st * TILE_BYTES;
+                const uint32_t vlo = st ? vlo1 : vlo0;
                 const uint32_t tP = tmem + (i ? COL_P1 : COL_P0), tO = tmem + (i ? COL_O1 : COL_O0);
                 if (!two || i == 0) {
                     if (!(ok = wait(BAR_V_FULL + st, (r / VST) & 1))) break;
@@ -549,14 +568,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     if (!(ok = wait(BAR_O_FREE + i, (uint32_t)((i ? au1 : au) - 1) & 1u))) break;
                 }
                 tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < BN / 32; ++ks)
-                    tc_mma_ts(tO, tP + ks * 8, desc_mnmajor(va + ks * 2048), kIdescPV, (!first || ks > 0) ? 1u : 0u);
+                tc_pv4(tO, tP, vlo, first ? 0u : 1u);
                 if (!(ok = wait(BAR_P_READY2 + i, par))) break;
                 tc_fence_after();
-#pragma unroll
-                for (int ks = BN / 32; ks < BN / 16; ++ks)
-                    tc_mma_ts(tO, tP + ks * 8, desc_mnmajor(va + ks * 2048), kIdescPV, 1u);
+                tc_pv4(tO, tP + 32, vlo + 4 * 128, 1u);
                 tc_commit(bar(BAR_P_FREE + i));
                 if (!two || i == 1) tc_commit(bar(BAR_V_EMPTY + st));
                 if (k + 2 >= njobs) tc_commit(bar(BAR_O_DONE + i));   // the stream's last job of the unit
