@@ -46,6 +46,7 @@ constexpr uint32_t TILE_BYTES = 2 * HALF_BYTES;   // a 128 x 128 bf16 tile (two 
 constexpr int kThreads = 384;
 constexpr uint32_t kSmemBytes = (2 + KST + VST) * TILE_BYTES + 2 * HALF_BYTES + 1024;  // tiles, output staging, alignment slack
 constexpr float kRescaleThreshold = 8.0f;         // log2 units
+constexpr int kUnitTable = 12;                    // units of work per CTA decoded in the prologue (one per warp)
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 // TMEM columns (32-bit words): one score tile, a bf16 P tile per stream, an accumulator per stream
@@ -395,6 +396,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     __shared__ float2 s_ml1[BM];      // (max, sum) of the odd-tile stream, one per row
+    __shared__ UnitInfo s_units[kUnitTable];   // the CTA's first units of work, decoded once up front
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int N = p.N, G = p.G, R = p.R;
@@ -430,11 +432,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&s_tmem_base)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    const int total_work = p.total_work;
+    // Decoding a unit costs two dependent trips to global memory (sequence length, mask rows).
+    // Each warp decodes one of the CTA's first units here, all at once, so that no role pays
+    // that latency between units.
+    for (int k = warp; k < kUnitTable; k += kThreads / 32) {
+        const int w = blockIdx.x + k * gridDim.x;
+        if (w < total_work) {
+            const UnitInfo u = unit_info(p, w, lane);
+            if (lane == 0) s_units[k] = u;
+        }
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem_base;
-    const int total_work = p.total_work;
+    auto unit_of = [&](int w, int it) -> UnitInfo { return it < kUnitTable ? s_units[it] : unit_info(p, w, lane); };
 
     if (warp >= 8) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 96;");
@@ -443,8 +456,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         int kvc = 0;          // key tiles loaded so far (ring position)
         int au = 0;           // non-empty units so far
         bool ok = true, q_pending = false;
-        for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
-            const UnitInfo u = unit_info(p, w, lane);
+        for (int w = blockIdx.x, it = 0; w < total_work && ok; w += gridDim.x, ++it) {
+            const UnitInfo u = unit_of(w, it);
             if (u.ntiles == 0) continue;
             if (lane == 0) {
                 // Q of the previous unit is free once its last QK^T has completed
@@ -507,8 +520,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         static_assert(KST == 2, "two K stages are selected by a flag");
         const uint32_t qlo0 = desc_lo_kmajor(sQ), qlo1 = desc_lo_kmajor(sQ + TILE_BYTES);
         const uint32_t klo0 = desc_lo_kmajor(sK), klo1 = desc_lo_kmajor(sK + TILE_BYTES);
-        for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
-            const UnitInfo u = unit_info(p, w, lane);
+        for (int w = blockIdx.x, it = 0; w < total_work && ok; w += gridDim.x, ++it) {
+            const UnitInfo u = unit_of(w, it);
             if (u.ntiles == 0) continue;
             const bool two = u.two;
             const int njobs = two ? 2 * u.ntiles : u.ntiles;
@@ -546,8 +559,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         auto wait = [&](int b, uint32_t par) -> bool { return mbar_wait_warp(bar(b), par, abort_flag, p.status); };
         static_assert(VST == 2, "two V stages are selected by a flag");
         const uint32_t vlo0 = desc_lo_mnmajor(sV), vlo1 = desc_lo_mnmajor(sV + TILE_BYTES);
-        for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
-            const UnitInfo u = unit_info(p, w, lane);
+        for (int w = blockIdx.x, it = 0; w < total_work && ok; w += gridDim.x, ++it) {
+            const UnitInfo u = unit_of(w, it);
             if (u.ntiles == 0) continue;
             const bool two = u.two;
             const int njobs = two ? 2 * u.ntiles : u.ntiles;
@@ -597,8 +610,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         int auc1 = 0;     // units in which stream 1 had jobs (phase of its barriers as seen by warpgroup 0)
         int mlc = 0;      // single-row-tile units whose odd-tile stream had tiles
         bool ok = true;
-        for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
-            const UnitInfo u = unit_info(p, w, lane);
+        for (int w = blockIdx.x, it = 0; w < total_work && ok; w += gridDim.x, ++it) {
+            const UnitInfo u = unit_of(w, it);
             const int ntiles = u.ntiles;
             // with one row tile only, the two warpgroups take the even / odd key tiles of the
             // same rows and warpgroup 0 merges the two partial results in the epilogue
@@ -654,13 +667,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
                     for (int e = 0; e < BN; ++e) sc[e] = ((mw[e >> 5] >> (e & 31)) & 1u) ? sc[e] : -CUDART_INF_F;
                 }
-                float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+                // row maximum: 16 independent chains of 3-input max, then a tree
+                float mx16[16];
 #pragma unroll
-                for (int e = 0; e < BN; e += 8) {
+                for (int k = 0; k < 16; ++k) mx16[k] = max3(sc[2 * k], sc[2 * k + 1], sc[32 + 2 * k]);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) mx4[k] = max3(mx4[k], sc[e + 2 * k], sc[e + 2 * k + 1]);
-                }
-                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                for (int k = 0; k < 16; ++k) mx16[k] = max3(mx16[k], sc[33 + 2 * k], sc[64 + 2 * k]);
+#pragma unroll
+                for (int k = 0; k < 16; ++k) mx16[k] = max3(mx16[k], sc[65 + 2 * k], sc[96 + 2 * k]);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) mx16[k] = max3(mx16[k], mx16[k + 8], sc[97 + 2 * k]);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) mx16[k] = fmaxf(mx16[k], sc[113 + 2 * k]);
+                const float mx = fmaxf(max3(mx16[0], mx16[1], mx16[2]), fmaxf(max3(mx16[3], mx16[4], mx16[5]), fmaxf(mx16[6], mx16[7])));
                 const float m_tile = mx * p.scale_log2;     // scale > 0 keeps the order
                 float m_new = m_ref, alpha = 1.f;
                 bool need = false;
