@@ -667,19 +667,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
                     for (int e = 0; e < BN; ++e) sc[e] = ((mw[e >> 5] >> (e & 31)) & 1u) ? sc[e] : -CUDART_INF_F;
                 }
-                // row maximum: 16 independent chains of 3-input max, then a tree
-                float mx16[16];
+                float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
-                for (int k = 0; k < 16; ++k) mx16[k] = max3(sc[2 * k], sc[2 * k + 1], sc[32 + 2 * k]);
+                for (int e = 0; e < BN; e += 8) {
 #pragma unroll
-                for (int k = 0; k < 16; ++k) mx16[k] = max3(mx16[k], sc[33 + 2 * k], sc[64 + 2 * k]);
-#pragma unroll
-                for (int k = 0; k < 16; ++k) mx16[k] = max3(mx16[k], sc[65 + 2 * k], sc[96 + 2 * k]);
-#pragma unroll
-                for (int k = 0; k < 8; ++k) mx16[k] = max3(mx16[k], mx16[k + 8], sc[97 + 2 * k]);
-#pragma unroll
-                for (int k = 0; k < 8; ++k) mx16[k] = fmaxf(mx16[k], sc[113 + 2 * k]);
-                const float mx = fmaxf(max3(mx16[0], mx16[1], mx16[2]), fmaxf(max3(mx16[3], mx16[4], mx16[5]), fmaxf(mx16[6], mx16[7])));
+                    for (int k = 0; k < 4; ++k) mx4[k] = max3(mx4[k], sc[e + 2 * k], sc[e + 2 * k + 1]);
+                }
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 const float m_tile = mx * p.scale_log2;     // scale > 0 keeps the order
                 float m_new = m_ref, alpha = 1.f;
                 bool need = false;
