@@ -726,14 +726,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 // -inf and comes out as exactly 0
                 const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
                 const float2 negm2 = make_float2(-m_use, -m_use);
-                float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                float2 sum2[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};   // four chains
                 uint32_t pk[4][16];
                 auto exp_chunk = [&](int ch) {
 #pragma unroll
                     for (int e = 0; e < 16; ++e) {
                         const float2 t = ffma2(make_float2(sc[ch * 32 + 2 * e], sc[ch * 32 + 2 * e + 1]), scale2, negm2);
                         const float2 pe = make_float2(fast_exp2(t.x), fast_exp2(t.y));
-                        sum2[e & 1] = fadd2(sum2[e & 1], pe);
+                        sum2[e & 3] = fadd2(sum2[e & 3], pe);
                         pk[ch][e] = pack_bf16(pe.x, pe.y);
                     }
                 };
@@ -757,7 +757,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 exp_chunk(3);
                 tc_st16(tP + 32, pk[2]);
                 tc_st16(tP + 48, pk[3]);
-                l_run += (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
+                l_run += ((sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y)) + ((sum2[2].x + sum2[2].y) + (sum2[3].x + sum2[3].y));
                 tc_wait_st();
                 tc_fence_before();
                 if (lane == 0) mbar_arrive(bar(BAR_P_READY2 + i));
