@@ -368,6 +368,9 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(MergeParams p) {
     const int row = (item % p.plan.tiles_per_unit) * p.rows_per_item + rloc;
     if (row >= p.R) return;
     const int b = unit / p.Hkv, c = unit % p.Hkv;
+    // Launched as a programmatic dependent of the attention kernel: the blocks may become
+    // resident while that kernel drains; its partial results are only visible after this wait.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // Loads are issued in groups of four before any of them is used, so that a row costs a few
     // memory round trips instead of two per split.
     const float* ml_base = p.part_ml + ((size_t)slot0 * p.rows_per_item + rloc) * 2;
@@ -467,8 +470,17 @@ int launch_attn_merge(const AttnArgs& a) {
     if (p.warps_total == 0) return GSD_OK;
     const int warps = 8;
     const long blocks = (p.warps_total + warps - 1) / warps;
-    attn_merge_kernel<<<(unsigned)blocks, warps * 32, 0, a.stream>>>(p);
-    GSD_CUDA_TRY(cudaGetLastError());
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(warps * 32);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = a.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    GSD_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_merge_kernel, p));
     return GSD_OK;
 }
 

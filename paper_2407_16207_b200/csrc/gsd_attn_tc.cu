@@ -411,6 +411,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     volatile int* abort_flag = &s_abort;
 
     if (tid == 0) {
+        // the merge pass (a programmatic dependent launch) may be made resident as CTAs retire
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
         s_abort = 0;
         mbar_init(bar(BAR_Q_FULL), 1);
         mbar_init(bar(BAR_Q_EMPTY), 1);
