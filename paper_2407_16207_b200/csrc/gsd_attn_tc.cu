@@ -43,7 +43,7 @@ constexpr int KST = 2;             // K ring stages
 constexpr int VST = 2;             // V ring stages
 constexpr uint32_t HALF_BYTES = 128 * 64 * 2;     // one [128 rows][64 bf16] swizzled block
 constexpr uint32_t TILE_BYTES = 2 * HALF_BYTES;   // a 128 x 128 bf16 tile (two column halves)
-constexpr int kThreads = 512;
+constexpr int kThreads = 384;
 constexpr uint32_t kSmemBytes = (2 + KST + VST) * TILE_BYTES + 2 * HALF_BYTES + 1024;  // tiles, output staging, alignment slack
 constexpr float kRescaleThreshold = 8.0f;         // log2 units
 constexpr int kUnitTable = 12;                    // units of work per CTA decoded in the prologue (one per warp)
@@ -66,9 +66,8 @@ enum Bar {
     BAR_O_DONE = BAR_P_FREE + 2,      // 2: every PV of the unit on stream i has completed
     BAR_O_FREE = BAR_O_DONE + 2,      // 2: the accumulator rows of the unit have been read out
     BAR_Q_EMPTY = BAR_O_FREE + 2,     // 1: every QK^T of the unit has completed
-    BAR_ML_DONE = BAR_Q_EMPTY + 1,    // 2: the softmax of stream i has published (max, sum) of the unit's rows
-    BAR_EPI_DONE = BAR_ML_DONE + 2,   // 2: the epilogue has finished with staging block i (and the (max, sum) in it)
-    BAR_COUNT = BAR_EPI_DONE + 2
+    BAR_ML_READY = BAR_Q_EMPTY + 1,   // 1: (max, sum) of the odd-tile stream are in shared memory
+    BAR_COUNT = BAR_ML_READY + 1
 };
 
 struct TcParams {
@@ -153,6 +152,7 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t sr
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void wg_barrier(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -202,15 +202,6 @@ __device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16])
         : "memory");
 }
 
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
-    uint32_t* r = reinterpret_cast<uint32_t*>(v);
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr) : "memory");
-}
 // pointer form: v[0..31] must be register-resident (constant indices after unrolling)
 __device__ __forceinline__ void tc_ld32p(uint32_t taddr, float* v) {
     uint32_t* r = reinterpret_cast<uint32_t*>(v);
@@ -404,6 +395,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     __shared__ __align__(8) unsigned long long s_bars[BAR_COUNT];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
+    __shared__ float2 s_ml1[BM];      // (max, sum) of the odd-tile stream, one per row
     __shared__ UnitInfo s_units[kUnitTable];   // the CTA's first units of work, decoded once up front
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -424,6 +416,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         s_abort = 0;
         mbar_init(bar(BAR_Q_FULL), 1);
         mbar_init(bar(BAR_Q_EMPTY), 1);
+        mbar_init(bar(BAR_ML_READY), 4);
         for (int s = 0; s < KST; ++s) { mbar_init(bar(BAR_K_FULL + s), 1); mbar_init(bar(BAR_K_EMPTY + s), 1); }
         for (int s = 0; s < VST; ++s) { mbar_init(bar(BAR_V_FULL + s), 1); mbar_init(bar(BAR_V_EMPTY + s), 1); }
         for (int i = 0; i < 2; ++i) {
@@ -433,9 +426,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             mbar_init(bar(BAR_P_READY2 + i), 4);
             mbar_init(bar(BAR_P_FREE + i), 1);
             mbar_init(bar(BAR_O_DONE + i), 1);
-            mbar_init(bar(BAR_O_FREE + i), 4);     // one arrival per epilogue warp
-            mbar_init(bar(BAR_ML_DONE + i), 4);    // one arrival per softmax warp of the stream
-            mbar_init(bar(BAR_EPI_DONE + i), 1);
+            mbar_init(bar(BAR_O_FREE + i), 4);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -461,7 +452,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     auto unit_of = [&](int w, int it) -> UnitInfo { return it < kUnitTable ? s_units[it] : unit_info(p, w, lane); };
 
     if (warp >= 8) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 96;");
     if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
         int kvc = 0;          // key tiles loaded so far (ring position)
@@ -605,162 +596,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             ++au;
             if (n1 > 0) ++au1;
         }
-    } else if (warp >= 12) {
-        // ------------------------------------------------------------ epilogue warps (thread = row = TMEM lane)
-        // They take the finished accumulators out of TMEM, normalise, and write the rows out,
-        // while the softmax warps are already on the next unit.  16 columns at a time keeps
-        // them inside their small register share.
-        const int q = warp - 12;                         // TMEM lane quarter
-        const int rloc = q * 32 + lane;
-        const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-        const bool issuer = warp == 12 && lane == 0;     // the thread that owns the output tile stores
-        int e0 = 0, e1 = 0;                              // units in which stream 0 / 1 had jobs so far (barrier phases)
-        bool ok = true;
-        auto wait = [&](int b, uint32_t par) -> bool { return mbar_wait_warp(bar(b), par, abort_flag, p.status); };
-        auto epi_barrier = [&]() { asm volatile("bar.sync 1, 128;" ::: "memory"); };
-        for (int w = blockIdx.x, it = 0; w < total_work && ok; w += gridDim.x, ++it) {
-            const UnitInfo u = unit_of(w, it);
-            const int ntiles = u.ntiles;
-            const bool alt = !u.two;
-            const int n0 = alt ? (ntiles + 1) / 2 : ntiles, n1 = alt ? ntiles / 2 : ntiles;
-            const int nout = alt ? 1 : 2;                // row tiles to write
-            for (int t = 0; t < nout && ok; ++t) {
-                const int row = u.row0 + t * BM + rloc;
-                const bool rvalid = row < R;
-                const int nj = t == 0 ? n0 : n1;         // jobs behind accumulator t
-                float m = -CUDART_INF_F, l = 0.f, w0 = 0.f, w1 = 0.f;
-                const bool merge = alt && n1 > 0;
-                if (nj > 0) {
-                    const int ph = t == 0 ? e0 : e1;
-                    if (!(ok = wait(BAR_ML_DONE + t, ph & 1))) break;
-                    const float2 ml = reinterpret_cast<const float2*>(smem_raw + (sStage - smem_u32(smem_raw)) + (uint32_t)t * HALF_BYTES)[rloc];
-                    m = ml.x; l = ml.y; w0 = 1.f;
-                    if (merge) {
-                        // single row tile: O = w0 O0 + w1 O1, l = w0 l0 + w1 l1 at the common maximum
-                        if (!(ok = wait(BAR_ML_DONE + 1, e1 & 1))) break;
-                        const float2 ml1 = reinterpret_cast<const float2*>(smem_raw + (sStage - smem_u32(smem_raw)) + HALF_BYTES)[rloc];
-                        const float mm = fmaxf(m, ml1.x);
-                        const float m_use = mm == -CUDART_INF_F ? 0.f : mm;
-                        w0 = fast_exp2(m - m_use); w1 = fast_exp2(ml1.x - m_use);
-                        l = w0 * l + w1 * ml1.y;
-                        m = mm;
-                        if (!(ok = wait(BAR_O_DONE + 1, e1 & 1))) break;
-                    }
-                    if (!(ok = wait(BAR_O_DONE + t, ph & 1))) break;
-                    tc_fence_after();
-                }
-                const uint32_t tO = tmem + lane_addr + (t ? COL_O1 : COL_O0);
-                const uint32_t tOm = tmem + lane_addr + COL_O1;      // the odd-tile stream's accumulator (merge)
-                if (u.nsplit == 1) {
-                    // Normalise, round to bf16 and stage the rows in shared memory in the swizzled
-                    // tile layout; one thread then writes each 64-column half with a TMA tile store
-                    // (rows of nodes >= N are clipped by the tensor map).
-                    const float inv = l > 0.f ? 1.f / l : 0.f;
-                    const float s0 = w0 * inv, s1 = w1 * inv;
-                    const uint32_t stage = sStage + (uint32_t)t * HALF_BYTES;
-                    unsigned char* srow = smem_raw + (stage - smem_u32(smem_raw)) + rloc * 128;
-#pragma unroll 1
-                    for (int h = 0; h < 2; ++h) {
-                        // every thread has its (max, sum); an earlier store has read the block
-                        if (issuer) bulk_wait_read();
-                        epi_barrier();
-#pragma unroll
-                        for (int c4 = 0; c4 < 4; ++c4) {
-                            float a[16];
-                            tc_ld16(tO + h * 64 + c4 * 16, a);
-                            tc_wait_ld();
-                            if (merge) {
-                                float b2[16];
-                                tc_ld16(tOm + h * 64 + c4 * 16, b2);
-                                tc_wait_ld();
-#pragma unroll
-                                for (int e = 0; e < 16; ++e) a[e] = s0 * a[e] + s1 * b2[e];
-                            } else {
-#pragma unroll
-                                for (int e = 0; e < 16; ++e) a[e] *= s0;
-                            }
-#pragma unroll
-                            for (int k2 = 0; k2 < 2; ++k2) {
-                                uint4 v;
-                                v.x = pack_bf16(a[k2 * 8 + 0], a[k2 * 8 + 1]);
-                                v.y = pack_bf16(a[k2 * 8 + 2], a[k2 * 8 + 3]);
-                                v.z = pack_bf16(a[k2 * 8 + 4], a[k2 * 8 + 5]);
-                                v.w = pack_bf16(a[k2 * 8 + 6], a[k2 * 8 + 7]);
-                                const int k = c4 * 2 + k2;          // 16-byte chunk of the 128-byte row
-                                *reinterpret_cast<uint4*>(srow + ((k ^ (rloc & 7)) << 4)) = v;
-                            }
-                        }
-                        if (h == 1 && nj > 0) {
-                            // the accumulators are out of TMEM: the next unit's first PV may overwrite them
-                            tc_fence_before();
-                            if (lane == 0) {
-                                mbar_arrive(bar(BAR_O_FREE + t));
-                                if (merge) mbar_arrive(bar(BAR_O_FREE + 1));
-                            }
-                        }
-                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                        epi_barrier();
-                        if (issuer) {
-                            tma_store_4d(&tm_out, stage, h * 64, u.c * G, (u.row0 + t * BM) / G, u.b);
-                            bulk_commit();
-                        }
-                    }
-                } else {
-                    // a piece of a cut item: unnormalised fp32 rows and (max, sum) for the merge pass
-                    const size_t prow = (size_t)u.slot * (2 * BM) + t * BM + rloc;
-                    float* dst = p.part_o + prow * HD;
-                    epi_barrier();                               // every thread has its (max, sum)
-#pragma unroll 1
-                    for (int c8 = 0; c8 < 8; ++c8) {
-                        float a[16];
-                        if (nj > 0) {
-                            tc_ld16(tO + c8 * 16, a);
-                            tc_wait_ld();
-                            if (merge) {
-                                float b2[16];
-                                tc_ld16(tOm + c8 * 16, b2);
-                                tc_wait_ld();
-#pragma unroll
-                                for (int e = 0; e < 16; ++e) a[e] = w0 * a[e] + w1 * b2[e];
-                            }
-                        } else {
-#pragma unroll
-                            for (int e = 0; e < 16; ++e) a[e] = 0.f;
-                        }
-                        if (rvalid) {
-#pragma unroll
-                            for (int k = 0; k < 4; ++k)
-                                *reinterpret_cast<float4*>(dst + c8 * 16 + k * 4) = make_float4(a[4 * k], a[4 * k + 1], a[4 * k + 2], a[4 * k + 3]);
-                        }
-                    }
-                    if (rvalid) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(m, l);
-                    if (nj > 0) {
-                        tc_fence_before();
-                        if (lane == 0) {
-                            mbar_arrive(bar(BAR_O_FREE + t));
-                            if (merge) mbar_arrive(bar(BAR_O_FREE + 1));
-                        }
-                    }
-                }
-                if (nj > 0) {
-                    // the staging block (and the (max, sum) in it) may be written again once the
-                    // stores have read it
-                    epi_barrier();
-                    if (issuer) {
-                        bulk_wait_read();
-                        mbar_arrive(bar(BAR_EPI_DONE + t));
-                        if (merge) mbar_arrive(bar(BAR_EPI_DONE + 1));
-                    }
-                }
-            }
-            if (n0 > 0) ++e0;
-            if (n1 > 0) ++e1;
-        }
-        if (issuer) bulk_wait_all();   // the output stores have landed
     }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
-        // ------------------------------------------------------------ softmax
+        // ------------------------------------------------------------ softmax + epilogue
         const int i = warp >> 2;                         // stream of this warpgroup
         const int rloc = (warp & 3) * 32 + lane;         // row inside the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
@@ -769,17 +608,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const uint32_t tO = tmem + lane_addr + (i ? COL_O1 : COL_O0);
         int kvc = 0;      // key tiles of all non-empty units so far (ring position of the V tiles)
         int tcnt = 0;     // jobs this stream has processed so far (barrier phase)
-        int auc = 0;      // units in which this stream had jobs so far (barrier phase)
+        int auc = 0;      // non-empty units this stream has finished so far (barrier phase)
+        int auc1 = 0;     // units in which stream 1 had jobs (phase of its barriers as seen by warpgroup 0)
+        int mlc = 0;      // single-row-tile units whose odd-tile stream had tiles
         bool ok = true;
         for (int w = blockIdx.x, it = 0; w < total_work && ok; w += gridDim.x, ++it) {
             const UnitInfo u = unit_of(w, it);
             const int ntiles = u.ntiles;
             // with one row tile only, the two warpgroups take the even / odd key tiles of the
-            // same rows and the epilogue warps merge the two partial results
+            // same rows and warpgroup 0 merges the two partial results in the epilogue
             const bool alt = !u.two;
             const int my_n = alt ? (i == 0 ? (ntiles + 1) / 2 : ntiles / 2) : ntiles;
             const int n1 = alt ? ntiles / 2 : ntiles;           // tiles of stream 1 in this unit
-            const int b = u.b;
+            const int b = u.b, c = u.c;
             const int row = u.row0 + (alt ? 0 : i * BM) + rloc;
             const bool rvalid = row < R;
             if (warp == 0 && lane == 0) {
@@ -925,24 +766,108 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
             if (!ok) break;
 
-            // ---- end of the unit: publish (max, sum) of this stream's rows for the epilogue warps
-            // and go on.  The two floats travel in the first KB of the stream's staging block,
-            // which the previous unit's output stores must have left.
-            if (my_n > 0) {
-                if (auc > 0) {
-                    ok = mbar_wait(bar(BAR_EPI_DONE + i), (uint32_t)((auc - 1) & 1), abort_flag, p.status);
+            if (alt && i == 1) {
+                // odd-tile stream: publish (max, sum); warpgroup 0 reads the accumulator itself
+                if (my_n > 0) {
+                    s_ml1[rloc] = make_float2(m_ref, l_run);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(BAR_ML_READY));
+                    ++mlc;
+                    ++auc;
+                }
+                kvc += ntiles;
+                tcnt += my_n;
+                continue;
+            }
+            // ---- epilogue: pull the accumulator row into registers, give TMEM back, then store
+            float acc[HD];
+            if (ntiles > 0) {
+                ok = mbar_wait(bar(BAR_O_DONE + i), (uint32_t)(auc & 1), abort_flag, p.status);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) tc_ld32p(tO + ch * 32, acc + ch * 32);
+                tc_wait_ld();
+                if (alt && n1 > 0) {
+                    // merge the odd-tile stream: O = w0 O0 + w1 O1, l = w0 l0 + w1 l1 at the common maximum
+                    ok = mbar_wait(bar(BAR_O_DONE + 1), (uint32_t)(auc1 & 1), abort_flag, p.status);
+                    if (ok) ok = mbar_wait(bar(BAR_ML_READY), (uint32_t)(mlc & 1), abort_flag, p.status);
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
+                    tc_fence_after();
+                    const float2 ml1 = s_ml1[rloc];
+                    const float m = fmaxf(m_ref, ml1.x);
+                    const float m_use = m == -CUDART_INF_F ? 0.f : m;
+                    const float w0 = fast_exp2(m_ref - m_use), w1 = fast_exp2(ml1.x - m_use);
+                    const uint32_t tO1 = tmem + lane_addr + COL_O1;
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        float v[32];
+                        tc_ld32(tO1 + ch * 32, v);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) acc[ch * 32 + e] = w0 * acc[ch * 32 + e] + w1 * v[e];
+                    }
+                    l_run = w0 * l_run + w1 * ml1.y;
+                    m_ref = m;
+                    tc_fence_before();
+                    if (lane == 0) mbar_arrive(bar(BAR_O_FREE + 1));
+                    ++mlc;
                 }
-                float2* ml = reinterpret_cast<float2*>(smem_raw + (sStage - smem_u32(smem_raw)) + (uint32_t)i * HALF_BYTES);
-                ml[rloc] = make_float2(m_ref, l_run);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_ML_DONE + i));
-                ++auc;
+                tc_fence_before();
+                if (lane == 0) mbar_arrive(bar(BAR_O_FREE + i));
+            } else {
+#pragma unroll
+                for (int e = 0; e < HD; ++e) acc[e] = 0.f;
+            }
+            if (u.nsplit == 1) {
+                // Normalise, round to bf16 and stage the rows in shared memory in the swizzled tile
+                // layout; one thread then writes each 64-column half with a TMA tile store (full
+                // 128-byte lines instead of 32 scattered 16-byte pieces per store instruction;
+                // rows of nodes >= N are clipped by the tensor map).
+                const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+                const uint32_t stage = sStage + (uint32_t)i * HALF_BYTES;
+                unsigned char* srow = smem_raw + (stage - smem_u32(smem_raw)) + rloc * 128;
+                const bool issuer = (warp & 3) == 0 && lane == 0;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const int e = h * 64 + k * 8;
+                        uint4 v;
+                        v.x = pack_bf16(acc[e + 0] * inv, acc[e + 1] * inv);
+                        v.y = pack_bf16(acc[e + 2] * inv, acc[e + 3] * inv);
+                        v.z = pack_bf16(acc[e + 4] * inv, acc[e + 5] * inv);
+                        v.w = pack_bf16(acc[e + 6] * inv, acc[e + 7] * inv);
+                        *reinterpret_cast<uint4*>(srow + ((k ^ (rloc & 7)) << 4)) = v;
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    wg_barrier(1 + i);
+                    if (issuer) {
+                        tma_store_4d(&tm_out, stage, h * 64, c * G, (u.row0 + (alt ? 0 : i * BM)) / G, b);
+                        bulk_commit();
+                        bulk_wait_read();          // the staging block may be overwritten again
+                    }
+                    wg_barrier(1 + i);
+                }
+            } else if (rvalid) {
+                {
+                    const size_t prow = (size_t)u.slot * (2 * BM) + (alt ? 0 : i * BM) + rloc;
+                    float* dst = p.part_o + prow * HD;
+#pragma unroll
+                    for (int k = 0; k < HD / 4; ++k)
+                        *reinterpret_cast<float4*>(dst + k * 4) =
+                            make_float4(acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]);
+                    *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(m_ref, l_run);
+                }
             }
             kvc += ntiles;
             tcnt += my_n;
+            if (ntiles > 0) ++auc;
+            if (n1 > 0) ++auc1;
         }
+        if ((warp & 3) == 0 && lane == 0) bulk_wait_all();   // the output stores have landed
     }
 
     // ---------------------------------------------------------------- teardown
