@@ -168,6 +168,25 @@ def test_sweep_points_sampled_rows(point):
     assert_close(np.stack([got[b, n, h] for b, n, h in rows]), want)
 
 
+def test_many_units_per_cta_sampled_rows():
+    # 4096 units of work for 148 persistent CTAs (about 28 each, more than the kernel decodes up
+    # front), short ragged prefix (one partial cache tile) and four draft tiles per unit
+    cfg = gi.sweep_config(32, 100, 512)
+    inp = gi.make_inputs(cfg, accept=False)
+    out = gpu_attn(inp)
+    rng = np.random.default_rng(77)
+    rows = []
+    for b0, c0 in ((0, 0), (31, 7), (17, 3)):          # first, last and a middle (sequence, kv head)
+        rows += [(b0, n, c0 * cfg.G + g) for n in range(0, cfg.N, 16) for g in range(cfg.G)]
+    rows += [(int(rng.integers(cfg.B)), int(rng.integers(cfg.N)), int(rng.integers(cfg.Hq)))
+             for _ in range(1024)]
+    want = oracle.attn_rows(inp["q"], inp["k_cache"], inp["v_cache"], inp["draft_k"],
+                            inp["draft_v"], inp["ancestor_mask"], inp["seq_lens"], rows)
+    idx = torch.tensor(rows, device=out.device, dtype=torch.long)
+    got = out_to_f64(out[idx[:, 0], idx[:, 1], idx[:, 2]])
+    assert_close(got, want)
+
+
 def test_dominant_key_and_large_score_jumps():
     # one cache key scores 2^k times above the rest from some tile on: the running maximum has
     # to be raised (accumulator rescale path) and nothing may overflow
