@@ -48,7 +48,7 @@ def _load() -> ctypes.CDLL:
         _lib = ctypes.CDLL(build())
         _lib.gsd_oracle_threads.restype = ctypes.c_int
         _lib.gsd_oracle_argmax_row.restype = ctypes.c_int32
-        for name in ("gsd_oracle_attn", "gsd_oracle_attn_rows", "gsd_oracle_accept",
+        for name in ("gsd_oracle_attn", "gsd_oracle_attn_rows", "gsd_oracle_accept", "gsd_oracle_accept_sampled",
                      "gsd_oracle_commit_kv", "gsd_oracle_build_mask"):
             getattr(_lib, name).restype = ctypes.c_int
         _lib.gsd_oracle_argmax.restype = None
@@ -141,6 +141,30 @@ def accept(logits, draft_tokens, parent_ptr, parent_idx, Tcap: int = 0, visit_ca
     if rc != 0:
         raise ValueError("oracle accept: malformed DAG or Tcap too small")
     return toks, lens, nodes, visited
+
+
+def accept_sampled(logits, draft_tokens, parent_ptr, parent_idx, draft_q, u_accept, u_sample, Tcap: int = 0):
+    """Non-deterministic verification with the random numbers passed in (see gsd_oracle_accept_sampled).
+
+    Returns (accepted_tokens [B,Tcap] padded with -1, accepted_len [B], accepted_nodes [B,Tcap])."""
+    logits = _c(logits, np.float32); draft_tokens = _c(draft_tokens, np.int32)
+    parent_ptr = _c(parent_ptr, np.int32); parent_idx = _c(parent_idx, np.int32)
+    draft_q = _c(draft_q, np.float32); u_accept = _c(u_accept, np.float32); u_sample = _c(u_sample, np.float32)
+    B, N, V = logits.shape
+    assert draft_tokens.shape == (B, N) and parent_ptr.shape == (B, N + 1)
+    assert draft_q.shape == (B, N) and u_accept.shape == (B, N) and u_sample.shape == (B,)
+    Ecap = parent_idx.shape[1]
+    Tcap = Tcap or N
+    toks = np.zeros((B, Tcap), dtype=np.int32)
+    lens = np.zeros((B,), dtype=np.int32)
+    nodes = np.zeros((B, Tcap), dtype=np.int32)
+    rc = _load().gsd_oracle_accept_sampled(_p(logits), _p(draft_tokens), _p(parent_ptr), _p(parent_idx),
+                                           _p(draft_q), _p(u_accept), _p(u_sample),
+                                           ctypes.c_int32(B), ctypes.c_int32(N), ctypes.c_int32(V),
+                                           ctypes.c_int32(Ecap), ctypes.c_int32(Tcap), _p(toks), _p(lens), _p(nodes))
+    if rc != 0:
+        raise ValueError("oracle accept_sampled: malformed DAG or Tcap too small")
+    return toks, lens, nodes
 
 
 def commit_kv(k_cache, v_cache, draft_k, draft_v, accepted_nodes, accepted_len, seq_lens):

@@ -25,6 +25,11 @@
  *    longest accepted path wins; among equally long ones the path whose node sequence,
  *    read from its last node backwards, is lexicographically smallest.  Output:
  *    tok[v1..vm] followed by a[vm], so accepted_len = m + 1.
+ *  - Non-deterministic acceptance (Sec. 3: accept with probability min(1, p/q); Sec. 6.4: on
+ *    the token graph), with the random numbers as inputs: the same walk with the step
+ *    p -> v accepted iff u_accept[v] * q_v < softmax(logits[p])[tok v], and the regenerated
+ *    token drawn from softmax(logits[end]) by inverting the cumulative distribution.
+ *  - The KV-cache commit of the accepted path and the ancestor-mask closure (see there).
  *
  * Readings where the paper is silent are listed in the repository's design notes
  * (scale default 1/sqrt(D), q-head h uses kv-head h / G, mask bits honoured literally,
@@ -203,6 +208,7 @@ typedef struct {
     int N;
     const int32_t *tok;   /* [N] */
     const int32_t *amax;  /* [N] */
+    const unsigned char *edge_ok; /* NULL, or [N*N]: edge_ok[p*N + v] = the step p -> v is accepted */
     const int *child_ptr; /* [N+1] */
     const int *child_idx;
     int *stack;           /* current path, stack[0] = 0 */
@@ -215,8 +221,13 @@ typedef struct {
 
 static int path_is_accepted(const walk_t *w, int len)
 {
-    for (int i = 1; i < len; ++i)
-        if (w->tok[w->stack[i]] != w->amax[w->stack[i - 1]]) return 0;
+    for (int i = 1; i < len; ++i) {
+        if (w->edge_ok) {
+            if (!w->edge_ok[(size_t)w->stack[i - 1] * w->N + w->stack[i]]) return 0;
+        } else if (w->tok[w->stack[i]] != w->amax[w->stack[i - 1]]) {
+            return 0;
+        }
+    }
     return 1;
 }
 
@@ -295,7 +306,7 @@ int gsd_oracle_accept(const float *logits, const int32_t *draft_tokens, const in
                     cidx[cptr[p] + fill[p]++] = v;
                 }
             walk_t w;
-            w.N = N; w.tok = tok; w.amax = amax; w.child_ptr = cptr; w.child_idx = cidx;
+            w.N = N; w.tok = tok; w.amax = amax; w.edge_ok = NULL; w.child_ptr = cptr; w.child_idx = cidx;
             w.stack = stack; w.best = best; w.best_edges = -1; w.visited = 0;
             w.visit_cap = visit_cap; w.pruned = 0;
             stack[0] = 0;
@@ -316,6 +327,106 @@ int gsd_oracle_accept(const float *logits, const int32_t *draft_tokens, const in
             }
         }
         free(amax); free(cptr); free(cidx); free(fill); free(stack); free(best);
+        if (rc != 0) return rc;
+    }
+    return 0;
+}
+
+/*
+ * Non-deterministic verification (Sec. 3: the i-th drafted token is accepted with probability
+ * min(1, p/q), the first rejection discards the rest of the hypothesis and the target model
+ * regenerates that token; Sec. 6.4 runs it on the token graph).  Readings taken here: the
+ * random numbers are inputs; the test is applied per step p -> v of the graph with
+ * p = softmax(logits[parent])[token of v] and q = draft_q[v]:
+ *     accepted(p -> v)  iff  u_accept[v] * q_v < p          (u < min(1, p/q) for q > 0)
+ * the accepted hypothesis is the longest root path whose steps are all accepted (ties as in
+ * gsd_oracle_accept); the regenerated token is drawn from softmax(logits[end node]) by
+ * inverting its cumulative distribution in index order: the smallest t with
+ * sum_{j<=t} P_j > u_sample[b] (the last t with P_t > 0 if rounding leaves none).
+ * All arithmetic in double.  logits must be finite or -inf with at least one finite entry per row.
+ *
+ * logits [B,N,V]; draft_q, u_accept [B,N]; u_sample [B]; the rest as gsd_oracle_accept.
+ * Returns 0, or -1 on malformed input or allocation failure.
+ */
+static void softmax_stats(const float *x, int V, double *m_out, double *s_out)
+{
+    double m = -INFINITY, s = 0.0;
+    for (int j = 0; j < V; ++j) if ((double)x[j] > m) m = (double)x[j];
+    for (int j = 0; j < V; ++j) s += exp((double)x[j] - m);
+    *m_out = m; *s_out = s;
+}
+
+int gsd_oracle_accept_sampled(const float *logits, const int32_t *draft_tokens,
+                              const int32_t *parent_ptr, const int32_t *parent_idx,
+                              const float *draft_q, const float *u_accept, const float *u_sample,
+                              int32_t B, int32_t N, int32_t V, int32_t Ecap, int32_t Tcap,
+                              int32_t *accepted_tokens, int32_t *accepted_len, int32_t *accepted_nodes)
+{
+    int rc = 0;
+    for (int b = 0; b < B; ++b) {
+        const int32_t *tok = draft_tokens + (size_t)b * N;
+        const int32_t *pp = parent_ptr + (size_t)b * (N + 1);
+        const int32_t *pi = parent_idx + (size_t)b * Ecap;
+        const float *lg = logits + (size_t)b * N * V;
+        double *mx = (double *)malloc(sizeof(double) * (size_t)N);
+        double *sm = (double *)malloc(sizeof(double) * (size_t)N);
+        unsigned char *ok = (unsigned char *)calloc((size_t)N * N, 1);
+        int *cptr = (int *)calloc((size_t)N + 2, sizeof(int));
+        int *cidx = (int *)malloc(sizeof(int) * (size_t)(pp[N] > 0 ? pp[N] : 1));
+        int *fill = (int *)calloc((size_t)N + 1, sizeof(int));
+        int *stack = (int *)malloc(sizeof(int) * (size_t)(N + 1));
+        int *best = (int *)malloc(sizeof(int) * (size_t)(N + 1));
+        if (!mx || !sm || !ok || !cptr || !cidx || !fill || !stack || !best) rc = -1;
+        if (rc == 0) {
+#pragma omp parallel for schedule(static)
+            for (int v = 0; v < N; ++v) softmax_stats(lg + (size_t)v * V, V, &mx[v], &sm[v]);
+            for (int v = 0; v < N && rc == 0; ++v)
+                for (int e = pp[v]; e < pp[v + 1]; ++e) {
+                    const int p = pi[e];
+                    if (p < 0 || p >= v || tok[v] < 0 || tok[v] >= V) { rc = -1; break; }
+                    const double prob = exp((double)lg[(size_t)p * V + tok[v]] - mx[p]) / sm[p];
+                    ok[(size_t)p * N + v] = ((double)u_accept[(size_t)b * N + v] * (double)draft_q[(size_t)b * N + v] < prob);
+                    cptr[p + 1]++;
+                }
+        }
+        if (rc == 0) {
+            for (int v = 0; v < N; ++v) cptr[v + 1] += cptr[v];
+            for (int v = 0; v < N; ++v)
+                for (int e = pp[v]; e < pp[v + 1]; ++e) cidx[cptr[pi[e]] + fill[pi[e]]++] = v;
+            walk_t w;
+            w.N = N; w.tok = tok; w.amax = NULL; w.edge_ok = ok; w.child_ptr = cptr; w.child_idx = cidx;
+            w.stack = stack; w.best = best; w.best_edges = -1; w.visited = 0;
+            w.visit_cap = 0; w.pruned = 0;
+            stack[0] = 0;
+            walk(&w, 1);
+            const int m = w.best_edges;
+            if (m + 1 > Tcap) rc = -1;
+            if (rc == 0) {
+                /* the regenerated token: inverse of the cumulative distribution at the end node */
+                const int end = best[m];
+                const float *x = lg + (size_t)end * V;
+                const double target = (double)u_sample[b];
+                double cum = 0.0;
+                int pick = -1, last_pos = -1;
+                for (int j = 0; j < V; ++j) {
+                    const double pj = exp((double)x[j] - mx[end]) / sm[end];
+                    if (pj > 0.0) last_pos = j;
+                    cum += pj;
+                    if (cum > target) { pick = j; break; }
+                }
+                if (pick < 0) pick = last_pos;
+                for (int i = 0; i < Tcap; ++i) {
+                    accepted_tokens[(size_t)b * Tcap + i] = -1;
+                    if (accepted_nodes) accepted_nodes[(size_t)b * Tcap + i] = -1;
+                }
+                for (int i = 1; i <= m; ++i) accepted_tokens[(size_t)b * Tcap + i - 1] = tok[best[i]];
+                accepted_tokens[(size_t)b * Tcap + m] = pick;
+                accepted_len[b] = m + 1;
+                if (accepted_nodes)
+                    for (int i = 0; i <= m; ++i) accepted_nodes[(size_t)b * Tcap + i] = best[i];
+            }
+        }
+        free(mx); free(sm); free(ok); free(cptr); free(cidx); free(fill); free(stack); free(best);
         if (rc != 0) return rc;
     }
     return 0;

@@ -31,6 +31,16 @@ MUTATIONS = [
      "test_oracle_accept.py"),
     ("commit_position", "k_cache + ((size_t)b * Lmax + pos) * row, draft_k",
      "k_cache + ((size_t)b * Lmax + pos + 1 - (pos + 1 >= Lmax)) * row, draft_k", "test_oracle_commit.py"),
+    ("sampled_le", "(double)draft_q[(size_t)b * N + v] < prob);", "(double)draft_q[(size_t)b * N + v] <= prob);",
+     "test_oracle_accept_sampled.py"),
+    ("sampled_without_q", "(double)u_accept[(size_t)b * N + v] * (double)draft_q[(size_t)b * N + v] < prob",
+     "(double)u_accept[(size_t)b * N + v] < prob", "test_oracle_accept_sampled.py"),
+    ("sampled_child_logits", "exp((double)lg[(size_t)p * V + tok[v]] - mx[p]) / sm[p]",
+     "exp((double)lg[(size_t)v * V + tok[v]] - mx[v]) / sm[v]", "test_oracle_accept_sampled.py"),
+    ("sampled_cdf_ge", "if (cum > target) { pick = j; break; }", "if (cum >= target) { pick = j; break; }",
+     "test_oracle_accept_sampled.py"),
+    ("sampled_regenerates_at_parent", "const int end = best[m];", "const int end = best[m > 0 ? m - 1 : 0];",
+     "test_oracle_accept_sampled.py"),
     ("mask_without_self", "row[v / 32] |= 1u << (v % 32);", "if (v != n) row[v / 32] |= 1u << (v % 32);",
      "test_oracle_mask.py"),
     ("mask_parents_only", "seen[p] = 1;\n                    todo[top++] = p;", "seen[p] = 1;\n                    if (v == n) todo[top++] = p;",
