@@ -56,6 +56,7 @@ typedef enum gsd_status {
 #define GSD_DEV_WAIT_EXPIRED 0x8u  /* a bounded in-kernel wait gave up; the output is not valid */
 #define GSD_DEV_BAD_SEQ_LEN  0x10u /* seq_lens[b] outside [0, Lmax]; it was clamped */
 #define GSD_DEV_CACHE_FULL   0x20u /* gsd_commit_kv: the accepted rows did not all fit below Lmax; the rest was dropped */
+#define GSD_DEV_BAD_LOGITS   0x40u /* gsd_accept_sampled: a logits row without a finite entry, or with +inf or NaN */
 
 #define GSD_MAX_NODES 512          /* largest supported N (draft nodes per sequence) */
 
@@ -168,6 +169,46 @@ int gsd_accept(const float* logits, const int32_t* draft_tokens, const int32_t* 
                size_t workspace_bytes, int32_t* status, void* stream);
 
 size_t gsd_accept_workspace_bytes(const gsd_accept_params* p);
+
+/*
+ * gsd_accept_sampled - non-deterministic verification of the token graph (Sec. 3: a drafted
+ * token is accepted with probability min(1, p/q); the first rejection discards the rest of the
+ * hypothesis and the target model regenerates that token; Sec. 6.4 runs this on the graph;
+ * longest-path selection as in Sec. 4.1).  The random numbers are inputs, so the call is a pure
+ * function.  Readings (the paper gives the rule for a single hypothesis only):
+ *   - the test is applied to every step parent -> v of the graph, with p the target
+ *     probability softmax(logits[b][parent])[draft_tokens[b][v]] and q = draft_q[b][v]:
+ *         accepted  iff  u_accept[b][v] * q < p        (u < min(1, p/q); q = 0 accepts iff p > 0)
+ *   - the hypothesis is the longest root path all of whose steps are accepted; ties as in
+ *     gsd_accept (lowest end node, then lowest predecessor walking back);
+ *   - the regenerated token is drawn from softmax(logits[b][end node]) by inverting its
+ *     cumulative distribution in index order: the smallest t with sum_{j<=t} P_j > u_sample[b]
+ *     (the last t with P_t > 0 if rounding leaves none).  The residual distribution
+ *     max(0, p - q) of the original sampling scheme would need the draft model's whole
+ *     distribution per node and is not formed.
+ * Temperature / nucleus filtering are the caller's: pass logits already divided by the
+ * temperature (and with filtered entries at -inf).
+ *
+ *   logits, draft_tokens, parent_ptr, parent_idx   device, as for gsd_accept; every logits row
+ *                    must hold at least one finite value, no +inf and no NaN (GSD_DEV_BAD_LOGITS)
+ *   draft_q          device const f32 [B,N]: the probability the draft model gave node v's token
+ *                    when it drafted it (entry 0, the root, is not read)
+ *   u_accept         device const f32 [B,N]: one number in [0,1) per node (entry 0 not read)
+ *   u_sample         device const f32 [B]: one number in [0,1) per sequence
+ *   accepted_tokens, accepted_len, accepted_nodes   device outputs as for gsd_accept; the entry
+ *                    after the drafted tokens of the path is the regenerated token
+ *   workspace        device scratch of gsd_accept_sampled_workspace_bytes(p) bytes, 8-byte
+ *                    aligned, arbitrary contents; the call clears what has to start at zero
+ * The softmax statistics are accumulated in fp32 (ex2.approx); a step whose two sides differ by
+ * less than a few 1e-6 relative may be decided differently from an exact evaluation.
+ * Errors and status bits as for gsd_accept, plus GSD_DEV_BAD_LOGITS.  Asynchronous on `stream`.
+ */
+size_t gsd_accept_sampled_workspace_bytes(const gsd_accept_params* p);
+int gsd_accept_sampled(const float* logits, const int32_t* draft_tokens, const int32_t* parent_ptr,
+                       const int32_t* parent_idx, const float* draft_q, const float* u_accept,
+                       const float* u_sample, int32_t* accepted_tokens, int32_t* accepted_len,
+                       int32_t* accepted_nodes, const gsd_accept_params* p, void* workspace,
+                       size_t workspace_bytes, int32_t* status, void* stream);
 
 /*
  * gsd_accept_static - gsd_accept without a workspace argument.  (The paper has no counterpart

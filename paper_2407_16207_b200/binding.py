@@ -46,7 +46,8 @@ class AcceptParams(ctypes.Structure):
 
 EXPORTS = ["gsd_version", "gsd_status_string", "gsd_last_cuda_error", "gsd_verify_attn",
            "gsd_verify_attn_workspace_bytes", "gsd_verify_attn_num_splits", "gsd_accept",
-           "gsd_accept_workspace_bytes", "gsd_accept_static", "gsd_commit_kv", "gsd_build_mask", "gsd_verify_step_host",
+           "gsd_accept_workspace_bytes", "gsd_accept_static", "gsd_accept_sampled",
+           "gsd_accept_sampled_workspace_bytes", "gsd_commit_kv", "gsd_build_mask", "gsd_verify_step_host",
            "gsd_verify_step_host_arena_bytes"]
 
 
@@ -75,6 +76,10 @@ def lib() -> ctypes.CDLL:
         L.gsd_verify_attn_num_splits.argtypes = [ctypes.POINTER(AttnParams)]
         L.gsd_accept.restype = i32
         L.gsd_accept.argtypes = [vp] * 7 + [ctypes.POINTER(AcceptParams), vp, sz, vp, vp]
+        L.gsd_accept_sampled.restype = i32
+        L.gsd_accept_sampled.argtypes = [vp] * 10 + [ctypes.POINTER(AcceptParams), vp, sz, vp, vp]
+        L.gsd_accept_sampled_workspace_bytes.restype = sz
+        L.gsd_accept_sampled_workspace_bytes.argtypes = [ctypes.POINTER(AcceptParams)]
         L.gsd_accept_static.restype = i32
         L.gsd_accept_static.argtypes = [vp] * 7 + [ctypes.POINTER(AcceptParams), vp, vp]
         L.gsd_build_mask.restype = i32
@@ -222,6 +227,44 @@ def gsd_accept(logits, draft_tokens, parent_ptr, parent_idx, *, Tcap: int = 0,
                             ctypes.byref(p), workspace.data_ptr(),
                             workspace.numel() * workspace.element_size(), _ptr(status),
                             _stream(logits)))
+    return toks, lens, nodes
+
+
+def gsd_accept_sampled(logits, draft_tokens, parent_ptr, parent_idx, draft_q, u_accept, u_sample, *,
+                       Tcap: int = 0, want_nodes: bool = True, workspace: Optional[torch.Tensor] = None,
+                       status: Optional[torch.Tensor] = None
+                       ) -> Tuple[torch.Tensor, torch.Tensor, Optional[torch.Tensor]]:
+    """Non-deterministic verification with the random numbers passed in; see gsd_accept_sampled in
+    include/gsd.h.  Returns (accepted_tokens [B,Tcap], accepted_len [B], accepted_nodes or None)."""
+    if logits.dim() != 3:
+        raise ValueError("logits must be [B,N,V]")
+    B, N, V = logits.shape
+    _want(logits, torch.float32, (B, N, V), "logits", True)
+    _want(draft_tokens, torch.int32, (B, N), "draft_tokens", True)
+    _want(parent_ptr, torch.int32, (B, N + 1), "parent_ptr", True)
+    if parent_idx.dim() != 2:
+        raise ValueError("parent_idx must be [B,Ecap]")
+    Ecap = parent_idx.shape[1]
+    _want(parent_idx, torch.int32, (B, Ecap), "parent_idx", True)
+    _want(draft_q, torch.float32, (B, N), "draft_q", True)
+    _want(u_accept, torch.float32, (B, N), "u_accept", True)
+    _want(u_sample, torch.float32, (B,), "u_sample", True)
+    Tcap = Tcap or N
+    toks = torch.empty((B, Tcap), dtype=torch.int32, device=logits.device)
+    lens = torch.empty((B,), dtype=torch.int32, device=logits.device)
+    nodes = torch.empty((B, Tcap), dtype=torch.int32, device=logits.device) if want_nodes else None
+    p = AcceptParams(B, N, V, Ecap, Tcap)
+    L = lib()
+    with torch.cuda.device(logits.device):
+        need = int(L.gsd_accept_sampled_workspace_bytes(ctypes.byref(p)))
+        if workspace is None:
+            workspace = torch.empty(max(need, 8), dtype=torch.uint8, device=logits.device)
+        _check(L.gsd_accept_sampled(logits.data_ptr(), draft_tokens.data_ptr(), parent_ptr.data_ptr(),
+                                    parent_idx.data_ptr(), draft_q.data_ptr(), u_accept.data_ptr(),
+                                    u_sample.data_ptr(), toks.data_ptr(), lens.data_ptr(), _ptr(nodes),
+                                    ctypes.byref(p), workspace.data_ptr(),
+                                    workspace.numel() * workspace.element_size(), _ptr(status),
+                                    _stream(logits)))
     return toks, lens, nodes
 
 

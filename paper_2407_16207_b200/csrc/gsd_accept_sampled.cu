@@ -1,0 +1,407 @@
+// gsd_accept_sampled: non-deterministic verification of the draft token graph (Sec. 3: a
+// drafted token is accepted with probability min(1, p/q), the first rejection ends the
+// hypothesis and the target model regenerates that token; Sec. 6.4: the same on the graph).
+// The random numbers are inputs.  A step parent -> v of the graph is accepted iff
+//     u_accept[v] * draft_q[v] < softmax(logits[parent])[token of v];
+// the hypothesis is the longest root path of accepted steps (ties as in gsd_accept), and the
+// regenerated token is drawn from softmax(logits[end node]) by inverting the cumulative
+// distribution in index order with u_sample.
+//
+// One launch.  Grid (slices, B*N): each CTA streams one slice of one logits row with 16-byte
+// loads and keeps a running (maximum, sum of exponentials) pair; the slices of a row leave
+// their pairs in scratch.  The CTA that finishes last for a sequence combines them, tests the
+// steps, runs the level-synchronous longest-path relaxation, walks back, and samples the
+// regenerated token with a block-wide scan over that one row.
+#include "gsd_internal.cuh"
+#include <math_constants.h>
+
+namespace gsd {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kNone = 0x7FFFFFFF;
+constexpr int kNodeSlots = (GSD_MAX_NODES + kThreads - 1) / kThreads;
+constexpr int kEdgeCache = 3 * GSD_MAX_NODES;   // parent edges of one sequence kept in shared memory
+constexpr int kMaxSlices = 16;
+constexpr float kLog2e = 1.4426950408889634f;
+
+// (maximum, sum of 2^((x - maximum) * log2 e)) of a set of logits; the empty set is (-inf, 0)
+struct Ms {
+    float m, s;
+};
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ Ms combine(Ms a, Ms b) {
+    const float m = fmaxf(a.m, b.m);
+    if (m == -CUDART_INF_F) return Ms{m, 0.f};
+    return Ms{m, a.s * ex2((a.m - m) * kLog2e) + b.s * ex2((b.m - m) * kLog2e)};
+}
+
+// sixteen values at once: one rescale of the running sum per group
+__device__ __forceinline__ void take16(Ms& r, const float4& a, const float4& b, const float4& c, const float4& d) {
+    const float m4 = fmaxf(fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)), fmaxf(fmaxf(b.x, b.y), fmaxf(b.z, b.w)));
+    const float m8 = fmaxf(fmaxf(fmaxf(c.x, c.y), fmaxf(c.z, c.w)), fmaxf(fmaxf(d.x, d.y), fmaxf(d.z, d.w)));
+    const float m = fmaxf(r.m, fmaxf(m4, m8));
+    if (m == -CUDART_INF_F) return;
+    const float k = -m * kLog2e;
+    float s = r.s * ex2(fmaf(r.m, kLog2e, k));
+    s += ex2(fmaf(a.x, kLog2e, k)) + ex2(fmaf(a.y, kLog2e, k)) + ex2(fmaf(a.z, kLog2e, k)) + ex2(fmaf(a.w, kLog2e, k));
+    s += ex2(fmaf(b.x, kLog2e, k)) + ex2(fmaf(b.y, kLog2e, k)) + ex2(fmaf(b.z, kLog2e, k)) + ex2(fmaf(b.w, kLog2e, k));
+    s += ex2(fmaf(c.x, kLog2e, k)) + ex2(fmaf(c.y, kLog2e, k)) + ex2(fmaf(c.z, kLog2e, k)) + ex2(fmaf(c.w, kLog2e, k));
+    s += ex2(fmaf(d.x, kLog2e, k)) + ex2(fmaf(d.y, kLog2e, k)) + ex2(fmaf(d.z, kLog2e, k)) + ex2(fmaf(d.w, kLog2e, k));
+    r.m = m;
+    r.s = s;
+}
+
+__device__ __forceinline__ void take1(Ms& r, float x) {
+    r = combine(r, Ms{x, x == -CUDART_INF_F ? 0.f : 1.f});
+}
+
+struct SampledArgs {
+    const float* logits;
+    const int32_t* tok;
+    const int32_t* pptr;
+    const int32_t* pidx;
+    const float* q;
+    const float* u;
+    const float* us;
+    int32_t* out_tok;
+    int32_t* out_len;
+    int32_t* out_nodes;
+    float2* part;     // [B*N*slices] (maximum, sum) per slice
+    unsigned* done;   // [B], zeroed before the launch
+    int32_t* status;
+    int B, N, V, Ecap, Tcap, slices;
+};
+
+__device__ void finish_sequence(const SampledArgs& a, int b) {
+    __shared__ float s_mx[GSD_MAX_NODES];
+    __shared__ float s_sum[GSD_MAX_NODES];
+    __shared__ int s_best[GSD_MAX_NODES];
+    __shared__ int s_tok[GSD_MAX_NODES];
+    __shared__ int s_ptr[GSD_MAX_NODES + 1];
+    __shared__ int s_edge[kEdgeCache];
+    __shared__ unsigned char s_eok[kEdgeCache];
+    __shared__ int s_red[kThreads / 32];
+    __shared__ float s_scan[kThreads / 32];
+    __shared__ unsigned s_flags;
+    __shared__ int s_m, s_end, s_pick;
+    const int N = a.N, V = a.V, tid = threadIdx.x;
+    const int32_t* tok = a.tok + (size_t)b * N;
+    const int32_t* pptr = a.pptr + (size_t)b * (N + 1);
+    const int32_t* pidx = a.pidx + (size_t)b * a.Ecap;
+    const float* lg = a.logits + (size_t)b * N * V;
+    const float* q = a.q + (size_t)b * N;
+    const float* u = a.u + (size_t)b * N;
+    unsigned flags = 0;
+    if (tid == 0) s_flags = 0;
+    for (int v = tid; v < N; v += kThreads) {
+        // the pairs were written by other CTAs: read them past L1
+        Ms r{-CUDART_INF_F, 0.f};
+        for (int k = 0; k < a.slices; ++k) {
+            const float2 p = __ldcg(a.part + ((size_t)b * N + v) * a.slices + k);
+            r = combine(r, Ms{p.x, p.y});
+        }
+        s_mx[v] = r.m;
+        s_sum[v] = r.s;
+        if (!(r.s > 0.f) || r.m == CUDART_INF_F) flags |= GSD_DEV_BAD_LOGITS;   // no finite entry, +inf or NaN
+        const int t = tok[v];
+        s_tok[v] = t;
+        if (t < 0 || t >= V) flags |= GSD_DEV_BAD_TOKEN;
+        s_best[v] = v == 0 ? 0 : -1;
+    }
+    for (int v = tid; v <= N; v += kThreads) {
+        int e = pptr[v];
+        if (e < 0 || e > a.Ecap) {
+            flags |= GSD_DEV_BAD_CSR;
+            e = e < 0 ? 0 : a.Ecap;
+        }
+        s_ptr[v] = e;
+    }
+    __syncthreads();
+    // the test of one step: the target's probability of v's token under its parent p
+    auto step_ok = [&](int p, int v) -> bool {
+        const int t = s_tok[v];
+        if (t < 0 || t >= V) return false;
+        const float prob = ex2((lg[(size_t)p * V + t] - s_mx[p]) * kLog2e) / s_sum[p];
+        return u[v] * q[v] < prob;
+    };
+    const int n_edges = s_ptr[N];
+    const bool cached = n_edges <= kEdgeCache;
+    if (cached) {
+        // parent lists and the outcome of every step once, on chip
+        for (int v = tid; v < N; v += kThreads)
+            for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
+                const int p = pidx[e];
+                s_edge[e] = p;
+                s_eok[e] = (p >= 0 && p < v) ? (unsigned char)step_ok(p, v) : 0;
+            }
+        __syncthreads();
+    }
+
+    // level-synchronous relaxation of best[v] = 1 + max over accepted steps into v
+    for (int round = 0; round < N; ++round) {
+        int nb[kNodeSlots];
+        int changed = 0;
+#pragma unroll
+        for (int k = 0; k < kNodeSlots; ++k) {
+            const int v = tid + k * kThreads;
+            nb[k] = -1;
+            if (v > 0 && v < N) {
+                int cur = s_best[v];
+                for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
+                    const int p = cached ? s_edge[e] : pidx[e];
+                    if (p < 0 || p >= v) {
+                        flags |= GSD_DEV_BAD_CSR;
+                        continue;
+                    }
+                    const int bp = s_best[p];
+                    if (bp >= 0 && bp + 1 > cur && (cached ? s_eok[e] != 0 : step_ok(p, v))) cur = bp + 1;
+                }
+                nb[k] = cur;
+                changed |= (cur != s_best[v]);
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < kNodeSlots; ++k) {
+            const int v = tid + k * kThreads;
+            if (v > 0 && v < N) s_best[v] = nb[k];
+        }
+        if (!__syncthreads_or(changed)) break;
+    }
+
+    // end node: longest, then lowest index
+    int key = -1;
+    for (int v = tid; v < N; v += kThreads)
+        if (s_best[v] >= 0) key = max(key, (s_best[v] << 10) | (1023 - v));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xFFFFFFFFu, key, o));
+    if ((tid & 31) == 0) s_red[tid >> 5] = key;
+    if (flags) atomicOr(&s_flags, flags);
+    __syncthreads();
+
+    int32_t* out_tok = a.out_tok + (size_t)b * a.Tcap;
+    int32_t* out_nodes = a.out_nodes ? a.out_nodes + (size_t)b * a.Tcap : nullptr;
+    if (tid == 0) {
+        for (int w = 1; w < kThreads / 32; ++w) key = max(key, s_red[w]);
+        const int m = key >> 10;
+        int v = 1023 - (key & 1023);
+        s_end = v;
+        unsigned fl = s_flags;
+        if (m + 1 > a.Tcap) fl |= GSD_DEV_TCAP;
+        // walk back: the lowest predecessor with an accepted step that carries length - 1
+        for (int len = m; len >= 0; --len) {
+            if (out_nodes && len < a.Tcap) out_nodes[len] = v;
+            if (len == 0) break;
+            if (len - 1 < a.Tcap) out_tok[len - 1] = s_tok[v];
+            int pred = kNone;
+            for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
+                const int p = cached ? s_edge[e] : pidx[e];
+                if (p < 0 || p >= v) continue;
+                if (s_best[p] == len - 1 && p < pred && (cached ? s_eok[e] != 0 : step_ok(p, v))) pred = p;
+            }
+            if (pred == kNone) break;  // cannot happen for a consistent best[]
+            v = pred;
+        }
+        a.out_len[b] = m + 1;
+        s_m = m;
+        if (fl && a.status) atomicOr((unsigned*)a.status, fl);
+    }
+    __syncthreads();
+
+    // The regenerated token: thread t owns a contiguous piece of the end node's row; an
+    // inclusive scan of the pieces' sums finds the piece in which the cumulative sum first
+    // exceeds u * total, and that thread walks its piece.
+    {
+        const float* x = lg + (size_t)s_end * V;
+        const float mx = s_mx[s_end];
+        const int per = (V + kThreads - 1) / kThreads;
+        const int j0 = min(tid * per, V), j1 = min(j0 + per, V);
+        float mine = 0.f;
+        int last_pos = -1;
+        for (int j = j0; j < j1; ++j) {
+            const float e = ex2((x[j] - mx) * kLog2e);
+            mine += e;
+            if (e > 0.f) last_pos = j;
+        }
+        // inclusive scan over the 256 pieces
+        float inc = mine;
+        const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+            if (lane >= o) inc += t;
+        }
+        if (lane == 31) s_scan[warp] = inc;
+        if (tid == 0) s_pick = kNone;
+        __syncthreads();
+        float base = 0.f, total = 0.f;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) {
+            if (w < warp) base += s_scan[w];
+            total += s_scan[w];
+        }
+        inc += base;
+        const float target = a.us[b] * total;
+        const float before = inc - mine;
+        if (mine > 0.f && inc > target && !(before > target)) {
+            // the crossing lies in this piece (exactly one piece qualifies: the sums grow)
+            float cum = before;
+            int pick = last_pos;
+            for (int j = j0; j < j1; ++j) {
+                cum += ex2((x[j] - mx) * kLog2e);
+                if (cum > target) { pick = j; break; }
+            }
+            atomicMin(&s_pick, pick);
+        }
+        // if rounding left no crossing: the last entry with any mass
+        int lp = last_pos;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) lp = max(lp, __shfl_xor_sync(0xFFFFFFFFu, lp, o));
+        if (lane == 0) s_red[warp] = lp;
+        __syncthreads();
+        if (tid == 0) {
+            int pick = s_pick;
+            if (pick == kNone) {
+                pick = -1;
+                for (int w = 0; w < kThreads / 32; ++w) pick = max(pick, s_red[w]);
+            }
+            if (s_m < a.Tcap) out_tok[s_m] = pick;
+        }
+    }
+    for (int i = s_m + 1 + tid; i < a.Tcap; i += kThreads) {
+        out_tok[i] = -1;
+        if (out_nodes) out_nodes[i] = -1;
+    }
+}
+
+template <bool kVec>
+__global__ void __launch_bounds__(kThreads) accept_sampled_kernel(SampledArgs a) {
+    __shared__ Ms sh[kThreads / 32];
+    __shared__ int s_last;
+    const int row = blockIdx.y;  // b * N + n
+    const int slice = blockIdx.x;
+    const float* x = a.logits + (size_t)row * a.V;
+    Ms r{-CUDART_INF_F, 0.f};
+    if (kVec) {
+        const int nvec = a.V >> 2;
+        const int per = (nvec + a.slices - 1) / a.slices;
+        const int v0 = min(slice * per, nvec), v1 = min(v0 + per, nvec);
+        const float4* x4 = reinterpret_cast<const float4*>(x);
+        int i = v0 + threadIdx.x;
+        // four independent 16-byte loads in flight per thread
+        for (; i + 3 * kThreads < v1; i += 4 * kThreads) {
+            const float4 r0 = __ldcs(x4 + i), r1 = __ldcs(x4 + i + kThreads);
+            const float4 r2 = __ldcs(x4 + i + 2 * kThreads), r3 = __ldcs(x4 + i + 3 * kThreads);
+            take16(r, r0, r1, r2, r3);
+        }
+        for (; i < v1; i += kThreads) {
+            const float4 t = __ldcs(x4 + i);
+            take1(r, t.x); take1(r, t.y); take1(r, t.z); take1(r, t.w);
+        }
+    } else {
+        const int per = (a.V + a.slices - 1) / a.slices;
+        const int lo = min(slice * per, a.V), hi = min(lo + per, a.V);
+        for (int i = lo + threadIdx.x; i < hi; i += kThreads) take1(r, __ldcs(x + i));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Ms t;
+        t.m = __shfl_xor_sync(0xFFFFFFFFu, r.m, o);
+        t.s = __shfl_xor_sync(0xFFFFFFFFu, r.s, o);
+        r = combine(r, t);
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) sh[warp] = r;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < kThreads / 32; ++w) r = combine(r, sh[w]);
+        a.part[(size_t)row * a.slices + slice] = make_float2(r.m, r.s);
+        __threadfence();
+        const int b = row / a.N;
+        const unsigned prev = atomicAdd(a.done + b, 1u);
+        s_last = (prev == (unsigned)(a.N * a.slices) - 1u);
+    }
+    __syncthreads();
+    if (s_last) {
+        __threadfence();
+        finish_sequence(a, row / a.N);
+    }
+}
+
+int pick_slices(long rows, int V, int sm_count) {
+    // enough CTAs to cover the machine a few times over, slices of at least 4096 floats
+    int slices = 1;
+    const long want = (long)sm_count * 8;
+    while (rows * slices < want && (V / (slices * 2)) >= 4096 && slices * 2 <= kMaxSlices) slices *= 2;
+    return slices;
+}
+
+}  // namespace
+}  // namespace gsd
+
+extern "C" size_t gsd_accept_sampled_workspace_bytes(const gsd_accept_params* p) {
+    if (!p || p->B < 1 || p->N < 1 || p->N > GSD_MAX_NODES) return 0;
+    return gsd::align_up((size_t)p->B * p->N * gsd::kMaxSlices * 8 + (size_t)p->B * 4, 256);
+}
+
+extern "C" int gsd_accept_sampled(const float* logits, const int32_t* draft_tokens,
+                                  const int32_t* parent_ptr, const int32_t* parent_idx,
+                                  const float* draft_q, const float* u_accept, const float* u_sample,
+                                  int32_t* accepted_tokens, int32_t* accepted_len,
+                                  int32_t* accepted_nodes, const gsd_accept_params* p,
+                                  void* workspace, size_t workspace_bytes, int32_t* status,
+                                  void* stream) {
+    using namespace gsd;
+    if (!p || !logits || !draft_tokens || !parent_ptr || !parent_idx || !draft_q || !u_accept ||
+        !u_sample || !accepted_tokens || !accepted_len)
+        return GSD_ERR_NULL_POINTER;
+    if (p->B < 1 || p->N < 1 || p->N > GSD_MAX_NODES || p->V < 1 || p->Ecap < 1 || p->Tcap < 1)
+        return GSD_ERR_BAD_SHAPE;
+    if ((long long)p->B * p->N > (1ll << 30)) return GSD_ERR_BAD_SHAPE;
+    if (((uintptr_t)logits & 3u) != 0) return GSD_ERR_MISALIGNED;
+    const size_t need = gsd_accept_sampled_workspace_bytes(p);
+    if (!workspace || workspace_bytes < need) return GSD_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 7u) != 0) return GSD_ERR_MISALIGNED;
+    DeviceInfo di;
+    if (device_info(&di) != 0) return GSD_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    SampledArgs a;
+    a.logits = logits; a.tok = draft_tokens; a.pptr = parent_ptr; a.pidx = parent_idx;
+    a.q = draft_q; a.u = u_accept; a.us = u_sample;
+    a.out_tok = accepted_tokens; a.out_len = accepted_len; a.out_nodes = accepted_nodes;
+    a.part = (float2*)workspace;
+    const size_t part_bytes = (size_t)p->B * p->N * kMaxSlices * 8;
+    a.done = (unsigned*)((char*)workspace + part_bytes);
+    a.status = status;
+    a.B = p->B; a.N = p->N; a.V = p->V; a.Ecap = p->Ecap; a.Tcap = p->Tcap;
+    const bool vec = (p->V % 4 == 0) && (((uintptr_t)logits & 15u) == 0);
+    a.slices = pick_slices((long)p->B * p->N, p->V, di.sm_count);
+
+    // only the completion counters have to start at zero; every pair is written before it is read
+    GSD_CUDA_TRY(cudaMemsetAsync(a.done, 0, (size_t)p->B * 4, st));
+    // grid.y holds at most 65535 rows: larger problems go out in blocks of whole sequences
+    const int seq_per = 65535 / p->N;
+    for (int b0 = 0; b0 < p->B; b0 += seq_per) {
+        const int nb = (p->B - b0 < seq_per) ? p->B - b0 : seq_per;
+        SampledArgs s = a;
+        s.logits += (size_t)b0 * p->N * p->V; s.tok += (size_t)b0 * p->N;
+        s.pptr += (size_t)b0 * (p->N + 1); s.pidx += (size_t)b0 * p->Ecap;
+        s.q += (size_t)b0 * p->N; s.u += (size_t)b0 * p->N; s.us += b0;
+        s.out_tok += (size_t)b0 * p->Tcap; s.out_len += b0;
+        if (s.out_nodes) s.out_nodes += (size_t)b0 * p->Tcap;
+        s.part += (size_t)b0 * p->N * a.slices; s.done += b0; s.B = nb;
+        dim3 grid(a.slices, (unsigned)(nb * p->N));
+        if (vec) accept_sampled_kernel<true><<<grid, kThreads, 0, st>>>(s);
+        else accept_sampled_kernel<false><<<grid, kThreads, 0, st>>>(s);
+    }
+    GSD_CUDA_TRY(cudaGetLastError());
+    return GSD_OK;
+}
