@@ -305,6 +305,28 @@ def main():
         commit_us = statistics.median(a.elapsed_time(b) for a, b in ev_c) * 1e3
         del kc2, vc2
 
+    # ---- non-deterministic verification (gsd_accept_sampled) on the same logits, timed on its
+    # own with the two input sets rotated; it is not part of `value`
+    sampled_us = None
+    if rank == 0:
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(7)
+        dq = torch.rand((cfg.B, cfg.N), device=dev, generator=gen) * 0.5 + 0.01
+        ua = torch.rand((cfg.B, cfg.N), device=dev, generator=gen)
+        usm = torch.rand((cfg.B,), device=dev, generator=gen)
+        ws_s = torch.empty(gsd.gsd_accept_sampled_workspace_bytes(cfg.B, cfg.N), dtype=torch.uint8, device=dev)
+        ev_s = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(20)]
+        for i in range(23):
+            ts = sets[i % len(sets)]
+            if i >= 3:
+                ev_s[i - 3][0].record()
+            gsd.gsd_accept_sampled(ts["logits"], ts["draft_tokens"], ts["parent_ptr"], ts["parent_idx"], dq, ua, usm,
+                                   workspace=ws_s, status=status)
+            if i >= 3:
+                ev_s[i - 3][1].record()
+        torch.cuda.synchronize()
+        sampled_us = statistics.median(a.elapsed_time(b) for a, b in ev_s) * 1e3
+
     # ---- end to end through the host-buffer C-ABI call (pinned host tensors)
     e2e = None
     if args.e2e_steps > 0:
@@ -391,7 +413,7 @@ def main():
                    "D": cfg.D, "L": cfg.L, "V": cfg.V, "depth": cfg.depth,
                    "l2": "two input sets rotated; each step reads more than the L2 size",
                    "replicas": world, "attn_kernel": args.kernel, "num_splits": splits},
-        "attn_us": attn_mean * 1e6, "accept_us": acc_mean * 1e6, "commit_kv_us": commit_us,
+        "attn_us": attn_mean * 1e6, "accept_us": acc_mean * 1e6, "commit_kv_us": commit_us, "accept_sampled_us": sampled_us,
         "attn_tokens_per_s": tokens / attn_mean,
         "accept_gbs": accept_bytes / acc_mean / 1e9,
         "accept_frac_of_hbm": accept_bytes / acc_mean / 1e9 / peaks["hbm_gbs"],

@@ -230,6 +230,11 @@ def gsd_accept(logits, draft_tokens, parent_ptr, parent_idx, *, Tcap: int = 0,
     return toks, lens, nodes
 
 
+def gsd_accept_sampled_workspace_bytes(B, N) -> int:
+    p = AcceptParams(B, N, 1, 1, 1)
+    return int(lib().gsd_accept_sampled_workspace_bytes(ctypes.byref(p)))
+
+
 def gsd_accept_sampled(logits, draft_tokens, parent_ptr, parent_idx, draft_q, u_accept, u_sample, *,
                        Tcap: int = 0, want_nodes: bool = True, workspace: Optional[torch.Tensor] = None,
                        status: Optional[torch.Tensor] = None
