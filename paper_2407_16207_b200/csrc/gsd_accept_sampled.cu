@@ -87,6 +87,7 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     __shared__ int s_ptr[GSD_MAX_NODES + 1];
     __shared__ int s_edge[kEdgeCache];
     __shared__ unsigned char s_eok[kEdgeCache];
+    __shared__ short s_enode[kEdgeCache];          // the node an edge leads into
     __shared__ int s_red[kThreads / 32];
     __shared__ float s_scan[kThreads / 32];
     __shared__ unsigned s_flags;
@@ -134,13 +135,16 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     const int n_edges = s_ptr[N];
     const bool cached = n_edges <= kEdgeCache;
     if (cached) {
-        // parent lists and the outcome of every step once, on chip
+        // parent lists and the outcome of every step once, on chip; the tests gather one logit
+        // each from global memory, so they go out one per thread, all at once
         for (int v = tid; v < N; v += kThreads)
-            for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
-                const int p = pidx[e];
-                s_edge[e] = p;
-                s_eok[e] = (p >= 0 && p < v) ? (unsigned char)step_ok(p, v) : 0;
-            }
+            for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) s_enode[e] = (short)v;
+        __syncthreads();
+        for (int e = tid; e < n_edges; e += kThreads) {
+            const int p = pidx[e], v = s_enode[e];
+            s_edge[e] = p;
+            s_eok[e] = (p >= 0 && p < v) ? (unsigned char)step_ok(p, v) : 0;
+        }
         __syncthreads();
     }
 
@@ -215,43 +219,68 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     }
     __syncthreads();
 
-    // The regenerated token: thread t owns a contiguous piece of the end node's row; an
-    // inclusive scan of the pieces' sums finds the piece in which the cumulative sum first
-    // exceeds u * total, and that thread walks its piece.
+    // The regenerated token.  Phase 1: warp w owns the contiguous range w of the end node's row
+    // and sums it with coalesced loads; an exclusive prefix over the 8 warp sums finds the range
+    // in which the cumulative sum first exceeds u * total.  Phase 2: the whole block splits that
+    // range into 256 contiguous pieces, scans the piece sums, and the thread whose piece holds
+    // the crossing walks it.
     {
         const float* x = lg + (size_t)s_end * V;
         const float mx = s_mx[s_end];
-        const int per = (V + kThreads - 1) / kThreads;
-        const int j0 = min(tid * per, V), j1 = min(j0 + per, V);
+        const int lane = tid & 31, warp = tid >> 5;
+        constexpr int kWarps = kThreads / 32;
+        const int wper = (V + kWarps - 1) / kWarps;
+        const int w0 = min(warp * wper, V), w1 = min(w0 + wper, V);
         float mine = 0.f;
+        for (int j = w0 + lane; j < w1; j += 32) mine += ex2((x[j] - mx) * kLog2e);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, o);
+        if (lane == 0) s_scan[warp] = mine;
+        if (tid == 0) s_pick = kNone;
+        __syncthreads();
+        float total = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) total += s_scan[w];
+        const float target = a.us[b] * total;
+        // the first range whose inclusive prefix exceeds the target (the last non-empty one if none does)
+        int rw = -1, last_w = 0;
+        float before_range = 0.f, run = 0.f, before_last = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            const float sw = s_scan[w];
+            if (rw < 0 && run + sw > target) { rw = w; before_range = run; }
+            if (sw > 0.f) { last_w = w; before_last = run; }
+            run += sw;
+        }
+        const bool crossing = rw >= 0;
+        if (!crossing) { rw = last_w; before_range = before_last; }
+        __syncthreads();                                  // s_scan is reused below
+        // phase 2 inside range rw
+        const int r0 = min(rw * wper, V), r1 = min(r0 + wper, V);
+        const int per = (r1 - r0 + kThreads - 1) / kThreads;
+        const int j0 = min(r0 + tid * per, r1), j1 = min(j0 + per, r1);
+        float piece = 0.f;
         int last_pos = -1;
         for (int j = j0; j < j1; ++j) {
             const float e = ex2((x[j] - mx) * kLog2e);
-            mine += e;
+            piece += e;
             if (e > 0.f) last_pos = j;
         }
-        // inclusive scan over the 256 pieces
-        float inc = mine;
-        const int lane = tid & 31, warp = tid >> 5;
+        float inc = piece;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const float t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
             if (lane >= o) inc += t;
         }
         if (lane == 31) s_scan[warp] = inc;
-        if (tid == 0) s_pick = kNone;
         __syncthreads();
-        float base = 0.f, total = 0.f;
+        float base = before_range;
 #pragma unroll
-        for (int w = 0; w < kThreads / 32; ++w) {
+        for (int w = 0; w < kWarps; ++w)
             if (w < warp) base += s_scan[w];
-            total += s_scan[w];
-        }
         inc += base;
-        const float target = a.us[b] * total;
-        const float before = inc - mine;
-        if (mine > 0.f && inc > target && !(before > target)) {
-            // the crossing lies in this piece (exactly one piece qualifies: the sums grow)
+        const float before = inc - piece;
+        if (crossing && piece > 0.f && inc > target && !(before > target)) {
             float cum = before;
             int pick = last_pos;
             for (int j = j0; j < j1; ++j) {
@@ -260,7 +289,7 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
             }
             atomicMin(&s_pick, pick);
         }
-        // if rounding left no crossing: the last entry with any mass
+        // if rounding left no crossing: the last entry with any mass (it lies in range rw)
         int lp = last_pos;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) lp = max(lp, __shfl_xor_sync(0xFFFFFFFFu, lp, o));
@@ -270,7 +299,7 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
             int pick = s_pick;
             if (pick == kNone) {
                 pick = -1;
-                for (int w = 0; w < kThreads / 32; ++w) pick = max(pick, s_red[w]);
+                for (int w = 0; w < kWarps; ++w) pick = max(pick, s_red[w]);
             }
             if (s_m < a.Tcap) out_tok[s_m] = pick;
         }
