@@ -77,6 +77,7 @@ struct SampledArgs {
     unsigned* done;   // [B], zeroed before the launch
     int32_t* status;
     int B, N, V, Ecap, Tcap, slices;
+    int vec;          // rows are read as float4 (decides where the slices of a row begin)
 };
 
 __device__ void finish_sequence(const SampledArgs& a, int b) {
@@ -219,18 +220,39 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     }
     __syncthreads();
 
-    // The regenerated token.  Phase 1: warp w owns the contiguous range w of the end node's row
-    // and sums it with coalesced loads; an exclusive prefix over the 8 warp sums finds the range
-    // in which the cumulative sum first exceeds u * total.  Phase 2: the whole block splits that
-    // range into 256 contiguous pieces, scans the piece sums, and the thread whose piece holds
-    // the crossing walks it.
+    // The regenerated token.  Phase 0: the per-slice sums of the streaming pass already say in
+    // which slice of the end node's row the cumulative sum first exceeds u * total.  Phase 1:
+    // warp w owns the contiguous range w of that slice and sums it with coalesced loads; an
+    // exclusive prefix over the 8 warp sums narrows the crossing down to one range.  Phase 2:
+    // the whole block splits that range into 256 contiguous pieces, scans the piece sums, and
+    // the thread whose piece holds the crossing walks it.
     {
         const float* x = lg + (size_t)s_end * V;
         const float mx = s_mx[s_end];
         const int lane = tid & 31, warp = tid >> 5;
         constexpr int kWarps = kThreads / 32;
-        const int wper = (V + kWarps - 1) / kWarps;
-        const int w0 = min(warp * wper, V), w1 = min(w0 + wper, V);
+        // phase 0 (every thread computes the same)
+        int lo = 0, hi = V;
+        float before_slice = 0.f;
+        {
+            const float tgt = a.us[b] * s_sum[s_end];
+            const int unit = a.vec ? 4 : 1, n = a.vec ? (V >> 2) : V;
+            const int sper = (n + a.slices - 1) / a.slices;
+            float run = 0.f;
+            for (int k = 0; k < a.slices; ++k) {
+                const float2 pr = __ldcg(a.part + ((size_t)b * N + s_end) * a.slices + k);
+                const float sk = pr.x == -CUDART_INF_F ? 0.f : pr.y * ex2((pr.x - mx) * kLog2e);
+                lo = min(k * sper, n) * unit;
+                hi = min(k * sper + sper, n) * unit;
+                before_slice = run;
+                run += sk;
+                if (run > tgt) break;
+            }
+            // a crossing that rounding leaves out of every slice is handled below (last entry with mass)
+            if (!(run > tgt)) { lo = 0; hi = V; before_slice = 0.f; }
+        }
+        const int wper = (hi - lo + kWarps - 1) / kWarps;
+        const int w0 = min(lo + warp * wper, hi), w1 = min(w0 + wper, hi);
         float mine = 0.f;
         for (int j = w0 + lane; j < w1; j += 32) mine += ex2((x[j] - mx) * kLog2e);
 #pragma unroll
@@ -238,13 +260,10 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
         if (lane == 0) s_scan[warp] = mine;
         if (tid == 0) s_pick = kNone;
         __syncthreads();
-        float total = 0.f;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) total += s_scan[w];
-        const float target = a.us[b] * total;
+        const float target = a.us[b] * s_sum[s_end];
         // the first range whose inclusive prefix exceeds the target (the last non-empty one if none does)
         int rw = -1, last_w = 0;
-        float before_range = 0.f, run = 0.f, before_last = 0.f;
+        float before_range = before_slice, run = before_slice, before_last = before_slice;
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) {
             const float sw = s_scan[w];
@@ -256,7 +275,7 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
         if (!crossing) { rw = last_w; before_range = before_last; }
         __syncthreads();                                  // s_scan is reused below
         // phase 2 inside range rw
-        const int r0 = min(rw * wper, V), r1 = min(r0 + wper, V);
+        const int r0 = min(lo + rw * wper, hi), r1 = min(r0 + wper, hi);
         const int per = (r1 - r0 + kThreads - 1) / kThreads;
         const int j0 = min(r0 + tid * per, r1), j1 = min(j0 + per, r1);
         float piece = 0.f;
@@ -413,6 +432,7 @@ extern "C" int gsd_accept_sampled(const float* logits, const int32_t* draft_toke
     a.B = p->B; a.N = p->N; a.V = p->V; a.Ecap = p->Ecap; a.Tcap = p->Tcap;
     const bool vec = (p->V % 4 == 0) && (((uintptr_t)logits & 15u) == 0);
     a.slices = pick_slices((long)p->B * p->N, p->V, di.sm_count);
+    a.vec = vec ? 1 : 0;
 
     // only the completion counters have to start at zero; every pair is written before it is read
     GSD_CUDA_TRY(cudaMemsetAsync(a.done, 0, (size_t)p->B * 4, st));
