@@ -23,6 +23,7 @@ constexpr int kNone = 0x7FFFFFFF;
 constexpr int kNodeSlots = (GSD_MAX_NODES + kThreads - 1) / kThreads;
 constexpr int kEdgeCache = 3 * GSD_MAX_NODES;   // parent edges of one sequence kept in shared memory
 constexpr int kMaxSlices = 16;
+constexpr int kWarps = kThreads / 32;   // each warp of a CTA sums a contiguous eighth of the CTA's slice
 constexpr float kLog2e = 1.4426950408889634f;
 
 // (maximum, sum of 2^((x - maximum) * log2 e)) of a set of logits; the empty set is (-inf, 0)
@@ -62,6 +63,19 @@ __device__ __forceinline__ void take1(Ms& r, float x) {
     r = combine(r, Ms{x, x == -CUDART_INF_F ? 0.f : 1.f});
 }
 
+// The row is cut into slices (one CTA each) and every slice into kWarps contiguous ranges (one
+// warp each); in units of float4 when the row is read that way.  Range r = slice * kWarps + warp.
+__device__ __forceinline__ void range_of(int V, int slices, int vec, int r, int& lo, int& hi) {
+    const int unit = vec ? 4 : 1, n = vec ? (V >> 2) : V;
+    const int per = (n + slices - 1) / slices;
+    const int slice = r / kWarps, warp = r % kWarps;
+    const int v0 = min(slice * per, n), v1 = min(v0 + per, n);
+    const int wlen = (v1 - v0 + kWarps - 1) / kWarps;
+    const int a0 = min(v0 + warp * wlen, v1), a1 = min(a0 + wlen, v1);
+    lo = a0 * unit;
+    hi = a1 * unit;
+}
+
 struct SampledArgs {
     const float* logits;
     const int32_t* tok;
@@ -73,7 +87,7 @@ struct SampledArgs {
     int32_t* out_tok;
     int32_t* out_len;
     int32_t* out_nodes;
-    float2* part;     // [B*N*slices] (maximum, sum) per slice
+    float2* part;     // [B*N][slices][kWarps] (maximum, sum) of contiguous ranges of the row, in order
     unsigned* done;   // [B], zeroed before the launch
     int32_t* status;
     int B, N, V, Ecap, Tcap, slices;
@@ -105,8 +119,8 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     for (int v = tid; v < N; v += kThreads) {
         // the pairs were written by other CTAs: read them past L1
         Ms r{-CUDART_INF_F, 0.f};
-        for (int k = 0; k < a.slices; ++k) {
-            const float2 p = __ldcg(a.part + ((size_t)b * N + v) * a.slices + k);
+        for (int k = 0; k < a.slices * kWarps; ++k) {
+            const float2 p = __ldcg(a.part + ((size_t)b * N + v) * a.slices * kWarps + k);
             r = combine(r, Ms{p.x, p.y});
         }
         s_mx[v] = r.m;
@@ -220,62 +234,35 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     }
     __syncthreads();
 
-    // The regenerated token.  Phase 0: the per-slice sums of the streaming pass already say in
-    // which slice of the end node's row the cumulative sum first exceeds u * total.  Phase 1:
-    // warp w owns the contiguous range w of that slice and sums it with coalesced loads; an
-    // exclusive prefix over the 8 warp sums narrows the crossing down to one range.  Phase 2:
-    // the whole block splits that range into 256 contiguous pieces, scans the piece sums, and
-    // the thread whose piece holds the crossing walks it.
+    // The regenerated token.  The sums of the streaming pass over the row's contiguous ranges
+    // (slices x warps, kept in scratch) say in which range the cumulative sum first exceeds
+    // u * total; the whole block then splits that range into 256 contiguous pieces, scans the
+    // piece sums, and the thread whose piece holds the crossing walks it.
     {
         const float* x = lg + (size_t)s_end * V;
         const float mx = s_mx[s_end];
         const int lane = tid & 31, warp = tid >> 5;
-        constexpr int kWarps = kThreads / 32;
-        // phase 0 (every thread computes the same)
-        int lo = 0, hi = V;
-        float before_slice = 0.f;
-        {
-            const float tgt = a.us[b] * s_sum[s_end];
-            const int unit = a.vec ? 4 : 1, n = a.vec ? (V >> 2) : V;
-            const int sper = (n + a.slices - 1) / a.slices;
-            float run = 0.f;
-            for (int k = 0; k < a.slices; ++k) {
-                const float2 pr = __ldcg(a.part + ((size_t)b * N + s_end) * a.slices + k);
-                const float sk = pr.x == -CUDART_INF_F ? 0.f : pr.y * ex2((pr.x - mx) * kLog2e);
-                lo = min(k * sper, n) * unit;
-                hi = min(k * sper + sper, n) * unit;
-                before_slice = run;
-                run += sk;
-                if (run > tgt) break;
-            }
-            // a crossing that rounding leaves out of every slice is handled below (last entry with mass)
-            if (!(run > tgt)) { lo = 0; hi = V; before_slice = 0.f; }
-        }
-        const int wper = (hi - lo + kWarps - 1) / kWarps;
-        const int w0 = min(lo + warp * wper, hi), w1 = min(w0 + wper, hi);
-        float mine = 0.f;
-        for (int j = w0 + lane; j < w1; j += 32) mine += ex2((x[j] - mx) * kLog2e);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, o);
-        if (lane == 0) s_scan[warp] = mine;
-        if (tid == 0) s_pick = kNone;
-        __syncthreads();
         const float target = a.us[b] * s_sum[s_end];
-        // the first range whose inclusive prefix exceeds the target (the last non-empty one if none does)
-        int rw = -1, last_w = 0;
-        float before_range = before_slice, run = before_slice, before_last = before_slice;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
-            const float sw = s_scan[w];
-            if (rw < 0 && run + sw > target) { rw = w; before_range = run; }
-            if (sw > 0.f) { last_w = w; before_last = run; }
-            run += sw;
+        // every thread walks the (at most 128) range sums: the first range whose inclusive
+        // prefix exceeds the target, or the last one with any mass if rounding leaves none
+        int rsel = -1, last_r = 0;
+        float before_range = 0.f, before_last = 0.f;
+        {
+            float run = 0.f;
+            const float2* pr = a.part + ((size_t)b * N + s_end) * a.slices * kWarps;
+            for (int r = 0; r < a.slices * kWarps; ++r) {
+                const float2 t = __ldcg(pr + r);
+                const float sr = t.x == -CUDART_INF_F ? 0.f : t.y * ex2((t.x - mx) * kLog2e);
+                if (rsel < 0 && run + sr > target) { rsel = r; before_range = run; }
+                if (sr > 0.f) { last_r = r; before_last = run; }
+                run += sr;
+            }
         }
-        const bool crossing = rw >= 0;
-        if (!crossing) { rw = last_w; before_range = before_last; }
-        __syncthreads();                                  // s_scan is reused below
-        // phase 2 inside range rw
-        const int r0 = min(lo + rw * wper, hi), r1 = min(r0 + wper, hi);
+        const bool crossing = rsel >= 0;
+        if (!crossing) { rsel = last_r; before_range = before_last; }
+        if (tid == 0) s_pick = kNone;
+        int r0, r1;
+        range_of(V, a.slices, a.vec, rsel, r0, r1);
         const int per = (r1 - r0 + kThreads - 1) / kThreads;
         const int j0 = min(r0 + tid * per, r1), j1 = min(j0 + per, r1);
         float piece = 0.f;
@@ -308,7 +295,7 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
             }
             atomicMin(&s_pick, pick);
         }
-        // if rounding left no crossing: the last entry with any mass (it lies in range rw)
+        // if rounding left no crossing: the last entry with any mass (it lies in the chosen range)
         int lp = last_pos;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) lp = max(lp, __shfl_xor_sync(0xFFFFFFFFu, lp, o));
@@ -331,32 +318,30 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
 
 template <bool kVec>
 __global__ void __launch_bounds__(kThreads) accept_sampled_kernel(SampledArgs a) {
-    __shared__ Ms sh[kThreads / 32];
     __shared__ int s_last;
     const int row = blockIdx.y;  // b * N + n
     const int slice = blockIdx.x;
     const float* x = a.logits + (size_t)row * a.V;
     Ms r{-CUDART_INF_F, 0.f};
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int lo, hi;
+    range_of(a.V, a.slices, kVec ? 1 : 0, slice * kWarps + warp, lo, hi);
     if (kVec) {
-        const int nvec = a.V >> 2;
-        const int per = (nvec + a.slices - 1) / a.slices;
-        const int v0 = min(slice * per, nvec), v1 = min(v0 + per, nvec);
         const float4* x4 = reinterpret_cast<const float4*>(x);
-        int i = v0 + threadIdx.x;
-        // four independent 16-byte loads in flight per thread
-        for (; i + 3 * kThreads < v1; i += 4 * kThreads) {
-            const float4 r0 = __ldcs(x4 + i), r1 = __ldcs(x4 + i + kThreads);
-            const float4 r2 = __ldcs(x4 + i + 2 * kThreads), r3 = __ldcs(x4 + i + 3 * kThreads);
+        const int a1 = hi >> 2;
+        int i = (lo >> 2) + lane;
+        // four independent 16-byte loads in flight per thread, each a 512-byte run per warp
+        for (; i + 3 * 32 < a1; i += 4 * 32) {
+            const float4 r0 = __ldcs(x4 + i), r1 = __ldcs(x4 + i + 32);
+            const float4 r2 = __ldcs(x4 + i + 64), r3 = __ldcs(x4 + i + 96);
             take16(r, r0, r1, r2, r3);
         }
-        for (; i < v1; i += kThreads) {
+        for (; i < a1; i += 32) {
             const float4 t = __ldcs(x4 + i);
             take1(r, t.x); take1(r, t.y); take1(r, t.z); take1(r, t.w);
         }
     } else {
-        const int per = (a.V + a.slices - 1) / a.slices;
-        const int lo = min(slice * per, a.V), hi = min(lo + per, a.V);
-        for (int i = lo + threadIdx.x; i < hi; i += kThreads) take1(r, __ldcs(x + i));
+        for (int i = lo + lane; i < hi; i += 32) take1(r, __ldcs(x + i));
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -365,13 +350,10 @@ __global__ void __launch_bounds__(kThreads) accept_sampled_kernel(SampledArgs a)
         t.s = __shfl_xor_sync(0xFFFFFFFFu, r.s, o);
         r = combine(r, t);
     }
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (lane == 0) sh[warp] = r;
+    if (lane == 0) a.part[((size_t)row * a.slices + slice) * kWarps + warp] = make_float2(r.m, r.s);
+    __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
-        for (int w = 1; w < kThreads / 32; ++w) r = combine(r, sh[w]);
-        a.part[(size_t)row * a.slices + slice] = make_float2(r.m, r.s);
-        __threadfence();
         const int b = row / a.N;
         const unsigned prev = atomicAdd(a.done + b, 1u);
         s_last = (prev == (unsigned)(a.N * a.slices) - 1u);
@@ -396,7 +378,7 @@ int pick_slices(long rows, int V, int sm_count) {
 
 extern "C" size_t gsd_accept_sampled_workspace_bytes(const gsd_accept_params* p) {
     if (!p || p->B < 1 || p->N < 1 || p->N > GSD_MAX_NODES) return 0;
-    return gsd::align_up((size_t)p->B * p->N * gsd::kMaxSlices * 8 + (size_t)p->B * 4, 256);
+    return gsd::align_up((size_t)p->B * p->N * gsd::kMaxSlices * gsd::kWarps * 8 + (size_t)p->B * 4, 256);
 }
 
 extern "C" int gsd_accept_sampled(const float* logits, const int32_t* draft_tokens,
@@ -426,7 +408,7 @@ extern "C" int gsd_accept_sampled(const float* logits, const int32_t* draft_toke
     a.q = draft_q; a.u = u_accept; a.us = u_sample;
     a.out_tok = accepted_tokens; a.out_len = accepted_len; a.out_nodes = accepted_nodes;
     a.part = (float2*)workspace;
-    const size_t part_bytes = (size_t)p->B * p->N * kMaxSlices * 8;
+    const size_t part_bytes = (size_t)p->B * p->N * kMaxSlices * kWarps * 8;
     a.done = (unsigned*)((char*)workspace + part_bytes);
     a.status = status;
     a.B = p->B; a.N = p->N; a.V = p->V; a.Ecap = p->Ecap; a.Tcap = p->Tcap;
@@ -446,7 +428,7 @@ extern "C" int gsd_accept_sampled(const float* logits, const int32_t* draft_toke
         s.q += (size_t)b0 * p->N; s.u += (size_t)b0 * p->N; s.us += b0;
         s.out_tok += (size_t)b0 * p->Tcap; s.out_len += b0;
         if (s.out_nodes) s.out_nodes += (size_t)b0 * p->Tcap;
-        s.part += (size_t)b0 * p->N * a.slices; s.done += b0; s.B = nb;
+        s.part += (size_t)b0 * p->N * a.slices * kWarps; s.done += b0; s.B = nb;
         dim3 grid(a.slices, (unsigned)(nb * p->N));
         if (vec) accept_sampled_kernel<true><<<grid, kThreads, 0, st>>>(s);
         else accept_sampled_kernel<false><<<grid, kThreads, 0, st>>>(s);
