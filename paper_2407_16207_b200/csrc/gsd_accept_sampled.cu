@@ -8,10 +8,11 @@
 // distribution in index order with u_sample.
 //
 // One launch.  Grid (slices, B*N): each CTA streams one slice of one logits row with 16-byte
-// loads and keeps a running (maximum, sum of exponentials) pair; the slices of a row leave
-// their pairs in scratch.  The CTA that finishes last for a sequence combines them, tests the
-// steps, runs the level-synchronous longest-path relaxation, walks back, and samples the
-// regenerated token with a block-wide scan over that one row.
+// loads; each of its warps owns a contiguous eighth of the slice and keeps a running
+// (maximum, sum of exponentials) pair, which it leaves in scratch.  The CTA that finishes last
+// for a sequence combines the pairs per node, tests the steps, runs the level-synchronous
+// longest-path relaxation, walks back, and finds the regenerated token: the range sums in
+// scratch give the range of the crossing, a block-wide scan over that range gives the index.
 #include "gsd_internal.cuh"
 #include <math_constants.h>
 
