@@ -168,6 +168,30 @@ def test_sweep_points_sampled_rows(point):
     assert_close(np.stack([got[b, n, h] for b, n, h in rows]), want)
 
 
+RANDOM_SHAPES = []
+_rng = np.random.default_rng(20240716)
+for _i in range(24):
+    _G = int(_rng.choice([1, 2, 4, 8, 16]))
+    _Hkv = int(_rng.choice([1, 2, 3]))
+    _N = int(_rng.integers(1, 330))
+    _lo = int(_rng.integers(0, 500))
+    RANDOM_SHAPES.append((int(_rng.integers(1, 4)), _G * _Hkv, _Hkv, (_lo, _lo + int(_rng.integers(0, 400))), _N,
+                          int(_rng.choice([0, 0, 1, 2, 3, 5]))))
+
+
+@pytest.mark.parametrize("shape", RANDOM_SHAPES, ids=[f"B{b}_Hq{hq}_Hkv{hk}_L{l[0]}-{l[1]}_N{n}_s{sp}" for b, hq, hk, l, n, sp in RANDOM_SHAPES])
+def test_random_shapes_full_compare(shape):
+    # odd sizes: rows that do not fill a tile, one- and two-row-tile units in one call, empty and
+    # ragged prefixes that differ per sequence, one to three draft tiles, forced split counts
+    B, Hq, Hkv, L, N, splits = shape
+    depth = max(1, min(N - 1, 12)) if N > 1 else 0
+    cfg = gi.VerifyConfig("r", 9, B, Hq, Hkv, 128, L, N, depth, 4, 3, 8, 8, 0.5)
+    inp = gi.make_inputs(cfg, 1000 + N, accept=False, pad_fill="nan")
+    want = cpu_attn(inp)
+    for kernel in (0, 2):
+        assert_close(out_to_f64(gpu_attn(inp, kernel=kernel, num_splits=splits)), want)
+
+
 def test_many_units_per_cta_sampled_rows():
     # 4096 units of work for 148 persistent CTAs (about 28 each, more than the kernel decodes up
     # front), short ragged prefix (one partial cache tile) and four draft tiles per unit
