@@ -306,6 +306,13 @@ int gsd_commit_kv(void* k_cache, void* v_cache, const void* draft_k, const void*
  * buffer of at least gsd_verify_step_host_arena_bytes(ap, cp) bytes, 256-byte aligned,
  * owned by the caller.  `device_status_out` (host, may be NULL) receives the device
  * status word of this step.  ap->B == cp->B and ap->N == cp->N are required.
+ *
+ * The inputs travel on a copy stream that the library creates at the first call on a device
+ * (with three events; all kept until the process exits), the attention inputs first: the
+ * attention runs on `stream` as soon as they have landed, and its output goes back to the host
+ * while the logits are still coming in.  The copy stream waits for the work already queued on
+ * `stream`, and the call returns after `stream` has drained, so the arena may be reused at once.
+ * Calls on one device must not be made from several host threads at the same time.
  */
 int gsd_verify_step_host(const void* q, const void* k_cache, const void* v_cache,
                          const void* draft_k, const void* draft_v,

@@ -212,6 +212,37 @@ extern "C" size_t gsd_verify_step_host_arena_bytes(const gsd_attn_params* ap, co
     return L.total;
 }
 
+namespace {
+// One copy stream and three events per device, created at the first host-step call on that
+// device and kept for the life of the process.
+struct HostStepStreams {
+    cudaStream_t copy = nullptr;
+    cudaEvent_t entered = nullptr, attn_in = nullptr, accept_in = nullptr;
+};
+HostStepStreams* host_step_streams() {
+    static HostStepStreams per_dev[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        gsd::set_error_text("gsd_verify_step_host: no current device");
+        return nullptr;
+    }
+    HostStepStreams* h = &per_dev[dev];
+    if (!h->copy) {
+        cudaStream_t s = nullptr;
+        cudaEvent_t e[3] = {nullptr, nullptr, nullptr};
+        cudaError_t err = cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking);
+        for (int i = 0; i < 3 && err == cudaSuccess; ++i) err = cudaEventCreateWithFlags(&e[i], cudaEventDisableTiming);
+        if (err != cudaSuccess) {
+            gsd::set_cuda_error(err, "gsd_verify_step_host: copy stream / events");
+            return nullptr;
+        }
+        h->entered = e[0]; h->attn_in = e[1]; h->accept_in = e[2];
+        h->copy = s;
+    }
+    return h;
+}
+}  // namespace
+
 extern "C" int gsd_verify_step_host(const void* q, const void* k_cache, const void* v_cache,
                                     const void* draft_k, const void* draft_v,
                                     const uint32_t* ancestor_mask, const int32_t* seq_lens, void* out,
@@ -233,8 +264,16 @@ extern "C" int gsd_verify_step_host(const void* q, const void* k_cache, const vo
     if (((uintptr_t)arena & 255u) != 0) return GSD_ERR_MISALIGNED;
     cudaStream_t st = (cudaStream_t)stream;
     char* base = (char*)arena;
+    // The host->device copies go out on a copy stream of the library's own, the attention inputs
+    // first; `stream` runs the attention as soon as those have landed and sends its output back
+    // (the other direction of the link) while the logits are still coming in.
+    HostStepStreams* hs = host_step_streams();
+    if (!hs) return GSD_ERR_CUDA;
+    cudaStream_t cs = hs->copy;
+    GSD_CUDA_TRY(cudaEventRecord(hs->entered, st));           // the arena may still be in use by earlier work on `stream`
+    GSD_CUDA_TRY(cudaStreamWaitEvent(cs, hs->entered, 0));
     auto h2d = [&](size_t off, const void* src, size_t bytes) {
-        return cudaMemcpyAsync(base + off, src, bytes, cudaMemcpyHostToDevice, st);
+        return cudaMemcpyAsync(base + off, src, bytes, cudaMemcpyHostToDevice, cs);
     };
     GSD_CUDA_TRY(h2d(L.q, q, L.b_q));
     GSD_CUDA_TRY(h2d(L.kc, k_cache, L.b_kv));
@@ -243,23 +282,27 @@ extern "C" int gsd_verify_step_host(const void* q, const void* k_cache, const vo
     GSD_CUDA_TRY(h2d(L.dv, draft_v, L.b_d));
     GSD_CUDA_TRY(h2d(L.mask, ancestor_mask, L.b_mask));
     GSD_CUDA_TRY(h2d(L.sl, seq_lens, L.b_sl));
+    GSD_CUDA_TRY(cudaEventRecord(hs->attn_in, cs));
     GSD_CUDA_TRY(h2d(L.logits, logits, L.b_logits));
     GSD_CUDA_TRY(h2d(L.tok, draft_tokens, L.b_tok));
     GSD_CUDA_TRY(h2d(L.pptr, parent_ptr, L.b_pptr));
     GSD_CUDA_TRY(h2d(L.pidx, parent_idx, L.b_pidx));
+    GSD_CUDA_TRY(cudaEventRecord(hs->accept_in, cs));
     GSD_CUDA_TRY(cudaMemsetAsync(base + L.status, 0, 4, st));
+    GSD_CUDA_TRY(cudaStreamWaitEvent(st, hs->attn_in, 0));
     int rc = gsd_verify_attn(base + L.q, base + L.kc, base + L.vc, base + L.dk, base + L.dv,
                              (const uint32_t*)(base + L.mask), (const int32_t*)(base + L.sl),
                              base + L.out, ap, base + L.ws_attn,
                              gsd_verify_attn_workspace_bytes(ap), (int32_t*)(base + L.status), stream);
     if (rc != GSD_OK) return rc;
+    GSD_CUDA_TRY(cudaMemcpyAsync(out, base + L.out, L.b_q, cudaMemcpyDeviceToHost, st));
+    GSD_CUDA_TRY(cudaStreamWaitEvent(st, hs->accept_in, 0));
     rc = gsd_accept((const float*)(base + L.logits), (const int32_t*)(base + L.tok),
                     (const int32_t*)(base + L.pptr), (const int32_t*)(base + L.pidx),
                     (int32_t*)(base + L.atok), (int32_t*)(base + L.alen),
                     (int32_t*)(base + L.anodes), cp, base + L.ws_acc,
                     gsd_accept_workspace_bytes(cp), (int32_t*)(base + L.status), stream);
     if (rc != GSD_OK) return rc;
-    GSD_CUDA_TRY(cudaMemcpyAsync(out, base + L.out, L.b_q, cudaMemcpyDeviceToHost, st));
     GSD_CUDA_TRY(cudaMemcpyAsync(accepted_tokens, base + L.atok, L.b_acc, cudaMemcpyDeviceToHost, st));
     GSD_CUDA_TRY(cudaMemcpyAsync(accepted_len, base + L.alen, L.b_len, cudaMemcpyDeviceToHost, st));
     if (accepted_nodes)
