@@ -383,8 +383,8 @@ __device__ __forceinline__ UnitInfo unit_info(const TcParams& p, int w, int lane
 }
 
 // Persistent kernel: CTA k walks the work indices k, k + gridDim.x, ...  Barrier phases are
-// counted across units, so the producer and the MMA issuer run ahead into the next unit
-// (Q, the first K/V tiles and the first QK^T) while the softmax warps still drain the
+// counted across units, so the producer and the QK^T issuer run ahead into the next unit
+// (Q, the first K/V tiles and the first QK^T) while the softmax warps still read out the
 // accumulators of the previous one.
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
