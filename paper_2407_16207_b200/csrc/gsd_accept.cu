@@ -4,19 +4,18 @@
 //
 // One launch.  Grid (splits, B*N): each CTA streams one slice of one logits row with
 // 16-byte loads and reduces (value, index) pairs; slices of a row meet in a packed 64-bit
-// atomicMax.  The CTA that finishes last for a sequence runs the path pass for it:
-// level-synchronous relaxation of best[v] = 1 + max over accepted parents, selection of
-// the end node, backtracking, emission.
+// atomicMax.  The CTA that finishes last for a sequence runs the path pass for it
+// (gsd_path.cuh: level-synchronous relaxation of best[v] = 1 + max over accepted parents,
+// selection of the end node, backtracking, emission).
 #include "gsd_internal.cuh"
+#include "gsd_path.cuh"
 #include <math_constants.h>
 
 namespace gsd {
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = kPathThreads;
 constexpr int kNone = 0x7FFFFFFF;
-constexpr int kNodeSlots = (GSD_MAX_NODES + kThreads - 1) / kThreads;
-constexpr int kEdgeCache = 3 * GSD_MAX_NODES;   // parent edges of one sequence kept in shared memory
 
 struct Best {
     float v;
@@ -92,121 +91,25 @@ struct AcceptArgs {
 };
 
 __device__ void path_pass(const AcceptArgs& a, int b) {
-    __shared__ int s_best[GSD_MAX_NODES];
     __shared__ int s_amax[GSD_MAX_NODES];
-    __shared__ int s_tok[GSD_MAX_NODES];
-    __shared__ int s_ptr[GSD_MAX_NODES + 1];
-    __shared__ int s_red[kThreads / 32];
-    __shared__ unsigned s_flags;
-    __shared__ int s_m;
-    __shared__ int s_edge[kEdgeCache];
     const int N = a.N, tid = threadIdx.x;
+    // the keys were written by other CTAs: read them past L1
+    for (int v = tid; v < N; v += kThreads) s_amax[v] = key_index(__ldcg(a.keys + (size_t)b * N + v));
+    __syncthreads();
     const int32_t* tok = a.tok + (size_t)b * N;
-    const int32_t* pptr = a.pptr + (size_t)b * (N + 1);
-    const int32_t* pidx = a.pidx + (size_t)b * a.Ecap;
-    unsigned flags = 0;
-    if (tid == 0) s_flags = 0;
-    for (int v = tid; v < N; v += kThreads) {
-        // the keys were written by other CTAs: read them past L1
-        s_amax[v] = key_index(__ldcg(a.keys + (size_t)b * N + v));
-        const int t = tok[v];
-        s_tok[v] = t;
-        if (t < 0 || t >= a.V) flags |= GSD_DEV_BAD_TOKEN;
-        s_best[v] = v == 0 ? 0 : -1;
-    }
-    for (int v = tid; v <= N; v += kThreads) {
-        int e = pptr[v];
-        if (e < 0 || e > a.Ecap) {
-            flags |= GSD_DEV_BAD_CSR;
-            e = e < 0 ? 0 : a.Ecap;
-        }
-        s_ptr[v] = e;
-    }
-    __syncthreads();
-    // the relaxation rounds walk the parent lists again and again: keep them on chip
-    const int n_edges = s_ptr[N];
-    const bool cached = n_edges <= kEdgeCache;
-    if (cached) {
-        for (int e = tid; e < n_edges; e += kThreads) s_edge[e] = pidx[e];
-        __syncthreads();
-    }
-
-    // level-synchronous relaxation: after round r every node whose longest accepted root
-    // path has <= r edges is final; values only grow, so it stops when nothing changed
-    for (int round = 0; round < N; ++round) {
-        int nb[kNodeSlots];
-        int changed = 0;
-#pragma unroll
-        for (int k = 0; k < kNodeSlots; ++k) {
-            const int v = tid + k * kThreads;
-            nb[k] = -1;
-            if (v > 0 && v < N) {
-                int cur = s_best[v];
-                const int t = s_tok[v];
-                for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
-                    const int p = cached ? s_edge[e] : pidx[e];
-                    if (p < 0 || p >= v) {
-                        flags |= GSD_DEV_BAD_CSR;
-                        continue;
-                    }
-                    const int bp = s_best[p];
-                    if (bp >= 0 && t == s_amax[p] && bp + 1 > cur) cur = bp + 1;
-                }
-                nb[k] = cur;
-                changed |= (cur != s_best[v]);
-            }
-        }
-        __syncthreads();
-#pragma unroll
-        for (int k = 0; k < kNodeSlots; ++k) {
-            const int v = tid + k * kThreads;
-            if (v > 0 && v < N) s_best[v] = nb[k];
-        }
-        if (!__syncthreads_or(changed)) break;
-    }
-
-    // end node: longest, then lowest index
-    int key = -1;
-    for (int v = tid; v < N; v += kThreads)
-        if (s_best[v] >= 0) key = max(key, (s_best[v] << 10) | (1023 - v));
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xFFFFFFFFu, key, o));
-    if ((tid & 31) == 0) s_red[tid >> 5] = key;
-    if (flags) atomicOr(&s_flags, flags);
-    __syncthreads();
-
-    int32_t* out_tok = a.out_tok + (size_t)b * a.Tcap;
-    int32_t* out_nodes = a.out_nodes ? a.out_nodes + (size_t)b * a.Tcap : nullptr;
-    if (tid == 0) {
-        for (int w = 1; w < kThreads / 32; ++w) key = max(key, s_red[w]);
-        const int m = key >> 10;
-        int v = 1023 - (key & 1023);
-        unsigned fl = s_flags;
-        if (m + 1 > a.Tcap) fl |= GSD_DEV_TCAP;
-        if (m < a.Tcap) out_tok[m] = s_amax[v];  // the target model's own next token
-        // walk back: the lowest predecessor that is accepted and carries length - 1
-        for (int len = m; len >= 0; --len) {
-            if (out_nodes && len < a.Tcap) out_nodes[len] = v;
-            if (len == 0) break;
-            if (len - 1 < a.Tcap) out_tok[len - 1] = s_tok[v];
-            int pred = kNone;
-            for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
-                const int p = cached ? s_edge[e] : pidx[e];
-                if (p < 0 || p >= v) continue;
-                if (s_best[p] == len - 1 && s_tok[v] == s_amax[p] && p < pred) pred = p;
-            }
-            if (pred == kNone) break;  // cannot happen for a consistent best[]
-            v = pred;
-        }
-        a.out_len[b] = m + 1;
-        s_m = m;
-        if (fl && a.status) atomicOr((unsigned*)a.status, fl);
-    }
-    __syncthreads();
-    for (int i = s_m + 1 + tid; i < a.Tcap; i += kThreads) {
-        out_tok[i] = -1;
-        if (out_nodes) out_nodes[i] = -1;
-    }
+    PathIo io;
+    io.tok = tok;
+    io.pptr = a.pptr + (size_t)b * (N + 1);
+    io.pidx = a.pidx + (size_t)b * a.Ecap;
+    io.out_tok = a.out_tok + (size_t)b * a.Tcap;
+    io.out_nodes = a.out_nodes ? a.out_nodes + (size_t)b * a.Tcap : nullptr;
+    io.out_len = a.out_len + b;
+    io.status = a.status;
+    io.N = N; io.V = a.V; io.Ecap = a.Ecap; io.Tcap = a.Tcap;
+    // a step parent -> v is accepted iff v's token is what the target model would emit after the parent
+    const PathResult res = longest_accepted_path(io, 0u, [&](int p, int v) { return tok[v] == s_amax[p]; });
+    // the target model's own next token
+    if (tid == 0 && res.edges < a.Tcap) io.out_tok[res.edges] = s_amax[res.end];
 }
 
 template <bool kVec>

@@ -14,15 +14,14 @@
 // longest-path relaxation, walks back, and finds the regenerated token: the range sums in
 // scratch give the range of the crossing, a block-wide scan over that range gives the index.
 #include "gsd_internal.cuh"
+#include "gsd_path.cuh"
 #include <math_constants.h>
 
 namespace gsd {
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = kPathThreads;
 constexpr int kNone = 0x7FFFFFFF;
-constexpr int kNodeSlots = (GSD_MAX_NODES + kThreads - 1) / kThreads;
-constexpr int kEdgeCache = 3 * GSD_MAX_NODES;   // parent edges of one sequence kept in shared memory
 constexpr int kMaxSlices = 16;
 constexpr int kWarps = kThreads / 32;   // each warp of a CTA sums a contiguous eighth of the CTA's slice
 constexpr float kLog2e = 1.4426950408889634f;
@@ -98,25 +97,15 @@ struct SampledArgs {
 __device__ void finish_sequence(const SampledArgs& a, int b) {
     __shared__ float s_mx[GSD_MAX_NODES];
     __shared__ float s_sum[GSD_MAX_NODES];
-    __shared__ int s_best[GSD_MAX_NODES];
-    __shared__ int s_tok[GSD_MAX_NODES];
-    __shared__ int s_ptr[GSD_MAX_NODES + 1];
-    __shared__ int s_edge[kEdgeCache];
-    __shared__ unsigned char s_eok[kEdgeCache];
-    __shared__ short s_enode[kEdgeCache];          // the node an edge leads into
     __shared__ int s_red[kThreads / 32];
     __shared__ float s_scan[kThreads / 32];
-    __shared__ unsigned s_flags;
-    __shared__ int s_m, s_end, s_pick;
+    __shared__ int s_pick;
     const int N = a.N, V = a.V, tid = threadIdx.x;
     const int32_t* tok = a.tok + (size_t)b * N;
-    const int32_t* pptr = a.pptr + (size_t)b * (N + 1);
-    const int32_t* pidx = a.pidx + (size_t)b * a.Ecap;
     const float* lg = a.logits + (size_t)b * N * V;
     const float* q = a.q + (size_t)b * N;
     const float* u = a.u + (size_t)b * N;
     unsigned flags = 0;
-    if (tid == 0) s_flags = 0;
     for (int v = tid; v < N; v += kThreads) {
         // the pairs were written by other CTAs: read them past L1
         Ms r{-CUDART_INF_F, 0.f};
@@ -127,113 +116,25 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
         s_mx[v] = r.m;
         s_sum[v] = r.s;
         if (!(r.s > 0.f) || r.m == CUDART_INF_F) flags |= GSD_DEV_BAD_LOGITS;   // no finite entry, +inf or NaN
-        const int t = tok[v];
-        s_tok[v] = t;
-        if (t < 0 || t >= V) flags |= GSD_DEV_BAD_TOKEN;
-        s_best[v] = v == 0 ? 0 : -1;
-    }
-    for (int v = tid; v <= N; v += kThreads) {
-        int e = pptr[v];
-        if (e < 0 || e > a.Ecap) {
-            flags |= GSD_DEV_BAD_CSR;
-            e = e < 0 ? 0 : a.Ecap;
-        }
-        s_ptr[v] = e;
     }
     __syncthreads();
-    // the test of one step: the target's probability of v's token under its parent p
-    auto step_ok = [&](int p, int v) -> bool {
-        const int t = s_tok[v];
-        if (t < 0 || t >= V) return false;
-        const float prob = ex2((lg[(size_t)p * V + t] - s_mx[p]) * kLog2e) / s_sum[p];
+    PathIo io;
+    io.tok = tok;
+    io.pptr = a.pptr + (size_t)b * (N + 1);
+    io.pidx = a.pidx + (size_t)b * a.Ecap;
+    io.out_tok = a.out_tok + (size_t)b * a.Tcap;
+    io.out_nodes = a.out_nodes ? a.out_nodes + (size_t)b * a.Tcap : nullptr;
+    io.out_len = a.out_len + b;
+    io.status = a.status;
+    io.N = N; io.V = V; io.Ecap = a.Ecap; io.Tcap = a.Tcap;
+    // the test of one step: the target's probability of v's token under its parent p (one
+    // logit gathered from global memory) against u q
+    const PathResult res = longest_accepted_path(io, flags, [&](int p, int v) {
+        const float prob = ex2((lg[(size_t)p * V + tok[v]] - s_mx[p]) * kLog2e) / s_sum[p];
         return u[v] * q[v] < prob;
-    };
-    const int n_edges = s_ptr[N];
-    const bool cached = n_edges <= kEdgeCache;
-    if (cached) {
-        // parent lists and the outcome of every step once, on chip; the tests gather one logit
-        // each from global memory, so they go out one per thread, all at once
-        for (int v = tid; v < N; v += kThreads)
-            for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) s_enode[e] = (short)v;
-        __syncthreads();
-        for (int e = tid; e < n_edges; e += kThreads) {
-            const int p = pidx[e], v = s_enode[e];
-            s_edge[e] = p;
-            s_eok[e] = (p >= 0 && p < v) ? (unsigned char)step_ok(p, v) : 0;
-        }
-        __syncthreads();
-    }
-
-    // level-synchronous relaxation of best[v] = 1 + max over accepted steps into v
-    for (int round = 0; round < N; ++round) {
-        int nb[kNodeSlots];
-        int changed = 0;
-#pragma unroll
-        for (int k = 0; k < kNodeSlots; ++k) {
-            const int v = tid + k * kThreads;
-            nb[k] = -1;
-            if (v > 0 && v < N) {
-                int cur = s_best[v];
-                for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
-                    const int p = cached ? s_edge[e] : pidx[e];
-                    if (p < 0 || p >= v) {
-                        flags |= GSD_DEV_BAD_CSR;
-                        continue;
-                    }
-                    const int bp = s_best[p];
-                    if (bp >= 0 && bp + 1 > cur && (cached ? s_eok[e] != 0 : step_ok(p, v))) cur = bp + 1;
-                }
-                nb[k] = cur;
-                changed |= (cur != s_best[v]);
-            }
-        }
-        __syncthreads();
-#pragma unroll
-        for (int k = 0; k < kNodeSlots; ++k) {
-            const int v = tid + k * kThreads;
-            if (v > 0 && v < N) s_best[v] = nb[k];
-        }
-        if (!__syncthreads_or(changed)) break;
-    }
-
-    // end node: longest, then lowest index
-    int key = -1;
-    for (int v = tid; v < N; v += kThreads)
-        if (s_best[v] >= 0) key = max(key, (s_best[v] << 10) | (1023 - v));
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xFFFFFFFFu, key, o));
-    if ((tid & 31) == 0) s_red[tid >> 5] = key;
-    if (flags) atomicOr(&s_flags, flags);
-    __syncthreads();
-
-    int32_t* out_tok = a.out_tok + (size_t)b * a.Tcap;
-    int32_t* out_nodes = a.out_nodes ? a.out_nodes + (size_t)b * a.Tcap : nullptr;
-    if (tid == 0) {
-        for (int w = 1; w < kThreads / 32; ++w) key = max(key, s_red[w]);
-        const int m = key >> 10;
-        int v = 1023 - (key & 1023);
-        s_end = v;
-        unsigned fl = s_flags;
-        if (m + 1 > a.Tcap) fl |= GSD_DEV_TCAP;
-        // walk back: the lowest predecessor with an accepted step that carries length - 1
-        for (int len = m; len >= 0; --len) {
-            if (out_nodes && len < a.Tcap) out_nodes[len] = v;
-            if (len == 0) break;
-            if (len - 1 < a.Tcap) out_tok[len - 1] = s_tok[v];
-            int pred = kNone;
-            for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
-                const int p = cached ? s_edge[e] : pidx[e];
-                if (p < 0 || p >= v) continue;
-                if (s_best[p] == len - 1 && p < pred && (cached ? s_eok[e] != 0 : step_ok(p, v))) pred = p;
-            }
-            if (pred == kNone) break;  // cannot happen for a consistent best[]
-            v = pred;
-        }
-        a.out_len[b] = m + 1;
-        s_m = m;
-        if (fl && a.status) atomicOr((unsigned*)a.status, fl);
-    }
-    __syncthreads();
+    });
+    const int s_m = res.edges, s_end = res.end;
+    int32_t* out_tok = io.out_tok;
 
     // The regenerated token.  The sums of the streaming pass over the row's contiguous ranges
     // (slices x warps, kept in scratch) say in which range the cumulative sum first exceeds
@@ -310,10 +211,6 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
             }
             if (s_m < a.Tcap) out_tok[s_m] = pick;
         }
-    }
-    for (int i = s_m + 1 + tid; i < a.Tcap; i += kThreads) {
-        out_tok[i] = -1;
-        if (out_nodes) out_nodes[i] = -1;
     }
 }
 

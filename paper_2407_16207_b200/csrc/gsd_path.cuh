@@ -1,0 +1,163 @@
+// Longest accepted root path through the draft DAG (Sec. 4.1 longest-path selection; Sec. 3
+// rejection cascade), shared by the deterministic and the non-deterministic verification.
+// One CTA of kPathThreads threads per sequence.  The caller supplies the test of one step
+// parent -> v; this file does the rest: parent lists on chip, level-synchronous relaxation of
+// best[v] = 1 + max over accepted steps into v, choice of the end node (longest, then lowest
+// index), walk back (lowest predecessor that carries length - 1), emission of the path's node
+// ids and drafted tokens.  The token the target model contributes at the end is the caller's.
+#pragma once
+#include "gsd_internal.cuh"
+
+namespace gsd {
+
+constexpr int kPathThreads = 256;
+constexpr int kPathNone = 0x7FFFFFFF;
+constexpr int kPathNodeSlots = (GSD_MAX_NODES + kPathThreads - 1) / kPathThreads;
+constexpr int kPathEdgeCache = 3 * GSD_MAX_NODES;   // parent edges of one sequence kept in shared memory
+
+struct PathIo {
+    const int32_t* tok;     // [N] drafted tokens of the sequence
+    const int32_t* pptr;    // [N+1]
+    const int32_t* pidx;    // [Ecap]
+    int32_t* out_tok;       // [Tcap]
+    int32_t* out_nodes;     // [Tcap] or nullptr
+    int32_t* out_len;       // one entry
+    int32_t* status;        // device status word or nullptr
+    int N, V, Ecap, Tcap;
+};
+
+struct PathResult {
+    int edges;   // m: the accepted path has m + 1 nodes
+    int end;     // its last node
+};
+
+// `step_ok(p, v)` is called once per step when the parent lists fit the on-chip cache (one
+// thread per step, all at once), else again on every use.  `flags` carries status bits the
+// caller has already found; the function adds its own and publishes them.  All threads of the
+// CTA must call it; all return the same result.  out_tok[edges] is left for the caller,
+// entries past it are set to -1.
+template <class StepOk>
+__device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, StepOk step_ok) {
+    __shared__ int s_best[GSD_MAX_NODES];
+    __shared__ int s_tok[GSD_MAX_NODES];
+    __shared__ int s_ptr[GSD_MAX_NODES + 1];
+    __shared__ int s_edge[kPathEdgeCache];
+    __shared__ unsigned char s_eok[kPathEdgeCache];
+    __shared__ short s_enode[kPathEdgeCache];   // the node a step leads into
+    __shared__ int s_red[kPathThreads / 32];
+    __shared__ unsigned s_flags;
+    __shared__ int s_m, s_end;
+    const int N = io.N, tid = threadIdx.x;
+    if (tid == 0) s_flags = 0;
+    for (int v = tid; v < N; v += kPathThreads) {
+        const int t = io.tok[v];
+        s_tok[v] = t;
+        if (t < 0 || t >= io.V) flags |= GSD_DEV_BAD_TOKEN;
+        s_best[v] = v == 0 ? 0 : -1;
+    }
+    for (int v = tid; v <= N; v += kPathThreads) {
+        int e = io.pptr[v];
+        if (e < 0 || e > io.Ecap) {
+            flags |= GSD_DEV_BAD_CSR;
+            e = e < 0 ? 0 : io.Ecap;
+        }
+        s_ptr[v] = e;
+    }
+    __syncthreads();
+    // the relaxation rounds walk the parent lists again and again: keep them, and the outcome
+    // of every step, on chip
+    const int n_edges = s_ptr[N];
+    const bool cached = n_edges <= kPathEdgeCache;
+    if (cached) {
+        for (int v = tid; v < N; v += kPathThreads)
+            for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) s_enode[e] = (short)v;
+        __syncthreads();
+        for (int e = tid; e < n_edges; e += kPathThreads) {
+            const int p = io.pidx[e], v = s_enode[e];
+            s_edge[e] = p;
+            s_eok[e] = (p >= 0 && p < v && s_tok[v] >= 0 && s_tok[v] < io.V) ? (unsigned char)step_ok(p, v) : 0;
+        }
+        __syncthreads();
+    }
+    auto ok_at = [&](int e, int p, int v) -> bool {
+        if (cached) return s_eok[e] != 0;
+        return s_tok[v] >= 0 && s_tok[v] < io.V && step_ok(p, v);
+    };
+
+    // level-synchronous relaxation: after round r every node whose longest accepted root
+    // path has <= r edges is final; values only grow, so it stops when nothing changed
+    for (int round = 0; round < N; ++round) {
+        int nb[kPathNodeSlots];
+        int changed = 0;
+#pragma unroll
+        for (int k = 0; k < kPathNodeSlots; ++k) {
+            const int v = tid + k * kPathThreads;
+            nb[k] = -1;
+            if (v > 0 && v < N) {
+                int cur = s_best[v];
+                for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
+                    const int p = cached ? s_edge[e] : io.pidx[e];
+                    if (p < 0 || p >= v) {
+                        flags |= GSD_DEV_BAD_CSR;
+                        continue;
+                    }
+                    const int bp = s_best[p];
+                    if (bp >= 0 && bp + 1 > cur && ok_at(e, p, v)) cur = bp + 1;
+                }
+                nb[k] = cur;
+                changed |= (cur != s_best[v]);
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < kPathNodeSlots; ++k) {
+            const int v = tid + k * kPathThreads;
+            if (v > 0 && v < N) s_best[v] = nb[k];
+        }
+        if (!__syncthreads_or(changed)) break;
+    }
+
+    // end node: longest, then lowest index
+    int key = -1;
+    for (int v = tid; v < N; v += kPathThreads)
+        if (s_best[v] >= 0) key = max(key, (s_best[v] << 10) | (1023 - v));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xFFFFFFFFu, key, o));
+    if ((tid & 31) == 0) s_red[tid >> 5] = key;
+    if (flags) atomicOr(&s_flags, flags);
+    __syncthreads();
+
+    if (tid == 0) {
+        for (int w = 1; w < kPathThreads / 32; ++w) key = max(key, s_red[w]);
+        const int m = key >> 10;
+        int v = 1023 - (key & 1023);
+        s_end = v;
+        unsigned fl = s_flags;
+        if (m + 1 > io.Tcap) fl |= GSD_DEV_TCAP;
+        // walk back: the lowest predecessor with an accepted step that carries length - 1
+        for (int len = m; len >= 0; --len) {
+            if (io.out_nodes && len < io.Tcap) io.out_nodes[len] = v;
+            if (len == 0) break;
+            if (len - 1 < io.Tcap) io.out_tok[len - 1] = s_tok[v];
+            int pred = kPathNone;
+            for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
+                const int p = cached ? s_edge[e] : io.pidx[e];
+                if (p < 0 || p >= v) continue;
+                if (s_best[p] == len - 1 && p < pred && ok_at(e, p, v)) pred = p;
+            }
+            if (pred == kPathNone) break;  // cannot happen for a consistent best[]
+            v = pred;
+        }
+        *io.out_len = m + 1;
+        s_m = m;
+        if (fl && io.status) atomicOr((unsigned*)io.status, fl);
+    }
+    __syncthreads();
+    for (int i = s_m + 1 + tid; i < io.Tcap; i += kPathThreads) {
+        io.out_tok[i] = -1;
+        if (io.out_nodes) io.out_nodes[i] = -1;
+    }
+    return PathResult{s_m, s_end};
+}
+
+}  // namespace gsd
