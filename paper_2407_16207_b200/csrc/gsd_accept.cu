@@ -107,7 +107,7 @@ __device__ void path_pass(const AcceptArgs& a, int b) {
     io.status = a.status;
     io.N = N; io.V = a.V; io.Ecap = a.Ecap; io.Tcap = a.Tcap;
     // a step parent -> v is accepted iff v's token is what the target model would emit after the parent
-    const PathResult res = longest_accepted_path(io, 0u, [&](int p, int v) { return tok[v] == s_amax[p]; });
+    const PathResult res = longest_accepted_path<false>(io, 0u, [&](int p, int v) { return tok[v] == s_amax[p]; });
     // the target model's own next token
     if (tid == 0 && res.edges < a.Tcap) io.out_tok[res.edges] = s_amax[res.end];
 }

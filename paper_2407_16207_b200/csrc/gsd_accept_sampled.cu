@@ -129,7 +129,7 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     io.N = N; io.V = V; io.Ecap = a.Ecap; io.Tcap = a.Tcap;
     // the test of one step: the target's probability of v's token under its parent p (one
     // logit gathered from global memory) against u q
-    const PathResult res = longest_accepted_path(io, flags, [&](int p, int v) {
+    const PathResult res = longest_accepted_path<true>(io, flags, [&](int p, int v) {
         const float prob = ex2((lg[(size_t)p * V + tok[v]] - s_mx[p]) * kLog2e) / s_sum[p];
         return u[v] * q[v] < prob;
     });

@@ -31,12 +31,13 @@ struct PathResult {
     int end;     // its last node
 };
 
-// `step_ok(p, v)` is called once per step when the parent lists fit the on-chip cache (one
-// thread per step, all at once), else again on every use.  `flags` carries status bits the
+// With kCacheOutcome, `step_ok(p, v)` is called once per step when the parent lists fit the
+// on-chip cache (one thread per step, all at once - for tests that touch global memory);
+// otherwise it is called again on every use (for tests that cost a comparison).  `flags` carries status bits the
 // caller has already found; the function adds its own and publishes them.  All threads of the
 // CTA must call it; all return the same result.  out_tok[edges] is left for the caller,
 // entries past it are set to -1.
-template <class StepOk>
+template <bool kCacheOutcome, class StepOk>
 __device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, StepOk step_ok) {
     __shared__ int s_best[GSD_MAX_NODES];
     __shared__ int s_tok[GSD_MAX_NODES];
@@ -68,7 +69,7 @@ __device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, St
     // of every step, on chip
     const int n_edges = s_ptr[N];
     const bool cached = n_edges <= kPathEdgeCache;
-    if (cached) {
+    if (cached && kCacheOutcome) {
         for (int v = tid; v < N; v += kPathThreads)
             for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) s_enode[e] = (short)v;
         __syncthreads();
@@ -78,9 +79,12 @@ __device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, St
             s_eok[e] = (p >= 0 && p < v && s_tok[v] >= 0 && s_tok[v] < io.V) ? (unsigned char)step_ok(p, v) : 0;
         }
         __syncthreads();
+    } else if (cached) {
+        for (int e = tid; e < n_edges; e += kPathThreads) s_edge[e] = io.pidx[e];
+        __syncthreads();
     }
     auto ok_at = [&](int e, int p, int v) -> bool {
-        if (cached) return s_eok[e] != 0;
+        if (cached && kCacheOutcome) return s_eok[e] != 0;
         return s_tok[v] >= 0 && s_tok[v] < io.V && step_ok(p, v);
     };
 
