@@ -48,7 +48,7 @@ def _load() -> ctypes.CDLL:
         _lib = ctypes.CDLL(build())
         _lib.gsd_oracle_threads.restype = ctypes.c_int
         _lib.gsd_oracle_argmax_row.restype = ctypes.c_int32
-        for name in ("gsd_oracle_attn", "gsd_oracle_attn_rows", "gsd_oracle_accept", "gsd_oracle_accept_sampled",
+        for name in ("gsd_oracle_attn", "gsd_oracle_attn_rows", "gsd_oracle_accept", "gsd_oracle_accept_sampled", "gsd_oracle_draft_expand",
                      "gsd_oracle_commit_kv", "gsd_oracle_build_mask"):
             getattr(_lib, name).restype = ctypes.c_int
         _lib.gsd_oracle_argmax.restype = None
@@ -165,6 +165,32 @@ def accept_sampled(logits, draft_tokens, parent_ptr, parent_idx, draft_q, u_acce
     if rc != 0:
         raise ValueError("oracle accept_sampled: malformed DAG or Tcap too small")
     return toks, lens, nodes
+
+
+def draft_expand(logits, frontier, frontier_len, tokens, tree_parent, merge_to, leaf, prob, num_nodes,
+                 k: int, tau: int, theta_prob: float, theta_sib: float):
+    """One growth step of the draft token graph (see gsd_oracle_draft_expand).  The graph arrays
+    are copied; returns (tokens, tree_parent, merge_to, leaf, prob, num_nodes, new_frontier
+    [B,F*k] padded with -1, new_frontier_len [B], out_of_capacity flag)."""
+    logits = _c(logits, np.float32); frontier = _c(frontier, np.int32); frontier_len = _c(frontier_len, np.int32)
+    tokens = _c(tokens, np.int32).copy(); tree_parent = _c(tree_parent, np.int32).copy()
+    merge_to = _c(merge_to, np.int32).copy(); leaf = _c(leaf, np.uint8).copy()
+    prob = _c(prob, np.float32).copy(); num_nodes = _c(num_nodes, np.int32).copy()
+    B, F, V = logits.shape
+    Ncap = tokens.shape[1]
+    assert frontier.shape == (B, F) and frontier_len.shape == (B,)
+    for a in (tree_parent, merge_to, leaf, prob):
+        assert a.shape == (B, Ncap)
+    nf = np.full((B, F * k), -1, dtype=np.int32)
+    nfl = np.zeros((B,), dtype=np.int32)
+    rc = _load().gsd_oracle_draft_expand(_p(logits), _p(frontier), _p(frontier_len), _p(tokens), _p(tree_parent),
+                                         _p(merge_to), _p(leaf), _p(prob), _p(num_nodes), _p(nf), _p(nfl),
+                                         ctypes.c_int32(B), ctypes.c_int32(F), ctypes.c_int32(V), ctypes.c_int32(Ncap),
+                                         ctypes.c_int32(k), ctypes.c_int32(tau), ctypes.c_double(theta_prob),
+                                         ctypes.c_double(theta_sib))
+    if rc < 0:
+        raise ValueError("oracle draft_expand: malformed input")
+    return tokens, tree_parent, merge_to, leaf, prob, num_nodes, nf, nfl, bool(rc & 1)
 
 
 def commit_kv(k_cache, v_cache, draft_k, draft_v, accepted_nodes, accepted_len, seq_lens):

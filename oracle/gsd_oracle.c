@@ -30,6 +30,8 @@
  *    p -> v accepted iff u_accept[v] * q_v < softmax(logits[p])[tok v], and the regenerated
  *    token drawn from softmax(logits[end]) by inverting the cumulative distribution.
  *  - The KV-cache commit of the accepted path and the ancestor-mask closure (see there).
+ *  - One growth step of the draft token graph: top-k children, probability and sibling
+ *    pruning (Sec. 4.2), tau-redundant nodes and their merge edges (Sec. 5.2, 5.3).
  *
  * Readings where the paper is silent are listed in the repository's design notes
  * (scale default 1/sqrt(D), q-head h uses kv-head h / G, mask bits honoured literally,
@@ -430,6 +432,92 @@ int gsd_oracle_accept_sampled(const float *logits, const int32_t *draft_tokens,
         if (rc != 0) return rc;
     }
     return 0;
+}
+
+/*
+ * One growth step of the draft token graph (Sec. 4 token tree with out-degree k; Sec. 4.2
+ * probability pruning and sibling pruning; Sec. 5.2 tau-redundant nodes; Sec. 5.3 merging).
+ * For sequence b the frontier nodes frontier[b][0..frontier_len[b]) are expanded in order; for
+ * a frontier node p with draft distribution P = softmax(logits[b][fi]) (double):
+ *   - its k children are the k most probable tokens (ties to the lowest token id), created in
+ *     that order as nodes n, n+1, ... with tokens[c] = token, tree_parent[c] = p, prob[c] = its
+ *     probability q, merge_to[c] = -1;
+ *   - a child is marked a leaf if q < theta_prob (probability pruning) or q < theta_sib * q_max
+ *     with q_max the largest of the k sibling probabilities (sibling pruning);
+ *   - a child is tau-redundant if the tau tokens ending at it along its tree path (itself and
+ *     tau - 1 tree ancestors; paths shorter than tau do not count) equal the tau tokens ending at
+ *     an earlier node (lower id, of this or an earlier step); it is then marked a leaf and
+ *     merge_to[c] is the lowest such id (the first occurrence).
+ * Creation stops when the node capacity Ncap is reached (return value bit 0).  The new
+ * frontier is the list of new nodes that are not leaves, in id order.
+ *
+ * logits [B,F,V] f32; frontier [B,F]; frontier_len [B]; tokens, tree_parent, merge_to [B,Ncap]
+ * i32, leaf [B,Ncap] u8, prob [B,Ncap] f32, num_nodes [B] (all in/out); new_frontier [B,F*k],
+ * new_frontier_len [B].  Returns 0, 1 if some sequence ran out of capacity, -1 on malformed input.
+ */
+static int same_gram(const int32_t *tok, const int32_t *par, int a, int b, int tau)
+{
+    for (int i = 0; i < tau; ++i) {
+        if (a < 0 || b < 0) return 0;          /* a path shorter than tau */
+        if (tok[a] != tok[b]) return 0;
+        a = par[a];
+        b = par[b];
+    }
+    return 1;
+}
+
+int gsd_oracle_draft_expand(const float *logits, const int32_t *frontier, const int32_t *frontier_len,
+                            int32_t *tokens, int32_t *tree_parent, int32_t *merge_to, uint8_t *leaf,
+                            float *prob, int32_t *num_nodes, int32_t *new_frontier,
+                            int32_t *new_frontier_len, int32_t B, int32_t F, int32_t V, int32_t Ncap,
+                            int32_t k, int32_t tau, double theta_prob, double theta_sib)
+{
+    int rc = 0;
+    if (k < 1 || k > V || tau < 1 || F < 0) return -1;
+    double *P = (double *)malloc(sizeof(double) * (size_t)V);
+    unsigned char *taken = (unsigned char *)malloc((size_t)V);
+    if (!P || !taken) { free(P); free(taken); return -1; }
+    for (int b = 0; b < B; ++b) {
+        int32_t *tok = tokens + (size_t)b * Ncap, *par = tree_parent + (size_t)b * Ncap;
+        int32_t *mt = merge_to + (size_t)b * Ncap;
+        uint8_t *lf = leaf + (size_t)b * Ncap;
+        float *pr = prob + (size_t)b * Ncap;
+        const int first_new = num_nodes[b];
+        int n = first_new;
+        if (frontier_len[b] < 0 || frontier_len[b] > F || n < 1 || n > Ncap) { rc = -1; break; }
+        for (int fi = 0; fi < frontier_len[b]; ++fi) {
+            const int p = frontier[(size_t)b * F + fi];
+            if (p < 0 || p >= first_new) { rc = -1; break; }
+            const float *x = logits + ((size_t)b * F + fi) * V;
+            double mx = -INFINITY, sum = 0.0;
+            for (int j = 0; j < V; ++j) if ((double)x[j] > mx) mx = (double)x[j];
+            for (int j = 0; j < V; ++j) { P[j] = exp((double)x[j] - mx); sum += P[j]; }
+            for (int j = 0; j < V; ++j) { P[j] /= sum; taken[j] = 0; }
+            double qmax = 0.0;
+            for (int i = 0; i < k; ++i) {
+                int best = -1;                 /* most probable token not taken yet, ties to the lowest id */
+                for (int j = 0; j < V; ++j)
+                    if (!taken[j] && (best < 0 || P[j] > P[best])) best = j;
+                taken[best] = 1;
+                if (i == 0) qmax = P[best];
+                if (n >= Ncap) { rc |= 1; continue; }
+                const int c = n++;
+                tok[c] = best; par[c] = p; mt[c] = -1; pr[c] = (float)P[best];
+                lf[c] = (P[best] < theta_prob) || (P[best] < theta_sib * qmax);
+            }
+        }
+        if (rc < 0) break;
+        int nf = 0;
+        for (int c = first_new; c < n; ++c) {
+            for (int e = 0; e < c; ++e)
+                if (same_gram(tok, par, c, e, tau)) { lf[c] = 1; mt[c] = e; break; }
+            if (!lf[c]) new_frontier[(size_t)b * F * k + nf++] = c;
+        }
+        new_frontier_len[b] = nf;
+        num_nodes[b] = n;
+    }
+    free(P); free(taken);
+    return rc;
 }
 
 /*

@@ -41,6 +41,17 @@ MUTATIONS = [
      "test_oracle_accept_sampled.py"),
     ("sampled_regenerates_at_parent", "const int end = best[m];", "const int end = best[m > 0 ? m - 1 : 0];",
      "test_oracle_accept_sampled.py"),
+    ("draft_tie_highest", "if (!taken[j] && (best < 0 || P[j] > P[best])) best = j;",
+     "if (!taken[j] && (best < 0 || P[j] >= P[best])) best = j;", "test_oracle_draft.py"),
+    ("draft_prob_le", "lf[c] = (P[best] < theta_prob) ||", "lf[c] = (P[best] <= theta_prob) ||", "test_oracle_draft.py"),
+    ("draft_sibling_vs_previous", "if (i == 0) qmax = P[best];", "qmax = (i == 0) ? P[best] : P[best] * 2.0;",
+     "test_oracle_draft.py"),
+    ("draft_gram_ignores_ancestors", "if (tok[a] != tok[b]) return 0;\n        a = par[a];",
+     "if (tok[a] != tok[b]) return 0;\n        if (i == 0) return 1;\n        a = par[a];", "test_oracle_draft.py"),
+    ("draft_last_occurrence", "for (int e = 0; e < c; ++e)\n                if (same_gram(tok, par, c, e, tau))",
+     "for (int e = c - 1; e >= 0; --e)\n                if (same_gram(tok, par, c, e, tau))", "test_oracle_draft.py"),
+    ("draft_short_paths_count", "if (a < 0 || b < 0) return 0;          /* a path shorter than tau */",
+     "if (a < 0 || b < 0) return a < 0 && b < 0;", "test_oracle_draft.py"),
     ("mask_without_self", "row[v / 32] |= 1u << (v % 32);", "if (v != n) row[v / 32] |= 1u << (v % 32);",
      "test_oracle_mask.py"),
     ("mask_parents_only", "seen[p] = 1;\n                    todo[top++] = p;", "seen[p] = 1;\n                    if (v == n) todo[top++] = p;",
