@@ -56,7 +56,9 @@ typedef enum gsd_status {
 #define GSD_DEV_WAIT_EXPIRED 0x8u  /* a bounded in-kernel wait gave up; the output is not valid */
 #define GSD_DEV_BAD_SEQ_LEN  0x10u /* seq_lens[b] outside [0, Lmax]; it was clamped */
 #define GSD_DEV_CACHE_FULL   0x20u /* gsd_commit_kv: the accepted rows did not all fit below Lmax; the rest was dropped */
-#define GSD_DEV_BAD_LOGITS   0x40u /* gsd_accept_sampled: a logits row without a finite entry, or with +inf or NaN */
+#define GSD_DEV_BAD_LOGITS   0x40u /* gsd_accept_sampled, gsd_draft_expand: a logits row without a finite entry (fewer than k for the draft step), or with +inf or NaN */
+#define GSD_DEV_DRAFT_FULL   0x80u /* gsd_draft_expand: the node capacity was reached; the remaining children were not created */
+#define GSD_DEV_BAD_FRONTIER 0x100u /* gsd_draft_expand: frontier_len, num_nodes or a frontier node id out of range */
 
 #define GSD_MAX_NODES 512          /* largest supported N (draft nodes per sequence) */
 
@@ -209,6 +211,56 @@ int gsd_accept_sampled(const float* logits, const int32_t* draft_tokens, const i
                        const float* u_sample, int32_t* accepted_tokens, int32_t* accepted_len,
                        int32_t* accepted_nodes, const gsd_accept_params* p, void* workspace,
                        size_t workspace_bytes, int32_t* status, void* stream);
+
+/*
+ * gsd_draft_expand - one growth step of the draft token graph on the device (Sec. 4: token
+ * tree of out-degree k; Sec. 4.2: probability pruning and sibling pruning; Sec. 5.2:
+ * tau-redundant nodes; Sec. 5.3: merging).  For every sequence b the frontier nodes
+ * frontier[b][0..frontier_len[b]) are expanded in order.  For a frontier node p with draft
+ * distribution P = softmax(logits[b][fi]):
+ *   - its k children are the k most probable tokens, best first, ties to the lowest token id;
+ *     they become the nodes num_nodes[b], num_nodes[b]+1, ... with tokens[c] = token,
+ *     tree_parent[c] = p, prob[c] = the token's probability q, merge_to[c] = -1;
+ *   - leaf[c] = 1 if q < theta_prob (probability pruning) or q < theta_sib * q_best with q_best
+ *     the largest of the k sibling probabilities (sibling pruning); pruned children are kept as
+ *     leaves, as the paper marks them;
+ *   - a child is tau-redundant if the tau tokens that end at it along its tree path (itself and
+ *     tau - 1 tree ancestors; a shorter path does not count) equal the tau tokens ending at a
+ *     node with a lower id (of this or an earlier step): then leaf[c] = 1 and merge_to[c] = the
+ *     lowest such id, the first occurrence (whose successors verification re-uses, Sec. 5.3).
+ * new_frontier[b] lists the new nodes that are not leaves, in id order.  Readings: the root's
+ * token is part of the paths; the first occurrence may itself be a pruned leaf; the merge edges
+ * are reported (merge_to), the verification DAG's parent lists are the caller's to derive:
+ * parents(x) = { tree_parent[x] } + { r : merge_to[r] == tree_parent[x] }.
+ *
+ *   logits        device const f32 [B,F,V], draft-model logits of the frontier nodes (rows at or
+ *                 past frontier_len[b] are not read); every row needs at least k entries above
+ *                 -inf, no +inf, no NaN (else GSD_DEV_BAD_LOGITS)
+ *   frontier      device const i32 [B,F] node ids < num_nodes[b];  frontier_len  device const i32 [B]
+ *   tokens, tree_parent, merge_to   device i32 [B,Ncap];  leaf  device u8 [B,Ncap];
+ *   prob          device f32 [B,Ncap];  num_nodes  device i32 [B]   - the graph, updated in place
+ *                 (node 0 is the root: tree_parent -1); Ncap <= GSD_MAX_NODES; when the capacity
+ *                 is reached the remaining children are dropped (GSD_DEV_DRAFT_FULL)
+ *   new_frontier  device i32 [B,F*k] (only the first new_frontier_len[b] entries are written);
+ *   new_frontier_len  device i32 [B]
+ *   workspace     device scratch of gsd_draft_expand_workspace_bytes(p) bytes, 8-byte aligned,
+ *                 arbitrary contents
+ * The probabilities are fp32 (ex2.approx); a pruning comparison whose two sides differ by less
+ * than a few 1e-6 relative may fall either way.  The order of the children never depends on
+ * arithmetic (it compares logits).  1 <= k <= GSD_DRAFT_MAX_K, k <= V, tau >= 1.
+ * Returns GSD_OK or a negative gsd_status; asynchronous on `stream`; allocates nothing.
+ */
+#define GSD_DRAFT_MAX_K 8
+typedef struct gsd_draft_params {
+    int32_t B, F, V, Ncap, k, tau;
+    float theta_prob, theta_sib;
+} gsd_draft_params;
+size_t gsd_draft_expand_workspace_bytes(const gsd_draft_params* p);
+int gsd_draft_expand(const float* logits, const int32_t* frontier, const int32_t* frontier_len,
+                     int32_t* tokens, int32_t* tree_parent, int32_t* merge_to, uint8_t* leaf,
+                     float* prob, int32_t* num_nodes, int32_t* new_frontier,
+                     int32_t* new_frontier_len, const gsd_draft_params* p, void* workspace,
+                     size_t workspace_bytes, int32_t* status, void* stream);
 
 /*
  * gsd_accept_static - gsd_accept without a workspace argument.  (The paper has no counterpart

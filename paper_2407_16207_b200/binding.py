@@ -44,10 +44,17 @@ class AcceptParams(ctypes.Structure):
                 ("Ecap", ctypes.c_int32), ("Tcap", ctypes.c_int32)]
 
 
+class DraftParams(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("F", ctypes.c_int32), ("V", ctypes.c_int32),
+                ("Ncap", ctypes.c_int32), ("k", ctypes.c_int32), ("tau", ctypes.c_int32),
+                ("theta_prob", ctypes.c_float), ("theta_sib", ctypes.c_float)]
+
+
 EXPORTS = ["gsd_version", "gsd_status_string", "gsd_last_cuda_error", "gsd_verify_attn",
            "gsd_verify_attn_workspace_bytes", "gsd_verify_attn_num_splits", "gsd_accept",
            "gsd_accept_workspace_bytes", "gsd_accept_static", "gsd_accept_sampled",
-           "gsd_accept_sampled_workspace_bytes", "gsd_commit_kv", "gsd_build_mask", "gsd_verify_step_host",
+           "gsd_accept_sampled_workspace_bytes", "gsd_draft_expand", "gsd_draft_expand_workspace_bytes",
+           "gsd_commit_kv", "gsd_build_mask", "gsd_verify_step_host",
            "gsd_verify_step_host_arena_bytes"]
 
 
@@ -80,6 +87,10 @@ def lib() -> ctypes.CDLL:
         L.gsd_accept_sampled.argtypes = [vp] * 10 + [ctypes.POINTER(AcceptParams), vp, sz, vp, vp]
         L.gsd_accept_sampled_workspace_bytes.restype = sz
         L.gsd_accept_sampled_workspace_bytes.argtypes = [ctypes.POINTER(AcceptParams)]
+        L.gsd_draft_expand.restype = i32
+        L.gsd_draft_expand.argtypes = [vp] * 11 + [ctypes.POINTER(DraftParams), vp, sz, vp, vp]
+        L.gsd_draft_expand_workspace_bytes.restype = sz
+        L.gsd_draft_expand_workspace_bytes.argtypes = [ctypes.POINTER(DraftParams)]
         L.gsd_accept_static.restype = i32
         L.gsd_accept_static.argtypes = [vp] * 7 + [ctypes.POINTER(AcceptParams), vp, vp]
         L.gsd_build_mask.restype = i32
@@ -271,6 +282,39 @@ def gsd_accept_sampled(logits, draft_tokens, parent_ptr, parent_idx, draft_q, u_
                                     workspace.numel() * workspace.element_size(), _ptr(status),
                                     _stream(logits)))
     return toks, lens, nodes
+
+
+def gsd_draft_expand(logits, frontier, frontier_len, tokens, tree_parent, merge_to, leaf, prob, num_nodes, *,
+                     k: int, tau: int, theta_prob: float, theta_sib: float,
+                     workspace: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None
+                     ) -> Tuple[torch.Tensor, torch.Tensor]:
+    """One growth step of the draft token graph, in place; see gsd_draft_expand in include/gsd.h.
+    Returns (new_frontier [B,F*k], new_frontier_len [B])."""
+    if logits.dim() != 3:
+        raise ValueError("logits must be [B,F,V]")
+    B, F, V = logits.shape
+    Ncap = tokens.shape[1]
+    _want(logits, torch.float32, (B, F, V), "logits", True)
+    _want(frontier, torch.int32, (B, F), "frontier", True)
+    _want(frontier_len, torch.int32, (B,), "frontier_len", True)
+    for name, t, dt in (("tokens", tokens, torch.int32), ("tree_parent", tree_parent, torch.int32),
+                        ("merge_to", merge_to, torch.int32), ("leaf", leaf, torch.uint8), ("prob", prob, torch.float32)):
+        _want(t, dt, (B, Ncap), name, True)
+    _want(num_nodes, torch.int32, (B,), "num_nodes", True)
+    nf = torch.full((B, F * k), -1, dtype=torch.int32, device=logits.device)
+    nfl = torch.zeros((B,), dtype=torch.int32, device=logits.device)
+    p = DraftParams(B, F, V, Ncap, int(k), int(tau), float(theta_prob), float(theta_sib))
+    L = lib()
+    with torch.cuda.device(logits.device):
+        need = int(L.gsd_draft_expand_workspace_bytes(ctypes.byref(p)))
+        if workspace is None:
+            workspace = torch.empty(max(need, 8), dtype=torch.uint8, device=logits.device)
+        _check(L.gsd_draft_expand(logits.data_ptr(), frontier.data_ptr(), frontier_len.data_ptr(),
+                                  tokens.data_ptr(), tree_parent.data_ptr(), merge_to.data_ptr(), leaf.data_ptr(),
+                                  prob.data_ptr(), num_nodes.data_ptr(), nf.data_ptr(), nfl.data_ptr(),
+                                  ctypes.byref(p), workspace.data_ptr(),
+                                  workspace.numel() * workspace.element_size(), _ptr(status), _stream(logits)))
+    return nf, nfl
 
 
 def gsd_build_mask(parent_ptr, parent_idx, out: Optional[torch.Tensor] = None, *,

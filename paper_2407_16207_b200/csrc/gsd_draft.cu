@@ -1,0 +1,327 @@
+// gsd_draft_expand: one growth step of the draft token graph (Sec. 4: token tree of out-degree
+// k; Sec. 4.2: probability pruning and sibling pruning; Sec. 5.2: tau-redundant nodes; Sec. 5.3:
+// merge edges to the first occurrence).
+//
+// One launch.  Grid (F, B): the CTA of frontier row (b, fi) streams that row of draft logits
+// once with 16-byte loads; every thread keeps the k best (value, index) pairs it has seen and a
+// running (maximum, sum of exponentials); a block-wide selection leaves the row's k best tokens
+// and their probabilities in scratch.  The CTA that finishes last for a sequence appends the
+// children (k per frontier node, in frontier order), applies the two pruning rules, looks for
+// an earlier node with the same tau-gram for every new node (first occurrence = lowest id),
+// and compacts the new frontier.
+#include "gsd_internal.cuh"
+#include <math_constants.h>
+
+namespace gsd {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int K = GSD_DRAFT_MAX_K;
+constexpr float kLog2e = 1.4426950408889634f;
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// a candidate ranks before another if its logit is larger, or equal with the lower token id
+__device__ __forceinline__ bool before(float va, int ia, float vb, int ib) {
+    return va > vb || (va == vb && ia < ib);
+}
+
+struct TopK {
+    float v[K];
+    int i[K];
+};
+
+// insertion into the thread's list (descending).  A thread meets its elements in ascending
+// index order, so an equal value never displaces an earlier one.
+__device__ __forceinline__ void offer(TopK& t, float x, int idx) {
+    if (!(x > t.v[K - 1])) return;
+#pragma unroll
+    for (int j = K - 1; j >= 0; --j) {
+        const bool up = j > 0 && x > t.v[j - 1];     // the slot above also has to move down
+        if (up) {
+            t.v[j] = t.v[j - 1];
+            t.i[j] = t.i[j - 1];
+        } else {
+            t.v[j] = x;
+            t.i[j] = idx;
+            break;
+        }
+    }
+}
+
+struct DraftArgs {
+    const float* logits;
+    const int32_t* frontier;
+    const int32_t* frontier_len;
+    int32_t* tokens;
+    int32_t* tree_parent;
+    int32_t* merge_to;
+    uint8_t* leaf;
+    float* prob;
+    int32_t* num_nodes;
+    int32_t* new_frontier;
+    int32_t* new_frontier_len;
+    int32_t* wk_tok;     // [B,F,K]
+    float* wk_q;         // [B,F,K]
+    unsigned* done;      // [B], zeroed before the launch
+    int32_t* status;
+    int B, F, V, Ncap, k, tau;
+    float theta_prob, theta_sib;
+};
+
+__device__ void grow_sequence(const DraftArgs& a, int b) {
+    __shared__ int s_tok[GSD_MAX_NODES];
+    __shared__ int s_par[GSD_MAX_NODES];
+    __shared__ unsigned char s_leaf[GSD_MAX_NODES];
+    __shared__ int s_cnt[kWarps];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int Ncap = a.Ncap, k = a.k;
+    int32_t* tok = a.tokens + (size_t)b * Ncap;
+    int32_t* par = a.tree_parent + (size_t)b * Ncap;
+    int32_t* mrg = a.merge_to + (size_t)b * Ncap;
+    uint8_t* leaf = a.leaf + (size_t)b * Ncap;
+    float* prob = a.prob + (size_t)b * Ncap;
+    unsigned flags = 0;
+    int n0 = a.num_nodes[b];
+    int fl = a.frontier_len[b];
+    if (n0 < 1 || n0 > Ncap || fl < 0 || fl > a.F) {
+        // nothing sensible can be appended: leave the graph as it is
+        if (tid == 0) {
+            a.new_frontier_len[b] = 0;
+            if (a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_FRONTIER);
+        }
+        return;
+    }
+    int want = fl * k;
+    if (n0 + want > Ncap) {
+        want = Ncap - n0;
+        flags |= GSD_DEV_DRAFT_FULL;
+    }
+    const int n1 = n0 + want;
+    for (int v = tid; v < n0; v += kThreads) {
+        s_tok[v] = tok[v];
+        s_par[v] = par[v];
+    }
+    // the children: k per frontier node, in frontier order, best first
+    for (int j = tid; j < want; j += kThreads) {
+        const int fi = j / k, i = j % k, c = n0 + j;
+        const size_t w = ((size_t)b * a.F + fi) * K;
+        int p = a.frontier[(size_t)b * a.F + fi];
+        if (p < 0 || p >= n0) {
+            flags |= GSD_DEV_BAD_FRONTIER;
+            p = 0;
+        }
+        const float q = a.wk_q[w + i], qmax = a.wk_q[w];
+        s_tok[c] = a.wk_tok[w + i];
+        s_par[c] = p;
+        // Sec. 4.2: below the probability threshold, or too far below the best sibling
+        s_leaf[c] = (q < a.theta_prob) || (q < a.theta_sib * qmax);
+        prob[c] = q;
+    }
+    __syncthreads();
+    // Sec. 5.2 / 5.3: a new node whose last tau tokens along its tree path equal those of an
+    // earlier node is redundant; it becomes a leaf that points at the first such node
+    for (int j = tid; j < want; j += kThreads) {
+        const int c = n0 + j;
+        int first = -1;
+        for (int e = 0; e < c && first < 0; ++e) {
+            int x = c, y = e, t = 0;
+            for (; t < a.tau; ++t) {
+                if (x < 0 || y < 0 || s_tok[x] != s_tok[y]) break;
+                x = s_par[x];
+                y = s_par[y];
+            }
+            if (t == a.tau) first = e;
+        }
+        if (first >= 0) s_leaf[c] = 1;
+        tok[c] = s_tok[c];
+        par[c] = s_par[c];
+        mrg[c] = first;
+        leaf[c] = s_leaf[c];
+    }
+    __syncthreads();
+    // the new frontier: the new nodes that are not leaves, in id order
+    int32_t* nf = a.new_frontier + (size_t)b * a.F * k;
+    int base = 0;
+    for (int j0 = 0; j0 < want; j0 += kThreads) {
+        const int j = j0 + tid;
+        const bool keep = j < want && !s_leaf[n0 + j];
+        const unsigned bal = __ballot_sync(0xFFFFFFFFu, keep);
+        if (lane == 0) s_cnt[warp] = __popc(bal);
+        __syncthreads();
+        int off = base;
+        for (int w = 0; w < warp; ++w) off += s_cnt[w];
+        if (keep) nf[off + __popc(bal & ((1u << lane) - 1u))] = n0 + j;
+        for (int w = 0; w < kWarps; ++w) base += s_cnt[w];
+        __syncthreads();
+    }
+    if (tid == 0) {
+        a.new_frontier_len[b] = base;
+        a.num_nodes[b] = n1;
+    }
+    if (flags && a.status) atomicOr((unsigned*)a.status, flags);
+}
+
+template <bool kVec>
+__global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
+    __shared__ float s_v[kThreads * K];
+    __shared__ int s_i[kThreads * K];
+    __shared__ float s_rv[kWarps];
+    __shared__ int s_ri[kWarps], s_rt[kWarps];
+    __shared__ float s_m[kWarps], s_s[kWarps];
+    __shared__ int s_last;
+    const int fi = blockIdx.x, b = blockIdx.y;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int V = a.V;
+    int fl = a.frontier_len[b];
+    if (fi < fl && fl <= a.F) {
+        const float* x = a.logits + ((size_t)b * a.F + fi) * V;
+        TopK t;
+#pragma unroll
+        for (int j = 0; j < K; ++j) {
+            t.v[j] = -CUDART_INF_F;
+            t.i[j] = 0x7FFFFFFF;
+        }
+        float m = -CUDART_INF_F, s = 0.f;
+        auto take = [&](float val, int idx) {
+            offer(t, val, idx);
+            // -inf entries (filtered tokens) add nothing; the first finite entry sets the scale
+            if (val > m) {
+                s = s * ex2((m - val) * kLog2e) + 1.f;
+                m = val;
+            } else if (val > -CUDART_INF_F) {
+                s += ex2((val - m) * kLog2e);
+            } else if (val != val) {
+                s = val;    // NaN poisons the sum and is reported below
+            }
+        };
+        if (kVec) {
+            const float4* x4 = reinterpret_cast<const float4*>(x);
+            const int nvec = V >> 2;
+            int i = tid;
+            for (; i + kThreads < nvec; i += 2 * kThreads) {
+                const float4 r0 = __ldcs(x4 + i), r1 = __ldcs(x4 + i + kThreads);
+                int e = i * 4;
+                take(r0.x, e); take(r0.y, e + 1); take(r0.z, e + 2); take(r0.w, e + 3);
+                e += 4 * kThreads;
+                take(r1.x, e); take(r1.y, e + 1); take(r1.z, e + 2); take(r1.w, e + 3);
+            }
+            for (; i < nvec; i += kThreads) {
+                const float4 r = __ldcs(x4 + i);
+                const int e = i * 4;
+                take(r.x, e); take(r.y, e + 1); take(r.z, e + 2); take(r.w, e + 3);
+            }
+        } else {
+            for (int i = tid; i < V; i += kThreads) take(__ldcs(x + i), i);
+        }
+        // (maximum, sum) of the row
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m, o), s2 = __shfl_xor_sync(0xFFFFFFFFu, s, o);
+            const float mm = fmaxf(m, m2);
+            s = (mm == -CUDART_INF_F) ? 0.f : s * ex2((m - mm) * kLog2e) + s2 * ex2((m2 - mm) * kLog2e);
+            m = mm;
+        }
+        if (lane == 0) { s_m[warp] = m; s_s[warp] = s; }
+#pragma unroll
+        for (int j = 0; j < K; ++j) {
+            s_v[tid * K + j] = t.v[j];
+            s_i[tid * K + j] = t.i[j];
+        }
+        __syncthreads();
+        float rm = -CUDART_INF_F, rs = 0.f;
+        for (int w = 0; w < kWarps; ++w) {
+            const float mm = fmaxf(rm, s_m[w]);
+            rs = (mm == -CUDART_INF_F) ? 0.f : rs * ex2((rm - mm) * kLog2e) + s_s[w] * ex2((s_m[w] - mm) * kLog2e);
+            rm = mm;
+        }
+        if (tid == 0 && (!(rs > 0.f) || rm == CUDART_INF_F) && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
+        // k rounds: every thread offers the head of its list, the block picks the best, its owner moves on
+        int head = 0;
+        const size_t w = ((size_t)b * a.F + fi) * K;
+        for (int r = 0; r < a.k; ++r) {
+            float bv = head < K ? s_v[tid * K + head] : -CUDART_INF_F;
+            int bi = head < K ? s_i[tid * K + head] : 0x7FFFFFFF;
+            int bt = tid;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float v2 = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
+                const int i2 = __shfl_xor_sync(0xFFFFFFFFu, bi, o), t2 = __shfl_xor_sync(0xFFFFFFFFu, bt, o);
+                if (before(v2, i2, bv, bi)) { bv = v2; bi = i2; bt = t2; }
+            }
+            if (lane == 0) { s_rv[warp] = bv; s_ri[warp] = bi; s_rt[warp] = bt; }
+            __syncthreads();
+            bv = s_rv[0]; bi = s_ri[0]; bt = s_rt[0];
+            for (int q = 1; q < kWarps; ++q)
+                if (before(s_rv[q], s_ri[q], bv, bi)) { bv = s_rv[q]; bi = s_ri[q]; bt = s_rt[q]; }
+            if (tid == bt) ++head;
+            if (tid == 0) {
+                if (bi == 0x7FFFFFFF && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);   // fewer than k entries above -inf
+                a.wk_tok[w + r] = bi == 0x7FFFFFFF ? -1 : bi;
+                a.wk_q[w + r] = bv == -CUDART_INF_F ? 0.f : ex2((bv - rm) * kLog2e) / rs;
+            }
+            __syncthreads();
+        }
+    }
+    if (tid == 0) {
+        __threadfence();
+        const unsigned prev = atomicAdd(a.done + b, 1u);
+        s_last = (prev == (unsigned)a.F - 1u);
+    }
+    __syncthreads();
+    if (s_last) {
+        __threadfence();
+        grow_sequence(a, b);
+    }
+}
+
+}  // namespace
+}  // namespace gsd
+
+extern "C" size_t gsd_draft_expand_workspace_bytes(const gsd_draft_params* p) {
+    if (!p || p->B < 1 || p->F < 1) return 0;
+    return gsd::align_up((size_t)p->B * p->F * GSD_DRAFT_MAX_K * 8 + (size_t)p->B * 4, 256);
+}
+
+extern "C" int gsd_draft_expand(const float* logits, const int32_t* frontier, const int32_t* frontier_len,
+                                int32_t* tokens, int32_t* tree_parent, int32_t* merge_to, uint8_t* leaf,
+                                float* prob, int32_t* num_nodes, int32_t* new_frontier,
+                                int32_t* new_frontier_len, const gsd_draft_params* p, void* workspace,
+                                size_t workspace_bytes, int32_t* status, void* stream) {
+    using namespace gsd;
+    if (!p || !logits || !frontier || !frontier_len || !tokens || !tree_parent || !merge_to || !leaf ||
+        !prob || !num_nodes || !new_frontier || !new_frontier_len)
+        return GSD_ERR_NULL_POINTER;
+    if (p->B < 1 || p->B > 65535 || p->F < 1 || p->V < 1 || p->Ncap < 1 || p->Ncap > GSD_MAX_NODES ||
+        p->k < 1 || p->k > GSD_DRAFT_MAX_K || p->k > p->V || p->tau < 1 || p->tau > GSD_MAX_NODES)
+        return GSD_ERR_BAD_SHAPE;
+    if (((uintptr_t)logits & 3u) != 0) return GSD_ERR_MISALIGNED;
+    const size_t need = gsd_draft_expand_workspace_bytes(p);
+    if (!workspace || workspace_bytes < need) return GSD_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 7u) != 0) return GSD_ERR_MISALIGNED;
+    cudaStream_t st = (cudaStream_t)stream;
+    DraftArgs a;
+    a.logits = logits; a.frontier = frontier; a.frontier_len = frontier_len;
+    a.tokens = tokens; a.tree_parent = tree_parent; a.merge_to = merge_to; a.leaf = leaf; a.prob = prob;
+    a.num_nodes = num_nodes; a.new_frontier = new_frontier; a.new_frontier_len = new_frontier_len;
+    const size_t rows = (size_t)p->B * p->F * GSD_DRAFT_MAX_K;
+    a.wk_tok = (int32_t*)workspace;
+    a.wk_q = (float*)((char*)workspace + rows * 4);
+    a.done = (unsigned*)((char*)workspace + rows * 8);
+    a.status = status;
+    a.B = p->B; a.F = p->F; a.V = p->V; a.Ncap = p->Ncap; a.k = p->k; a.tau = p->tau;
+    a.theta_prob = p->theta_prob; a.theta_sib = p->theta_sib;
+    // only the completion counters have to start at zero
+    GSD_CUDA_TRY(cudaMemsetAsync(a.done, 0, (size_t)p->B * 4, st));
+    const bool vec = (p->V % 4 == 0) && (((uintptr_t)logits & 15u) == 0);
+    dim3 grid((unsigned)p->F, (unsigned)p->B);
+    if (vec) draft_expand_kernel<true><<<grid, kThreads, 0, st>>>(a);
+    else draft_expand_kernel<false><<<grid, kThreads, 0, st>>>(a);
+    GSD_CUDA_TRY(cudaGetLastError());
+    return GSD_OK;
+}
