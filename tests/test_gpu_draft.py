@@ -56,7 +56,7 @@ def compare(got, want, nf_g, nfl_g, nf_w, nfl_w):
         assert nfl_g[b] == nfl_w[b] and np.array_equal(nf_g[b, :nfl_g[b]], nf_w[b, :nfl_w[b]])
 
 
-def grow_levels(B, V, k, tau, levels, Ncap, seed, logit_scale=3.0, round_to=None, drop=0.0):
+def grow_levels(B, V, k, tau, levels, Ncap, seed, logit_scale=3.0, round_to=None, drop=0.0, tp_range=(0.02, 0.4), ts_range=(0.05, 0.6)):
     rng = np.random.default_rng(seed)
     state = fresh(B, Ncap)
     frontier = [[0] for _ in range(B)]
@@ -64,6 +64,10 @@ def grow_levels(B, V, k, tau, levels, Ncap, seed, logit_scale=3.0, round_to=None
     for level in range(levels):
         F = max(1, max(len(f) for f in frontier))
         lg = (rng.normal(size=(B, F, V)) * logit_scale).astype(np.float32)
+        if V > 4 * k:
+            # a peaked draft distribution: a handful of tokens well above the rest
+            hot = rng.integers(0, V, size=(B, F, 2 * k))
+            np.put_along_axis(lg, hot, (rng.uniform(4, 7, size=hot.shape) * logit_scale + 4).astype(np.float32), axis=-1)
         if round_to:
             lg = np.round(lg / round_to).astype(np.float32) * np.float32(round_to)     # exact ties between logits
         if drop > 0:
@@ -74,7 +78,7 @@ def grow_levels(B, V, k, tau, levels, Ncap, seed, logit_scale=3.0, round_to=None
         fr = np.full((B, F), -1, np.int32); fl = np.zeros((B,), np.int32)
         for b, f in enumerate(frontier):
             fr[b, :len(f)] = f; fl[b] = len(f)
-        tp, ts = decisive_thresholds(lg, fl, k, rng)
+        tp, ts = decisive_thresholds(lg, fl, k, rng, tp_range, ts_range)
         status = torch.zeros(1, dtype=torch.int32, device="cuda")
         got, nf_g, nfl_g = gpu_step(state, lg, fr, fl, k, tau, tp, ts, status=status)
         out = oracle.draft_expand(lg, fr, fl, *state, k=k, tau=tau, theta_prob=tp, theta_sib=ts)
@@ -91,8 +95,8 @@ def grow_levels(B, V, k, tau, levels, Ncap, seed, logit_scale=3.0, round_to=None
 
 
 def test_llama_vocabulary_four_levels():
-    state, _ = grow_levels(B=3, V=32000, k=4, tau=2, levels=4, Ncap=512, seed=1)
-    assert state[5].min() > 5
+    state, _ = grow_levels(B=3, V=32000, k=4, tau=2, levels=5, Ncap=512, seed=1, tp_range=(0.005, 0.05), ts_range=(0.02, 0.2))
+    assert state[5].min() > 40
 
 
 @pytest.mark.parametrize("tau", [1, 2, 3])
