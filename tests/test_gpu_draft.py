@@ -1,6 +1,6 @@
 """gsd_draft_expand on the GPU against the CPU oracle, level by level.  The order of the children
 compares logits (exact on both sides); the pruning flags compare fp32 probabilities with
-thresholds, so the thresholds of these tests are placed at least 2 % (relative) away from every
+thresholds, so the thresholds of these tests are placed at least 0.2 % (relative) away from every
 probability (and probability ratio) they are compared with - taken from a numpy fp64 softmax."""
 import numpy as np
 import pytest
@@ -29,11 +29,13 @@ def decisive_thresholds(lg, fl, k, rng, tp_range=(0.02, 0.4), ts_range=(0.05, 0.
     rows = [top[b, f] for b in range(lg.shape[0]) for f in range(fl[b])]
     q = np.concatenate(rows) if rows else np.zeros(0)
     ratio = np.concatenate([r / r[0] for r in rows]) if rows else np.zeros(0)
-    for _ in range(1000):
-        tp, ts = rng.uniform(*tp_range), rng.uniform(*ts_range)
-        if (np.abs(q - tp) > 0.02 * tp).all() and (np.abs(ratio - ts) > 0.02 * ts).all():
-            return float(np.float32(tp)), float(np.float32(ts))
-    raise AssertionError("no decisive thresholds found")
+    def pick(values, lo_hi):
+        for _ in range(4000):
+            t = rng.uniform(*lo_hi)
+            if (np.abs(values - t) > 0.002 * t).all():
+                return float(np.float32(t))
+        raise AssertionError("no decisive threshold found")
+    return pick(q, tp_range), pick(ratio, ts_range)
 
 
 def gpu_step(state, lg, fr, fl, k, tau, tp, ts, status=None):
