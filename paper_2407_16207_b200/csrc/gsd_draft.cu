@@ -188,6 +188,7 @@ __global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
             t.i[j] = 0x7FFFFFFF;
         }
         float m = -CUDART_INF_F, s = 0.f;
+        // one value: into the list if it beats the thread's k-th, and into the running sum
         auto take = [&](float val, int idx) {
             offer(t, val, idx);
             // -inf entries (filtered tokens) add nothing; the first finite entry sets the scale
@@ -200,16 +201,45 @@ __global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
                 s = val;    // NaN poisons the sum and is reported below
             }
         };
+        // sixteen values: one comparison of their maximum against the k-th best decides whether
+        // any of them has to be offered at all, and the running sum is rescaled once
+        auto take16 = [&](const float4& r0, const float4& r1, const float4& r2, const float4& r3, int e0) {
+            const float a = fmaxf(fmaxf(fmaxf(r0.x, r0.y), fmaxf(r0.z, r0.w)), fmaxf(fmaxf(r1.x, r1.y), fmaxf(r1.z, r1.w)));
+            const float c = fmaxf(fmaxf(fmaxf(r2.x, r2.y), fmaxf(r2.z, r2.w)), fmaxf(fmaxf(r3.x, r3.y), fmaxf(r3.z, r3.w)));
+            const float g = fmaxf(a, c);
+            if (g > t.v[K - 1]) {
+                offer(t, r0.x, e0); offer(t, r0.y, e0 + 1); offer(t, r0.z, e0 + 2); offer(t, r0.w, e0 + 3);
+                const int e1 = e0 + 4 * kThreads;
+                offer(t, r1.x, e1); offer(t, r1.y, e1 + 1); offer(t, r1.z, e1 + 2); offer(t, r1.w, e1 + 3);
+                const int e2 = e1 + 4 * kThreads;
+                offer(t, r2.x, e2); offer(t, r2.y, e2 + 1); offer(t, r2.z, e2 + 2); offer(t, r2.w, e2 + 3);
+                const int e3 = e2 + 4 * kThreads;
+                offer(t, r3.x, e3); offer(t, r3.y, e3 + 1); offer(t, r3.z, e3 + 2); offer(t, r3.w, e3 + 3);
+            }
+            const float mn = fmaxf(m, g);
+            if (mn == -CUDART_INF_F) {
+                // nothing finite yet; a NaN among the sixteen still has to poison the sum
+                s += (r0.x + r0.y + r0.z + r0.w) + (r1.x + r1.y + r1.z + r1.w) + (r2.x + r2.y + r2.z + r2.w) + (r3.x + r3.y + r3.z + r3.w) == -CUDART_INF_F ? 0.f : CUDART_NAN_F;
+                return;
+            }
+            const float kk = -mn * kLog2e;
+            float acc = s * ex2(fmaf(m, kLog2e, kk));
+            acc += ex2(fmaf(r0.x, kLog2e, kk)) + ex2(fmaf(r0.y, kLog2e, kk)) + ex2(fmaf(r0.z, kLog2e, kk)) + ex2(fmaf(r0.w, kLog2e, kk));
+            acc += ex2(fmaf(r1.x, kLog2e, kk)) + ex2(fmaf(r1.y, kLog2e, kk)) + ex2(fmaf(r1.z, kLog2e, kk)) + ex2(fmaf(r1.w, kLog2e, kk));
+            acc += ex2(fmaf(r2.x, kLog2e, kk)) + ex2(fmaf(r2.y, kLog2e, kk)) + ex2(fmaf(r2.z, kLog2e, kk)) + ex2(fmaf(r2.w, kLog2e, kk));
+            acc += ex2(fmaf(r3.x, kLog2e, kk)) + ex2(fmaf(r3.y, kLog2e, kk)) + ex2(fmaf(r3.z, kLog2e, kk)) + ex2(fmaf(r3.w, kLog2e, kk));
+            s = acc;
+            m = mn;
+        };
         if (kVec) {
             const float4* x4 = reinterpret_cast<const float4*>(x);
             const int nvec = V >> 2;
             int i = tid;
-            for (; i + kThreads < nvec; i += 2 * kThreads) {
+            // four independent 16-byte loads in flight per thread
+            for (; i + 3 * kThreads < nvec; i += 4 * kThreads) {
                 const float4 r0 = __ldcs(x4 + i), r1 = __ldcs(x4 + i + kThreads);
-                int e = i * 4;
-                take(r0.x, e); take(r0.y, e + 1); take(r0.z, e + 2); take(r0.w, e + 3);
-                e += 4 * kThreads;
-                take(r1.x, e); take(r1.y, e + 1); take(r1.z, e + 2); take(r1.w, e + 3);
+                const float4 r2 = __ldcs(x4 + i + 2 * kThreads), r3 = __ldcs(x4 + i + 3 * kThreads);
+                take16(r0, r1, r2, r3, i * 4);
             }
             for (; i < nvec; i += kThreads) {
                 const float4 r = __ldcs(x4 + i);
