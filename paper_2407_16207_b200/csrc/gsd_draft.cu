@@ -31,6 +31,15 @@ __device__ __forceinline__ bool before(float va, int ia, float vb, int ib) {
     return va > vb || (va == vb && ia < ib);
 }
 
+// monotone map of non-NaN floats to unsigned and back (for an atomicMax on a float)
+__device__ __forceinline__ unsigned ordered_bits(float v) {
+    const unsigned u = __float_as_uint(v);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_bits(unsigned o) {
+    return __uint_as_float((o & 0x80000000u) ? (o & 0x7FFFFFFFu) : ~o);
+}
+
 struct TopK {
     float v[K];
     int i[K];
@@ -175,10 +184,17 @@ __global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
     __shared__ int s_ri[kWarps], s_rt[kWarps];
     __shared__ float s_m[kWarps], s_s[kWarps];
     __shared__ int s_last;
+    // A lower bound on the row's k-th best logit, shared by the block: the k-th best of any one
+    // thread is such a bound, so every thread publishes its own and skips what lies below the
+    // largest published one.  (A thread alone sees too few values for its own k-th best to
+    // reject much.)  Values equal to the bound are kept: ties are decided by the token id.
+    __shared__ unsigned s_bound;
     const int fi = blockIdx.x, b = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int V = a.V;
     int fl = a.frontier_len[b];
+    if (threadIdx.x == 0) s_bound = ordered_bits(-CUDART_INF_F);
+    __syncthreads();
     if (fi < fl && fl <= a.F) {
         const float* x = a.logits + ((size_t)b * a.F + fi) * V;
         TopK t;
@@ -207,7 +223,8 @@ __global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
             const float a = fmaxf(fmaxf(fmaxf(r0.x, r0.y), fmaxf(r0.z, r0.w)), fmaxf(fmaxf(r1.x, r1.y), fmaxf(r1.z, r1.w)));
             const float c = fmaxf(fmaxf(fmaxf(r2.x, r2.y), fmaxf(r2.z, r2.w)), fmaxf(fmaxf(r3.x, r3.y), fmaxf(r3.z, r3.w)));
             const float g = fmaxf(a, c);
-            if (g > t.v[K - 1]) {
+            const float bound = from_ordered_bits(*(volatile unsigned*)&s_bound);
+            if (g >= bound && g > t.v[K - 1]) {
                 offer(t, r0.x, e0); offer(t, r0.y, e0 + 1); offer(t, r0.z, e0 + 2); offer(t, r0.w, e0 + 3);
                 const int e1 = e0 + 4 * kThreads;
                 offer(t, r1.x, e1); offer(t, r1.y, e1 + 1); offer(t, r1.z, e1 + 2); offer(t, r1.w, e1 + 3);
@@ -215,6 +232,11 @@ __global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
                 offer(t, r2.x, e2); offer(t, r2.y, e2 + 1); offer(t, r2.z, e2 + 2); offer(t, r2.w, e2 + 3);
                 const int e3 = e2 + 4 * kThreads;
                 offer(t, r3.x, e3); offer(t, r3.y, e3 + 1); offer(t, r3.z, e3 + 2); offer(t, r3.w, e3 + 3);
+                // this thread's k-th best (k <= K) is a bound for everybody
+                float kth = t.v[0];
+#pragma unroll
+                for (int j = 1; j < K; ++j) kth = (j < a.k) ? t.v[j] : kth;
+                if (kth > bound) atomicMax(&s_bound, ordered_bits(kth));
             }
             const float mn = fmaxf(m, g);
             if (mn == -CUDART_INF_F) {
