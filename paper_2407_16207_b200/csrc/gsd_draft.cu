@@ -220,9 +220,9 @@ __global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
         // sixteen values: one comparison of their maximum against the k-th best decides whether
         // any of them has to be offered at all, and the running sum is rescaled once
         auto take16 = [&](const float4& r0, const float4& r1, const float4& r2, const float4& r3, int e0) {
-            const float a = fmaxf(fmaxf(fmaxf(r0.x, r0.y), fmaxf(r0.z, r0.w)), fmaxf(fmaxf(r1.x, r1.y), fmaxf(r1.z, r1.w)));
-            const float c = fmaxf(fmaxf(fmaxf(r2.x, r2.y), fmaxf(r2.z, r2.w)), fmaxf(fmaxf(r3.x, r3.y), fmaxf(r3.z, r3.w)));
-            const float g = fmaxf(a, c);
+            const float g01 = fmaxf(fmaxf(fmaxf(r0.x, r0.y), fmaxf(r0.z, r0.w)), fmaxf(fmaxf(r1.x, r1.y), fmaxf(r1.z, r1.w)));
+            const float g23 = fmaxf(fmaxf(fmaxf(r2.x, r2.y), fmaxf(r2.z, r2.w)), fmaxf(fmaxf(r3.x, r3.y), fmaxf(r3.z, r3.w)));
+            const float g = fmaxf(g01, g23);
             const float bound = from_ordered_bits(*(volatile unsigned*)&s_bound);
             if (g >= bound && g > t.v[K - 1]) {
                 offer(t, r0.x, e0); offer(t, r0.y, e0 + 1); offer(t, r0.z, e0 + 2); offer(t, r0.w, e0 + 3);
