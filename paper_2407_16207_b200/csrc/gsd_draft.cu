@@ -3,9 +3,9 @@
 // merge edges to the first occurrence).
 //
 // One launch.  Grid (F, B): the CTA of frontier row (b, fi) streams that row of draft logits
-// once with 16-byte loads; every thread keeps the k best (value, index) pairs it has seen and a
-// running (maximum, sum of exponentials); a block-wide selection leaves the row's k best tokens
-// and their probabilities in scratch.  The CTA that finishes last for a sequence appends the
+// with 16-byte loads for the softmax statistics and a lower bound on the k-th best logit, reads
+// it once more (from L2) to collect the few entries above the bound, and leaves the row's k best
+// tokens and their probabilities in scratch.  The CTA that finishes last for a sequence appends the
 // children (k per frontier node, in frontier order), applies the two pruning rules, looks for
 // an earlier node with the same tau-gram for every new node (first occurrence = lowest id),
 // and compacts the new frontier.
@@ -29,15 +29,6 @@ __device__ __forceinline__ float ex2(float x) {
 // a candidate ranks before another if its logit is larger, or equal with the lower token id
 __device__ __forceinline__ bool before(float va, int ia, float vb, int ib) {
     return va > vb || (va == vb && ia < ib);
-}
-
-// monotone map of non-NaN floats to unsigned and back (for an atomicMax on a float)
-__device__ __forceinline__ unsigned ordered_bits(float v) {
-    const unsigned u = __float_as_uint(v);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-__device__ __forceinline__ float from_ordered_bits(unsigned o) {
-    return __uint_as_float((o & 0x80000000u) ? (o & 0x7FFFFFFFu) : ~o);
 }
 
 struct TopK {
@@ -176,38 +167,52 @@ __device__ void grow_sequence(const DraftArgs& a, int b) {
     if (flags && a.status) atomicOr((unsigned*)a.status, flags);
 }
 
+constexpr int kCand = 1024;   // candidates (logit >= bound) a row may have before the exact fallback takes over
+
+// Block-wide pick of the best remaining (value, index) pair, ranked by `before`; every thread
+// passes its own proposal and gets the winner (and the proposing thread) back.
+__device__ __forceinline__ void block_best(float& v, int& i, int& owner, float* s_rv, int* s_ri, int* s_rt) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float v2 = __shfl_xor_sync(0xFFFFFFFFu, v, o);
+        const int i2 = __shfl_xor_sync(0xFFFFFFFFu, i, o), t2 = __shfl_xor_sync(0xFFFFFFFFu, owner, o);
+        if (before(v2, i2, v, i)) { v = v2; i = i2; owner = t2; }
+    }
+    if (lane == 0) { s_rv[warp] = v; s_ri[warp] = i; s_rt[warp] = owner; }
+    __syncthreads();
+    v = s_rv[0]; i = s_ri[0]; owner = s_rt[0];
+    for (int q = 1; q < kWarps; ++q)
+        if (before(s_rv[q], s_ri[q], v, i)) { v = s_rv[q]; i = s_ri[q]; owner = s_rt[q]; }
+    __syncthreads();
+}
+
+// The k best tokens of one row of logits and their probabilities.
+// Pass 1 streams the row: running (maximum, sum of exponentials) per thread, and each thread's
+// own largest value.  The k-th largest of those 256 thread maxima is a lower bound on the row's
+// k-th best logit (they are k different entries).  Pass 2 reads the row again (it is still in
+// L2) and collects the entries >= that bound - a few dozen at most for any peaked or random row;
+// the k best of them, ties to the lower token id, are the answer.  A row with more than kCand
+// such entries (long runs of equal logits) takes the exact fallback: every thread keeps the K
+// best pairs it meets and the block merges the 256 lists.
 template <bool kVec>
 __global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
-    __shared__ float s_v[kThreads * K];
-    __shared__ int s_i[kThreads * K];
+    __shared__ float s_cv[kCand];
+    __shared__ int s_ci[kCand];
     __shared__ float s_rv[kWarps];
     __shared__ int s_ri[kWarps], s_rt[kWarps];
     __shared__ float s_m[kWarps], s_s[kWarps];
-    __shared__ int s_last;
-    // A lower bound on the row's k-th best logit, shared by the block: the k-th best of any one
-    // thread is such a bound, so every thread publishes its own and skips what lies below the
-    // largest published one.  (A thread alone sees too few values for its own k-th best to
-    // reject much.)  Values equal to the bound are kept: ties are decided by the token id.
-    __shared__ unsigned s_bound;
+    __shared__ int s_last, s_count;
     const int fi = blockIdx.x, b = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int V = a.V;
-    int fl = a.frontier_len[b];
-    if (threadIdx.x == 0) s_bound = ordered_bits(-CUDART_INF_F);
-    __syncthreads();
+    const int fl = a.frontier_len[b];
     if (fi < fl && fl <= a.F) {
         const float* x = a.logits + ((size_t)b * a.F + fi) * V;
-        TopK t;
-#pragma unroll
-        for (int j = 0; j < K; ++j) {
-            t.v[j] = -CUDART_INF_F;
-            t.i[j] = 0x7FFFFFFF;
-        }
-        float m = -CUDART_INF_F, s = 0.f;
-        // one value: into the list if it beats the thread's k-th, and into the running sum
-        auto take = [&](float val, int idx) {
-            offer(t, val, idx);
-            // -inf entries (filtered tokens) add nothing; the first finite entry sets the scale
+        const float4* x4 = reinterpret_cast<const float4*>(x);
+        const int nvec = V >> 2;
+        float m = -CUDART_INF_F, s = 0.f;        // running maximum (= this thread's best) and sum
+        auto take = [&](float val) {
             if (val > m) {
                 s = s * ex2((m - val) * kLog2e) + 1.f;
                 m = val;
@@ -217,60 +222,37 @@ __global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
                 s = val;    // NaN poisons the sum and is reported below
             }
         };
-        // sixteen values: one comparison of their maximum against the k-th best decides whether
-        // any of them has to be offered at all, and the running sum is rescaled once
-        auto take16 = [&](const float4& r0, const float4& r1, const float4& r2, const float4& r3, int e0) {
-            const float g01 = fmaxf(fmaxf(fmaxf(r0.x, r0.y), fmaxf(r0.z, r0.w)), fmaxf(fmaxf(r1.x, r1.y), fmaxf(r1.z, r1.w)));
-            const float g23 = fmaxf(fmaxf(fmaxf(r2.x, r2.y), fmaxf(r2.z, r2.w)), fmaxf(fmaxf(r3.x, r3.y), fmaxf(r3.z, r3.w)));
-            const float g = fmaxf(g01, g23);
-            const float bound = from_ordered_bits(*(volatile unsigned*)&s_bound);
-            if (g >= bound && g > t.v[K - 1]) {
-                offer(t, r0.x, e0); offer(t, r0.y, e0 + 1); offer(t, r0.z, e0 + 2); offer(t, r0.w, e0 + 3);
-                const int e1 = e0 + 4 * kThreads;
-                offer(t, r1.x, e1); offer(t, r1.y, e1 + 1); offer(t, r1.z, e1 + 2); offer(t, r1.w, e1 + 3);
-                const int e2 = e1 + 4 * kThreads;
-                offer(t, r2.x, e2); offer(t, r2.y, e2 + 1); offer(t, r2.z, e2 + 2); offer(t, r2.w, e2 + 3);
-                const int e3 = e2 + 4 * kThreads;
-                offer(t, r3.x, e3); offer(t, r3.y, e3 + 1); offer(t, r3.z, e3 + 2); offer(t, r3.w, e3 + 3);
-                // this thread's k-th best (k <= K) is a bound for everybody
-                float kth = t.v[0];
-#pragma unroll
-                for (int j = 1; j < K; ++j) kth = (j < a.k) ? t.v[j] : kth;
-                if (kth > bound) atomicMax(&s_bound, ordered_bits(kth));
-            }
-            const float mn = fmaxf(m, g);
-            if (mn == -CUDART_INF_F) {
-                // nothing finite yet; a NaN among the sixteen still has to poison the sum
-                s += (r0.x + r0.y + r0.z + r0.w) + (r1.x + r1.y + r1.z + r1.w) + (r2.x + r2.y + r2.z + r2.w) + (r3.x + r3.y + r3.z + r3.w) == -CUDART_INF_F ? 0.f : CUDART_NAN_F;
-                return;
-            }
-            const float kk = -mn * kLog2e;
-            float acc = s * ex2(fmaf(m, kLog2e, kk));
-            acc += ex2(fmaf(r0.x, kLog2e, kk)) + ex2(fmaf(r0.y, kLog2e, kk)) + ex2(fmaf(r0.z, kLog2e, kk)) + ex2(fmaf(r0.w, kLog2e, kk));
-            acc += ex2(fmaf(r1.x, kLog2e, kk)) + ex2(fmaf(r1.y, kLog2e, kk)) + ex2(fmaf(r1.z, kLog2e, kk)) + ex2(fmaf(r1.w, kLog2e, kk));
-            acc += ex2(fmaf(r2.x, kLog2e, kk)) + ex2(fmaf(r2.y, kLog2e, kk)) + ex2(fmaf(r2.z, kLog2e, kk)) + ex2(fmaf(r2.w, kLog2e, kk));
-            acc += ex2(fmaf(r3.x, kLog2e, kk)) + ex2(fmaf(r3.y, kLog2e, kk)) + ex2(fmaf(r3.z, kLog2e, kk)) + ex2(fmaf(r3.w, kLog2e, kk));
-            s = acc;
-            m = mn;
-        };
         if (kVec) {
-            const float4* x4 = reinterpret_cast<const float4*>(x);
-            const int nvec = V >> 2;
             int i = tid;
-            // four independent 16-byte loads in flight per thread
+            // four independent 16-byte loads in flight per thread; one rescale per sixteen values
             for (; i + 3 * kThreads < nvec; i += 4 * kThreads) {
-                const float4 r0 = __ldcs(x4 + i), r1 = __ldcs(x4 + i + kThreads);
-                const float4 r2 = __ldcs(x4 + i + 2 * kThreads), r3 = __ldcs(x4 + i + 3 * kThreads);
-                take16(r0, r1, r2, r3, i * 4);
+                const float4 r0 = x4[i], r1 = x4[i + kThreads], r2 = x4[i + 2 * kThreads], r3 = x4[i + 3 * kThreads];
+                const float g01 = fmaxf(fmaxf(fmaxf(r0.x, r0.y), fmaxf(r0.z, r0.w)), fmaxf(fmaxf(r1.x, r1.y), fmaxf(r1.z, r1.w)));
+                const float g23 = fmaxf(fmaxf(fmaxf(r2.x, r2.y), fmaxf(r2.z, r2.w)), fmaxf(fmaxf(r3.x, r3.y), fmaxf(r3.z, r3.w)));
+                const float mn = fmaxf(m, fmaxf(g01, g23));
+                if (mn == -CUDART_INF_F) {
+                    // nothing finite yet; a NaN among the sixteen still has to poison the sum
+                    const float t16 = (r0.x + r0.y + r0.z + r0.w) + (r1.x + r1.y + r1.z + r1.w) + (r2.x + r2.y + r2.z + r2.w) + (r3.x + r3.y + r3.z + r3.w);
+                    if (t16 != t16) s = t16;
+                    continue;
+                }
+                const float kk = -mn * kLog2e;
+                float acc = s * ex2(fmaf(m, kLog2e, kk));
+                acc += ex2(fmaf(r0.x, kLog2e, kk)) + ex2(fmaf(r0.y, kLog2e, kk)) + ex2(fmaf(r0.z, kLog2e, kk)) + ex2(fmaf(r0.w, kLog2e, kk));
+                acc += ex2(fmaf(r1.x, kLog2e, kk)) + ex2(fmaf(r1.y, kLog2e, kk)) + ex2(fmaf(r1.z, kLog2e, kk)) + ex2(fmaf(r1.w, kLog2e, kk));
+                acc += ex2(fmaf(r2.x, kLog2e, kk)) + ex2(fmaf(r2.y, kLog2e, kk)) + ex2(fmaf(r2.z, kLog2e, kk)) + ex2(fmaf(r2.w, kLog2e, kk));
+                acc += ex2(fmaf(r3.x, kLog2e, kk)) + ex2(fmaf(r3.y, kLog2e, kk)) + ex2(fmaf(r3.z, kLog2e, kk)) + ex2(fmaf(r3.w, kLog2e, kk));
+                s = acc;
+                m = mn;
             }
             for (; i < nvec; i += kThreads) {
-                const float4 r = __ldcs(x4 + i);
-                const int e = i * 4;
-                take(r.x, e); take(r.y, e + 1); take(r.z, e + 2); take(r.w, e + 3);
+                const float4 r = x4[i];
+                take(r.x); take(r.y); take(r.z); take(r.w);
             }
         } else {
-            for (int i = tid; i < V; i += kThreads) take(__ldcs(x + i), i);
+            for (int i = tid; i < V; i += kThreads) take(x[i]);
         }
+        const float my_best = m;
         // (maximum, sum) of the row
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -280,11 +262,7 @@ __global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
             m = mm;
         }
         if (lane == 0) { s_m[warp] = m; s_s[warp] = s; }
-#pragma unroll
-        for (int j = 0; j < K; ++j) {
-            s_v[tid * K + j] = t.v[j];
-            s_i[tid * K + j] = t.i[j];
-        }
+        if (tid == 0) s_count = 0;
         __syncthreads();
         float rm = -CUDART_INF_F, rs = 0.f;
         for (int w = 0; w < kWarps; ++w) {
@@ -293,31 +271,81 @@ __global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
             rm = mm;
         }
         if (tid == 0 && (!(rs > 0.f) || rm == CUDART_INF_F) && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
-        // k rounds: every thread offers the head of its list, the block picks the best, its owner moves on
-        int head = 0;
+        // the k-th largest of the 256 thread maxima
+        float bound = -CUDART_INF_F;
+        {
+            bool taken = false;
+            for (int r = 0; r < a.k; ++r) {
+                float v = taken ? -CUDART_INF_F : my_best;
+                int i = tid, owner = tid;
+                block_best(v, i, owner, s_rv, s_ri, s_rt);
+                if (owner == tid) taken = true;
+                bound = v;
+            }
+        }
+        // pass 2: everything >= bound (and above -inf) is a candidate
+        auto consider = [&](float val, int idx) {
+            if (val >= bound && val > -CUDART_INF_F) {
+                const int slot = atomicAdd(&s_count, 1);
+                if (slot < kCand) { s_cv[slot] = val; s_ci[slot] = idx; }
+            }
+        };
+        if (kVec) {
+            for (int i = tid; i < nvec; i += kThreads) {
+                const float4 r = x4[i];
+                const int e = i * 4;
+                if (fmaxf(fmaxf(r.x, r.y), fmaxf(r.z, r.w)) >= bound) {
+                    consider(r.x, e); consider(r.y, e + 1); consider(r.z, e + 2); consider(r.w, e + 3);
+                }
+            }
+        } else {
+            for (int i = tid; i < V; i += kThreads) consider(x[i], i);
+        }
+        __syncthreads();
+        const int count = s_count;
         const size_t w = ((size_t)b * a.F + fi) * K;
-        for (int r = 0; r < a.k; ++r) {
-            float bv = head < K ? s_v[tid * K + head] : -CUDART_INF_F;
-            int bi = head < K ? s_i[tid * K + head] : 0x7FFFFFFF;
-            int bt = tid;
+        if (count <= kCand) {
+            // k rounds over the candidate list: each thread proposes the best of its strided share
+            for (int r = 0; r < a.k; ++r) {
+                float v = -CUDART_INF_F;
+                int i = 0x7FFFFFFF, owner = -1;
+                for (int c = tid; c < count; c += kThreads)
+                    if (before(s_cv[c], s_ci[c], v, i)) { v = s_cv[c]; i = s_ci[c]; owner = c; }
+                block_best(v, i, owner, s_rv, s_ri, s_rt);
+                if (tid == 0) {
+                    if (i == 0x7FFFFFFF && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);   // fewer than k entries above -inf
+                    a.wk_tok[w + r] = i == 0x7FFFFFFF ? -1 : i;
+                    a.wk_q[w + r] = v == -CUDART_INF_F ? 0.f : ex2((v - rm) * kLog2e) / rs;
+                    if (owner >= 0) s_cv[owner] = -CUDART_INF_F;      // taken (an entry at -inf is never a candidate)
+                    if (owner >= 0) s_ci[owner] = 0x7FFFFFFF;
+                }
+                __syncthreads();
+            }
+        } else {
+            // exact fallback: per-thread lists of the K best pairs, merged by the block
+            TopK t;
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const float v2 = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
-                const int i2 = __shfl_xor_sync(0xFFFFFFFFu, bi, o), t2 = __shfl_xor_sync(0xFFFFFFFFu, bt, o);
-                if (before(v2, i2, bv, bi)) { bv = v2; bi = i2; bt = t2; }
+            for (int j = 0; j < K; ++j) {
+                t.v[j] = -CUDART_INF_F;
+                t.i[j] = 0x7FFFFFFF;
             }
-            if (lane == 0) { s_rv[warp] = bv; s_ri[warp] = bi; s_rt[warp] = bt; }
-            __syncthreads();
-            bv = s_rv[0]; bi = s_ri[0]; bt = s_rt[0];
-            for (int q = 1; q < kWarps; ++q)
-                if (before(s_rv[q], s_ri[q], bv, bi)) { bv = s_rv[q]; bi = s_ri[q]; bt = s_rt[q]; }
-            if (tid == bt) ++head;
-            if (tid == 0) {
-                if (bi == 0x7FFFFFFF && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);   // fewer than k entries above -inf
-                a.wk_tok[w + r] = bi == 0x7FFFFFFF ? -1 : bi;
-                a.wk_q[w + r] = bv == -CUDART_INF_F ? 0.f : ex2((bv - rm) * kLog2e) / rs;
+            for (int i = tid; i < V; i += kThreads) offer(t, x[i], i);
+            int head = 0;
+            for (int r = 0; r < a.k; ++r) {
+                float v = -CUDART_INF_F;
+                int i = 0x7FFFFFFF;
+#pragma unroll
+                for (int j = 0; j < K; ++j)
+                    if (j == head) { v = t.v[j]; i = t.i[j]; }
+                int owner = tid;
+                block_best(v, i, owner, s_rv, s_ri, s_rt);
+                if (owner == tid) ++head;
+                if (tid == 0) {
+                    if (i == 0x7FFFFFFF && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
+                    a.wk_tok[w + r] = i == 0x7FFFFFFF ? -1 : i;
+                    a.wk_q[w + r] = v == -CUDART_INF_F ? 0.f : ex2((v - rm) * kLog2e) / rs;
+                }
             }
-            __syncthreads();
         }
     }
     if (tid == 0) {

@@ -112,6 +112,23 @@ def test_scalar_loads_filtered_entries_and_k8():
     grow_levels(B=2, V=1003, k=8, tau=2, levels=3, Ncap=512, seed=3, drop=0.6)
 
 
+def test_long_runs_of_equal_logits():
+    # thousands of entries tie with the k-th best: the order is decided by the token id alone
+    # (on the GPU this is the path that keeps per-thread lists instead of a candidate buffer)
+    rng = np.random.default_rng(8)
+    B, F, V, k = 2, 3, 5000, 6
+    lg = rng.integers(0, 2, size=(B, F, V)).astype(np.float32)       # values 0 and 1 only
+    lg[0, 0, :] = 0.0                                                 # one row entirely flat
+    fr = np.zeros((B, F), np.int32); fl = np.full((B,), F, np.int32)
+    state = fresh(B, 64)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got, nf_g, nfl_g = gpu_step(state, lg, fr, fl, k, 9, 0.0, 0.0, status=status)
+    out = oracle.draft_expand(lg, fr, fl, *state, k=k, tau=9, theta_prob=0.0, theta_sib=0.0)
+    compare(got, list(out[:6]), nf_g, nfl_g, out[6], out[7])
+    assert int(status.item()) == 0
+    assert list(got[0][0, 1:1 + k]) == list(range(k))
+
+
 def test_capacity_is_reported_and_respected():
     state, _ = grow_levels(B=2, V=64, k=4, tau=4, levels=8, Ncap=50, seed=5)
     assert (state[5] == 50).any()
