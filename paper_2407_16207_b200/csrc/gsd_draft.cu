@@ -78,6 +78,7 @@ __device__ void grow_sequence(const DraftArgs& a, int b) {
     __shared__ int s_tok[GSD_MAX_NODES];
     __shared__ int s_par[GSD_MAX_NODES];
     __shared__ unsigned char s_leaf[GSD_MAX_NODES];
+    __shared__ __align__(16) unsigned s_key[GSD_MAX_NODES];   // hash of the tau-gram that ends at a node (kNoGram: none)
     __shared__ int s_cnt[kWarps];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int Ncap = a.Ncap, k = a.k;
@@ -125,18 +126,43 @@ __device__ void grow_sequence(const DraftArgs& a, int b) {
     }
     __syncthreads();
     // Sec. 5.2 / 5.3: a new node whose last tau tokens along its tree path equal those of an
-    // earlier node is redundant; it becomes a leaf that points at the first such node
+    // earlier node is redundant; it becomes a leaf that points at the first such node.
+    // A 32-bit hash of every node's tau-gram makes the scan over the earlier nodes one
+    // comparison per node; equal hashes are confirmed token by token.
+    constexpr unsigned kNoGram = 0xFFFFFFFFu;
+    for (int v = tid; v < n1; v += kThreads) {
+        unsigned h = 2166136261u;
+        int x = v, t = 0;
+        for (; t < a.tau && x >= 0; ++t) {
+            h = (h ^ (unsigned)s_tok[x]) * 16777619u;
+            h ^= h >> 15;
+            x = s_par[x];
+        }
+        s_key[v] = (t == a.tau) ? (h == kNoGram ? 0u : h) : kNoGram;
+    }
+    __syncthreads();
+    auto same_gram = [&](int x, int y) -> bool {
+        for (int t = 0; t < a.tau; ++t) {
+            if (x < 0 || y < 0 || s_tok[x] != s_tok[y]) return false;
+            x = s_par[x];
+            y = s_par[y];
+        }
+        return true;
+    };
     for (int j = tid; j < want; j += kThreads) {
         const int c = n0 + j;
+        const unsigned kc = s_key[c];
         int first = -1;
-        for (int e = 0; e < c && first < 0; ++e) {
-            int x = c, y = e, t = 0;
-            for (; t < a.tau; ++t) {
-                if (x < 0 || y < 0 || s_tok[x] != s_tok[y]) break;
-                x = s_par[x];
-                y = s_par[y];
+        if (kc != kNoGram) {
+            const uint4* k4 = reinterpret_cast<const uint4*>(s_key);
+            for (int e4 = 0; e4 * 4 < c && first < 0; ++e4) {
+                const uint4 q = k4[e4];
+                const int e = e4 * 4;
+                if (q.x == kc && e < c && same_gram(c, e)) first = e;
+                else if (q.y == kc && e + 1 < c && same_gram(c, e + 1)) first = e + 1;
+                else if (q.z == kc && e + 2 < c && same_gram(c, e + 2)) first = e + 2;
+                else if (q.w == kc && e + 3 < c && same_gram(c, e + 3)) first = e + 3;
             }
-            if (t == a.tau) first = e;
         }
         if (first >= 0) s_leaf[c] = 1;
         tok[c] = s_tok[c];
