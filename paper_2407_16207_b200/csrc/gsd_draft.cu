@@ -229,7 +229,6 @@ __global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
     __shared__ int s_ri[kWarps], s_rt[kWarps];
     __shared__ float s_m[kWarps], s_s[kWarps];
     __shared__ int s_last, s_count;
-    __shared__ float s_bound;
     const int fi = blockIdx.x, b = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int V = a.V;
@@ -298,18 +297,18 @@ __global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
             rm = mm;
         }
         if (tid == 0 && (!(rs > 0.f) || rm == CUDART_INF_F) && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
-        // the k-th largest of the 256 thread maxima: every thread ranks its own maximum among
-        // all of them (ties by thread id); the one with rank k-1 holds the bound
-        s_cv[tid] = my_best;
-        if (tid == 0) s_bound = -CUDART_INF_F;
-        __syncthreads();
+        // the k-th largest of the 256 thread maxima
+        float bound = -CUDART_INF_F;
         {
-            int rank = 0;
-            for (int j = 0; j < kThreads; ++j) rank += before(s_cv[j], j, my_best, tid) ? 1 : 0;
-            if (rank == a.k - 1) s_bound = my_best;
+            bool taken = false;
+            for (int r = 0; r < a.k; ++r) {
+                float v = taken ? -CUDART_INF_F : my_best;
+                int i = tid, owner = tid;
+                block_best(v, i, owner, s_rv, s_ri, s_rt);
+                if (owner == tid) taken = true;
+                bound = v;
+            }
         }
-        __syncthreads();
-        const float bound = s_bound;
         // pass 2: everything >= bound (and above -inf) is a candidate
         auto consider = [&](float val, int idx) {
             if (val >= bound && val > -CUDART_INF_F) {
@@ -332,21 +331,21 @@ __global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
         const int count = s_count;
         const size_t w = ((size_t)b * a.F + fi) * K;
         if (count <= kCand) {
-            // every candidate ranks itself among the candidates; ranks 0..k-1 are the children
-            for (int c = tid; c < count; c += kThreads) {
-                const float v = s_cv[c];
-                const int i = s_ci[c];
-                int rank = 0;
-                for (int j = 0; j < count; ++j) rank += before(s_cv[j], s_ci[j], v, i) ? 1 : 0;
-                if (rank < a.k) {
-                    a.wk_tok[w + rank] = i;
-                    a.wk_q[w + rank] = ex2((v - rm) * kLog2e) / rs;
+            // k rounds over the candidate list: each thread proposes the best of its strided share
+            for (int r = 0; r < a.k; ++r) {
+                float v = -CUDART_INF_F;
+                int i = 0x7FFFFFFF, owner = -1;
+                for (int c = tid; c < count; c += kThreads)
+                    if (before(s_cv[c], s_ci[c], v, i)) { v = s_cv[c]; i = s_ci[c]; owner = c; }
+                block_best(v, i, owner, s_rv, s_ri, s_rt);
+                if (tid == 0) {
+                    if (i == 0x7FFFFFFF && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);   // fewer than k entries above -inf
+                    a.wk_tok[w + r] = i == 0x7FFFFFFF ? -1 : i;
+                    a.wk_q[w + r] = v == -CUDART_INF_F ? 0.f : ex2((v - rm) * kLog2e) / rs;
+                    if (owner >= 0) s_cv[owner] = -CUDART_INF_F;      // taken (an entry at -inf is never a candidate)
+                    if (owner >= 0) s_ci[owner] = 0x7FFFFFFF;
                 }
-            }
-            if (count < a.k && tid == 0) {
-                // fewer than k entries above -inf
-                if (a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
-                for (int r = count; r < a.k; ++r) { a.wk_tok[w + r] = -1; a.wk_q[w + r] = 0.f; }
+                __syncthreads();
             }
         } else {
             // exact fallback: per-thread lists of the K best pairs, merged by the block
