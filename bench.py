@@ -327,6 +327,38 @@ def main():
         torch.cuda.synchronize()
         sampled_us = statistics.median(a.elapsed_time(b) for a, b in ev_s) * 1e3
 
+    # ---- one growth step of the draft token graph (gsd_draft_expand): 64 frontier rows per
+    # sequence of random draft logits over the same vocabulary, on a graph of 104 earlier nodes;
+    # timed on its own, not part of `value`
+    draft_us = None
+    if rank == 0:
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(11)
+        Fr, Ncap, n_old = 64, 512, 104
+        dl = [torch.randn((cfg.B, Fr, cfg.V), device=dev, generator=gen) * 3 for _ in range(2)]
+        g_tok = torch.randint(0, cfg.V, (cfg.B, Ncap), device=dev, generator=gen, dtype=torch.int32)
+        g_par = (torch.arange(Ncap, device=dev, dtype=torch.int32) - 1).clamp(min=0).repeat(cfg.B, 1).contiguous()
+        g_par[:, 0] = -1
+        g_mrg = torch.full((cfg.B, Ncap), -1, dtype=torch.int32, device=dev)
+        g_leaf = torch.zeros((cfg.B, Ncap), dtype=torch.uint8, device=dev)
+        g_prob = torch.zeros((cfg.B, Ncap), dtype=torch.float32, device=dev)
+        n_ref = torch.full((cfg.B,), n_old, dtype=torch.int32, device=dev)
+        g_n = n_ref.clone()
+        fr = (torch.arange(Fr, device=dev, dtype=torch.int32) % n_old).repeat(cfg.B, 1).contiguous()
+        fl = torch.full((cfg.B,), Fr, dtype=torch.int32, device=dev)
+        ev_d = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(20)]
+        for i in range(23):
+            g_n.copy_(n_ref)
+            if i >= 3:
+                ev_d[i - 3][0].record()
+            gsd.gsd_draft_expand(dl[i % 2], fr, fl, g_tok, g_par, g_mrg, g_leaf, g_prob, g_n, k=4, tau=2,
+                                 theta_prob=0.01, theta_sib=0.1, status=status)
+            if i >= 3:
+                ev_d[i - 3][1].record()
+        torch.cuda.synchronize()
+        draft_us = statistics.median(a.elapsed_time(b) for a, b in ev_d) * 1e3
+        del dl
+
     # ---- end to end through the host-buffer C-ABI call (pinned host tensors)
     e2e = None
     if args.e2e_steps > 0:
@@ -413,7 +445,7 @@ def main():
                    "D": cfg.D, "L": cfg.L, "V": cfg.V, "depth": cfg.depth,
                    "l2": "two input sets rotated; each step reads more than the L2 size",
                    "replicas": world, "attn_kernel": args.kernel, "num_splits": splits},
-        "attn_us": attn_mean * 1e6, "accept_us": acc_mean * 1e6, "commit_kv_us": commit_us, "accept_sampled_us": sampled_us,
+        "attn_us": attn_mean * 1e6, "accept_us": acc_mean * 1e6, "commit_kv_us": commit_us, "accept_sampled_us": sampled_us, "draft_expand_us": draft_us,
         "attn_tokens_per_s": tokens / attn_mean,
         "accept_gbs": accept_bytes / acc_mean / 1e9,
         "accept_frac_of_hbm": accept_bytes / acc_mean / 1e9 / peaks["hbm_gbs"],
