@@ -40,6 +40,11 @@
  * Every function here is pinned by tests that do not re-use it: closed forms (uniform
  * softmax, two-key sigmoid), library attention on chain / tree / full-mask special
  * cases, numpy argmax, hand-built DAGs with hand-derived answers, and invariants.
+ * Three choices are readings of a silent paper, not facts the pins can settle; for these the
+ * parity is unpinned: a node merged from several branches attends to the union of its
+ * ancestors (the paper un-merges the graph before verification, Sec. 5.4); the target
+ * model's own next token is counted in accepted_len; the regenerated token of the
+ * non-deterministic rule is drawn from the target distribution itself, not from a residual.
  */
 #include <math.h>
 #include <stdint.h>
