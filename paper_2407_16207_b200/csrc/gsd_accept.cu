@@ -112,6 +112,13 @@ __device__ void path_pass(const AcceptArgs& a, int b) {
     if (tid == 0 && res.edges < a.Tcap) io.out_tok[res.edges] = s_amax[res.end];
 }
 
+// Zeroes scratch words.  The kernel that uses them is launched as a programmatic dependent: it
+// may start streaming its input at once and only waits for these zeros before its first atomic.
+__global__ void clear_words_kernel(unsigned* words, int n) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) words[i] = 0u;
+}
+
 template <bool kVec>
 __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a) {
     __shared__ Best sh[kThreads / 32];
@@ -165,6 +172,8 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a) {
         best.v = -CUDART_INF_F;
     }
     if (threadIdx.x == 0) {
+        // the scratch is zeroed by the launch before this one; everything above ran beside it
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         if (best.i != kNone) atomicMax(a.keys + row, pack_key(best.v, best.i));
         __threadfence();
         const int b = row / a.N;
@@ -179,6 +188,14 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a) {
 }
 
 }  // namespace
+
+int launch_clear_words(unsigned* words, int n, cudaStream_t stream) {
+    const int blocks = (n + 1023) / 1024;
+    clear_words_kernel<<<blocks < 64 ? blocks : 64, 256, 0, stream>>>(words, n);
+    GSD_CUDA_TRY(cudaGetLastError());
+    return GSD_OK;
+}
+
 }  // namespace gsd
 
 extern "C" size_t gsd_accept_workspace_bytes(const gsd_accept_params* p) {
@@ -221,7 +238,9 @@ extern "C" int gsd_accept(const float* logits, const int32_t* draft_tokens,
     while (rows * splits < want && (p->V / (splits * 2)) >= 4096) splits *= 2;
     a.splits = splits;
 
-    GSD_CUDA_TRY(cudaMemsetAsync(workspace, 0, (size_t)p->B * p->N * 8 + (size_t)p->B * 4, st));
+    if (launch_clear_words((unsigned*)workspace, p->B * p->N * 2 + p->B, st) != GSD_OK) return GSD_ERR_CUDA;
+    cudaLaunchAttribute attr[1];
+    dependent_launch_attr(attr);
     // grid.y holds at most 65535 rows: larger problems go out in blocks of whole sequences
     // so that the per-sequence completion counter still works
     const int seq_per = 65535 / p->N;
@@ -233,9 +252,14 @@ extern "C" int gsd_accept(const float* logits, const int32_t* draft_tokens,
         s.out_tok += (size_t)b0 * p->Tcap; s.out_len += b0;
         if (s.out_nodes) s.out_nodes += (size_t)b0 * p->Tcap;
         s.keys += (size_t)b0 * p->N; s.done += b0; s.B = nb;
-        dim3 grid(splits, (unsigned)(nb * p->N));
-        if (vec) accept_kernel<true><<<grid, kThreads, 0, st>>>(s);
-        else accept_kernel<false><<<grid, kThreads, 0, st>>>(s);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(splits, (unsigned)(nb * p->N));
+        cfg.blockDim = dim3(kThreads);
+        cfg.stream = st;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (vec) GSD_CUDA_TRY(cudaLaunchKernelEx(&cfg, accept_kernel<true>, s));
+        else GSD_CUDA_TRY(cudaLaunchKernelEx(&cfg, accept_kernel<false>, s));
     }
     GSD_CUDA_TRY(cudaGetLastError());
     return GSD_OK;

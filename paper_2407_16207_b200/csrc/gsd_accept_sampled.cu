@@ -253,6 +253,8 @@ __global__ void __launch_bounds__(kThreads) accept_sampled_kernel(SampledArgs a)
     __syncthreads();
     if (threadIdx.x == 0) {
         const int b = row / a.N;
+        // the counters are zeroed by the launch before this one; everything above ran beside it
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         const unsigned prev = atomicAdd(a.done + b, 1u);
         s_last = (prev == (unsigned)(a.N * a.slices) - 1u);
     }
@@ -315,7 +317,9 @@ extern "C" int gsd_accept_sampled(const float* logits, const int32_t* draft_toke
     a.vec = vec ? 1 : 0;
 
     // only the completion counters have to start at zero; every pair is written before it is read
-    GSD_CUDA_TRY(cudaMemsetAsync(a.done, 0, (size_t)p->B * 4, st));
+    if (launch_clear_words(a.done, p->B, st) != GSD_OK) return GSD_ERR_CUDA;
+    cudaLaunchAttribute attr[1];
+    dependent_launch_attr(attr);
     // grid.y holds at most 65535 rows: larger problems go out in blocks of whole sequences
     const int seq_per = 65535 / p->N;
     for (int b0 = 0; b0 < p->B; b0 += seq_per) {
@@ -327,9 +331,14 @@ extern "C" int gsd_accept_sampled(const float* logits, const int32_t* draft_toke
         s.out_tok += (size_t)b0 * p->Tcap; s.out_len += b0;
         if (s.out_nodes) s.out_nodes += (size_t)b0 * p->Tcap;
         s.part += (size_t)b0 * p->N * a.slices * kWarps; s.done += b0; s.B = nb;
-        dim3 grid(a.slices, (unsigned)(nb * p->N));
-        if (vec) accept_sampled_kernel<true><<<grid, kThreads, 0, st>>>(s);
-        else accept_sampled_kernel<false><<<grid, kThreads, 0, st>>>(s);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(a.slices, (unsigned)(nb * p->N));
+        cfg.blockDim = dim3(kThreads);
+        cfg.stream = st;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (vec) GSD_CUDA_TRY(cudaLaunchKernelEx(&cfg, accept_sampled_kernel<true>, s));
+        else GSD_CUDA_TRY(cudaLaunchKernelEx(&cfg, accept_sampled_kernel<false>, s));
     }
     GSD_CUDA_TRY(cudaGetLastError());
     return GSD_OK;

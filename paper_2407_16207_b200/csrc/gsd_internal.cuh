@@ -87,4 +87,14 @@ int launch_attn_tcgen05(const AttnArgs& a);
 bool attn_tcgen05_supports(int D, int G);
 int launch_attn_merge(const AttnArgs& a);
 
+// ---- scratch words that must start at zero ----
+// Enqueues a small kernel that zeroes `n` 32-bit words and lets the next launch on the stream
+// start beside it.  That next kernel has to be launched with the attribute set up by
+// dependent_launch_attr() and to execute griddepcontrol.wait before it first touches the words.
+int launch_clear_words(unsigned* words, int n, cudaStream_t stream);
+inline void dependent_launch_attr(cudaLaunchAttribute* attr) {
+    attr->id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr->val.programmaticStreamSerializationAllowed = 1;
+}
+
 }  // namespace gsd
