@@ -450,7 +450,9 @@ def main():
         "accept_gbs": accept_bytes / acc_mean / 1e9,
         "accept_frac_of_hbm": accept_bytes / acc_mean / 1e9 / peaks["hbm_gbs"],
         "roofline": roof, "cpu_baseline": cpu, "e2e": e2e,
-        "gpu_launches": args.steps * ((2 if splits > 1 else 1) + 1),
+        # per step: the attention kernel (+ its merge pass when key ranges are cut), the scratch
+        # clear of gsd_accept and the accept kernel
+        "gpu_launches": args.steps * ((2 if splits > 1 else 1) + 2),
         "clocks": clocks,
     }
     print(json.dumps(line), flush=True)
