@@ -282,7 +282,7 @@ int gsd_draft_expand(const float* logits, const int32_t* frontier, const int32_t
  * The first call on each device looks up the array's device address (the device must be
  * current, as for every call here); make that first call outside any stream capture.
  * All calls on a device share the one array: it keeps whatever the last call left in it, the
- * part a call uses is cleared on `stream` before its kernel runs, and two calls that can
+ * part a call uses is cleared on `stream` before its kernel touches it, and two calls that can
  * overlap on the GPU (different streams, no dependency) race on it - serialise them.
  */
 #define GSD_STATIC_MAX_ROWS 16384
