@@ -143,8 +143,11 @@ def accept(logits, draft_tokens, parent_ptr, parent_idx, Tcap: int = 0, visit_ca
     return toks, lens, nodes, visited
 
 
-def accept_sampled(logits, draft_tokens, parent_ptr, parent_idx, draft_q, u_accept, u_sample, Tcap: int = 0):
+def accept_sampled(logits, draft_tokens, parent_ptr, parent_idx, draft_q, u_accept, u_sample, Tcap: int = 0,
+                   draft_logits=None):
     """Non-deterministic verification with the random numbers passed in (see gsd_oracle_accept_sampled).
+    With `draft_logits` [B,N,V] the regenerated token after a rejection comes from the residual
+    max(0, P - Q) of the end node; without it, from the target distribution P.
 
     Returns (accepted_tokens [B,Tcap] padded with -1, accepted_len [B], accepted_nodes [B,Tcap])."""
     logits = _c(logits, np.float32); draft_tokens = _c(draft_tokens, np.int32)
@@ -153,12 +156,16 @@ def accept_sampled(logits, draft_tokens, parent_ptr, parent_idx, draft_q, u_acce
     B, N, V = logits.shape
     assert draft_tokens.shape == (B, N) and parent_ptr.shape == (B, N + 1)
     assert draft_q.shape == (B, N) and u_accept.shape == (B, N) and u_sample.shape == (B,)
+    if draft_logits is not None:
+        draft_logits = _c(draft_logits, np.float32)
+        assert draft_logits.shape == (B, N, V)
     Ecap = parent_idx.shape[1]
     Tcap = Tcap or N
     toks = np.zeros((B, Tcap), dtype=np.int32)
     lens = np.zeros((B,), dtype=np.int32)
     nodes = np.zeros((B, Tcap), dtype=np.int32)
     rc = _load().gsd_oracle_accept_sampled(_p(logits), _p(draft_tokens), _p(parent_ptr), _p(parent_idx),
+                                           _p(draft_logits) if draft_logits is not None else None,
                                            _p(draft_q), _p(u_accept), _p(u_sample),
                                            ctypes.c_int32(B), ctypes.c_int32(N), ctypes.c_int32(V),
                                            ctypes.c_int32(Ecap), ctypes.c_int32(Tcap), _p(toks), _p(lens), _p(nodes))

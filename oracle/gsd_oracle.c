@@ -28,7 +28,8 @@
  *  - Non-deterministic acceptance (Sec. 3: accept with probability min(1, p/q); Sec. 6.4: on
  *    the token graph), with the random numbers as inputs: the same walk with the step
  *    p -> v accepted iff u_accept[v] * q_v < softmax(logits[p])[tok v], and the regenerated
- *    token drawn from softmax(logits[end]) by inverting the cumulative distribution.
+ *    token drawn by inverting the cumulative distribution of the residual max(0, P - Q) at the
+ *    end node when a drafted continuation was rejected there, of P itself otherwise.
  *  - The KV-cache commit of the accepted path and the ancestor-mask closure (see there).
  *  - One growth step of the draft token graph: top-k children, probability and sibling
  *    pruning (Sec. 4.2), tau-redundant nodes and their merge edges (Sec. 5.2, 5.3).
@@ -43,8 +44,9 @@
  * Three choices are readings of a silent paper, not facts the pins can settle; for these the
  * parity is unpinned: a node merged from several branches attends to the union of its
  * ancestors (the paper un-merges the graph before verification, Sec. 5.4); the target
- * model's own next token is counted in accepted_len; the regenerated token of the
- * non-deterministic rule is drawn from the target distribution itself, not from a residual.
+ * model's own next token is counted in accepted_len; in the non-deterministic rule every step
+ * of the graph is tested against the target distribution of its parent, and several rejected
+ * siblings share the single residual max(0, P - Q) of their parent.
  */
 #include <math.h>
 #include <stdint.h>
@@ -342,18 +344,27 @@ int gsd_oracle_accept(const float *logits, const int32_t *draft_tokens, const in
 /*
  * Non-deterministic verification (Sec. 3: the i-th drafted token is accepted with probability
  * min(1, p/q), the first rejection discards the rest of the hypothesis and the target model
- * regenerates that token; Sec. 6.4 runs it on the token graph).  Readings taken here: the
- * random numbers are inputs; the test is applied per step p -> v of the graph with
+ * regenerates that token, so that the accepted tokens follow the target model's distribution;
+ * Sec. 6.4 runs it on the token graph).  Readings taken here: the random numbers are inputs;
+ * the test is applied per step p -> v of the graph with
  * p = softmax(logits[parent])[token of v] and q = draft_q[v]:
  *     accepted(p -> v)  iff  u_accept[v] * q_v < p          (u < min(1, p/q) for q > 0)
  * the accepted hypothesis is the longest root path whose steps are all accepted (ties as in
- * gsd_oracle_accept); the regenerated token is drawn from softmax(logits[end node]) by
- * inverting its cumulative distribution in index order: the smallest t with
- * sum_{j<=t} P_j > u_sample[b] (the last t with P_t > 0 if rounding leaves none).
- * All arithmetic in double.  logits must be finite or -inf with at least one finite entry per row.
+ * gsd_oracle_accept).  The regenerated token follows the sampling scheme that Sec. 3 cites:
+ * with P = softmax(logits[end node]) and Q = softmax(draft_logits[end node]) (the distribution
+ * the end node's children were drafted from),
+ *   - if the end node has at least one child in the graph (its drafted continuations were all
+ *     rejected) it is drawn from the residual  r_j = max(0, P_j - Q_j) / sum_i max(0, P_i - Q_i);
+ *   - if the end node has no child (nothing was rejected there), or draft_logits is NULL, or the
+ *     residual has no mass, it is drawn from P itself.
+ * Several rejected siblings share the one residual P - Q (the paper gives no rule for them).
+ * The draw inverts the cumulative distribution in index order: the smallest t with
+ * sum_{j<=t} w_j > u_sample[b] * sum_j w_j  (the last t with w_t > 0 if rounding leaves none),
+ * w = P or max(0, P - Q).  All arithmetic in double.  logits (and draft_logits) must be finite
+ * or -inf with at least one finite entry per row.
  *
- * logits [B,N,V]; draft_q, u_accept [B,N]; u_sample [B]; the rest as gsd_oracle_accept.
- * Returns 0, or -1 on malformed input or allocation failure.
+ * logits [B,N,V]; draft_logits [B,N,V] or NULL; draft_q, u_accept [B,N]; u_sample [B]; the rest
+ * as gsd_oracle_accept.  Returns 0, or -1 on malformed input or allocation failure.
  */
 static void softmax_stats(const float *x, int V, double *m_out, double *s_out)
 {
@@ -365,7 +376,8 @@ static void softmax_stats(const float *x, int V, double *m_out, double *s_out)
 
 int gsd_oracle_accept_sampled(const float *logits, const int32_t *draft_tokens,
                               const int32_t *parent_ptr, const int32_t *parent_idx,
-                              const float *draft_q, const float *u_accept, const float *u_sample,
+                              const float *draft_logits, const float *draft_q,
+                              const float *u_accept, const float *u_sample,
                               int32_t B, int32_t N, int32_t V, int32_t Ecap, int32_t Tcap,
                               int32_t *accepted_tokens, int32_t *accepted_len, int32_t *accepted_nodes)
 {
@@ -383,7 +395,9 @@ int gsd_oracle_accept_sampled(const float *logits, const int32_t *draft_tokens,
         int *fill = (int *)calloc((size_t)N + 1, sizeof(int));
         int *stack = (int *)malloc(sizeof(int) * (size_t)(N + 1));
         int *best = (int *)malloc(sizeof(int) * (size_t)(N + 1));
-        if (!mx || !sm || !ok || !cptr || !cidx || !fill || !stack || !best) rc = -1;
+        double *wgt = (double *)malloc(sizeof(double) * (size_t)V);
+        double *res = (double *)malloc(sizeof(double) * (size_t)V);
+        if (!mx || !sm || !ok || !cptr || !cidx || !fill || !stack || !best || !wgt || !res) rc = -1;
         if (rc == 0) {
 #pragma omp parallel for schedule(static)
             for (int v = 0; v < N; ++v) softmax_stats(lg + (size_t)v * V, V, &mx[v], &sm[v]);
@@ -409,16 +423,31 @@ int gsd_oracle_accept_sampled(const float *logits, const int32_t *draft_tokens,
             const int m = w.best_edges;
             if (m + 1 > Tcap) rc = -1;
             if (rc == 0) {
-                /* the regenerated token: inverse of the cumulative distribution at the end node */
+                /* the regenerated token: weights w over the vocabulary at the end node, then the
+                 * inverse of their cumulative distribution */
                 const int end = best[m];
                 const float *x = lg + (size_t)end * V;
-                const double target = (double)u_sample[b];
+                const int rejected_children = cptr[end + 1] - cptr[end];
+                double total = 0.0;
+                for (int j = 0; j < V; ++j) wgt[j] = exp((double)x[j] - mx[end]) / sm[end];
+                if (draft_logits && rejected_children > 0) {
+                    const float *y = draft_logits + ((size_t)b * N + end) * V;
+                    double mq, sq, mass = 0.0;
+                    softmax_stats(y, V, &mq, &sq);
+                    for (int j = 0; j < V; ++j) {
+                        const double r = wgt[j] - exp((double)y[j] - mq) / sq;
+                        res[j] = r > 0.0 ? r : 0.0;
+                        mass += res[j];
+                    }
+                    if (mass > 0.0) memcpy(wgt, res, sizeof(double) * (size_t)V);
+                }
+                for (int j = 0; j < V; ++j) total += wgt[j];
+                const double target = (double)u_sample[b] * total;
                 double cum = 0.0;
                 int pick = -1, last_pos = -1;
                 for (int j = 0; j < V; ++j) {
-                    const double pj = exp((double)x[j] - mx[end]) / sm[end];
-                    if (pj > 0.0) last_pos = j;
-                    cum += pj;
+                    if (wgt[j] > 0.0) last_pos = j;
+                    cum += wgt[j];
                     if (cum > target) { pick = j; break; }
                 }
                 if (pick < 0) pick = last_pos;
@@ -434,6 +463,7 @@ int gsd_oracle_accept_sampled(const float *logits, const int32_t *draft_tokens,
             }
         }
         free(mx); free(sm); free(ok); free(cptr); free(cidx); free(fill); free(stack); free(best);
+        free(wgt); free(res);
         if (rc != 0) return rc;
     }
     return 0;

@@ -142,3 +142,115 @@ def test_acceptance_frequency_matches_min_one_p_over_q():
         for u in rng.uniform(0, 1, size=n):
             acc += len(run(LOG(P), [0, 0], ptr, idx, q=[1, q], u=[0, u], us=.3)[1]) == 2
         assert abs(acc / n - want) < 0.03
+
+
+# ---- the regenerated token: residual of the sampling scheme that Sec. 3 cites ----
+
+def run_res(logits, dlogits, tok, ptr, idx, q, u, us):
+    t, l, nd = oracle.accept_sampled(np.asarray(logits, np.float32)[None], np.asarray(tok, np.int32)[None], ptr, idx,
+                                     np.asarray(q, np.float32)[None], np.asarray(u, np.float32)[None],
+                                     np.asarray([us], np.float32),
+                                     draft_logits=None if dlogits is None else np.asarray(dlogits, np.float32)[None])
+    n = int(l[0])
+    return list(t[0, :n]), list(nd[0, :n])
+
+
+def test_worked_residual():
+    # root: P = [.4,.3,.2,.1], Q = [.1,.2,.3,.4]: max(0, P - Q) = [.3,.1,0,0], mass .4
+    P = np.array([[.4, .3, .2, .1], [.25, .25, .25, .25]])
+    Q = np.array([[.1, .2, .3, .4], [.25, .25, .25, .25]])
+    ptr, idx = chain(2)
+    # the child carries token 3 (p = .1, q = .4): u q = .9 * .4 = .36 is not below .1 -> rejected
+    for us, want in ((.7, 0), (.74, 0), (.76, 1), (.99, 1), (0.0, 0)):
+        toks, nodes = run_res(LOG(P), LOG(Q), [0, 3], ptr, idx, q=[1, .4], u=[0, .9], us=us)
+        assert nodes == [0] and toks == [want], (us, toks)
+    # without the draft distribution the token comes from P itself: cumulative .4, .7, .9, 1
+    for us, want in ((.39, 0), (.41, 1), (.71, 2), (.95, 3)):
+        assert run_res(LOG(P), None, [0, 3], ptr, idx, q=[1, .4], u=[0, .9], us=us)[0] == [want]
+    # and the residual never yields a token to which the draft gives at least the target's mass
+    for us in np.linspace(0, 0.999, 23):
+        assert run_res(LOG(P), LOG(Q), [0, 3], ptr, idx, q=[1, .4], u=[0, .9], us=us)[0][0] in (0, 1)
+
+
+def test_residual_is_formed_at_the_end_node():
+    # chain 0 -> 1 -> 2: the first step is accepted, the second rejected; the residual is that of
+    # node 1 (P1 - Q1 = [0, 0, .2, .2] -> tokens 2, 3), not of the root (tokens 0, 1)
+    P = np.array([[.4, .3, .2, .1], [.1, .1, .4, .4], [.25] * 4])
+    Q = np.array([[.1, .2, .3, .4], [.3, .3, .2, .2], [.25] * 4])
+    ptr, idx = chain(3)
+    for us, want in ((.3, 2), (.49, 2), (.51, 3), (.9, 3)):
+        toks, nodes = run_res(LOG(P), LOG(Q), [0, 0, 1], ptr, idx, q=[1, .1, .3], u=[0, .5, .9], us=us)
+        assert nodes == [0, 1] and toks == [0, want]
+
+
+def test_no_rejection_at_the_end_node_draws_from_the_target():
+    # the step 0 -> 1 is accepted and node 1 has no child: nothing was rejected there, so the
+    # next token comes from P of node 1 whatever the draft distribution says
+    P = np.array([[.4, .3, .2, .1], [.1, .2, .3, .4]])
+    Q = np.array([[.1, .2, .3, .4], [.7, .1, .1, .1]])
+    ptr, idx = chain(2)
+    for us, want in ((.05, 0), (.2, 1), (.5, 2), (.7, 3)):
+        toks, nodes = run_res(LOG(P), LOG(Q), [0, 0], ptr, idx, q=[1, .1], u=[0, .5], us=us)
+        assert nodes == [0, 1] and toks == [0, want]
+
+
+def test_residual_without_mass_falls_back_to_the_target():
+    # draft distribution == target distribution: P - Q is zero everywhere; a rejection forced
+    # through an inconsistent draft_q then regenerates from P
+    P = np.array([[.5, .25, .125, .125], [.25, .25, .25, .25]])
+    ptr, idx = chain(2)
+    for us, want in ((.4, 0), (.6, 1), (.8, 2), (.9, 3)):
+        toks, nodes = run_res(LOG(P), LOG(P), [0, 2], ptr, idx, q=[1, 1.0], u=[0, .5], us=us)
+        assert nodes == [0] and toks == [want]
+
+
+def test_rejected_siblings_share_one_residual():
+    # the root has two children (tokens 2 and 3), both rejected; the residual is max(0, P - Q) of
+    # the root, formed once: [.3, .1, 0, 0] / .4
+    P = np.array([[.4, .3, .2, .1], [.25] * 4, [.25] * 4])
+    Q = np.array([[.1, .2, .3, .4], [.25] * 4, [.25] * 4])
+    ptr = np.array([[0, 0, 1, 2]], dtype=np.int32)
+    idx = np.array([[0, 0]], dtype=np.int32)
+    for us, want in ((.7, 0), (.8, 1)):
+        toks, nodes = run_res(LOG(P), LOG(Q), [0, 2, 3], ptr, idx, q=[1, .3, .4], u=[0, .9, .9], us=us)
+        assert nodes == [0] and toks == [want]
+    # one of them accepted (u small): the hypothesis goes on and the leaf draws from its own P
+    toks, nodes = run_res(LOG(P), LOG(Q), [0, 2, 3], ptr, idx, q=[1, .3, .4], u=[0, .9, .1], us=.6)
+    assert nodes == [0, 2] and toks == [3, 2]
+
+
+def chi_square(counts, probs):
+    n = counts.sum()
+    return float((((counts - n * probs) ** 2) / (n * probs)).sum())
+
+
+def test_emitted_token_follows_the_target_distribution():
+    # Sec. 3: the scheme "ensures that the tokens ultimately accepted are representative of the
+    # output distribution of M_p".  One drafted token x ~ Q per sequence, seeded uniform numbers:
+    # the first emitted token (x if accepted, else the regenerated one) must be distributed as P.
+    # Bound: the 99.9 % point of chi-square with V - 1 = 5 degrees of freedom is 20.5.
+    V, n = 6, 60000
+    rng = np.random.default_rng(20240716)
+    P = np.array([.30, .05, .25, .10, .02, .28])
+    Q = np.array([.10, .25, .05, .30, .20, .10])
+    x = rng.choice(V, size=n, p=Q)
+    lg = np.empty((n, 2, V), dtype=np.float32)
+    dl = np.empty((n, 2, V), dtype=np.float32)
+    lg[:, 0] = LOG(P); lg[:, 1] = 0.0
+    dl[:, 0] = LOG(Q); dl[:, 1] = 0.0
+    tok = np.stack([np.zeros(n, np.int32), x.astype(np.int32)], axis=1)
+    ptr = np.tile(np.array([0, 0, 1], dtype=np.int32), (n, 1))
+    idx = np.zeros((n, 1), dtype=np.int32)
+    q = np.stack([np.ones(n), Q[x]], axis=1).astype(np.float32)
+    u = rng.uniform(0, 1, size=(n, 2)).astype(np.float32)
+    us = rng.uniform(0, 1, size=n).astype(np.float32)
+    t, l, _ = oracle.accept_sampled(lg, tok, ptr, idx, q, u, us, draft_logits=dl)
+    first = t[:, 0]
+    counts = np.bincount(first, minlength=V).astype(np.float64)
+    assert chi_square(counts, P) < 20.5
+    # the accepted fraction is sum_x min(P, Q) and the rejected ones never emit a token with Q >= P
+    assert abs((l == 2).mean() - np.minimum(P, Q).sum()) < 0.01
+    assert set(np.unique(first[l == 1])) <= {0, 2, 5}
+    # the same stream with the regenerated token drawn from P itself is visibly NOT distributed as P
+    t2, _, _ = oracle.accept_sampled(lg, tok, ptr, idx, q, u, us)
+    assert chi_square(np.bincount(t2[:, 0], minlength=V).astype(np.float64), P) > 1000

@@ -41,6 +41,16 @@ MUTATIONS = [
      "test_oracle_accept_sampled.py"),
     ("sampled_regenerates_at_parent", "const int end = best[m];", "const int end = best[m > 0 ? m - 1 : 0];",
      "test_oracle_accept_sampled.py"),
+    ("sampled_regenerates_from_target", "if (mass > 0.0) memcpy(wgt, res, sizeof(double) * (size_t)V);", "(void)mass;",
+     "test_oracle_accept_sampled.py"),
+    ("sampled_residual_sign", "const double r = wgt[j] - exp((double)y[j] - mq) / sq;",
+     "const double r = exp((double)y[j] - mq) / sq - wgt[j];", "test_oracle_accept_sampled.py"),
+    ("sampled_residual_at_a_leaf", "if (draft_logits && rejected_children > 0) {", "if (draft_logits) {",
+     "test_oracle_accept_sampled.py"),
+    ("sampled_residual_of_the_root", "const float *y = draft_logits + ((size_t)b * N + end) * V;",
+     "const float *y = draft_logits + ((size_t)b * N) * V;", "test_oracle_accept_sampled.py"),
+    ("sampled_residual_unclamped", "res[j] = r > 0.0 ? r : 0.0;", "res[j] = r > 0.0 ? r : -r;",
+     "test_oracle_accept_sampled.py"),
     ("draft_tie_highest", "if (!taken[j] && (best < 0 || P[j] > P[best])) best = j;",
      "if (!taken[j] && (best < 0 || P[j] >= P[best])) best = j;", "test_oracle_draft.py"),
     ("draft_prob_le", "lf[c] = (P[best] < theta_prob) ||", "lf[c] = (P[best] <= theta_prob) ||", "test_oracle_draft.py"),
