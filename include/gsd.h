@@ -37,7 +37,7 @@
 extern "C" {
 #endif
 
-#define GSD_VERSION 100
+#define GSD_VERSION 101
 
 typedef enum gsd_status {
     GSD_OK = 0,
@@ -183,16 +183,24 @@ size_t gsd_accept_workspace_bytes(const gsd_accept_params* p);
  *         accepted  iff  u_accept[b][v] * q < p        (u < min(1, p/q); q = 0 accepts iff p > 0)
  *   - the hypothesis is the longest root path all of whose steps are accepted; ties as in
  *     gsd_accept (lowest end node, then lowest predecessor walking back);
- *   - the regenerated token is drawn from softmax(logits[b][end node]) by inverting its
- *     cumulative distribution in index order: the smallest t with sum_{j<=t} P_j > u_sample[b]
- *     (the last t with P_t > 0 if rounding leaves none).  The residual distribution
- *     max(0, p - q) of the original sampling scheme would need the draft model's whole
- *     distribution per node and is not formed.
+ *   - the regenerated token follows the sampling scheme that Sec. 3 cites, which is what makes
+ *     the accepted tokens follow the target model's distribution: with P = softmax(logits[b][end
+ *     node]) and Q = softmax(draft_logits[b][end node]) it is drawn from the residual
+ *     max(0, P_j - Q_j) / sum_i max(0, P_i - Q_i) when the end node has a child in the graph (its
+ *     drafted continuations were all rejected; several rejected siblings share the one
+ *     residual), and from P itself when the end node has no child, when the residual has no
+ *     mass (sum <= 1e-6) or when draft_logits is NULL.  The draw inverts the cumulative weights
+ *     in index order: the smallest t with sum_{j<=t} w_j > u_sample[b] * sum_j w_j (the last t
+ *     with w_t > 0 if rounding leaves none).
  * Temperature / nucleus filtering are the caller's: pass logits already divided by the
  * temperature (and with filtered entries at -inf).
  *
  *   logits, draft_tokens, parent_ptr, parent_idx   device, as for gsd_accept; every logits row
  *                    must hold at least one finite value, no +inf and no NaN (GSD_DEV_BAD_LOGITS)
+ *   draft_logits     device const f32 [B,N,V] or NULL: the draft model's logits at every node (the
+ *                    distribution the node's children were drafted from); only the row of the end
+ *                    node of each sequence is read.  NULL: the regenerated token is always drawn
+ *                    from P (no residual)
  *   draft_q          device const f32 [B,N]: the probability the draft model gave node v's token
  *                    when it drafted it (entry 0, the root, is not read)
  *   u_accept         device const f32 [B,N]: one number in [0,1) per node (entry 0 not read)
@@ -207,8 +215,9 @@ size_t gsd_accept_workspace_bytes(const gsd_accept_params* p);
  */
 size_t gsd_accept_sampled_workspace_bytes(const gsd_accept_params* p);
 int gsd_accept_sampled(const float* logits, const int32_t* draft_tokens, const int32_t* parent_ptr,
-                       const int32_t* parent_idx, const float* draft_q, const float* u_accept,
-                       const float* u_sample, int32_t* accepted_tokens, int32_t* accepted_len,
+                       const int32_t* parent_idx, const float* draft_logits, const float* draft_q,
+                       const float* u_accept, const float* u_sample, int32_t* accepted_tokens,
+                       int32_t* accepted_len,
                        int32_t* accepted_nodes, const gsd_accept_params* p, void* workspace,
                        size_t workspace_bytes, int32_t* status, void* stream);
 

@@ -356,7 +356,9 @@ int gsd_oracle_accept(const float *logits, const int32_t *draft_tokens, const in
  *   - if the end node has at least one child in the graph (its drafted continuations were all
  *     rejected) it is drawn from the residual  r_j = max(0, P_j - Q_j) / sum_i max(0, P_i - Q_i);
  *   - if the end node has no child (nothing was rejected there), or draft_logits is NULL, or the
- *     residual has no mass, it is drawn from P itself.
+ *     residual has no mass (sum_i max(0, P_i - Q_i) <= 1e-6: the two distributions agree to
+ *     single-precision rounding, and a rejection then has probability <= 1e-6), it is drawn from
+ *     P itself.
  * Several rejected siblings share the one residual P - Q (the paper gives no rule for them).
  * The draw inverts the cumulative distribution in index order: the smallest t with
  * sum_{j<=t} w_j > u_sample[b] * sum_j w_j  (the last t with w_t > 0 if rounding leaves none),
@@ -439,7 +441,7 @@ int gsd_oracle_accept_sampled(const float *logits, const int32_t *draft_tokens,
                         res[j] = r > 0.0 ? r : 0.0;
                         mass += res[j];
                     }
-                    if (mass > 0.0) memcpy(wgt, res, sizeof(double) * (size_t)V);
+                    if (mass > 1e-6) memcpy(wgt, res, sizeof(double) * (size_t)V);
                 }
                 for (int j = 0; j < V; ++j) total += wgt[j];
                 const double target = (double)u_sample[b] * total;

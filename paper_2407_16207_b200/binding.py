@@ -84,7 +84,7 @@ def lib() -> ctypes.CDLL:
         L.gsd_accept.restype = i32
         L.gsd_accept.argtypes = [vp] * 7 + [ctypes.POINTER(AcceptParams), vp, sz, vp, vp]
         L.gsd_accept_sampled.restype = i32
-        L.gsd_accept_sampled.argtypes = [vp] * 10 + [ctypes.POINTER(AcceptParams), vp, sz, vp, vp]
+        L.gsd_accept_sampled.argtypes = [vp] * 11 + [ctypes.POINTER(AcceptParams), vp, sz, vp, vp]
         L.gsd_accept_sampled_workspace_bytes.restype = sz
         L.gsd_accept_sampled_workspace_bytes.argtypes = [ctypes.POINTER(AcceptParams)]
         L.gsd_draft_expand.restype = i32
@@ -247,11 +247,14 @@ def gsd_accept_sampled_workspace_bytes(B, N) -> int:
 
 
 def gsd_accept_sampled(logits, draft_tokens, parent_ptr, parent_idx, draft_q, u_accept, u_sample, *,
+                       draft_logits: Optional[torch.Tensor] = None,
                        Tcap: int = 0, want_nodes: bool = True, workspace: Optional[torch.Tensor] = None,
                        status: Optional[torch.Tensor] = None
                        ) -> Tuple[torch.Tensor, torch.Tensor, Optional[torch.Tensor]]:
     """Non-deterministic verification with the random numbers passed in; see gsd_accept_sampled in
-    include/gsd.h.  Returns (accepted_tokens [B,Tcap], accepted_len [B], accepted_nodes or None)."""
+    include/gsd.h.  `draft_logits` [B,N,V] (optional) makes the regenerated token come from the
+    residual max(0, P - Q).  Returns (accepted_tokens [B,Tcap], accepted_len [B], accepted_nodes
+    or None)."""
     if logits.dim() != 3:
         raise ValueError("logits must be [B,N,V]")
     B, N, V = logits.shape
@@ -265,6 +268,8 @@ def gsd_accept_sampled(logits, draft_tokens, parent_ptr, parent_idx, draft_q, u_
     _want(draft_q, torch.float32, (B, N), "draft_q", True)
     _want(u_accept, torch.float32, (B, N), "u_accept", True)
     _want(u_sample, torch.float32, (B,), "u_sample", True)
+    if draft_logits is not None:
+        _want(draft_logits, torch.float32, (B, N, V), "draft_logits", True)
     Tcap = Tcap or N
     toks = torch.empty((B, Tcap), dtype=torch.int32, device=logits.device)
     lens = torch.empty((B,), dtype=torch.int32, device=logits.device)
@@ -276,7 +281,8 @@ def gsd_accept_sampled(logits, draft_tokens, parent_ptr, parent_idx, draft_q, u_
         if workspace is None:
             workspace = torch.empty(max(need, 8), dtype=torch.uint8, device=logits.device)
         _check(L.gsd_accept_sampled(logits.data_ptr(), draft_tokens.data_ptr(), parent_ptr.data_ptr(),
-                                    parent_idx.data_ptr(), draft_q.data_ptr(), u_accept.data_ptr(),
+                                    parent_idx.data_ptr(), _ptr(draft_logits), draft_q.data_ptr(),
+                                    u_accept.data_ptr(),
                                     u_sample.data_ptr(), toks.data_ptr(), lens.data_ptr(), _ptr(nodes),
                                     ctypes.byref(p), workspace.data_ptr(),
                                     workspace.numel() * workspace.element_size(), _ptr(status),

@@ -4,15 +4,18 @@
 // The random numbers are inputs.  A step parent -> v of the graph is accepted iff
 //     u_accept[v] * draft_q[v] < softmax(logits[parent])[token of v];
 // the hypothesis is the longest root path of accepted steps (ties as in gsd_accept), and the
-// regenerated token is drawn from softmax(logits[end node]) by inverting the cumulative
-// distribution in index order with u_sample.
+// regenerated token is drawn by inverting a cumulative distribution in index order with
+// u_sample: that of the residual max(0, P - Q) at the end node (P the target's, Q the draft
+// model's distribution there) when drafted continuations of the end node were rejected, that of
+// P itself when the end node is a leaf of the graph or no draft logits are given.
 //
 // One launch.  Grid (slices, B*N): each CTA streams one slice of one logits row with 16-byte
 // loads; each of its warps owns a contiguous eighth of the slice and keeps a running
 // (maximum, sum of exponentials) pair, which it leaves in scratch.  The CTA that finishes last
 // for a sequence combines the pairs per node, tests the steps, runs the level-synchronous
 // longest-path relaxation, walks back, and finds the regenerated token: the range sums in
-// scratch give the range of the crossing, a block-wide scan over that range gives the index.
+// scratch (for the residual: range sums formed on the spot from the two rows of the end node)
+// give the range of the crossing, a block-wide scan over that range gives the index.
 #include "gsd_internal.cuh"
 #include "gsd_path.cuh"
 #include <math_constants.h>
@@ -25,6 +28,7 @@ constexpr int kNone = 0x7FFFFFFF;
 constexpr int kMaxSlices = 16;
 constexpr int kWarps = kThreads / 32;   // each warp of a CTA sums a contiguous eighth of the CTA's slice
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kResidualFloor = 1e-6f;   // a residual mass at or below this is rounding noise
 
 // (maximum, sum of 2^((x - maximum) * log2 e)) of a set of logits; the empty set is (-inf, 0)
 struct Ms {
@@ -78,6 +82,7 @@ __device__ __forceinline__ void range_of(int V, int slices, int vec, int r, int&
 
 struct SampledArgs {
     const float* logits;
+    const float* dlogits;  // draft-model logits [B,N,V] or nullptr (then no residual is formed)
     const int32_t* tok;
     const int32_t* pptr;
     const int32_t* pidx;
@@ -99,6 +104,7 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     __shared__ float s_sum[GSD_MAX_NODES];
     __shared__ int s_red[kThreads / 32];
     __shared__ float s_scan[kThreads / 32];
+    __shared__ float s_rm[kThreads / 32];
     __shared__ int s_pick;
     const int N = a.N, V = a.V, tid = threadIdx.x;
     const int32_t* tok = a.tok + (size_t)b * N;
@@ -136,81 +142,155 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     const int s_m = res.edges, s_end = res.end;
     int32_t* out_tok = io.out_tok;
 
-    // The regenerated token.  The sums of the streaming pass over the row's contiguous ranges
-    // (slices x warps, kept in scratch) say in which range the cumulative sum first exceeds
-    // u * total; the whole block then splits that range into 256 contiguous pieces, scans the
-    // piece sums, and the thread whose piece holds the crossing walks it.
+    // The regenerated token: weights w_j over the vocabulary at the end node, then the smallest
+    // t whose cumulative weight exceeds u * (total weight).  First the contiguous range of the
+    // row that holds the crossing is found from range sums, then the whole block splits that
+    // range into 256 contiguous pieces, scans the piece sums, and the thread whose piece holds
+    // the crossing walks it.
+    const float* x = lg + (size_t)s_end * V;
+    const float mx = s_mx[s_end];
+    const int lane = tid & 31, warp = tid >> 5;
+
+    // Residual of the sampling scheme: when drafted continuations of the end node were rejected
+    // (it has a child in the graph) the weights are max(0, P_j - Q_j), Q the draft model's
+    // distribution at that node.  Its range sums are formed here: each warp takes a contiguous
+    // eighth of the row with coalesced loads.
+    bool residual = false;
+    float q_m = 0.f, inv_sp = 0.f, inv_sq = 0.f, res_total = 0.f;
+    const float* y = nullptr;
+    if (a.dlogits) {
+        int has_child = 0;
+        const int ne = min(max(io.pptr[N], 0), a.Ecap);
+        for (int e = tid; e < ne; e += kThreads) has_child |= (io.pidx[e] == s_end);
+        has_child = __syncthreads_or(has_child);
+        if (has_child) {
+            y = a.dlogits + ((size_t)b * N + s_end) * V;
+            Ms r{-CUDART_INF_F, 0.f};
+            for (int j = tid; j < V; j += kThreads) take1(r, __ldg(y + j));
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                Ms t;
+                t.m = __shfl_xor_sync(0xFFFFFFFFu, r.m, o);
+                t.s = __shfl_xor_sync(0xFFFFFFFFu, r.s, o);
+                r = combine(r, t);
+            }
+            if (lane == 0) { s_rm[warp] = r.m; s_scan[warp] = r.s; }
+            __syncthreads();
+            r = Ms{-CUDART_INF_F, 0.f};
+            for (int w = 0; w < kWarps; ++w) r = combine(r, Ms{s_rm[w], s_scan[w]});
+            __syncthreads();
+            if (!(r.s > 0.f) || r.m == CUDART_INF_F) {
+                if (tid == 0 && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
+            } else {
+                q_m = r.m;
+                inv_sp = 1.f / s_sum[s_end];
+                inv_sq = 1.f / r.s;
+                const int per = (V + kWarps - 1) / kWarps;
+                const int w0 = min(warp * per, V), w1 = min(w0 + per, V);
+                float part = 0.f;
+                for (int j = w0 + lane; j < w1; j += 32)
+                    part += fmaxf(ex2((x[j] - mx) * kLog2e) * inv_sp - ex2((y[j] - q_m) * kLog2e) * inv_sq, 0.f);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+                if (lane == 0) s_scan[warp] = part;
+                __syncthreads();
+                for (int w = 0; w < kWarps; ++w) res_total += s_scan[w];
+                // a residual without mass (the two distributions agree to rounding) leaves P
+                residual = res_total > kResidualFloor;
+            }
+        }
+    }
+    auto weight = [&](int j) -> float {
+        const float e = ex2((x[j] - mx) * kLog2e);
+        return residual ? fmaxf(e * inv_sp - ex2((y[j] - q_m) * kLog2e) * inv_sq, 0.f) : e;
+    };
+    const float target = a.us[b] * (residual ? res_total : s_sum[s_end]);
+    // every thread walks the range sums: the first range whose inclusive prefix exceeds the
+    // target, or the last one with any mass if rounding leaves none
+    int rsel = -1, last_r = 0;
+    float before_range = 0.f, before_last = 0.f;
     {
-        const float* x = lg + (size_t)s_end * V;
-        const float mx = s_mx[s_end];
-        const int lane = tid & 31, warp = tid >> 5;
-        const float target = a.us[b] * s_sum[s_end];
-        // every thread walks the (at most 128) range sums: the first range whose inclusive
-        // prefix exceeds the target, or the last one with any mass if rounding leaves none
-        int rsel = -1, last_r = 0;
-        float before_range = 0.f, before_last = 0.f;
-        {
-            float run = 0.f;
-            const float2* pr = a.part + ((size_t)b * N + s_end) * a.slices * kWarps;
-            for (int r = 0; r < a.slices * kWarps; ++r) {
+        float run = 0.f;
+        const int nr = residual ? kWarps : a.slices * kWarps;
+        const float2* pr = a.part + ((size_t)b * N + s_end) * a.slices * kWarps;
+        for (int r = 0; r < nr; ++r) {
+            float sr;
+            if (residual) {
+                sr = s_scan[r];
+            } else {
                 const float2 t = __ldcg(pr + r);
-                const float sr = t.x == -CUDART_INF_F ? 0.f : t.y * ex2((t.x - mx) * kLog2e);
-                if (rsel < 0 && run + sr > target) { rsel = r; before_range = run; }
-                if (sr > 0.f) { last_r = r; before_last = run; }
-                run += sr;
+                sr = t.x == -CUDART_INF_F ? 0.f : t.y * ex2((t.x - mx) * kLog2e);
             }
+            if (rsel < 0 && run + sr > target) { rsel = r; before_range = run; }
+            if (sr > 0.f) { last_r = r; before_last = run; }
+            run += sr;
         }
-        const bool crossing = rsel >= 0;
-        if (!crossing) { rsel = last_r; before_range = before_last; }
-        if (tid == 0) s_pick = kNone;
-        int r0, r1;
+    }
+    __syncthreads();   // s_scan is reused below
+    const bool crossing = rsel >= 0;
+    if (!crossing) { rsel = last_r; before_range = before_last; }
+    if (tid == 0) s_pick = kNone;
+    int r0, r1;
+    if (residual) {
+        const int per = (V + kWarps - 1) / kWarps;
+        r0 = min(rsel * per, V);
+        r1 = min(r0 + per, V);
+    } else {
         range_of(V, a.slices, a.vec, rsel, r0, r1);
-        const int per = (r1 - r0 + kThreads - 1) / kThreads;
-        const int j0 = min(r0 + tid * per, r1), j1 = min(j0 + per, r1);
-        float piece = 0.f;
-        int last_pos = -1;
+    }
+    const int per = (r1 - r0 + kThreads - 1) / kThreads;
+    const int j0 = min(r0 + tid * per, r1), j1 = min(j0 + per, r1);
+    float piece = 0.f;
+    int last_pos = -1;
+    for (int j = j0; j < j1; ++j) {
+        const float e = weight(j);
+        piece += e;
+        if (e > 0.f) last_pos = j;
+    }
+    float inc = piece;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) s_scan[warp] = inc;
+    __syncthreads();
+    float base = before_range;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w)
+        if (w < warp) base += s_scan[w];
+    inc += base;
+    // The pieces partition the cumulative axis exactly: a piece begins where the one before it
+    // ends (its predecessor's inclusive value, not inc - piece, which rounding could move past a
+    // target that the predecessor had not reached).  The first piece whose inclusive value exceeds
+    // the target holds the crossing.
+    float before = __shfl_up_sync(0xFFFFFFFFu, inc, 1);
+    if (lane == 0) before = base;
+    if (crossing && inc > target) atomicMin(&s_pick, tid);
+    __syncthreads();
+    const int first = s_pick;           // kNone: rounding left no crossing in this range
+    __syncthreads();
+    if (tid == first) {
+        float cum = before;
+        int pick = -1;
         for (int j = j0; j < j1; ++j) {
-            const float e = ex2((x[j] - mx) * kLog2e);
-            piece += e;
-            if (e > 0.f) last_pos = j;
+            cum += weight(j);
+            if (cum > target) { pick = j; break; }
         }
-        float inc = piece;
+        s_pick = pick;                  // -1: the serial sum stayed at or below the target
+    }
+    // without a crossing the draw is the last entry with any mass at or before that piece (in
+    // the whole range if no piece claimed the target)
+    int lp = (first == kNone || tid <= first) ? last_pos : -1;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const float t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-            if (lane >= o) inc += t;
-        }
-        if (lane == 31) s_scan[warp] = inc;
-        __syncthreads();
-        float base = before_range;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w)
-            if (w < warp) base += s_scan[w];
-        inc += base;
-        const float before = inc - piece;
-        if (crossing && piece > 0.f && inc > target && !(before > target)) {
-            float cum = before;
-            int pick = last_pos;
-            for (int j = j0; j < j1; ++j) {
-                cum += ex2((x[j] - mx) * kLog2e);
-                if (cum > target) { pick = j; break; }
-            }
-            atomicMin(&s_pick, pick);
-        }
-        // if rounding left no crossing: the last entry with any mass (it lies in the chosen range)
-        int lp = last_pos;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) lp = max(lp, __shfl_xor_sync(0xFFFFFFFFu, lp, o));
-        if (lane == 0) s_red[warp] = lp;
-        __syncthreads();
-        if (tid == 0) {
-            int pick = s_pick;
-            if (pick == kNone) {
-                pick = -1;
-                for (int w = 0; w < kWarps; ++w) pick = max(pick, s_red[w]);
-            }
-            if (s_m < a.Tcap) out_tok[s_m] = pick;
-        }
+    for (int o = 16; o > 0; o >>= 1) lp = max(lp, __shfl_xor_sync(0xFFFFFFFFu, lp, o));
+    if (lane == 0) s_red[warp] = lp;
+    __syncthreads();
+    if (tid == 0) {
+        int pick = first == kNone ? -1 : s_pick;
+        if (pick < 0)
+            for (int w = 0; w < kWarps; ++w) pick = max(pick, s_red[w]);
+        if (s_m < a.Tcap) out_tok[s_m] = pick;
     }
 }
 
@@ -283,7 +363,8 @@ extern "C" size_t gsd_accept_sampled_workspace_bytes(const gsd_accept_params* p)
 
 extern "C" int gsd_accept_sampled(const float* logits, const int32_t* draft_tokens,
                                   const int32_t* parent_ptr, const int32_t* parent_idx,
-                                  const float* draft_q, const float* u_accept, const float* u_sample,
+                                  const float* draft_logits, const float* draft_q,
+                                  const float* u_accept, const float* u_sample,
                                   int32_t* accepted_tokens, int32_t* accepted_len,
                                   int32_t* accepted_nodes, const gsd_accept_params* p,
                                   void* workspace, size_t workspace_bytes, int32_t* status,
@@ -295,7 +376,7 @@ extern "C" int gsd_accept_sampled(const float* logits, const int32_t* draft_toke
     if (p->B < 1 || p->N < 1 || p->N > GSD_MAX_NODES || p->V < 1 || p->Ecap < 1 || p->Tcap < 1)
         return GSD_ERR_BAD_SHAPE;
     if ((long long)p->B * p->N > (1ll << 30)) return GSD_ERR_BAD_SHAPE;
-    if (((uintptr_t)logits & 3u) != 0) return GSD_ERR_MISALIGNED;
+    if (((uintptr_t)logits & 3u) != 0 || ((uintptr_t)draft_logits & 3u) != 0) return GSD_ERR_MISALIGNED;
     const size_t need = gsd_accept_sampled_workspace_bytes(p);
     if (!workspace || workspace_bytes < need) return GSD_ERR_WORKSPACE;
     if (((uintptr_t)workspace & 7u) != 0) return GSD_ERR_MISALIGNED;
@@ -304,7 +385,7 @@ extern "C" int gsd_accept_sampled(const float* logits, const int32_t* draft_toke
     cudaStream_t st = (cudaStream_t)stream;
 
     SampledArgs a;
-    a.logits = logits; a.tok = draft_tokens; a.pptr = parent_ptr; a.pidx = parent_idx;
+    a.logits = logits; a.dlogits = draft_logits; a.tok = draft_tokens; a.pptr = parent_ptr; a.pidx = parent_idx;
     a.q = draft_q; a.u = u_accept; a.us = u_sample;
     a.out_tok = accepted_tokens; a.out_len = accepted_len; a.out_nodes = accepted_nodes;
     a.part = (float2*)workspace;
@@ -326,6 +407,7 @@ extern "C" int gsd_accept_sampled(const float* logits, const int32_t* draft_toke
         const int nb = (p->B - b0 < seq_per) ? p->B - b0 : seq_per;
         SampledArgs s = a;
         s.logits += (size_t)b0 * p->N * p->V; s.tok += (size_t)b0 * p->N;
+        if (s.dlogits) s.dlogits += (size_t)b0 * p->N * p->V;
         s.pptr += (size_t)b0 * (p->N + 1); s.pidx += (size_t)b0 * p->Ecap;
         s.q += (size_t)b0 * p->N; s.u += (size_t)b0 * p->N; s.us += b0;
         s.out_tok += (size_t)b0 * p->Tcap; s.out_len += b0;

@@ -65,6 +65,26 @@ __device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, St
         s_ptr[v] = e;
     }
     __syncthreads();
+    // Row pointers must start at zero and never decrease.  Otherwise they are replaced by their
+    // running maximum (a row whose pointer goes backwards becomes empty, the rows stay disjoint
+    // and every edge below the last pointer has exactly one owner) and the status bit is set.
+    {
+        int bad = 0;
+        for (int v = tid; v < N; v += kPathThreads) bad |= (s_ptr[v] > s_ptr[v + 1]);
+        if (tid == 0 && s_ptr[0] != 0) bad = 1;
+        if (__syncthreads_or(bad)) {
+            flags |= GSD_DEV_BAD_CSR;
+            if (tid == 0) {
+                int run = 0;
+                s_ptr[0] = 0;
+                for (int v = 1; v <= N; ++v) {
+                    run = max(run, s_ptr[v]);
+                    s_ptr[v] = run;
+                }
+            }
+            __syncthreads();
+        }
+    }
     // the relaxation rounds walk the parent lists again and again: keep them, and the outcome
     // of every step, on chip
     const int n_edges = s_ptr[N];

@@ -40,7 +40,7 @@ def test_binding_lists_the_same_symbols():
 
 def test_version_and_status_strings(library):
     library.gsd_status_string.restype = ctypes.c_char_p
-    assert library.gsd_version() == 100
+    assert library.gsd_version() == 101
     assert library.gsd_status_string(0) == b"ok"
     for code in range(-6, 0):
         assert library.gsd_status_string(code) not in (b"ok", b"unknown status")

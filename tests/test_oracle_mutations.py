@@ -41,7 +41,7 @@ MUTATIONS = [
      "test_oracle_accept_sampled.py"),
     ("sampled_regenerates_at_parent", "const int end = best[m];", "const int end = best[m > 0 ? m - 1 : 0];",
      "test_oracle_accept_sampled.py"),
-    ("sampled_regenerates_from_target", "if (mass > 0.0) memcpy(wgt, res, sizeof(double) * (size_t)V);", "(void)mass;",
+    ("sampled_regenerates_from_target", "if (mass > 1e-6) memcpy(wgt, res, sizeof(double) * (size_t)V);", "(void)mass;",
      "test_oracle_accept_sampled.py"),
     ("sampled_residual_sign", "const double r = wgt[j] - exp((double)y[j] - mq) / sq;",
      "const double r = exp((double)y[j] - mq) / sq - wgt[j];", "test_oracle_accept_sampled.py"),
