@@ -18,8 +18,10 @@ Random numbers come from numpy's Philox counter-based generator keyed by the see
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
 from dataclasses import dataclass, replace
-from typing import Dict, List, Sequence, Tuple, Union
+from typing import Dict, List, Optional, Sequence, Tuple, Union
 
 import numpy as np
 
@@ -206,16 +208,34 @@ def parents_to_csr(parents_per_seq: Sequence[Sequence[Sequence[int]]], Ecap: int
 
 
 # ----------------------------------------------------------------------------- tensors
-def _normal_bf16(rng: np.random.Generator, shape: Tuple[int, ...]) -> np.ndarray:
+def _normal_bf16(seed: int, stream: int, shape: Tuple[int, ...]) -> np.ndarray:
+    """N(0,1) values rounded to bf16.  Slice i along the first axis is drawn from the Philox
+    stream (seed, stream) jumped i times, so the slices can be filled by several host threads
+    and the result does not depend on how many there are."""
     out = np.empty(shape, dtype=np.uint16)
     flat = out.reshape(shape[0], -1) if len(shape) > 1 else out.reshape(1, -1)
-    for i in range(flat.shape[0]):          # chunked so the fp32 temporary stays small
-        flat[i] = f32_to_bf16_bits(rng.standard_normal(flat.shape[1], dtype=np.float32))
+    base = np.random.Philox(key=[seed & 0xFFFFFFFFFFFFFFFF, stream])
+    step = 1 << 22                          # the fp32 temporary of a piece stays at 16 MB
+
+    def fill(i: int) -> None:
+        g = np.random.Generator(base.jumped(i))
+        for a in range(0, flat.shape[1], step):
+            b = min(a + step, flat.shape[1])
+            flat[i, a:b] = f32_to_bf16_bits(g.standard_normal(b - a, dtype=np.float32))
+
+    workers = min(flat.shape[0], os.cpu_count() or 1)
+    if workers <= 1 or flat.size < (1 << 22):
+        for i in range(flat.shape[0]):
+            fill(i)
+    else:
+        with ThreadPoolExecutor(max_workers=workers) as ex:
+            list(ex.map(fill, range(flat.shape[0])))
     return out
 
 
 def make_inputs(cfg: VerifyConfig, seed: int | None = None, *, attn: bool = True,
-                accept: bool = True, pad_fill: str = "junk") -> Dict[str, object]:
+                accept: bool = True, pad_fill: str = "junk",
+                kv_from: Optional[Dict[str, object]] = None) -> Dict[str, object]:
     """Draw one batch for `cfg`.
 
     Keys: cfg, seed, parents (list per sequence), levels, draft_tokens [B,N] i32,
@@ -225,6 +245,9 @@ def make_inputs(cfg: VerifyConfig, seed: int | None = None, *, attn: bool = True
 
     pad_fill: what cache rows at positions >= seq_lens[b] hold: "junk" (large finite
     values of random sign), "nan" (quiet-NaN patterns) or "zero".
+    kv_from: an earlier batch drawn with the same seed, B, Hkv, D, prefix lengths and pad_fill;
+    its k_cache / v_cache arrays are used as they are instead of being drawn a second time
+    (the draw depends on nothing else, so they would come out identical).
     """
     if seed is None:
         seed = seed_for(cfg)
@@ -247,13 +270,19 @@ def make_inputs(cfg: VerifyConfig, seed: int | None = None, *, attn: bool = True
                                   draft_tokens=tokens, parent_ptr=ptr, parent_idx=idx,
                                   ancestor_mask=mask, seq_lens=seq_lens, Lmax=Lmax)
     if attn:
-        out["q"] = _normal_bf16(_rng(seed, 4), (B, N, Hq, D))
-        kc = _normal_bf16(_rng(seed, 5), (B, max(Lmax, 1), Hkv, D))
-        vc = _normal_bf16(_rng(seed, 6), (B, max(Lmax, 1), Hkv, D))
+        out["q"] = _normal_bf16(seed, 4, (B, N, Hq, D))
+        if kv_from is not None:
+            kc, vc = kv_from["k_cache"], kv_from["v_cache"]
+            if (kv_from["seed"] != seed or kc.shape != (B, max(Lmax, 1), Hkv, D)
+                    or not np.array_equal(kv_from["seq_lens"], seq_lens)):
+                raise ValueError("kv_from was drawn for another cache shape or seed")
+        else:
+            kc = _normal_bf16(seed, 5, (B, max(Lmax, 1), Hkv, D))
+            vc = _normal_bf16(seed, 6, (B, max(Lmax, 1), Hkv, D))
         g_pad = _rng(seed, 9)
         for b in range(B):
             n_pad = kc.shape[1] - int(seq_lens[b])
-            if n_pad <= 0:
+            if n_pad <= 0 or kv_from is not None:
                 continue
             shp = (n_pad, Hkv, D)
             if pad_fill == "junk":
@@ -268,8 +297,8 @@ def make_inputs(cfg: VerifyConfig, seed: int | None = None, *, attn: bool = True
             kc[b, int(seq_lens[b]):] = fill
             vc[b, int(seq_lens[b]):] = fill
         out["k_cache"], out["v_cache"] = kc, vc
-        out["draft_k"] = _normal_bf16(_rng(seed, 7), (B, N, Hkv, D))
-        out["draft_v"] = _normal_bf16(_rng(seed, 8), (B, N, Hkv, D))
+        out["draft_k"] = _normal_bf16(seed, 7, (B, N, Hkv, D))
+        out["draft_v"] = _normal_bf16(seed, 8, (B, N, Hkv, D))
     if accept:
         g_log = _rng(seed, 10)
         logits = np.empty((B, N, V), dtype=np.float32)

@@ -159,11 +159,7 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     float q_m = 0.f, inv_sp = 0.f, inv_sq = 0.f, res_total = 0.f;
     const float* y = nullptr;
     if (a.dlogits) {
-        int has_child = 0;
-        const int ne = min(max(io.pptr[N], 0), a.Ecap);
-        for (int e = tid; e < ne; e += kThreads) has_child |= (io.pidx[e] == s_end);
-        has_child = __syncthreads_or(has_child);
-        if (has_child) {
+        if (res.end_has_child) {
             y = a.dlogits + ((size_t)b * N + s_end) * V;
             Ms r{-CUDART_INF_F, 0.f};
             for (int j = tid; j < V; j += kThreads) take1(r, __ldg(y + j));

@@ -27,8 +27,9 @@ struct PathIo {
 };
 
 struct PathResult {
-    int edges;   // m: the accepted path has m + 1 nodes
-    int end;     // its last node
+    int edges;           // m: the accepted path has m + 1 nodes
+    int end;             // its last node
+    bool end_has_child;  // some node lists `end` as a parent (only filled in with kCacheOutcome)
 };
 
 // With kCacheOutcome, `step_ok(p, v)` is called once per step when the parent lists fit the
@@ -181,7 +182,15 @@ __device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, St
         io.out_tok[i] = -1;
         if (io.out_nodes) io.out_nodes[i] = -1;
     }
-    return PathResult{s_m, s_end};
+    bool end_has_child = false;
+    if (kCacheOutcome) {
+        int has = 0;
+        const int end = s_end;
+        for (int v = end + 1 + tid; v < N; v += kPathThreads)
+            for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) has |= ((cached ? s_edge[e] : io.pidx[e]) == end);
+        end_has_child = __syncthreads_or(has) != 0;
+    }
+    return PathResult{s_m, s_end, end_has_child};
 }
 
 }  // namespace gsd

@@ -132,3 +132,44 @@ def test_repeated_calls_are_identical():
     b = run_gpu(inp)
     for x, y in zip(a, b):
         assert np.array_equal(x, y)
+
+
+def test_more_rows_than_one_launch_holds():
+    # B * N = 70400 rows: the library sends them out as two launches of whole sequences (a grid
+    # dimension holds 65535 rows); results and the per-sequence completion counters must not care
+    cfg = gi.VerifyConfig("many", 6, 1100, 1, 1, 64, 8, 64, 8, 3, 2, 128, 128, 0.7)
+    inp = gi.make_inputs(cfg, attn=False)
+    assert cfg.B * cfg.N > 65535
+    check_against_oracle(inp)
+
+
+def sanitised_parents(ptr, idx, N):
+    """What the library documents for row pointers that do not start at zero or go backwards:
+    they are replaced by their running maximum (from zero), and parent indices outside [0, v)
+    are ignored.  Written out here in plain Python."""
+    run, sp = 0, [0]
+    for v in range(1, N + 1):
+        run = max(run, min(max(int(ptr[v]), 0), len(idx)))
+        sp.append(run)
+    return [[int(p) for p in idx[sp[v]:sp[v + 1]] if 0 <= p < v] for v in range(N)]
+
+
+@pytest.mark.parametrize("ptr", [
+    [0, 0, 1, 5, 3, 4, 6],        # an interior pointer above the last one, then going backwards
+    [2, 2, 3, 4, 5, 6, 6],        # does not start at zero: edges 0, 1 belong to the root's row and are ignored
+    [0, 0, 4, 2, 3, 9, 5],        # a pointer past the capacity (clamped) and non-monotone ones
+])
+def test_row_pointers_that_go_backwards_are_flagged_and_made_safe(ptr):
+    N, Ecap = 6, 8
+    idx = np.array([[0, 0, 1, 1, 2, 3, 4, 2]], dtype=np.int32)
+    tok = np.array([[0, 5, 6, 7, 8, 9]], dtype=np.int32)
+    logits = logits_with_argmax([5, 6, 7, 8, 9, 3], 16)[None]          # node v's argmax is the token of node v+1
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    inp = dict(logits=logits, draft_tokens=tok, parent_ptr=np.array([ptr], dtype=np.int32), parent_idx=idx)
+    got = run_gpu(inp, status=status)
+    assert int(status.item()) & 0x1
+    parents = sanitised_parents(ptr, idx[0], N)
+    cptr, cidx = gi.parents_to_csr([parents], Ecap)
+    want = oracle.accept(logits, tok, cptr, cidx)
+    for g, w in zip(got, want[:3]):
+        assert np.array_equal(g, w)

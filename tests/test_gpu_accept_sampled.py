@@ -292,3 +292,39 @@ def test_row_without_mass_is_flagged_and_repeat_calls_agree():
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     run_gpu(bad, q, u, us, status=status)
     assert int(status.item()) & 0x40
+
+
+def test_more_rows_than_one_launch_holds():
+    # B * N = 70400 rows go out as two launches of whole sequences
+    cfg = gi.VerifyConfig("many", 6, 1100, 1, 1, 64, 8, 64, 8, 3, 2, 128, 128, 0.7)
+    inp = gi.make_inputs(cfg, attn=False)
+    dl = draft_logits_for(inp["logits"], 17)
+    check(inp, 31, dl=dl)
+
+
+def test_row_pointers_that_go_backwards_are_flagged_and_made_safe():
+    # the same sanitising rule as gsd_accept (running maximum from zero, bad parents ignored);
+    # with every u = 0 each surviving step is accepted
+    from test_gpu_accept import sanitised_parents
+    N, Ecap, V = 6, 8, 16
+    ptr = [0, 0, 1, 5, 3, 4, 6]
+    idx = np.array([[0, 0, 1, 1, 2, 3, 4, 2]], dtype=np.int32)
+    rng = np.random.default_rng(3)
+    inp = dict(logits=rng.standard_normal((1, N, V)).astype(np.float32),
+               draft_tokens=rng.integers(0, V, size=(1, N)).astype(np.int32),
+               parent_ptr=np.array([ptr], dtype=np.int32), parent_idx=idx)
+    q = np.ones((1, N), dtype=np.float32)
+    u = np.zeros((1, N), dtype=np.float32)
+    end_w = None
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    parents = sanitised_parents(ptr, idx[0], N)
+    cptr, cidx = gi.parents_to_csr([parents], Ecap)
+    us = np.array([0.5], dtype=np.float32)
+    _, lens, nodes = oracle.accept_sampled(inp["logits"], inp["draft_tokens"], cptr, cidx, q, u, us)
+    w = softmax64(inp["logits"][0, nodes[0, lens[0] - 1]]); t = int(np.argmax(w))
+    us[0] = np.float32(np.cumsum(w)[t] - 0.5 * w[t])
+    want = oracle.accept_sampled(inp["logits"], inp["draft_tokens"], cptr, cidx, q, u, us)
+    got = run_gpu(inp, q, u, us, status=status)
+    assert int(status.item()) & 0x1
+    for g, w_ in zip(got, want):
+        assert np.array_equal(g, w_)

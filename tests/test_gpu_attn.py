@@ -54,21 +54,25 @@ def test_configs_full_compare(name, kernel):
         assert_close(out_to_f64(gpu_attn(inp, kernel=kernel)), cpu_attn(inp))
 
 
-@pytest.mark.parametrize("kernel", [0] + KERNELS)
-def test_llama70b_sampled_rows_and_one_full_unit(kernel):
-    # full-size configuration: the oracle recomputes one whole (sequence, kv head) unit and
-    # 1024 random rows one by one
+@pytest.fixture(scope="module")
+def llama70b_all_rows():
+    """The full-size configuration with the oracle's answer for ALL 131072 rows, computed once
+    (some tens of seconds on the host cores) and shared by the three kernel selections."""
     cfg = gi.CONFIGS["llama70b"]
     inp = gi.make_inputs(cfg, accept=False)
+    return inp, cpu_attn(inp)
+
+
+@pytest.mark.parametrize("kernel", [0] + KERNELS)
+def test_llama70b_every_row(kernel, llama70b_all_rows):
+    inp, want = llama70b_all_rows
     got = out_to_f64(gpu_attn(inp, kernel=kernel))
-    rng = np.random.default_rng(4)
-    rows = [(3, n, 5 * cfg.G + g) for n in range(cfg.N) for g in range(cfg.G)]
-    rows += [(int(rng.integers(cfg.B)), int(rng.integers(cfg.N)), int(rng.integers(cfg.Hq)))
-             for _ in range(1024)]
-    want = oracle.attn_rows(inp["q"], inp["k_cache"], inp["v_cache"], inp["draft_k"],
-                            inp["draft_v"], inp["ancestor_mask"], inp["seq_lens"], rows)
-    g = np.stack([got[b, n, h] for b, n, h in rows])
-    assert_close(g, want)
+    assert got.shape == want.shape
+    assert_close(got, want)
+    # no single (sequence, kv head) unit hides behind the global mean
+    cfg = inp["cfg"]
+    err = np.abs(got - want).reshape(cfg.B, cfg.N, cfg.Hkv, cfg.G, cfg.D)
+    assert err.mean(axis=(1, 3, 4)).max() <= MEAN_ABS
 
 
 @pytest.mark.parametrize("kernel", KERNELS)
@@ -150,22 +154,42 @@ def test_bad_seq_len_is_clamped_and_flagged():
     assert_close(got, want)          # clamped to Lmax == the true length here
 
 
-@pytest.mark.parametrize("point", [(1, 512, 32), (8, 2048, 128), (1, 8192, 512)])
-def test_sweep_points_sampled_rows(point):
-    # 70B-shaped sweep (64 q heads over 8 kv heads, D 128): one whole (sequence, kv head) unit
-    # of stacked rows plus 256 random rows, each recomputed one by one by the oracle
-    B, L, N = point
-    cfg = gi.sweep_config(B, L, N)
-    inp = gi.make_inputs(cfg, accept=False)
-    got = out_to_f64(gpu_attn(inp))
-    rng = np.random.default_rng(B * 1000 + N)
-    b0, c0 = int(rng.integers(cfg.B)), int(rng.integers(cfg.Hkv))
-    rows = [(b0, n, c0 * cfg.G + g) for n in range(0, cfg.N, max(1, cfg.N // 64)) for g in range(cfg.G)]
+def sampled_rows_check(inp, out, rng, n_random=256, node_step=0, units=None):
+    """Rows the oracle recomputes one by one: every `node_step`-th node (all GQA heads) of the
+    listed (sequence, kv head) units plus `n_random` random rows."""
+    cfg = inp["cfg"]
+    if units is None:
+        units = [(int(rng.integers(cfg.B)), int(rng.integers(cfg.Hkv)))]
+    node_step = node_step or max(1, cfg.N // 64)
+    rows = [(b0, n, c0 * cfg.G + g) for b0, c0 in units for n in range(0, cfg.N, node_step) for g in range(cfg.G)]
     rows += [(int(rng.integers(cfg.B)), int(rng.integers(cfg.N)), int(rng.integers(cfg.Hq)))
-             for _ in range(256)]
+             for _ in range(n_random)]
     want = oracle.attn_rows(inp["q"], inp["k_cache"], inp["v_cache"], inp["draft_k"],
                             inp["draft_v"], inp["ancestor_mask"], inp["seq_lens"], rows)
-    assert_close(np.stack([got[b, n, h] for b, n, h in rows]), want)
+    idx = torch.tensor(rows, device=out.device, dtype=torch.long)
+    assert_close(out_to_f64(out[idx[:, 0], idx[:, 1], idx[:, 2]]), want)
+
+
+SWEEP_B, SWEEP_L, SWEEP_N = (1, 8, 32), (512, 2048, 8192, 32768), (32, 128, 512)
+
+
+@pytest.mark.parametrize("L", SWEEP_L)
+@pytest.mark.parametrize("B", SWEEP_B)
+def test_sweep_points_sampled_rows(B, L):
+    # every point of the 70B-shaped sweep (64 q heads over 8 kv heads, D 128; 3 x 4 x 3 = 36
+    # points, up to 4.3 GB of KV cache): one whole (sequence, kv head) unit of stacked rows
+    # (every node for N = 32, every N/64-th node otherwise, all 8 heads of each) plus 256 random
+    # rows, recomputed one by one by the oracle.  The three graph sizes of a (B, L) pair share
+    # one KV cache (it is drawn from (seed, B, L) alone).
+    first = None
+    for N in SWEEP_N:
+        cfg = gi.sweep_config(B, L, N)
+        inp = gi.make_inputs(cfg, accept=False, kv_from=first)
+        first = first or inp
+        out = gpu_attn(inp)
+        sampled_rows_check(inp, out, np.random.default_rng(B * 1000 + N + L))
+        del out
+        torch.cuda.empty_cache()
 
 
 RANDOM_SHAPES = []
@@ -198,17 +222,9 @@ def test_many_units_per_cta_sampled_rows():
     cfg = gi.sweep_config(32, 100, 512)
     inp = gi.make_inputs(cfg, accept=False)
     out = gpu_attn(inp)
-    rng = np.random.default_rng(77)
-    rows = []
-    for b0, c0 in ((0, 0), (31, 7), (17, 3)):          # first, last and a middle (sequence, kv head)
-        rows += [(b0, n, c0 * cfg.G + g) for n in range(0, cfg.N, 16) for g in range(cfg.G)]
-    rows += [(int(rng.integers(cfg.B)), int(rng.integers(cfg.N)), int(rng.integers(cfg.Hq)))
-             for _ in range(1024)]
-    want = oracle.attn_rows(inp["q"], inp["k_cache"], inp["v_cache"], inp["draft_k"],
-                            inp["draft_v"], inp["ancestor_mask"], inp["seq_lens"], rows)
-    idx = torch.tensor(rows, device=out.device, dtype=torch.long)
-    got = out_to_f64(out[idx[:, 0], idx[:, 1], idx[:, 2]])
-    assert_close(got, want)
+    # first, last and a middle (sequence, kv head)
+    sampled_rows_check(inp, out, np.random.default_rng(77), n_random=1024, node_step=16,
+                       units=[(0, 0), (31, 7), (17, 3)])
 
 
 def test_dominant_key_and_large_score_jumps():

@@ -10,6 +10,7 @@ import pytest
 import torch
 
 import gsd_inputs as gi
+import oracle
 from gpu_util import accept_tensors
 
 pytestmark = pytest.mark.gpu
@@ -33,6 +34,42 @@ def test_two_calls_in_a_row_match_gsd_accept():
         want, got = both(inp)
         for w, g in zip(want, got):
             assert np.array_equal(w, g)
+        # and against the CPU oracle directly, so that this file stands on its own
+        ref = oracle.accept(inp["logits"], inp["draft_tokens"], inp["parent_ptr"], inp["parent_idx"])
+        for r, g in zip(ref[:3], got):
+            assert np.array_equal(r, g)
+
+
+def test_free_device_memory_does_not_move():
+    # the call's promise is that it allocates nothing: with the outputs allocated up front, the
+    # driver's free-byte count (cudaMemGetInfo) is the same after twenty more calls
+    import ctypes
+    import paper_2407_16207_b200 as gsd
+    inp = gi.make_inputs(gi.CONFIGS["llama7b"], attn=False)
+    t = accept_tensors(inp)
+    B, N, V = t["logits"].shape
+    toks = torch.empty((B, N), dtype=torch.int32, device="cuda")
+    lens = torch.empty((B,), dtype=torch.int32, device="cuda")
+    nodes = torch.empty((B, N), dtype=torch.int32, device="cuda")
+    p = gsd.binding.AcceptParams(B, N, V, t["parent_idx"].shape[1], N)
+    L = gsd.lib()
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def call():
+        rc = L.gsd_accept_static(t["logits"].data_ptr(), t["draft_tokens"].data_ptr(), t["parent_ptr"].data_ptr(),
+                                 t["parent_idx"].data_ptr(), toks.data_ptr(), lens.data_ptr(), nodes.data_ptr(),
+                                 ctypes.byref(p), None, stream)
+        assert rc == 0
+
+    call()                                   # the first call on a device looks the array up
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    for _ in range(20):
+        call()
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    ref = oracle.accept(inp["logits"], inp["draft_tokens"], inp["parent_ptr"], inp["parent_idx"])
+    assert np.array_equal(toks.cpu().numpy(), ref[0]) and np.array_equal(lens.cpu().numpy(), ref[1])
 
 
 def test_size_limit_is_refused_cleanly():
