@@ -1,20 +1,23 @@
 #!/usr/bin/env python
 """Benchmark of the GSD verification step (gsd_verify_attn + gsd_accept) on B200.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama70b] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+  python bench.py --sweep [--points B1_L512_N32,...]      one JSON line per point of the 70B-shaped sweep
 
 A step is one pass of the whole hot path over one batch of synthetic LLaMA-2-shaped input:
 DAG-masked attention of all draft nodes, then vocabulary argmax and longest accepted path.
+NAME is tiny, llama7b, llama13b, llama70b (default) or a sweep point sweep_B{b}_L{l}_N{n}.
 Prints ONE JSON line (rank 0).  With N > 1 every rank runs an independent replica of the
 workload (the path has no cross-GPU exchange), timed as the max over ranks.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import re
 import statistics
-import subprocess
 import sys
 import time
 
@@ -23,13 +26,15 @@ import torch
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
-sys.path.insert(0, os.path.join(ROOT, "tests"))
 
 import gsd_inputs as gi  # noqa: E402
 
 METRIC = "draft_tokens_verified_per_s_per_attn_layer"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
+L2_BYTES = 126 << 20
+SWEEP_B, SWEEP_L, SWEEP_N = (1, 8, 32), (512, 2048, 8192, 32768), (32, 128, 512)
 
 
 def load_peaks():
@@ -40,6 +45,15 @@ def load_peaks():
         return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
     except Exception:
         return dict(FALLBACK_PEAKS), "fallback"
+
+
+def config_by_name(name: str) -> gi.VerifyConfig:
+    if name in gi.CONFIGS:
+        return gi.CONFIGS[name]
+    m = re.fullmatch(r"(?:sweep_)?B(\d+)_L(\d+)_N(\d+)", name)
+    if not m:
+        raise SystemExit(f"unknown workload {name!r}: one of {sorted(gi.CONFIGS)} or sweep_B<b>_L<l>_N<n>")
+    return gi.sweep_config(int(m.group(1)), int(m.group(2)), int(m.group(3)))
 
 
 def algorithmic_work(cfg, inp):
@@ -58,6 +72,51 @@ def algorithmic_work(cfg, inp):
     mask_bytes = inp["ancestor_mask"].nbytes
     accept_bytes = 4.0 * B * N * cfg.V
     return flops, kv_bytes + qo_bytes + mask_bytes, accept_bytes
+
+
+def roofline_of(flops, attn_bytes, seconds, peaks, peak_src):
+    """The roofline object of one gsd_verify_attn call that took `seconds`.  One fixed pair of
+    denominators: the measured burst bf16 throughput and the measured copy bandwidth."""
+    t_tc = flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = attn_bytes / (peaks["hbm_gbs"] * 1e9)
+    if t_tc >= t_hbm:
+        achieved = flops / seconds / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["bf16_tflops"], "traffic": None,
+                "peak_kind": f"burst bf16, of {peak_src}",
+                "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+                "frac_of_nominal": achieved / NOMINAL["bf16_tflops"]}
+    else:
+        achieved = attn_bytes / seconds / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                "peak_kind": f"copy bandwidth, of {peak_src}",
+                "frac_of_nominal": achieved / NOMINAL["hbm_gbs"]}
+    roof["roofline_us"] = max(t_tc, t_hbm) * 1e6
+    roof["algorithmic_flops"] = flops
+    roof["algorithmic_bytes"] = attn_bytes
+    return roof
+
+
+def recorded_traffic(kernel_name: str, workload: str):
+    """DRAM bytes per launch of `kernel_name` on `workload` as recorded beside the ncu summaries
+    (kernel, workload, bytes, and the SHA-256 of the kernel's source at capture time).  None when
+    there is no record or the source has changed since: the counters then describe other code."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    try:
+        lines = open(path).read().splitlines()
+    except OSError:
+        return None
+    for line in lines:
+        f = line.split()
+        if len(f) == 5 and not line.startswith("#") and f[0] == kernel_name and f[1] == workload:
+            src = os.path.join(ROOT, "paper_2407_16207_b200", "csrc", f[3])
+            try:
+                digest = hashlib.sha256(open(src, "rb").read()).hexdigest()
+            except OSError:
+                return None
+            return float(f[2]) if digest == f[4] else None
+    return None
 
 
 class ClockSampler:
@@ -101,7 +160,7 @@ class ClockSampler:
             except Exception as e:  # pragma: no cover
                 self.err = str(e)
                 return
-            self._stop.wait(0.02)
+            self._stop.wait(0.01)
 
     def stop(self):
         self._stop.set()
@@ -137,98 +196,231 @@ def aggregate_over_ranks(ms_per_step, tokens_per_step, world, dist, device):
     return {"ms_per_step": ms_per_step, "value": world * tokens_per_step / (ms_per_step * 1e-3)}
 
 
-def cpu_oracle_sample(cfg, inp, budget_rows: int, accept_seqs: int = 0):
-    """Times the CPU oracle (as it stands) on a bounded sample of the workload: `budget_rows`
-    random attention rows plus the acceptance step of `accept_seqs` sequences (0 = all).
-    Returns (tokens/s extrapolated to the whole step, threads, description)."""
+# ------------------------------------------------------------------------------ CPU oracle legs
+def cpu_oracle_time(cfg, inp, rows: int, accept_seqs: int = 0):
+    """Times the CPU oracle (as it stands) on the workload: `rows` consecutive attention rows
+    (all of them when rows >= B*N*Hq; otherwise a block starting at a seeded offset, the same
+    access pattern as the full run) plus the acceptance of `accept_seqs` sequences (0 = all).
+    Returns a cpu_baseline object; anything not run in full is scaled up and says so."""
     import oracle
-    rng = np.random.default_rng(0)
     total_rows = cfg.B * cfg.N * cfg.Hq
-    n = min(budget_rows, total_rows)
-    rows = np.stack([rng.integers(cfg.B, size=n), rng.integers(cfg.N, size=n),
-                     rng.integers(cfg.Hq, size=n)], axis=1).astype(np.int32)
+    n = int(min(max(rows, 1), total_rows))
     t0 = time.perf_counter()
-    oracle.attn_rows(inp["q"], inp["k_cache"], inp["v_cache"], inp["draft_k"], inp["draft_v"],
-                     inp["ancestor_mask"], inp["seq_lens"], rows)
+    if n == total_rows:
+        oracle.attn(inp["q"], inp["k_cache"], inp["v_cache"], inp["draft_k"], inp["draft_v"],
+                    inp["ancestor_mask"], inp["seq_lens"])
+    else:
+        r0 = int(np.random.default_rng(0).integers(0, total_rows - n + 1))
+        r = np.arange(r0, r0 + n)
+        rows_bnh = np.stack([r // (cfg.N * cfg.Hq), (r // cfg.Hq) % cfg.N, r % cfg.Hq], axis=1).astype(np.int32)
+        oracle.attn_rows(inp["q"], inp["k_cache"], inp["v_cache"], inp["draft_k"], inp["draft_v"],
+                         inp["ancestor_mask"], inp["seq_lens"], rows_bnh)
     t_attn = time.perf_counter() - t0
     nb = cfg.B if accept_seqs <= 0 else min(accept_seqs, cfg.B)
     t0 = time.perf_counter()
-    oracle.accept(inp["logits"][:nb], inp["draft_tokens"][:nb], inp["parent_ptr"][:nb], inp["parent_idx"][:nb])
-    t_acc = (time.perf_counter() - t0) * (cfg.B / nb)
-    t_step = t_attn * (total_rows / n) + t_acc
-    desc = (f"{n} of {total_rows} attention rows (random (b,n,h), {t_attn:.3f} s, scaled to all rows) "
-            f"+ acceptance of {nb} of {cfg.B} sequences ({t_acc:.3f} s scaled to all)")
-    return cfg.B * cfg.N / t_step, oracle.threads(), desc
+    oracle.accept(inp["logits"][:nb], inp["draft_tokens"][:nb], inp["parent_ptr"][:nb], inp["parent_idx"][:nb],
+                  visit_cap=5_000_000)
+    t_acc = time.perf_counter() - t0
+    t_step = t_attn * (total_rows / n) + t_acc * (cfg.B / nb)
+    full = n == total_rows and nb == cfg.B
+    desc = (f"{'all' if n == total_rows else n} of {total_rows} attention rows ({t_attn:.3f} s) + acceptance of "
+            f"{nb} of {cfg.B} sequences ({t_acc:.3f} s)" + ("" if full else "; scaled to the whole step"))
+    return {"value": cfg.B * cfg.N / t_step, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": desc, "extrapolated": not full, "sampled_fraction": n / total_rows,
+            "seconds_per_step": t_step}
 
 
 def run_reference(args, cfg):
-    """The reference arm: the CPU oracle, timed on the host cores.  Each of the K steps is a
-    bounded sample of the workload, sized so that the whole run takes about a minute whatever K is."""
+    """The reference arm: the CPU oracle, timed on the host cores.  A step is the whole workload
+    when K + W such steps fit in about two minutes; otherwise each step is a block of rows sized
+    for that budget and the line says that its value is extrapolated."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     inp = gi.make_inputs(cfg)
     total_rows = cfg.B * cfg.N * cfg.Hq
     n_steps = args.warmup + args.steps
-    # ~2e5 rows/min on 16 threads at this size: spread ~40000 rows over the run, at least 16 per step
-    rows_per_step = int(min(total_rows, max(16, 40000 // max(1, n_steps))))
-    accept_seqs = 0 if n_steps <= 50 else 1
-    vals = []
-    desc, threads = "", 1
+    probe = cpu_oracle_time(cfg, inp, min(total_rows, 8192), 1)          # calibration, not reported
+    budget_s = 120.0
+    rows_per_step = int(min(total_rows, max(64, total_rows * budget_s / (n_steps * probe["seconds_per_step"]))))
+    if rows_per_step > 0.9 * total_rows:
+        rows_per_step = total_rows
+    accept_seqs = 0 if rows_per_step == total_rows else 1
+    runs = []
     for i in range(n_steps):
-        v, threads, desc = cpu_oracle_sample(cfg, inp, rows_per_step, accept_seqs)
+        r = cpu_oracle_time(cfg, inp, rows_per_step, accept_seqs)
         if i >= args.warmup:
-            vals.append(v)
-    value = cfg.B * cfg.N * len(vals) / sum(cfg.B * cfg.N / v for v in vals)
+            runs.append(r)
+    sec = sum(r["seconds_per_step"] for r in runs) / len(runs)
+    value = cfg.B * cfg.N / sec
+    last = runs[-1]
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": 1e3 * cfg.B * cfg.N / value, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "extrapolated": last["extrapolated"],
+            "sampled_fraction": last["sampled_fraction"],
             "config": {"workload": cfg.name, "B": cfg.B, "N": cfg.N, "Hq": cfg.Hq, "Hkv": cfg.Hkv,
                        "D": cfg.D, "L": cfg.L, "V": cfg.V},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
-                             "sample": "per step: " + desc},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"], "kind": "oracle",
+                             "sample": "per step: " + last["sample"], "extrapolated": last["extrapolated"],
+                             "sampled_fraction": last["sampled_fraction"]},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------------------ the 70B-shaped sweep
+def run_sweep(args):
+    """One JSON line per point: gsd_verify_attn (automatic kernel choice) and gsd_accept on the
+    seeded inputs of that point, timed cold (a buffer larger than L2 is written between calls)
+    and warm (the same resident set called back to back), each against the roofline."""
+    import paper_2407_16207_b200 as gsd
+    from gsd_inputs.torch_io import accept_tensors, attn_tensors
+    gsd.lib()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peaks, peak_src = load_peaks()
+    if args.points:
+        names = args.points.split(",")
+    else:
+        names = ["llama7b", "llama13b", "llama70b"] + [f"sweep_B{b}_L{l}_N{n}" for b in SWEEP_B for l in SWEEP_L
+                                                       for n in SWEEP_N]
+    flush = torch.empty(4 * L2_BYTES, dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    reps = max(args.steps if args.steps_given else 20, 3)
+    prev = None
+    for name in names:
+        cfg = config_by_name(name)
+        reuse = prev if (prev is not None and prev["cfg"].name.startswith("sweep") and name.startswith("sweep")
+                         and (prev["cfg"].B, prev["cfg"].L) == (cfg.B, cfg.L)) else None
+        inp = gi.make_inputs(cfg, kv_from=reuse)
+        prev = inp
+        t = {**attn_tensors(inp, dev), **accept_tensors(inp, dev)}
+        out = torch.empty_like(t["q"])
+        Lmax = inp["Lmax"]
+        ws = torch.empty(max(gsd.gsd_verify_attn_workspace_bytes(cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.D, Lmax), 256),
+                         dtype=torch.uint8, device=dev)
+        ws_acc = torch.empty(gsd.gsd_accept_workspace_bytes(cfg.B, cfg.N), dtype=torch.uint8, device=dev)
+        acc_out = (torch.empty((cfg.B, cfg.N), dtype=torch.int32, device=dev),
+                   torch.empty((cfg.B,), dtype=torch.int32, device=dev),
+                   torch.empty((cfg.B, cfg.N), dtype=torch.int32, device=dev))
+
+        def attn():
+            gsd.gsd_verify_attn(t["q"], t["k_cache"], t["v_cache"], t["draft_k"], t["draft_v"],
+                                t["ancestor_mask"], t["seq_lens"], out=out, workspace=ws, status=status)
+
+        def accept():
+            gsd.gsd_accept(t["logits"], t["draft_tokens"], t["parent_ptr"], t["parent_idx"],
+                           workspace=ws_acc, status=status, out=acc_out)
+
+        for _ in range(3):
+            attn(); accept()
+        torch.cuda.synchronize()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(reps)]
+        for i in range(reps):                       # cold: L2 holds the flush buffer's lines
+            flush.fill_(i & 0xFF)
+            ev[i][0].record(); attn(); ev[i][1].record(); accept(); ev[i][2].record()
+        torch.cuda.synchronize()
+        attn_cold = statistics.median(e[0].elapsed_time(e[1]) for e in ev) * 1e-3
+        acc_cold = statistics.median(e[1].elapsed_time(e[2]) for e in ev) * 1e-3
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        e0.record()
+        for _ in range(reps):
+            attn()
+        e1.record()
+        for _ in range(reps):
+            accept()
+        e2.record()
+        torch.cuda.synchronize()
+        attn_warm = e0.elapsed_time(e1) * 1e-3 / reps
+        acc_warm = e1.elapsed_time(e2) * 1e-3 / reps
+        if int(status.item()) != 0:
+            raise RuntimeError(f"device status {int(status.item()):#x} on {name}")
+        flops, attn_bytes, accept_bytes = algorithmic_work(cfg, inp)
+        roof = roofline_of(flops, attn_bytes, attn_cold, peaks, peak_src)
+        roof["kernel"] = "gsd_verify_attn"
+        roof["frac_warm"] = roofline_of(flops, attn_bytes, attn_warm, peaks, peak_src)["frac"]
+        tokens = cfg.B * cfg.N
+        line = {"mode": "sweep", "metric": METRIC, "value": tokens / (attn_cold + acc_cold), "unit": UNIT,
+                "n_gpus": 1, "steps": reps, "warmup": 3, "higher_is_better": True, "dtype": "bf16",
+                "data": "synthetic",
+                "config": {"workload": cfg.name, "B": cfg.B, "N": cfg.N, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
+                           "L": cfg.L, "V": cfg.V, "depth": cfg.depth, "R": cfg.N * cfg.G,
+                           "l2": "cold = a 504 MB buffer written between calls; warm = one resident set, back to back",
+                           "num_splits": gsd.gsd_verify_attn_num_splits(cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.D, Lmax)},
+                "attn_us_cold": attn_cold * 1e6, "attn_us_warm": attn_warm * 1e6,
+                "accept_us_cold": acc_cold * 1e6, "accept_us_warm": acc_warm * 1e6,
+                "accept_frac_of_hbm_cold": accept_bytes / acc_cold / 1e9 / peaks["hbm_gbs"],
+                "accept_frac_of_hbm_warm": accept_bytes / acc_warm / 1e9 / peaks["hbm_gbs"],
+                "roofline": roof}
+        print(json.dumps(line), flush=True)
+        del t, out, ws, ws_acc
+        torch.cuda.empty_cache()
+
+
+def timed_calls(fn, before=None, n=20, warm=3):
+    """Median CUDA-event time in microseconds of `fn(i)` over n calls after `warm` untimed ones;
+    `before(i)` runs ahead of each call, outside its pair of events."""
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+    for i in range(n + warm):
+        if before:
+            before(i)
+        if i >= warm:
+            ev[i - warm][0].record()
+        fn(i)
+        if i >= warm:
+            ev[i - warm][1].record()
+    torch.cuda.synchronize()
+    return statistics.median(a.elapsed_time(b) for a, b in ev) * 1e3
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=6000)
+    ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="llama70b", choices=sorted(gi.CONFIGS))
+    ap.add_argument("--workload", default="llama70b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 mma.sync, 2 tcgen05")
     ap.add_argument("--num-splits", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=5)
-    ap.add_argument("--cpu-rows", type=int, default=16384,
-                    help="attention rows in the CPU-oracle sample (0 = skip the CPU baseline)")
+    ap.add_argument("--cpu-baseline", default="auto", choices=["auto", "full", "sample", "off"],
+                    help="auto: the whole step on the named configurations, a sample on sweep points")
+    ap.add_argument("--sweep", action="store_true", help="one JSON line per point of the 70B-shaped sweep")
+    ap.add_argument("--points", default="", help="with --sweep: comma-separated workload names")
     args = ap.parse_args()
-    cfg = gi.CONFIGS[args.workload]
+    args.steps_given = args.steps is not None
+    if args.steps is None:
+        args.steps = 6000
+    if args.sweep:
+        run_sweep(args)
+        return
+    cfg = config_by_name(args.workload)
     if args.impl == "reference":
         run_reference(args, cfg)
         return
 
     import paper_2407_16207_b200 as gsd
-    from gpu_util import accept_tensors, attn_tensors
+    from gsd_inputs.torch_io import accept_tensors, attn_tensors
     gsd.lib()  # fail loudly if the CUDA library is missing
     rank, world, local, dist = dist_setup(args.gpus)
     dev = torch.device("cuda", local)
 
-    # inputs: two independent sets, rotated, so that every step reads ~0.5 GB it has not just
-    # touched (more than the 126 MB L2)
-    NSETS = 2
-    host_sets = [gi.make_inputs(cfg, gi.seed_for(cfg, 10 * rank + s)) for s in range(NSETS)]
+    # inputs: independent sets, rotated, so that every step reads more than the L2 holds
+    # (126 MB) of data it has not just touched
+    probe = gi.make_inputs(cfg, gi.seed_for(cfg, 10 * rank))
+    set_bytes = sum(v.nbytes for v in probe.values() if isinstance(v, np.ndarray))
+    NSETS = int(min(16, max(2, -(-3 * L2_BYTES // set_bytes))))
+    host_sets = [probe] + [gi.make_inputs(cfg, gi.seed_for(cfg, 10 * rank + s)) for s in range(1, NSETS)]
     sets = []
     for inp in host_sets:
         t = {**attn_tensors(inp, dev), **accept_tensors(inp, dev)}
         t["out"] = torch.empty_like(t["q"])
         sets.append(t)
-    Lmax = host_sets[0]["Lmax"]
-    ws_bytes = gsd.gsd_verify_attn_workspace_bytes(cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.D,
-                                                   max(h["Lmax"] for h in host_sets),
+    Lmax = max(h["Lmax"] for h in host_sets)
+    if any(h["Lmax"] != Lmax for h in host_sets):
+        raise SystemExit("the rotated input sets must share one padded cache length")
+    ws_bytes = gsd.gsd_verify_attn_workspace_bytes(cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.D, Lmax,
                                                    args.num_splits, args.kernel)
     ws_attn = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=dev)
     ws_acc = torch.empty(gsd.gsd_accept_workspace_bytes(cfg.B, cfg.N), dtype=torch.uint8, device=dev)
@@ -283,56 +475,42 @@ def main():
     ms_per_step, value = agg["ms_per_step"], agg["value"]
     total_ms = ms_per_step * args.steps
 
-    # ---- the cache update that follows the step (gsd_commit_kv), timed on its own on a cache with
-    # head room; it is not part of `value`
-    commit_us = None
+    # ---- side timings on rank 0, each call between its own CUDA events; none is part of `value`
+    commit_us = sampled_us = draft_us = None
+    sampled_bytes = draft_bytes = 0.0
     if rank == 0:
+        # the cache update that follows the step (gsd_commit_kv) on a cache with head room
         t0s = sets[0]
         grow = cfg.depth + 1
-        kc2 = torch.cat([t0s["k_cache"], torch.zeros((cfg.B, grow, cfg.Hkv, cfg.D), dtype=torch.bfloat16, device=dev)], dim=1).contiguous()
-        vc2 = torch.cat([t0s["v_cache"], torch.zeros((cfg.B, grow, cfg.Hkv, cfg.D), dtype=torch.bfloat16, device=dev)], dim=1).contiguous()
+        pad = torch.zeros((cfg.B, grow, cfg.Hkv, cfg.D), dtype=torch.bfloat16, device=dev)
+        kc2 = torch.cat([t0s["k_cache"], pad], dim=1).contiguous()
+        vc2 = torch.cat([t0s["v_cache"], pad], dim=1).contiguous()
         sl0 = t0s["seq_lens"].clone()
         sl2 = sl0.clone()
-        ev_c = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(20)]
-        for i in range(23):
-            sl2.copy_(sl0)
-            if i >= 3:
-                ev_c[i - 3][0].record()
-            gsd.gsd_commit_kv(kc2, vc2, t0s["draft_k"], t0s["draft_v"], acc_out[2], acc_out[1], sl2, status=status)
-            if i >= 3:
-                ev_c[i - 3][1].record()
-        torch.cuda.synchronize()
-        commit_us = statistics.median(a.elapsed_time(b) for a, b in ev_c) * 1e3
-        del kc2, vc2
 
-    # ---- non-deterministic verification (gsd_accept_sampled) on the same logits, timed on its
-    # own with the two input sets rotated; it is not part of `value`
-    sampled_us = None
-    if rank == 0:
+        def commit(i):
+            gsd.gsd_commit_kv(kc2, vc2, t0s["draft_k"], t0s["draft_v"], acc_out[2], acc_out[1], sl2, status=status)
+        commit_us = timed_calls(commit, before=lambda i: sl2.copy_(sl0))
+        del kc2, vc2, pad
+
+        # non-deterministic verification (gsd_accept_sampled): the rotated logits as the target's,
+        # the next set's logits as the draft model's (one row per sequence is read for the residual)
         gen = torch.Generator(device=dev)
         gen.manual_seed(7)
         dq = torch.rand((cfg.B, cfg.N), device=dev, generator=gen) * 0.5 + 0.01
         ua = torch.rand((cfg.B, cfg.N), device=dev, generator=gen)
         usm = torch.rand((cfg.B,), device=dev, generator=gen)
         ws_s = torch.empty(gsd.gsd_accept_sampled_workspace_bytes(cfg.B, cfg.N), dtype=torch.uint8, device=dev)
-        ev_s = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(20)]
-        for i in range(23):
-            ts = sets[i % len(sets)]
-            if i >= 3:
-                ev_s[i - 3][0].record()
-            gsd.gsd_accept_sampled(ts["logits"], ts["draft_tokens"], ts["parent_ptr"], ts["parent_idx"], dq, ua, usm,
-                                   workspace=ws_s, status=status)
-            if i >= 3:
-                ev_s[i - 3][1].record()
-        torch.cuda.synchronize()
-        sampled_us = statistics.median(a.elapsed_time(b) for a, b in ev_s) * 1e3
 
-    # ---- one growth step of the draft token graph (gsd_draft_expand): 64 frontier rows per
-    # sequence of random draft logits over the same vocabulary, on a graph of 104 earlier nodes;
-    # timed on its own, not part of `value`
-    draft_us = None
-    if rank == 0:
-        gen = torch.Generator(device=dev)
+        def sampled(i):
+            ts, td = sets[i % NSETS], sets[(i + 1) % NSETS]
+            gsd.gsd_accept_sampled(ts["logits"], ts["draft_tokens"], ts["parent_ptr"], ts["parent_idx"], dq, ua, usm,
+                                   draft_logits=td["logits"], workspace=ws_s, status=status)
+        sampled_us = timed_calls(sampled)
+        sampled_bytes = 4.0 * cfg.V * (cfg.B * cfg.N + cfg.B)
+
+        # one growth step of the draft token graph (gsd_draft_expand): 64 frontier rows per
+        # sequence of random draft logits over the same vocabulary, on a graph of 104 earlier nodes
         gen.manual_seed(11)
         Fr, Ncap, n_old = 64, 512, 104
         dl = [torch.randn((cfg.B, Fr, cfg.V), device=dev, generator=gen) * 3 for _ in range(2)]
@@ -346,17 +524,12 @@ def main():
         g_n = n_ref.clone()
         fr = (torch.arange(Fr, device=dev, dtype=torch.int32) % n_old).repeat(cfg.B, 1).contiguous()
         fl = torch.full((cfg.B,), Fr, dtype=torch.int32, device=dev)
-        ev_d = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(20)]
-        for i in range(23):
-            g_n.copy_(n_ref)
-            if i >= 3:
-                ev_d[i - 3][0].record()
+
+        def draft(i):
             gsd.gsd_draft_expand(dl[i % 2], fr, fl, g_tok, g_par, g_mrg, g_leaf, g_prob, g_n, k=4, tau=2,
                                  theta_prob=0.01, theta_sib=0.1, status=status)
-            if i >= 3:
-                ev_d[i - 3][1].record()
-        torch.cuda.synchronize()
-        draft_us = statistics.median(a.elapsed_time(b) for a, b in ev_d) * 1e3
+        draft_us = timed_calls(draft, before=lambda i: g_n.copy_(n_ref))
+        draft_bytes = 4.0 * cfg.B * Fr * cfg.V
         del dl
 
     # ---- end to end through the host-buffer C-ABI call (pinned host tensors)
@@ -404,51 +577,43 @@ def main():
     attn_med = statistics.median(attn_ms) * 1e-3
     attn_mean = sum(attn_ms) / len(attn_ms) * 1e-3
     acc_mean = sum(acc_ms) / len(acc_ms) * 1e-3
-    t_tc = flops / (peaks["bf16_tflops_sustained"] * 1e12)
-    t_hbm = attn_bytes / (peaks["hbm_gbs"] * 1e9)
-    sustained = total_ms >= 2000.0
-    if t_tc >= t_hbm:
-        peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
-        achieved = flops / attn_mean / 1e12
-        roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": None,
-                "peak_kind": f"{'sustained' if sustained else 'burst'} bf16, of {peak_src}",
-                "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
-                "frac_of_burst": achieved / peaks["bf16_tflops"],
-                "frac_of_nominal_2250": achieved / 2250.0}
-    else:
-        peak = peaks["hbm_gbs"]
-        achieved = attn_bytes / attn_mean / 1e9
-        roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": None, "peak_kind": f"copy bandwidth, of {peak_src}",
-                "frac_of_nominal_8000": achieved / 8000.0}
-    # DRAM bytes of one launch of the dominant kernel from the committed ncu capture
-    # (profiles/attn_tcgen05_llama70b.md); only valid for that kernel on that workload
-    if cfg.name == "llama70b" and args.kernel in (0, 2) and args.num_splits == 0:
-        roof["traffic"] = 197.7e6
+    roof = roofline_of(flops, attn_bytes, attn_mean, peaks, peak_src)
     roof["kernel"] = "gsd_verify_attn" + (" (split pass + merge pass)" if splits > 1 else "")
-    roof["algorithmic_flops"] = flops
-    roof["algorithmic_bytes"] = attn_bytes
+    if args.kernel in (0, 2) and args.num_splits == 0:
+        # recorded only for workloads whose capture ran the tcgen05 kernel under the automatic choice
+        roof["traffic"] = recorded_traffic("attn_tc_kernel", cfg.name)
     roof["launch_us_mean"] = attn_mean * 1e6
     roof["launch_us_median"] = attn_med * 1e6
+    if clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz"):
+        # the same time scaled to the maximum SM clock (clock cycles are what the kernel costs)
+        roof["launch_us_mean_at_max_clock"] = attn_mean * 1e6 * clocks["sm_mhz"] / clocks["sm_max_mhz"]
 
     cpu = None
-    if args.cpu_rows > 0 and world == 1:
-        v, threads, desc = cpu_oracle_sample(cfg, host_sets[0], args.cpu_rows)
-        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+    mode = args.cpu_baseline
+    if mode == "auto":
+        mode = "full" if cfg.name in gi.CONFIGS else "sample"
+    if mode != "off" and world == 1:
+        total_rows = cfg.B * cfg.N * cfg.Hq
+        cpu = cpu_oracle_time(cfg, host_sets[0], total_rows if mode == "full" else 16384, 0)
 
+    hbm = peaks["hbm_gbs"]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "B": cfg.B, "N": cfg.N, "Hq": cfg.Hq, "Hkv": cfg.Hkv,
                    "D": cfg.D, "L": cfg.L, "V": cfg.V, "depth": cfg.depth,
-                   "l2": "two input sets rotated; each step reads more than the L2 size",
+                   "l2": (f"{NSETS} input sets of {set_bytes / 1e6:.0f} MB rotated"
+                          + ("; together larger than L2" if NSETS * set_bytes > 2 * L2_BYTES else
+                             "; together NOT larger than L2 (L2-warm numbers)")),
                    "replicas": world, "attn_kernel": args.kernel, "num_splits": splits},
-        "attn_us": attn_mean * 1e6, "accept_us": acc_mean * 1e6, "commit_kv_us": commit_us, "accept_sampled_us": sampled_us, "draft_expand_us": draft_us,
+        "attn_us": attn_mean * 1e6, "accept_us": acc_mean * 1e6, "commit_kv_us": commit_us,
+        "accept_sampled_us": sampled_us, "draft_expand_us": draft_us,
         "attn_tokens_per_s": tokens / attn_mean,
         "accept_gbs": accept_bytes / acc_mean / 1e9,
-        "accept_frac_of_hbm": accept_bytes / acc_mean / 1e9 / peaks["hbm_gbs"],
+        "accept_frac_of_hbm": accept_bytes / acc_mean / 1e9 / hbm,
+        "accept_sampled_frac_of_hbm": (sampled_bytes / (sampled_us * 1e-6) / 1e9 / hbm) if sampled_us else None,
+        "draft_expand_frac_of_hbm": (draft_bytes / (draft_us * 1e-6) / 1e9 / hbm) if draft_us else None,
         "roofline": roof, "cpu_baseline": cpu, "e2e": e2e,
         # per step: the attention kernel (+ its merge pass when key ranges are cut), the scratch
         # clear of gsd_accept and the accept kernel

@@ -14,7 +14,9 @@ they stand in for the paper's GSM8K / XSum / Alpaca / WMT-14 workloads, which ar
 used here.
 
 Everything is numpy; bf16 tensors are carried as uint16 bit patterns.
-Random numbers come from numpy's Philox counter-based generator keyed by the seed.
+Random numbers come from numpy's Philox counter-based generator keyed by the seed; the
+large tensors are drawn slice by slice from jumped copies of their stream, so several host
+threads can fill them and the values do not depend on the thread count.
 """
 from __future__ import annotations
 
@@ -300,10 +302,18 @@ def make_inputs(cfg: VerifyConfig, seed: int | None = None, *, attn: bool = True
         out["draft_k"] = _normal_bf16(seed, 7, (B, N, Hkv, D))
         out["draft_v"] = _normal_bf16(seed, 8, (B, N, Hkv, D))
     if accept:
-        g_log = _rng(seed, 10)
         logits = np.empty((B, N, V), dtype=np.float32)
-        for b in range(B):
-            logits[b] = g_log.standard_normal((N, V), dtype=np.float32)
+        base = np.random.Philox(key=[seed & 0xFFFFFFFFFFFFFFFF, 10])
+
+        def fill_logits(b: int) -> None:      # sequence b: the stream (seed, 10) jumped b times
+            np.random.Generator(base.jumped(b)).standard_normal((N, V), dtype=np.float32, out=logits[b])
+
+        if B > 1 and logits.size >= (1 << 22):
+            with ThreadPoolExecutor(max_workers=min(B, os.cpu_count() or 1)) as ex:
+                list(ex.map(fill_logits, range(B)))
+        else:
+            for b in range(B):
+                fill_logits(b)
         g_pl = _rng(seed, 11)
         for b in range(B):
             ch = children_of(parents_all[b])
