@@ -49,7 +49,7 @@ def _load() -> ctypes.CDLL:
         _lib.gsd_oracle_threads.restype = ctypes.c_int
         _lib.gsd_oracle_argmax_row.restype = ctypes.c_int32
         for name in ("gsd_oracle_attn", "gsd_oracle_attn_rows", "gsd_oracle_accept", "gsd_oracle_accept_sampled", "gsd_oracle_draft_expand",
-                     "gsd_oracle_commit_kv", "gsd_oracle_build_mask"):
+                     "gsd_oracle_commit_kv", "gsd_oracle_build_mask", "gsd_oracle_unmerge_tree"):
             getattr(_lib, name).restype = ctypes.c_int
         _lib.gsd_oracle_argmax.restype = None
     return _lib
@@ -229,3 +229,22 @@ def build_mask(parent_ptr, parent_idx) -> np.ndarray:
     if rc != 0:
         raise RuntimeError("oracle build_mask failed")
     return mask
+
+
+def unmerge_tree(draft_tokens, parent_ptr, parent_idx, Ucap: int, max_depth: int):
+    """The token graph unfolded into a tree, one node per root path (see gsd_oracle_unmerge_tree).
+    Returns (tree_tokens, tree_parent, tree_source [B,Ucap] padded with -1, tree_count [B],
+    out_of_capacity flag)."""
+    draft_tokens = _c(draft_tokens, np.int32); parent_ptr = _c(parent_ptr, np.int32)
+    parent_idx = _c(parent_idx, np.int32)
+    B, N = draft_tokens.shape
+    assert parent_ptr.shape == (B, N + 1)
+    tt = np.zeros((B, Ucap), dtype=np.int32); tp = np.zeros((B, Ucap), dtype=np.int32)
+    ts = np.zeros((B, Ucap), dtype=np.int32); cnt = np.zeros((B,), dtype=np.int32)
+    rc = _load().gsd_oracle_unmerge_tree(_p(draft_tokens), _p(parent_ptr), _p(parent_idx), ctypes.c_int32(B),
+                                         ctypes.c_int32(N), ctypes.c_int32(parent_idx.shape[1]),
+                                         ctypes.c_int32(Ucap), ctypes.c_int32(max_depth), _p(tt), _p(tp), _p(ts),
+                                         _p(cnt))
+    if rc < 0:
+        raise ValueError("oracle unmerge_tree: malformed input")
+    return tt, tp, ts, cnt, bool(rc)

@@ -634,3 +634,58 @@ int gsd_oracle_build_mask(const int32_t *parent_ptr, const int32_t *parent_idx, 
     free(todo);
     return 0;
 }
+
+/*
+ * Unmerging the token graph into a tree (Sec. 5.4, Fig. 4: before verification the graph is
+ * reverted to a tree; the successors of every redundant node are replicated from the node it was
+ * merged into, and the tree is then verified as in tree-structured decoding).  In terms of the
+ * verification DAG (parent lists; a node merged into f has f's children as its own) this is the
+ * unfolding of the DAG from the root: one tree node per root path.  Readings: tree nodes are
+ * numbered level by level, inside a level by (tree index of the parent, then id of the copied DAG
+ * node), so a parent always precedes its children; a repeating pattern makes the unfolding
+ * endless, so it is cut at max_depth edges from the root; when Ucap nodes have been created
+ * the rest is dropped (return value 1).
+ *
+ * draft_tokens [B,N]; parent_ptr [B,N+1]; parent_idx [B,Ecap] (parents below their child);
+ * tree_tokens, tree_parent (tree index of the parent, -1 for the root), tree_source (the DAG
+ * node a tree node copies) [B,Ucap], unused entries -1; tree_count [B].
+ * Returns 0, 1 if some sequence ran out of capacity, -1 on malformed input.
+ */
+int gsd_oracle_unmerge_tree(const int32_t *draft_tokens, const int32_t *parent_ptr,
+                            const int32_t *parent_idx, int32_t B, int32_t N, int32_t Ecap,
+                            int32_t Ucap, int32_t max_depth, int32_t *tree_tokens,
+                            int32_t *tree_parent, int32_t *tree_source, int32_t *tree_count)
+{
+    int rc = 0;
+    if (N < 1 || Ucap < 1 || max_depth < 0) return -1;
+    int *depth = (int *)malloc(sizeof(int) * (size_t)Ucap);
+    if (!depth) return -1;
+    for (int b = 0; b < B; ++b) {
+        const int32_t *tok = draft_tokens + (size_t)b * N;
+        const int32_t *pp = parent_ptr + (size_t)b * (N + 1);
+        const int32_t *pi = parent_idx + (size_t)b * Ecap;
+        int32_t *tt = tree_tokens + (size_t)b * Ucap, *tp = tree_parent + (size_t)b * Ucap;
+        int32_t *ts = tree_source + (size_t)b * Ucap;
+        for (int u = 0; u < Ucap; ++u) tt[u] = tp[u] = ts[u] = -1;
+        for (int v = 0; v < N; ++v)
+            for (int e = pp[v]; e < pp[v + 1]; ++e)
+                if (pi[e] < 0 || pi[e] >= v) { free(depth); return -1; }
+        int count = 1;
+        tt[0] = tok[0]; tp[0] = -1; ts[0] = 0; depth[0] = 0;
+        /* tree nodes are expanded in the order they were created (a queue): level order */
+        for (int u = 0; u < count; ++u) {
+            if (depth[u] >= max_depth) continue;
+            for (int v = 0; v < N; ++v) {          /* children of the copied node, ascending id */
+                int is_child = 0;
+                for (int e = pp[v]; e < pp[v + 1]; ++e) is_child |= (pi[e] == ts[u]);
+                if (!is_child) continue;
+                if (count >= Ucap) { rc = 1; continue; }
+                tt[count] = tok[v]; tp[count] = u; ts[count] = v; depth[count] = depth[u] + 1;
+                ++count;
+            }
+        }
+        tree_count[b] = count;
+    }
+    free(depth);
+    return rc;
+}

@@ -68,3 +68,36 @@ def dp_longest_accepted(tok, amax, parents):
         path.append(min(p for p in parents[v]
                         if best[p] == best[v] - 1 and tok[v] == amax[p]))
     return path[::-1]
+
+
+def verification_parents(tree_parent, merge_to, n):
+    """Parent lists of the verification DAG of a grown token graph: a node reaches the children
+    of its tree parent's merged copies too, i.e. parents(x) = {tree_parent[x]} + {r : merge_to[r]
+    == tree_parent[x]} (sorted; node 0 is the root)."""
+    merged_into = {}
+    for r in range(n):
+        if merge_to[r] >= 0:
+            merged_into.setdefault(int(merge_to[r]), []).append(r)
+    parents = [[]]
+    for x in range(1, n):
+        p = int(tree_parent[x])
+        parents.append(sorted([p] + [r for r in merged_into.get(p, []) if r < x]))
+    return parents
+
+
+def root_paths(parents, max_depth):
+    """Every root path (as a tuple of node ids) of a DAG given by parent lists, up to max_depth
+    edges, by explicit depth-first enumeration over child lists."""
+    n = len(parents)
+    children = [[] for _ in range(n)]
+    for v, ps in enumerate(parents):
+        for p in ps:
+            children[p].append(v)
+    out, stack = [], [(0,)]
+    while stack:
+        path = stack.pop()
+        out.append(path)
+        if len(path) - 1 < max_depth:
+            for c in children[path[-1]]:
+                stack.append(path + (c,))
+    return out

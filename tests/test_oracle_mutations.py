@@ -62,6 +62,13 @@ MUTATIONS = [
      "for (int e = c - 1; e >= 0; --e)\n                if (same_gram(tok, par, c, e, tau))", "test_oracle_draft.py"),
     ("draft_short_paths_count", "if (a < 0 || b < 0) return 0;          /* a path shorter than tau */",
      "if (a < 0 || b < 0) return a < 0 && b < 0;", "test_oracle_draft.py"),
+    ("unmerge_children_descending", "for (int v = 0; v < N; ++v) {          /* children of the copied node, ascending id */",
+     "for (int v = N - 1; v >= 0; --v) {", "test_oracle_unmerge.py"),
+    ("unmerge_parent_is_the_source", "tp[count] = u;", "tp[count] = ts[u];", "test_oracle_unmerge.py"),
+    ("unmerge_depth_off_by_one", "if (depth[u] >= max_depth) continue;", "if (depth[u] > max_depth) continue;",
+     "test_oracle_unmerge.py"),
+    ("unmerge_token_of_the_parent", "tt[count] = tok[v]; tp[count] = u;", "tt[count] = tok[ts[u]]; tp[count] = u;",
+     "test_oracle_unmerge.py"),
     ("mask_without_self", "row[v / 32] |= 1u << (v % 32);", "if (v != n) row[v / 32] |= 1u << (v % 32);",
      "test_oracle_mask.py"),
     ("mask_parents_only", "seen[p] = 1;\n                    todo[top++] = p;", "seen[p] = 1;\n                    if (v == n) todo[top++] = p;",
