@@ -60,6 +60,8 @@ typedef enum gsd_status {
 #define GSD_DEV_DRAFT_FULL   0x80u /* gsd_draft_expand: the node capacity was reached; the remaining children were not created */
 #define GSD_DEV_BAD_FRONTIER 0x100u /* gsd_draft_expand: frontier_len, num_nodes or a frontier node id out of range */
 
+#define GSD_DEV_TREE_FULL    0x200u /* gsd_unmerge_tree: the tree capacity was reached; the rest of the level order was dropped */
+
 #define GSD_MAX_NODES 512          /* largest supported N (draft nodes per sequence) */
 
 /* kernel selection for gsd_verify_attn */
@@ -320,6 +322,37 @@ int gsd_accept_static(const float* logits, const int32_t* draft_tokens, const in
  */
 int gsd_build_mask(const int32_t* parent_ptr, const int32_t* parent_idx, uint32_t* ancestor_mask,
                    int32_t B, int32_t N, int32_t Ecap, int32_t* status, void* stream);
+
+/*
+ * gsd_unmerge_tree - the token graph reverted to a tree for verification (Sec. 5.4, Fig. 4: before
+ * verification the merged nodes are "unmerged": the successors of a redundant node are replicated
+ * from the node it was merged into, and the tree is verified as in tree-structured decoding).
+ * On the verification DAG, given by parent lists, this is its unfolding from the root: one tree
+ * node per root path.  The tree can then be fed to gsd_build_mask / gsd_verify_attn / gsd_accept
+ * (gather q, draft K/V and logits rows by tree_source) as an alternative to verifying the DAG
+ * directly.
+ *
+ *   tree node 0 is the root.  Tree nodes are numbered level by level, inside a level by (tree
+ *   index of the parent, then id of the copied DAG node), so a parent precedes its children.
+ *   Nodes deeper than max_depth edges below the root are not created (a merge pattern that
+ *   repeats along one path could otherwise unfold without end); when Ucap nodes exist the rest
+ *   of the level order is dropped (GSD_DEV_TREE_FULL).
+ *
+ *   draft_tokens  [B, N] int32 device in      parent_ptr [B, N+1], parent_idx [B, Ecap] int32
+ *                 device in, as for gsd_accept (at most GSD_UNMERGE_MAX_EDGES edges per sequence
+ *                 are read; a parent listed twice in one row counts once)
+ *   tree_tokens, tree_parent, tree_source  [B, Ucap] int32 device out: token, tree index of the
+ *                 parent (-1 for the root) and copied DAG node of every tree node; -1 past the end
+ *   tree_count    [B] int32 device out: tree nodes created
+ *   status        device int32 word or NULL (GSD_DEV_BAD_CSR, GSD_DEV_TREE_FULL);  stream: cudaStream_t
+ *
+ * N <= GSD_MAX_NODES.  No workspace, no allocation, asynchronous on `stream`.
+ */
+#define GSD_UNMERGE_MAX_EDGES 4096
+int gsd_unmerge_tree(const int32_t* draft_tokens, const int32_t* parent_ptr, const int32_t* parent_idx,
+                     int32_t* tree_tokens, int32_t* tree_parent, int32_t* tree_source, int32_t* tree_count,
+                     int32_t B, int32_t N, int32_t Ecap, int32_t Ucap, int32_t max_depth, int32_t* status,
+                     void* stream);
 
 typedef struct gsd_commit_params {
     int32_t B;     /* sequences */

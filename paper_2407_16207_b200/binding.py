@@ -54,7 +54,7 @@ EXPORTS = ["gsd_version", "gsd_status_string", "gsd_last_cuda_error", "gsd_verif
            "gsd_verify_attn_workspace_bytes", "gsd_verify_attn_num_splits", "gsd_accept",
            "gsd_accept_workspace_bytes", "gsd_accept_static", "gsd_accept_sampled",
            "gsd_accept_sampled_workspace_bytes", "gsd_draft_expand", "gsd_draft_expand_workspace_bytes",
-           "gsd_commit_kv", "gsd_build_mask", "gsd_verify_step_host",
+           "gsd_commit_kv", "gsd_build_mask", "gsd_unmerge_tree", "gsd_verify_step_host",
            "gsd_verify_step_host_arena_bytes"]
 
 
@@ -95,6 +95,8 @@ def lib() -> ctypes.CDLL:
         L.gsd_accept_static.argtypes = [vp] * 7 + [ctypes.POINTER(AcceptParams), vp, vp]
         L.gsd_build_mask.restype = i32
         L.gsd_build_mask.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp]
+        L.gsd_unmerge_tree.restype = i32
+        L.gsd_unmerge_tree.argtypes = [vp] * 7 + [ctypes.c_int32] * 5 + [vp, vp]
         L.gsd_commit_kv.restype = i32
         L.gsd_commit_kv.argtypes = [vp] * 7 + [ctypes.POINTER(CommitParams), vp, vp]
         L.gsd_accept_workspace_bytes.restype = sz
@@ -339,6 +341,28 @@ def gsd_build_mask(parent_ptr, parent_idx, out: Optional[torch.Tensor] = None, *
         _check(lib().gsd_build_mask(parent_ptr.data_ptr(), parent_idx.data_ptr(), out.data_ptr(),
                                     B, N, Ecap, _ptr(status), _stream(parent_ptr)))
     return out
+
+
+def gsd_unmerge_tree(draft_tokens, parent_ptr, parent_idx, *, Ucap: int, max_depth: int,
+                     status: Optional[torch.Tensor] = None
+                     ) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor, torch.Tensor]:
+    """The token graph unfolded into a tree (one node per root path); see gsd_unmerge_tree in
+    include/gsd.h.  Returns (tree_tokens, tree_parent, tree_source [B,Ucap], tree_count [B])."""
+    B, N = draft_tokens.shape
+    Ecap = parent_idx.shape[1]
+    _want(draft_tokens, torch.int32, (B, N), "draft_tokens", True)
+    _want(parent_ptr, torch.int32, (B, N + 1), "parent_ptr", True)
+    _want(parent_idx, torch.int32, (B, Ecap), "parent_idx", True)
+    dev = draft_tokens.device
+    tt = torch.empty((B, Ucap), dtype=torch.int32, device=dev)
+    tp = torch.empty((B, Ucap), dtype=torch.int32, device=dev)
+    ts = torch.empty((B, Ucap), dtype=torch.int32, device=dev)
+    cnt = torch.empty((B,), dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        _check(lib().gsd_unmerge_tree(draft_tokens.data_ptr(), parent_ptr.data_ptr(), parent_idx.data_ptr(),
+                                      tt.data_ptr(), tp.data_ptr(), ts.data_ptr(), cnt.data_ptr(), B, N, Ecap,
+                                      int(Ucap), int(max_depth), _ptr(status), _stream(draft_tokens)))
+    return tt, tp, ts, cnt
 
 
 def gsd_commit_kv(k_cache, v_cache, draft_k, draft_v, accepted_nodes, accepted_len, seq_lens, *,
