@@ -9,13 +9,14 @@
 // model's distribution there) when drafted continuations of the end node were rejected, that of
 // P itself when the end node is a leaf of the graph or no draft logits are given.
 //
-// One launch.  Grid (slices, B*N): each CTA streams one slice of one logits row with 16-byte
+// Two launches.  Grid (slices, B*N): each CTA streams one slice of one logits row with 16-byte
 // loads; each of its warps owns a contiguous eighth of the slice and keeps a running
-// (maximum, sum of exponentials) pair, which it leaves in scratch.  The CTA that finishes last
-// for a sequence combines the pairs per node, tests the steps, runs the level-synchronous
-// longest-path relaxation, walks back, and finds the regenerated token: the range sums in
-// scratch (for the residual: range sums formed on the spot from the two rows of the end node)
-// give the range of the crossing, a block-wide scan over that range gives the index.
+// (maximum, sum of exponentials) pair, which it leaves in scratch.  The second launch (one CTA
+// per sequence, a programmatic dependent of the first, so it is resident when the stream ends)
+// combines the pairs per node, tests the steps, runs the level-synchronous longest-path
+// relaxation, walks back, and finds the regenerated token: range sums (for P those in scratch;
+// for the residual eight range sums formed on the spot from the two rows of the end node) give
+// the range of the crossing, a block-wide scan over that range gives the index.
 #include "gsd_internal.cuh"
 #include "gsd_path.cuh"
 #include <math_constants.h>
@@ -93,18 +94,20 @@ struct SampledArgs {
     int32_t* out_len;
     int32_t* out_nodes;
     float2* part;     // [B*N][slices][kWarps] (maximum, sum) of contiguous ranges of the row, in order
-    unsigned* done;   // [B], zeroed before the launch
     int32_t* status;
     int B, N, V, Ecap, Tcap, slices;
     int vec;          // rows are read as float4 (decides where the slices of a row begin)
+    int dvec;         // the rows of the draft logits can be read as float4 too
 };
 
 __device__ void finish_sequence(const SampledArgs& a, int b) {
     __shared__ float s_mx[GSD_MAX_NODES];
     __shared__ float s_sum[GSD_MAX_NODES];
+    __shared__ float s_uq[GSD_MAX_NODES];
     __shared__ int s_red[kThreads / 32];
     __shared__ float s_scan[kThreads / 32];
     __shared__ float s_rm[kThreads / 32];
+    __shared__ float s_rsum[kMaxSlices * kWarps];
     __shared__ int s_pick;
     const int N = a.N, V = a.V, tid = threadIdx.x;
     const int32_t* tok = a.tok + (size_t)b * N;
@@ -115,12 +118,20 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     for (int v = tid; v < N; v += kThreads) {
         // the pairs were written by other CTAs: read them past L1
         Ms r{-CUDART_INF_F, 0.f};
-        for (int k = 0; k < a.slices * kWarps; ++k) {
-            const float2 p = __ldcg(a.part + ((size_t)b * N + v) * a.slices * kWarps + k);
-            r = combine(r, Ms{p.x, p.y});
+        const float4* pp = reinterpret_cast<const float4*>(a.part + ((size_t)b * N + v) * a.slices * kWarps);
+        for (int k = 0; k < a.slices * (kWarps / 2); k += 4) {     // eight pairs (64 bytes) per round, loaded at once
+            float4 t[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) t[i] = __ldcg(pp + k + i);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                r = combine(r, Ms{t[i].x, t[i].y});
+                r = combine(r, Ms{t[i].z, t[i].w});
+            }
         }
         s_mx[v] = r.m;
         s_sum[v] = r.s;
+        s_uq[v] = u[v] * q[v];       // the left side of the step test, fetched beside the pairs
         if (!(r.s > 0.f) || r.m == CUDART_INF_F) flags |= GSD_DEV_BAD_LOGITS;   // no finite entry, +inf or NaN
     }
     __syncthreads();
@@ -137,7 +148,7 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     // logit gathered from global memory) against u q
     const PathResult res = longest_accepted_path<true>(io, flags, [&](int p, int v) {
         const float prob = ex2((lg[(size_t)p * V + tok[v]] - s_mx[p]) * kLog2e) / s_sum[p];
-        return u[v] * q[v] < prob;
+        return s_uq[v] < prob;
     });
     const int s_m = res.edges, s_end = res.end;
     int32_t* out_tok = io.out_tok;
@@ -158,47 +169,99 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     bool residual = false;
     float q_m = 0.f, inv_sp = 0.f, inv_sq = 0.f, res_total = 0.f;
     const float* y = nullptr;
-    if (a.dlogits) {
-        if (res.end_has_child) {
-            y = a.dlogits + ((size_t)b * N + s_end) * V;
-            Ms r{-CUDART_INF_F, 0.f};
+    // both rows readable as float4 (decides where the residual's ranges begin)
+    const bool rvec = a.vec && a.dvec;
+    const int runit = rvec ? 4 : 1, rn = rvec ? (V >> 2) : V;
+    const int rper = (rn + kWarps - 1) / kWarps;
+    if (a.dlogits && res.end_has_child) {
+        y = a.dlogits + ((size_t)b * N + s_end) * V;
+        // softmax statistics of the draft row: the row comes from DRAM, so every thread keeps
+        // sixteen 16-byte loads in flight (a 32000-entry row is two trips to memory)
+        Ms r{-CUDART_INF_F, 0.f};
+        if (a.dvec) {
+            const float4* y4 = reinterpret_cast<const float4*>(y);
+            const int n4 = V >> 2;
+            const float4 none = make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
+            for (int i = tid; i < n4; i += 16 * kThreads) {
+                float4 t[16];
+#pragma unroll
+                for (int k = 0; k < 16; ++k) t[k] = i + k * kThreads < n4 ? __ldg(y4 + i + k * kThreads) : none;
+#pragma unroll
+                for (int k = 0; k < 16; k += 4) take16(r, t[k], t[k + 1], t[k + 2], t[k + 3]);
+            }
+        } else {
             for (int j = tid; j < V; j += kThreads) take1(r, __ldg(y + j));
+        }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                Ms t;
-                t.m = __shfl_xor_sync(0xFFFFFFFFu, r.m, o);
-                t.s = __shfl_xor_sync(0xFFFFFFFFu, r.s, o);
-                r = combine(r, t);
-            }
-            if (lane == 0) { s_rm[warp] = r.m; s_scan[warp] = r.s; }
-            __syncthreads();
-            r = Ms{-CUDART_INF_F, 0.f};
-            for (int w = 0; w < kWarps; ++w) r = combine(r, Ms{s_rm[w], s_scan[w]});
-            __syncthreads();
-            if (!(r.s > 0.f) || r.m == CUDART_INF_F) {
-                if (tid == 0 && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
+        for (int o = 16; o > 0; o >>= 1) {
+            Ms t;
+            t.m = __shfl_xor_sync(0xFFFFFFFFu, r.m, o);
+            t.s = __shfl_xor_sync(0xFFFFFFFFu, r.s, o);
+            r = combine(r, t);
+        }
+        if (lane == 0) { s_rm[warp] = r.m; s_scan[warp] = r.s; }
+        __syncthreads();
+        r = Ms{-CUDART_INF_F, 0.f};
+        for (int w = 0; w < kWarps; ++w) r = combine(r, Ms{s_rm[w], s_scan[w]});
+        __syncthreads();
+        if (!(r.s > 0.f) || r.m == CUDART_INF_F) {
+            if (tid == 0 && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
+        } else {
+            q_m = r.m;
+            inv_sp = 1.f / s_sum[s_end];
+            inv_sq = 1.f / r.s;
+            auto res1 = [&](float xv, float yv) -> float {
+                return fmaxf(ex2((xv - mx) * kLog2e) * inv_sp - ex2((yv - q_m) * kLog2e) * inv_sq, 0.f);
+            };
+            // range sums of the residual: warp w takes the w-th eighth of the row
+            const int w0 = min(warp * rper, rn), w1 = min(w0 + rper, rn);
+            float part = 0.f;
+            if (rvec) {
+                const float4* x4 = reinterpret_cast<const float4*>(x);
+                const float4* y4 = reinterpret_cast<const float4*>(y);
+                const float4 none = make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
+                for (int i = w0 + lane; i < w1; i += 8 * 32) {
+                    float4 xv[8], yv[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const bool in = i + k * 32 < w1;
+                        xv[k] = in ? __ldg(x4 + i + k * 32) : none;
+                        yv[k] = in ? __ldg(y4 + i + k * 32) : none;
+                    }
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        part += (res1(xv[k].x, yv[k].x) + res1(xv[k].y, yv[k].y)) + (res1(xv[k].z, yv[k].z) + res1(xv[k].w, yv[k].w));
+                }
             } else {
-                q_m = r.m;
-                inv_sp = 1.f / s_sum[s_end];
-                inv_sq = 1.f / r.s;
-                const int per = (V + kWarps - 1) / kWarps;
-                const int w0 = min(warp * per, V), w1 = min(w0 + per, V);
-                float part = 0.f;
-                for (int j = w0 + lane; j < w1; j += 32)
-                    part += fmaxf(ex2((x[j] - mx) * kLog2e) * inv_sp - ex2((y[j] - q_m) * kLog2e) * inv_sq, 0.f);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
-                if (lane == 0) s_scan[warp] = part;
-                __syncthreads();
-                for (int w = 0; w < kWarps; ++w) res_total += s_scan[w];
-                // a residual without mass (the two distributions agree to rounding) leaves P
-                residual = res_total > kResidualFloor;
+                for (int j = w0 + lane; j < w1; j += 32) part += res1(x[j], y[j]);
             }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+            if (lane == 0) s_scan[warp] = part;
+            __syncthreads();
+            for (int w = 0; w < kWarps; ++w) res_total += s_scan[w];
+            // a residual without mass (the two distributions agree to rounding) leaves P
+            residual = res_total > kResidualFloor;
         }
     }
-    auto weight = [&](int j) -> float {
-        const float e = ex2((x[j] - mx) * kLog2e);
-        return residual ? fmaxf(e * inv_sp - ex2((y[j] - q_m) * kLog2e) * inv_sq, 0.f) : e;
+    // weight of one entry from its two logits (-inf stands for "past the end": weight 0)
+    auto weight = [&](float xv, float yv) -> float {
+        const float e = ex2((xv - mx) * kLog2e);
+        return residual ? fmaxf(e * inv_sp - ex2((yv - q_m) * kLog2e) * inv_sq, 0.f) : e;
+    };
+    // sixteen consecutive entries of a row, all loads issued before any is used
+    auto load16 = [&](const float* row, bool vec16, int j, int jend, float (&v)[16]) {
+        if (vec16 && (j & 3) == 0 && j + 16 <= jend) {
+            const float4* r4 = reinterpret_cast<const float4*>(row + j);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float4 t = r4[k];
+                v[4 * k] = t.x; v[4 * k + 1] = t.y; v[4 * k + 2] = t.z; v[4 * k + 3] = t.w;
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < 16; ++k) v[k] = j + k < jend ? row[j + k] : -CUDART_INF_F;
+        }
     };
     const float target = a.us[b] * (residual ? res_total : s_sum[s_end]);
     // every thread walks the range sums: the first range whose inclusive prefix exceeds the
@@ -206,17 +269,19 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     int rsel = -1, last_r = 0;
     float before_range = 0.f, before_last = 0.f;
     {
-        float run = 0.f;
         const int nr = residual ? kWarps : a.slices * kWarps;
-        const float2* pr = a.part + ((size_t)b * N + s_end) * a.slices * kWarps;
-        for (int r = 0; r < nr; ++r) {
-            float sr;
+        if (tid < nr) {          // one range sum per thread, brought to the row's maximum
             if (residual) {
-                sr = s_scan[r];
+                s_rsum[tid] = s_scan[tid];
             } else {
-                const float2 t = __ldcg(pr + r);
-                sr = t.x == -CUDART_INF_F ? 0.f : t.y * ex2((t.x - mx) * kLog2e);
+                const float2 t = __ldcg(a.part + ((size_t)b * N + s_end) * a.slices * kWarps + tid);
+                s_rsum[tid] = t.x == -CUDART_INF_F ? 0.f : t.y * ex2((t.x - mx) * kLog2e);
             }
+        }
+        __syncthreads();
+        float run = 0.f;
+        for (int r = 0; r < nr; ++r) {
+            const float sr = s_rsum[r];
             if (rsel < 0 && run + sr > target) { rsel = r; before_range = run; }
             if (sr > 0.f) { last_r = r; before_last = run; }
             run += sr;
@@ -228,9 +293,8 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     if (tid == 0) s_pick = kNone;
     int r0, r1;
     if (residual) {
-        const int per = (V + kWarps - 1) / kWarps;
-        r0 = min(rsel * per, V);
-        r1 = min(r0 + per, V);
+        r0 = min(rsel * rper, rn) * runit;
+        r1 = min(rsel * rper + rper, rn) * runit;
     } else {
         range_of(V, a.slices, a.vec, rsel, r0, r1);
     }
@@ -238,10 +302,16 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     const int j0 = min(r0 + tid * per, r1), j1 = min(j0 + per, r1);
     float piece = 0.f;
     int last_pos = -1;
-    for (int j = j0; j < j1; ++j) {
-        const float e = weight(j);
-        piece += e;
-        if (e > 0.f) last_pos = j;
+    for (int c0 = j0; c0 < j1; c0 += 16) {
+        float xv[16], yv[16];
+        load16(x, a.vec != 0, c0, j1, xv);
+        if (residual) load16(y, a.dvec != 0, c0, j1, yv);
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const float e = weight(xv[k], residual ? yv[k] : 0.f);
+            piece += e;
+            if (e > 0.f) last_pos = c0 + k;
+        }
     }
     float inc = piece;
 #pragma unroll
@@ -269,9 +339,15 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     if (tid == first) {
         float cum = before;
         int pick = -1;
-        for (int j = j0; j < j1; ++j) {
-            cum += weight(j);
-            if (cum > target) { pick = j; break; }
+        for (int c0 = j0; c0 < j1 && pick < 0; c0 += 16) {
+            float xv[16], yv[16];
+            load16(x, a.vec != 0, c0, j1, xv);
+            if (residual) load16(y, a.dvec != 0, c0, j1, yv);
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                cum += weight(xv[k], residual ? yv[k] : 0.f);
+                if (pick < 0 && cum > target) pick = c0 + k;
+            }
         }
         s_pick = pick;                  // -1: the serial sum stayed at or below the target
     }
@@ -290,9 +366,12 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     }
 }
 
+// First launch: one CTA per (slice, row) streams its part of the row and leaves the warps'
+// (maximum, sum) pairs in scratch.
 template <bool kVec>
 __global__ void __launch_bounds__(kThreads) accept_sampled_kernel(SampledArgs a) {
-    __shared__ int s_last;
+    // the per-sequence pass (a programmatic dependent launch) may become resident as CTAs retire
+    if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int row = blockIdx.y;  // b * N + n
     const int slice = blockIdx.x;
     const float* x = a.logits + (size_t)row * a.V;
@@ -325,20 +404,13 @@ __global__ void __launch_bounds__(kThreads) accept_sampled_kernel(SampledArgs a)
         r = combine(r, t);
     }
     if (lane == 0) a.part[((size_t)row * a.slices + slice) * kWarps + warp] = make_float2(r.m, r.s);
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const int b = row / a.N;
-        // the counters are zeroed by the launch before this one; everything above ran beside it
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        const unsigned prev = atomicAdd(a.done + b, 1u);
-        s_last = (prev == (unsigned)(a.N * a.slices) - 1u);
-    }
-    __syncthreads();
-    if (s_last) {
-        __threadfence();
-        finish_sequence(a, row / a.N);
-    }
+}
+
+// Second launch: one CTA per sequence does the rest (statistics per node, step tests, longest
+// path, regenerated token) once every pair of the first launch is visible.
+__global__ void __launch_bounds__(kThreads, 1) accept_sampled_tail_kernel(SampledArgs a) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    finish_sequence(a, blockIdx.x);
 }
 
 int pick_slices(long rows, int V, int sm_count) {
@@ -354,7 +426,7 @@ int pick_slices(long rows, int V, int sm_count) {
 
 extern "C" size_t gsd_accept_sampled_workspace_bytes(const gsd_accept_params* p) {
     if (!p || p->B < 1 || p->N < 1 || p->N > GSD_MAX_NODES) return 0;
-    return gsd::align_up((size_t)p->B * p->N * gsd::kMaxSlices * gsd::kWarps * 8 + (size_t)p->B * 4, 256);
+    return gsd::align_up((size_t)p->B * p->N * gsd::kMaxSlices * gsd::kWarps * 8, 256);
 }
 
 extern "C" int gsd_accept_sampled(const float* logits, const int32_t* draft_tokens,
@@ -385,19 +457,15 @@ extern "C" int gsd_accept_sampled(const float* logits, const int32_t* draft_toke
     a.q = draft_q; a.u = u_accept; a.us = u_sample;
     a.out_tok = accepted_tokens; a.out_len = accepted_len; a.out_nodes = accepted_nodes;
     a.part = (float2*)workspace;
-    const size_t part_bytes = (size_t)p->B * p->N * kMaxSlices * kWarps * 8;
-    a.done = (unsigned*)((char*)workspace + part_bytes);
     a.status = status;
     a.B = p->B; a.N = p->N; a.V = p->V; a.Ecap = p->Ecap; a.Tcap = p->Tcap;
     const bool vec = (p->V % 4 == 0) && (((uintptr_t)logits & 15u) == 0);
     a.slices = pick_slices((long)p->B * p->N, p->V, di.sm_count);
     a.vec = vec ? 1 : 0;
+    a.dvec = (draft_logits && (p->V % 4 == 0) && (((uintptr_t)draft_logits & 15u) == 0)) ? 1 : 0;
 
-    // only the completion counters have to start at zero; every pair is written before it is read
-    if (launch_clear_words(a.done, p->B, st) != GSD_OK) return GSD_ERR_CUDA;
-    cudaLaunchAttribute attr[1];
-    dependent_launch_attr(attr);
-    // grid.y holds at most 65535 rows: larger problems go out in blocks of whole sequences
+    // every pair is written before it is read: nothing in the scratch has to start at zero.
+    // grid.y holds at most 65535 rows: larger problems go out in blocks of whole sequences.
     const int seq_per = 65535 / p->N;
     for (int b0 = 0; b0 < p->B; b0 += seq_per) {
         const int nb = (p->B - b0 < seq_per) ? p->B - b0 : seq_per;
@@ -408,15 +476,20 @@ extern "C" int gsd_accept_sampled(const float* logits, const int32_t* draft_toke
         s.q += (size_t)b0 * p->N; s.u += (size_t)b0 * p->N; s.us += b0;
         s.out_tok += (size_t)b0 * p->Tcap; s.out_len += b0;
         if (s.out_nodes) s.out_nodes += (size_t)b0 * p->Tcap;
-        s.part += (size_t)b0 * p->N * a.slices * kWarps; s.done += b0; s.B = nb;
+        s.part += (size_t)b0 * p->N * a.slices * kWarps; s.B = nb;
+        const dim3 grid(a.slices, (unsigned)(nb * p->N));
+        if (vec) accept_sampled_kernel<true><<<grid, kThreads, 0, st>>>(s);
+        else accept_sampled_kernel<false><<<grid, kThreads, 0, st>>>(s);
+        GSD_CUDA_TRY(cudaGetLastError());
+        cudaLaunchAttribute attr[1];
+        dependent_launch_attr(attr);
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(a.slices, (unsigned)(nb * p->N));
+        cfg.gridDim = dim3((unsigned)nb);
         cfg.blockDim = dim3(kThreads);
         cfg.stream = st;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        if (vec) GSD_CUDA_TRY(cudaLaunchKernelEx(&cfg, accept_sampled_kernel<true>, s));
-        else GSD_CUDA_TRY(cudaLaunchKernelEx(&cfg, accept_sampled_kernel<false>, s));
+        GSD_CUDA_TRY(cudaLaunchKernelEx(&cfg, accept_sampled_tail_kernel, s));
     }
     GSD_CUDA_TRY(cudaGetLastError());
     return GSD_OK;

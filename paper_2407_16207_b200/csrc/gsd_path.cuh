@@ -5,6 +5,12 @@
 // best[v] = 1 + max over accepted steps into v, choice of the end node (longest, then lowest
 // index), walk back (lowest predecessor that carries length - 1), emission of the path's node
 // ids and drafted tokens.  The token the target model contributes at the end is the caller's.
+//
+// The pass runs on one SM while the rest of the device may already be idle, so it is laid out
+// for few dependent trips to memory: tokens, row pointers and the parent indices are fetched in
+// one go; the relaxation costs one barrier per round (two copies of best[]); every node picks
+// its predecessor in parallel, after which the walk back is a pointer chase in shared memory
+// and the outputs are written by the whole block.
 #pragma once
 #include "gsd_internal.cuh"
 
@@ -40,22 +46,25 @@ struct PathResult {
 // entries past it are set to -1.
 template <bool kCacheOutcome, class StepOk>
 __device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, StepOk step_ok) {
-    __shared__ int s_best[GSD_MAX_NODES];
+    __shared__ int s_best[2][GSD_MAX_NODES];      // two copies: a round reads one and writes the other
     __shared__ int s_tok[GSD_MAX_NODES];
     __shared__ int s_ptr[GSD_MAX_NODES + 1];
     __shared__ int s_edge[kPathEdgeCache];
     __shared__ unsigned char s_eok[kPathEdgeCache];
     __shared__ short s_enode[kPathEdgeCache];   // the node a step leads into
+    __shared__ short s_path[GSD_MAX_NODES];     // the chosen path, root first
     __shared__ int s_red[kPathThreads / 32];
     __shared__ unsigned s_flags;
     __shared__ int s_m, s_end;
     const int N = io.N, tid = threadIdx.x;
     if (tid == 0) s_flags = 0;
+    // tokens, row pointers and (speculatively: the row holds Ecap entries whatever the pointers
+    // say) the parent indices, all in one trip to memory
     for (int v = tid; v < N; v += kPathThreads) {
         const int t = io.tok[v];
         s_tok[v] = t;
         if (t < 0 || t >= io.V) flags |= GSD_DEV_BAD_TOKEN;
-        s_best[v] = v == 0 ? 0 : -1;
+        s_best[0][v] = v == 0 ? 0 : -1;
     }
     for (int v = tid; v <= N; v += kPathThreads) {
         int e = io.pptr[v];
@@ -65,6 +74,8 @@ __device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, St
         }
         s_ptr[v] = e;
     }
+    const int n_prefetch = min(io.Ecap, kPathEdgeCache);
+    for (int e = tid; e < n_prefetch; e += kPathThreads) s_edge[e] = io.pidx[e];
     __syncthreads();
     // Row pointers must start at zero and never decrease.  Otherwise they are replaced by their
     // running maximum (a row whose pointer goes backwards becomes empty, the rows stay disjoint
@@ -95,15 +106,12 @@ __device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, St
             for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) s_enode[e] = (short)v;
         __syncthreads();
         for (int e = tid; e < n_edges; e += kPathThreads) {
-            const int p = io.pidx[e], v = s_enode[e];
-            s_edge[e] = p;
+            const int p = s_edge[e], v = s_enode[e];
             s_eok[e] = (p >= 0 && p < v && s_tok[v] >= 0 && s_tok[v] < io.V) ? (unsigned char)step_ok(p, v) : 0;
         }
         __syncthreads();
-    } else if (cached) {
-        for (int e = tid; e < n_edges; e += kPathThreads) s_edge[e] = io.pidx[e];
-        __syncthreads();
     }
+    auto parent_at = [&](int e) -> int { return cached ? s_edge[e] : io.pidx[e]; };
     auto ok_at = [&](int e, int p, int v) -> bool {
         if (cached && kCacheOutcome) return s_eok[e] != 0;
         return s_tok[v] >= 0 && s_tok[v] < io.V && step_ok(p, v);
@@ -111,41 +119,54 @@ __device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, St
 
     // level-synchronous relaxation: after round r every node whose longest accepted root
     // path has <= r edges is final; values only grow, so it stops when nothing changed
+    int cur_buf = 0;
     for (int round = 0; round < N; ++round) {
-        int nb[kPathNodeSlots];
+        const int* rd = s_best[cur_buf];
+        int* wr = s_best[cur_buf ^ 1];
         int changed = 0;
 #pragma unroll
         for (int k = 0; k < kPathNodeSlots; ++k) {
             const int v = tid + k * kPathThreads;
-            nb[k] = -1;
-            if (v > 0 && v < N) {
-                int cur = s_best[v];
-                for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
-                    const int p = cached ? s_edge[e] : io.pidx[e];
-                    if (p < 0 || p >= v) {
-                        flags |= GSD_DEV_BAD_CSR;
-                        continue;
+            if (v < N) {
+                int cur = rd[v];
+                if (v > 0) {
+                    for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
+                        const int p = parent_at(e);
+                        if (p < 0 || p >= v) {
+                            flags |= GSD_DEV_BAD_CSR;
+                            continue;
+                        }
+                        const int bp = rd[p];
+                        if (bp >= 0 && bp + 1 > cur && ok_at(e, p, v)) cur = bp + 1;
                     }
-                    const int bp = s_best[p];
-                    if (bp >= 0 && bp + 1 > cur && ok_at(e, p, v)) cur = bp + 1;
                 }
-                nb[k] = cur;
-                changed |= (cur != s_best[v]);
+                wr[v] = cur;
+                changed |= (cur != rd[v]);
             }
         }
-        __syncthreads();
-#pragma unroll
-        for (int k = 0; k < kPathNodeSlots; ++k) {
-            const int v = tid + k * kPathThreads;
-            if (v > 0 && v < N) s_best[v] = nb[k];
-        }
+        cur_buf ^= 1;
         if (!__syncthreads_or(changed)) break;
     }
+    const int* best = s_best[cur_buf];
+    int* pred = s_best[cur_buf ^ 1];   // the other copy now takes every node's predecessor on its best path
+    __syncthreads();                   // (every thread has left the last round's reads of it)
 
-    // end node: longest, then lowest index
+    // every node: the lowest predecessor with an accepted step that carries length - 1
     int key = -1;
-    for (int v = tid; v < N; v += kPathThreads)
-        if (s_best[v] >= 0) key = max(key, (s_best[v] << 10) | (1023 - v));
+    for (int v = tid; v < N; v += kPathThreads) {
+        const int bv = best[v];
+        int pr = kPathNone;
+        if (v > 0 && bv > 0) {
+            for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
+                const int p = parent_at(e);
+                if (p < 0 || p >= v) continue;
+                if (best[p] == bv - 1 && p < pr && ok_at(e, p, v)) pr = p;
+            }
+        }
+        pred[v] = pr;
+        // end node: longest, then lowest index
+        if (bv >= 0) key = max(key, (bv << 10) | (1023 - v));
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xFFFFFFFFu, key, o));
     if ((tid & 31) == 0) s_red[tid >> 5] = key;
@@ -159,35 +180,35 @@ __device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, St
         s_end = v;
         unsigned fl = s_flags;
         if (m + 1 > io.Tcap) fl |= GSD_DEV_TCAP;
-        // walk back: the lowest predecessor with an accepted step that carries length - 1
+        // walk back along the predecessors (cannot break off for a consistent best[])
         for (int len = m; len >= 0; --len) {
-            if (io.out_nodes && len < io.Tcap) io.out_nodes[len] = v;
+            s_path[len] = (short)v;
             if (len == 0) break;
-            if (len - 1 < io.Tcap) io.out_tok[len - 1] = s_tok[v];
-            int pred = kPathNone;
-            for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) {
-                const int p = cached ? s_edge[e] : io.pidx[e];
-                if (p < 0 || p >= v) continue;
-                if (s_best[p] == len - 1 && p < pred && ok_at(e, p, v)) pred = p;
-            }
-            if (pred == kPathNone) break;  // cannot happen for a consistent best[]
-            v = pred;
+            const int pr = pred[v];
+            v = pr == kPathNone ? 0 : pr;
         }
         *io.out_len = m + 1;
         s_m = m;
         if (fl && io.status) atomicOr((unsigned*)io.status, fl);
     }
     __syncthreads();
-    for (int i = s_m + 1 + tid; i < io.Tcap; i += kPathThreads) {
-        io.out_tok[i] = -1;
-        if (io.out_nodes) io.out_nodes[i] = -1;
+    const int m = s_m;
+    for (int i = tid; i <= io.Tcap; i += kPathThreads) {
+        if (i <= m) {
+            const int node = s_path[i];
+            if (io.out_nodes && i < io.Tcap) io.out_nodes[i] = node;
+            if (i >= 1) io.out_tok[i - 1] = s_tok[node];    // i - 1 < Tcap
+        } else if (i < io.Tcap) {
+            io.out_tok[i] = -1;
+            if (io.out_nodes) io.out_nodes[i] = -1;
+        }
     }
     bool end_has_child = false;
     if (kCacheOutcome) {
         int has = 0;
         const int end = s_end;
         for (int v = end + 1 + tid; v < N; v += kPathThreads)
-            for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) has |= ((cached ? s_edge[e] : io.pidx[e]) == end);
+            for (int e = s_ptr[v]; e < s_ptr[v + 1]; ++e) has |= (parent_at(e) == end);
         end_has_child = __syncthreads_or(has) != 0;
     }
     return PathResult{s_m, s_end, end_has_child};
