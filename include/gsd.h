@@ -62,6 +62,8 @@ typedef enum gsd_status {
 
 #define GSD_DEV_TREE_FULL    0x200u /* gsd_unmerge_tree: the tree capacity was reached; the rest of the level order was dropped */
 
+#define GSD_DEV_BOUNDS       0x400u /* checking build (libgsd_check.so) only: a kernel formed an index outside its tensor; the access was skipped */
+
 #define GSD_MAX_NODES 512          /* largest supported N (draft nodes per sequence) */
 
 /* kernel selection for gsd_verify_attn */
@@ -129,6 +131,20 @@ int gsd_verify_attn(const void* q, const void* k_cache, const void* v_cache,
                     const void* draft_k, const void* draft_v, const uint32_t* ancestor_mask,
                     const int32_t* seq_lens, void* out, const gsd_attn_params* p,
                     void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+
+/*
+ * gsd_debug_attn_wait - test hook for the bounded waits of the tcgen05 back end of
+ * gsd_verify_attn (no counterpart in the paper).  Every in-kernel wait (on a copy, on a tensor
+ * core result, on another warp) gives up after a time limit, 2 s by default: the kernel then ORs
+ * GSD_DEV_WAIT_EXPIRED into *status, all its warps leave their loops, copies and tensor-core
+ * work already under way are awaited (again with the limit), the tensor memory is released and
+ * the launch ends normally; `out` is not valid, the next call works as usual.
+ *   limit_ns          new limit for later launches of this process (0 = back to the default)
+ *   withhold_first_k  non-zero: every CTA of later launches announces but never issues the copy of
+ *                     its first key tile, so that a wait really runs out - for tests of the path
+ *                     above; zero switches it off again
+ */
+void gsd_debug_attn_wait(uint64_t limit_ns, int32_t withhold_first_k);
 
 /* Bytes of workspace gsd_verify_attn needs for *p on the current device (0 on invalid
  * parameters or when none is needed). */

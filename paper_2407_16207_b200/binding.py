@@ -50,7 +50,7 @@ class DraftParams(ctypes.Structure):
                 ("theta_prob", ctypes.c_float), ("theta_sib", ctypes.c_float)]
 
 
-EXPORTS = ["gsd_version", "gsd_status_string", "gsd_last_cuda_error", "gsd_verify_attn",
+EXPORTS = ["gsd_version", "gsd_status_string", "gsd_last_cuda_error", "gsd_debug_attn_wait", "gsd_verify_attn",
            "gsd_verify_attn_workspace_bytes", "gsd_verify_attn_num_splits", "gsd_accept",
            "gsd_accept_workspace_bytes", "gsd_accept_static", "gsd_accept_sampled",
            "gsd_accept_sampled_workspace_bytes", "gsd_draft_expand", "gsd_draft_expand_workspace_bytes",
@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
         L.gsd_status_string.restype = ctypes.c_char_p
         L.gsd_status_string.argtypes = [i32]
         L.gsd_last_cuda_error.restype = ctypes.c_char_p
+        L.gsd_debug_attn_wait.restype = None
+        L.gsd_debug_attn_wait.argtypes = [ctypes.c_uint64, ctypes.c_int32]
         L.gsd_verify_attn.restype = i32
         L.gsd_verify_attn.argtypes = [vp] * 8 + [ctypes.POINTER(AttnParams), vp, sz, vp, vp]
         L.gsd_verify_attn_workspace_bytes.restype = sz
@@ -123,6 +125,12 @@ def _check(rc: int) -> None:
 
 def gsd_version() -> int:
     return int(lib().gsd_version())
+
+
+def gsd_debug_attn_wait(limit_ns: int = 0, withhold_first_k: bool = False) -> None:
+    """Test hook for the bounded in-kernel waits of the tcgen05 attention kernel; see
+    gsd_debug_attn_wait in include/gsd.h.  (0, False) restores the defaults."""
+    lib().gsd_debug_attn_wait(int(limit_ns), 1 if withhold_first_k else 0)
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -251,7 +259,8 @@ def gsd_accept_sampled_workspace_bytes(B, N) -> int:
 def gsd_accept_sampled(logits, draft_tokens, parent_ptr, parent_idx, draft_q, u_accept, u_sample, *,
                        draft_logits: Optional[torch.Tensor] = None,
                        Tcap: int = 0, want_nodes: bool = True, workspace: Optional[torch.Tensor] = None,
-                       status: Optional[torch.Tensor] = None
+                       status: Optional[torch.Tensor] = None,
+                       out: Optional[Tuple[torch.Tensor, torch.Tensor, Optional[torch.Tensor]]] = None
                        ) -> Tuple[torch.Tensor, torch.Tensor, Optional[torch.Tensor]]:
     """Non-deterministic verification with the random numbers passed in; see gsd_accept_sampled in
     include/gsd.h.  `draft_logits` [B,N,V] (optional) makes the regenerated token come from the
@@ -273,9 +282,14 @@ def gsd_accept_sampled(logits, draft_tokens, parent_ptr, parent_idx, draft_q, u_
     if draft_logits is not None:
         _want(draft_logits, torch.float32, (B, N, V), "draft_logits", True)
     Tcap = Tcap or N
-    toks = torch.empty((B, Tcap), dtype=torch.int32, device=logits.device)
-    lens = torch.empty((B,), dtype=torch.int32, device=logits.device)
-    nodes = torch.empty((B, Tcap), dtype=torch.int32, device=logits.device) if want_nodes else None
+    if out is None:
+        toks = torch.empty((B, Tcap), dtype=torch.int32, device=logits.device)
+        lens = torch.empty((B,), dtype=torch.int32, device=logits.device)
+        nodes = torch.empty((B, Tcap), dtype=torch.int32, device=logits.device) if want_nodes else None
+    else:
+        toks, lens, nodes = out
+        _want(toks, torch.int32, (B, Tcap), "accepted_tokens", True)
+        _want(lens, torch.int32, (B,), "accepted_len", True)
     p = AcceptParams(B, N, V, Ecap, Tcap)
     L = lib()
     with torch.cuda.device(logits.device):
@@ -294,7 +308,8 @@ def gsd_accept_sampled(logits, draft_tokens, parent_ptr, parent_idx, draft_q, u_
 
 def gsd_draft_expand(logits, frontier, frontier_len, tokens, tree_parent, merge_to, leaf, prob, num_nodes, *,
                      k: int, tau: int, theta_prob: float, theta_sib: float,
-                     workspace: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None
+                     workspace: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None,
+                     out: Optional[Tuple[torch.Tensor, torch.Tensor]] = None
                      ) -> Tuple[torch.Tensor, torch.Tensor]:
     """One growth step of the draft token graph, in place; see gsd_draft_expand in include/gsd.h.
     Returns (new_frontier [B,F*k], new_frontier_len [B])."""
@@ -309,8 +324,13 @@ def gsd_draft_expand(logits, frontier, frontier_len, tokens, tree_parent, merge_
                         ("merge_to", merge_to, torch.int32), ("leaf", leaf, torch.uint8), ("prob", prob, torch.float32)):
         _want(t, dt, (B, Ncap), name, True)
     _want(num_nodes, torch.int32, (B,), "num_nodes", True)
-    nf = torch.full((B, F * k), -1, dtype=torch.int32, device=logits.device)
-    nfl = torch.zeros((B,), dtype=torch.int32, device=logits.device)
+    if out is None:
+        nf = torch.full((B, F * k), -1, dtype=torch.int32, device=logits.device)
+        nfl = torch.zeros((B,), dtype=torch.int32, device=logits.device)
+    else:
+        nf, nfl = out
+        _want(nf, torch.int32, (B, F * k), "new_frontier", True)
+        _want(nfl, torch.int32, (B,), "new_frontier_len", True)
     p = DraftParams(B, F, V, Ncap, int(k), int(tau), float(theta_prob), float(theta_sib))
     L = lib()
     with torch.cuda.device(logits.device):
@@ -344,7 +364,8 @@ def gsd_build_mask(parent_ptr, parent_idx, out: Optional[torch.Tensor] = None, *
 
 
 def gsd_unmerge_tree(draft_tokens, parent_ptr, parent_idx, *, Ucap: int, max_depth: int,
-                     status: Optional[torch.Tensor] = None
+                     status: Optional[torch.Tensor] = None,
+                     out: Optional[Tuple[torch.Tensor, torch.Tensor, torch.Tensor, torch.Tensor]] = None
                      ) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor, torch.Tensor]:
     """The token graph unfolded into a tree (one node per root path); see gsd_unmerge_tree in
     include/gsd.h.  Returns (tree_tokens, tree_parent, tree_source [B,Ucap], tree_count [B])."""
@@ -354,10 +375,16 @@ def gsd_unmerge_tree(draft_tokens, parent_ptr, parent_idx, *, Ucap: int, max_dep
     _want(parent_ptr, torch.int32, (B, N + 1), "parent_ptr", True)
     _want(parent_idx, torch.int32, (B, Ecap), "parent_idx", True)
     dev = draft_tokens.device
-    tt = torch.empty((B, Ucap), dtype=torch.int32, device=dev)
-    tp = torch.empty((B, Ucap), dtype=torch.int32, device=dev)
-    ts = torch.empty((B, Ucap), dtype=torch.int32, device=dev)
-    cnt = torch.empty((B,), dtype=torch.int32, device=dev)
+    if out is None:
+        tt = torch.empty((B, Ucap), dtype=torch.int32, device=dev)
+        tp = torch.empty((B, Ucap), dtype=torch.int32, device=dev)
+        ts = torch.empty((B, Ucap), dtype=torch.int32, device=dev)
+        cnt = torch.empty((B,), dtype=torch.int32, device=dev)
+    else:
+        tt, tp, ts, cnt = out
+        for name, t in (("tree_tokens", tt), ("tree_parent", tp), ("tree_source", ts)):
+            _want(t, torch.int32, (B, Ucap), name, True)
+        _want(cnt, torch.int32, (B,), "tree_count", True)
     with torch.cuda.device(dev):
         _check(lib().gsd_unmerge_tree(draft_tokens.data_ptr(), parent_ptr.data_ptr(), parent_idx.data_ptr(),
                                       tt.data_ptr(), tp.data_ptr(), ts.data_ptr(), cnt.data_ptr(), B, N, Ecap,

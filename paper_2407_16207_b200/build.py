@@ -10,6 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libgsd.so")
+LIB_CHECK = os.path.join(PKG, "libgsd_check.so")
 OBJ_DIR = os.path.join(PKG, "_build")
 SOURCES = ["gsd_api.cu", "gsd_accept.cu", "gsd_accept_sampled.cu", "gsd_draft.cu", "gsd_attn_mma.cu", "gsd_attn_tc.cu", "gsd_commit.cu", "gsd_mask.cu", "gsd_unmerge.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
@@ -30,18 +31,24 @@ def _stale(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile the sources that changed and link libgsd.so next to this file."""
-    os.makedirs(OBJ_DIR, exist_ok=True)
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """Compile the sources that changed and link libgsd.so next to this file.  With `checked`
+    the same sources are compiled with -DGSD_BOUNDS_CHECK into libgsd_check.so: the build whose
+    kernels check the indices they form and report GSD_DEV_BOUNDS instead of accessing memory
+    outside a tensor (used by the tests in place of a memory sanitizer)."""
+    obj_dir = OBJ_DIR + ("_check" if checked else "")
+    lib = LIB_CHECK if checked else LIB
+    extra = ["-DGSD_BOUNDS_CHECK"] if checked else []
+    os.makedirs(obj_dir, exist_ok=True)
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]
     headers.append(os.path.join(ROOT, "include", "gsd.h"))
     jobs, objs = [], []
     for src in SOURCES:
         s = os.path.join(CSRC, src)
-        o = os.path.join(OBJ_DIR, src.replace(".cu", ".o"))
+        o = os.path.join(obj_dir, src.replace(".cu", ".o"))
         objs.append(o)
         if force or _stale(o, [s] + headers):
-            jobs.append([_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else [])
+            jobs.append([_nvcc()] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else [])
                         + ["-c", s, "-o", o])
 
     def run(cmd):
@@ -53,13 +60,13 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
     with ThreadPoolExecutor(max_workers=4) as ex:
         list(ex.map(run, jobs))
-    if force or jobs or _stale(LIB, objs):
-        tmp = LIB + f".tmp{os.getpid()}"
+    if force or jobs or _stale(lib, objs):
+        tmp = lib + f".tmp{os.getpid()}"
         run([_nvcc(), "-shared", "-o", tmp] + objs
             + ["-gencode", "arch=compute_100a,code=sm_100a", "-Xcompiler", "-fPIC"])
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, checked="--checked" in sys.argv))

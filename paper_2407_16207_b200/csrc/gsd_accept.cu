@@ -109,7 +109,8 @@ __device__ void path_pass(const AcceptArgs& a, int b) {
     // a step parent -> v is accepted iff v's token is what the target model would emit after the parent
     const PathResult res = longest_accepted_path<false>(io, 0u, [&](int p, int v) { return tok[v] == s_amax[p]; });
     // the target model's own next token
-    if (tid == 0 && res.edges < a.Tcap) io.out_tok[res.edges] = s_amax[res.end];
+    if (tid == 0 && res.edges < a.Tcap && GSD_IN_BOUNDS(res.end >= 0 && res.end < N && res.edges >= 0, a.status))
+        io.out_tok[res.edges] = s_amax[res.end];
 }
 
 // Zeroes scratch words.  The kernel that uses them is launched as a programmatic dependent: it
@@ -174,7 +175,8 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a) {
     if (threadIdx.x == 0) {
         // the scratch is zeroed by the launch before this one; everything above ran beside it
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        if (best.i != kNone) atomicMax(a.keys + row, pack_key(best.v, best.i));
+        if (best.i != kNone && GSD_IN_BOUNDS(row < a.B * a.N && best.i >= 0 && best.i < a.V, a.status))
+            atomicMax(a.keys + row, pack_key(best.v, best.i));
         __threadfence();
         const int b = row / a.N;
         const unsigned prev = atomicAdd(a.done + b, 1u);

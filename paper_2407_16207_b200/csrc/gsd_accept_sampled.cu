@@ -147,6 +147,7 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     // the test of one step: the target's probability of v's token under its parent p (one
     // logit gathered from global memory) against u q
     const PathResult res = longest_accepted_path<true>(io, flags, [&](int p, int v) {
+        if (!GSD_IN_BOUNDS(p >= 0 && p < N && tok[v] >= 0 && tok[v] < V, a.status)) return false;
         const float prob = ex2((lg[(size_t)p * V + tok[v]] - s_mx[p]) * kLog2e) / s_sum[p];
         return s_uq[v] < prob;
     });
@@ -362,7 +363,7 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
         int pick = first == kNone ? -1 : s_pick;
         if (pick < 0)
             for (int w = 0; w < kWarps; ++w) pick = max(pick, s_red[w]);
-        if (s_m < a.Tcap) out_tok[s_m] = pick;
+        if (s_m < a.Tcap && GSD_IN_BOUNDS(s_m >= 0 && pick < V, a.status)) out_tok[s_m] = pick;
     }
 }
 

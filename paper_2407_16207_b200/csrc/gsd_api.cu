@@ -103,6 +103,10 @@ using namespace gsd;
 
 extern "C" int gsd_version(void) { return GSD_VERSION; }
 
+extern "C" void gsd_debug_attn_wait(uint64_t limit_ns, int32_t withhold_first_k) {
+    debug_attn_wait((unsigned long long)limit_ns, (int)withhold_first_k);
+}
+
 extern "C" const char* gsd_status_string(int s) {
     switch (s) {
         case GSD_OK: return "ok";

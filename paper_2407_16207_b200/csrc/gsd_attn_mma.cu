@@ -74,6 +74,7 @@ struct MmaParams {
     PlanDev plan;
     int32_t* status;
     int B, N, Hq, Hkv, Lmax, G, W, R;
+    int slots;       // partial-result slots of the plan
     float scale_log2;
 };
 
@@ -315,6 +316,7 @@ __global__ void __launch_bounds__(kThreads) attn_mma_kernel(MmaParams p) {
         for (int h = 0; h < 2; ++h) {
             if (!rvalid[h]) continue;
             const int row = row0 + rloc[h];
+            if (!GSD_IN_BOUNDS(b < p.B && c < p.Hkv && row < p.R, p.status)) continue;
             const float inv = l_run[h] > 0.f ? 1.f / l_run[h] : 0.f;
             __nv_bfloat16* dst = p.out + (((size_t)b * N + row / G) * p.Hq + c * G + row % G) * D;
 #pragma unroll
@@ -328,6 +330,7 @@ __global__ void __launch_bounds__(kThreads) attn_mma_kernel(MmaParams p) {
         for (int h = 0; h < 2; ++h) {
             if (!rvalid[h]) continue;
             const size_t prow = (size_t)slot * BM + rloc[h];
+            if (!GSD_IN_BOUNDS(slot >= 0 && slot < p.slots, p.status)) continue;
             float* dst = p.part_o + prow * D;
 #pragma unroll
             for (int dt = 0; dt < DT; ++dt) {
@@ -429,7 +432,7 @@ int launch_mma_t(const AttnArgs& a) {
     p.draft_v = (const __nv_bfloat16*)a.draft_v; p.mask = a.mask; p.seq_lens = a.seq_lens;
     p.out = (__nv_bfloat16*)a.out; p.status = a.status;
     p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv; p.Lmax = a.Lmax; p.G = a.G; p.W = a.W;
-    p.R = a.N * a.G; p.scale_log2 = a.scale_log2; p.plan = a.plan.dev;
+    p.R = a.N * a.G; p.scale_log2 = a.scale_log2; p.plan = a.plan.dev; p.slots = a.plan.slots;
     p.part_o = (float*)a.workspace;
     p.part_ml = (float*)((char*)a.workspace + plan_part_o_bytes(a.plan, a.D));
     const int smem = 4 * BN * D * 2;

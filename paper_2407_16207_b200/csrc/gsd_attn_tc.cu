@@ -47,7 +47,20 @@ constexpr int kThreads = 384;
 constexpr uint32_t kSmemBytes = (2 + KST + VST) * TILE_BYTES + 2 * HALF_BYTES + 1024;  // tiles, output staging, alignment slack
 constexpr float kRescaleThreshold = 8.0f;         // log2 units
 constexpr int kUnitTable = 12;                    // units of work per CTA decoded in the prologue (one per warp)
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // default limit of every in-kernel wait
+
+// Test hook (see gsd_debug_attn_wait): a shorter limit and, optionally, a CTA's first K tile
+// withheld so that a wait really runs out.
+unsigned long long g_wait_limit_ns = kWaitLimitNs;
+int g_withhold_first_k = 0;
+
+// What every bounded wait looks at, in shared memory: word 0 is raised by the first wait that
+// gives up (all other waits then return within a few polls), words 2-3 hold the time limit.
+struct WaitCtl {
+    int abort;
+    int pad;
+    unsigned long long limit_ns;
+};
 
 // TMEM columns (32-bit words): one score tile, a bf16 P tile per stream, an accumulator per stream
 constexpr uint32_t COL_S = 0, COL_P0 = 128, COL_P1 = 192, COL_O0 = 256, COL_O1 = 384;
@@ -67,7 +80,8 @@ enum Bar {
     BAR_O_FREE = BAR_O_DONE + 2,      // 2: the accumulator rows of the unit have been read out
     BAR_Q_EMPTY = BAR_O_FREE + 2,     // 1: every QK^T of the unit has completed
     BAR_ML_READY = BAR_Q_EMPTY + 1,   // 1: (max, sum) of the odd-tile stream are in shared memory
-    BAR_COUNT = BAR_ML_READY + 1
+    BAR_DRAIN = BAR_ML_READY + 1,     // 2: every MMA issued by the QK^T / PV warp has completed
+    BAR_COUNT = BAR_DRAIN + 2
 };
 
 struct TcParams {
@@ -81,6 +95,9 @@ struct TcParams {
     float scale_log2;
     PlanDev plan;
     int total_work;   // CTAs of the plan = units of work
+    int slots;        // partial-result slots of the plan
+    unsigned long long wait_limit_ns;
+    int withhold_first_k;   // test hook: every CTA leaves out the K copy of its first key tile
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -113,11 +130,12 @@ __device__ __forceinline__ unsigned long long global_ns() {
 __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                             int32_t* status, bool ignore_abort) {
     const unsigned long long t0 = global_ns();
+    const unsigned long long limit = reinterpret_cast<const volatile WaitCtl*>(abort_flag)->limit_ns;
     for (unsigned it = 0;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 63u) {
             if (!ignore_abort && *abort_flag) return false;
-            if (global_ns() - t0 > kWaitLimitNs) {
+            if (global_ns() - t0 > limit) {
                 *abort_flag = 1;
                 if (status) atomicOr((unsigned*)status, GSD_DEV_WAIT_EXPIRED);
                 return false;
@@ -152,8 +170,16 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t sr
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void wg_barrier(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
 
+__device__ __forceinline__ void wg_barrier(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
+// the same hardware barrier of a warpgroup with an AND over a flag: every thread gets the answer
+__device__ __forceinline__ bool wg_all(int id, bool flag) {
+    uint32_t r;
+    asm volatile(
+        "{\n .reg .pred p, q;\n setp.ne.u32 q, %2, 0;\n bar.red.and.pred p, %1, 128, q;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(r) : "r"(id), "r"((uint32_t)flag) : "memory");
+    return r != 0;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -342,6 +368,9 @@ __device__ __forceinline__ UnitInfo unit_info(const TcParams& p, int w, int lane
     u.b = unit / p.Hkv;
     u.c = unit % p.Hkv;
     u.two = u.row0 + BM < p.R;
+    if (!GSD_IN_BOUNDS(u.b >= 0 && u.b < p.B && u.c < p.Hkv && u.row0 < p.R, p.status)) {
+        u.b = 0; u.c = 0; u.row0 = 0; u.two = false;      // checking build only: a unit outside the problem
+    }
     int L = p.seq_lens[u.b];
     L = L < 0 ? 0 : (L > p.Lmax ? p.Lmax : L);
     u.L = L;
@@ -394,7 +423,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     extern __shared__ unsigned char smem_raw[];
     __shared__ __align__(8) unsigned long long s_bars[BAR_COUNT];
     __shared__ uint32_t s_tmem_base;
-    __shared__ int s_abort;
+    __shared__ __align__(8) WaitCtl s_wait;
     __shared__ float2 s_ml1[BM];      // (max, sum) of the odd-tile stream, one per row
     __shared__ UnitInfo s_units[kUnitTable];   // the CTA's first units of work, decoded once up front
 
@@ -408,12 +437,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const uint32_t sStage = sV + VST * TILE_BYTES;                   // one [128][64] bf16 block per softmax warpgroup
     const uint32_t bar0 = smem_u32(s_bars);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
-    volatile int* abort_flag = &s_abort;
+    volatile int* abort_flag = &s_wait.abort;
 
     if (tid == 0) {
         // the merge pass (a programmatic dependent launch) may be made resident as CTAs retire
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-        s_abort = 0;
+        s_wait.abort = 0;
+        s_wait.limit_ns = p.wait_limit_ns;
         mbar_init(bar(BAR_Q_FULL), 1);
         mbar_init(bar(BAR_Q_EMPTY), 1);
         mbar_init(bar(BAR_ML_READY), 4);
@@ -427,6 +457,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             mbar_init(bar(BAR_P_FREE + i), 1);
             mbar_init(bar(BAR_O_DONE + i), 1);
             mbar_init(bar(BAR_O_FREE + i), 4);
+            mbar_init(bar(BAR_DRAIN + i), 1);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -482,8 +513,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     ok = mbar_wait(bar(BAR_K_EMPTY + s), par, abort_flag, p.status);
                     if (!ok) break;
                     mbar_expect_tx(bar(BAR_K_FULL + s), TILE_BYTES);
-                    for (int h = 0; h < 2; ++h)
-                        tma_load_4d(sK + s * TILE_BYTES + h * HALF_BYTES, mk, bar(BAR_K_FULL + s), h * 64, u.c, ti.key0, u.b);
+                    if (!(p.withhold_first_k && kvc == 0))   // (test hook: the bytes announced above never arrive)
+                        for (int h = 0; h < 2; ++h)
+                            tma_load_4d(sK + s * TILE_BYTES + h * HALF_BYTES, mk, bar(BAR_K_FULL + s), h * 64, u.c, ti.key0, u.b);
                     ok = mbar_wait(bar(BAR_V_EMPTY + s), par, abort_flag, p.status);
                     if (!ok) {
                         // the K copy just issued is still in flight: let it land
@@ -549,6 +581,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             kvc += u.ntiles;
             ++au;
         }
+        // after an abort nothing this warp issued may still be running when TMEM is given back
+        // (at a regular end the epilogues have waited for every MMA already)
+        if (!ok) {
+            tc_commit(bar(BAR_DRAIN + 0));
+            mbar_wait_slow(bar(BAR_DRAIN + 0), 0, abort_flag, nullptr, true);
+        }
     } else if (warp == 11) {
         // ------------------------------------------------------------ PV issuer (all lanes converged)
         // O_i += P_i V job by job: 8 k-steps of 16 keys, P (bf16 pairs) read from TMEM.  The
@@ -595,6 +633,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             kvc += u.ntiles;
             ++au;
             if (n1 > 0) ++au1;
+        }
+        if (!ok) {
+            tc_commit(bar(BAR_DRAIN + 1));
+            mbar_wait_slow(bar(BAR_DRAIN + 1), 0, abort_flag, nullptr, true);
         }
     }
     } else {
@@ -764,8 +806,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 tc_fence_before();
                 if (lane == 0) mbar_arrive(bar(BAR_P_READY2 + i));
             }
-            if (!ok) break;
-
+            if (!ok) {
+                // gave up inside the key loop: the warpgroup's decision barrier of this unit (below)
+                // still has to see this warp, or the neighbours would wait there for ever
+                if (u.nsplit == 1 && !(alt && i == 1)) wg_all(1 + i, false);
+                break;
+            }
             if (alt && i == 1) {
                 // odd-tile stream: publish (max, sum); warpgroup 0 reads the accumulator itself
                 if (my_n > 0) {
@@ -780,22 +826,31 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 continue;
             }
             // ---- epilogue: pull the accumulator row into registers, give TMEM back, then store
-            float acc[HD];
+            // every wait of the epilogue first ...
             if (ntiles > 0) {
                 ok = mbar_wait(bar(BAR_O_DONE + i), (uint32_t)(auc & 1), abort_flag, p.status);
+                if (ok && alt && n1 > 0) {
+                    ok = mbar_wait(bar(BAR_O_DONE + 1), (uint32_t)(auc1 & 1), abort_flag, p.status);
+                    if (ok) ok = mbar_wait(bar(BAR_ML_READY), (uint32_t)(mlc & 1), abort_flag, p.status);
+                }
                 ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok) break;
+            }
+            if (u.nsplit == 1) {
+                // ... then the four warps decide together whether to go on: the store section below
+                // meets at hardware barriers, which have no time limit, so no warp may enter it while
+                // a neighbour has given up.  Every warp of the warpgroup takes part in this barrier
+                // once per unit, here or where it gave up.
+                ok = wg_all(1 + i, ok);
+            }
+            if (!ok) break;
+            float acc[HD];
+            if (ntiles > 0) {
                 tc_fence_after();
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) tc_ld32p(tO + ch * 32, acc + ch * 32);
                 tc_wait_ld();
                 if (alt && n1 > 0) {
                     // merge the odd-tile stream: O = w0 O0 + w1 O1, l = w0 l0 + w1 l1 at the common maximum
-                    ok = mbar_wait(bar(BAR_O_DONE + 1), (uint32_t)(auc1 & 1), abort_flag, p.status);
-                    if (ok) ok = mbar_wait(bar(BAR_ML_READY), (uint32_t)(mlc & 1), abort_flag, p.status);
-                    ok = __all_sync(0xFFFFFFFFu, ok);
-                    if (!ok) break;
-                    tc_fence_after();
                     const float2 ml1 = s_ml1[rloc];
                     const float m = fmaxf(m_ref, ml1.x);
                     const float m_use = m == -CUDART_INF_F ? 0.f : m;
@@ -854,12 +909,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             } else if (rvalid) {
                 {
                     const size_t prow = (size_t)u.slot * (2 * BM) + (alt ? 0 : i * BM) + rloc;
+                    if (GSD_IN_BOUNDS(u.slot >= 0 && u.slot < p.slots, p.status)) {
                     float* dst = p.part_o + prow * HD;
 #pragma unroll
                     for (int k = 0; k < HD / 4; ++k)
                         *reinterpret_cast<float4*>(dst + k * 4) =
                             make_float4(acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]);
                     *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(m_ref, l_run);
+                    }
                 }
             }
             kvc += ntiles;
@@ -954,12 +1011,20 @@ int launch_attn_tcgen05(const AttnArgs& a) {
         }
     }
     p.total_work = a.plan.ctas;
+    p.slots = a.plan.slots;
+    p.wait_limit_ns = g_wait_limit_ns;
+    p.withhold_first_k = g_withhold_first_k;
     DeviceInfo di;
     if (device_info(&di) != 0) return GSD_ERR_CUDA;
     dim3 grid(a.plan.ctas < di.sm_count ? a.plan.ctas : di.sm_count);
     attn_tc_kernel<<<grid, kThreads, kSmemBytes, a.stream>>>(tq, tk, tv, tdk, tdv, tout, p);
     GSD_CUDA_TRY(cudaGetLastError());
     return GSD_OK;
+}
+
+void debug_attn_wait(unsigned long long limit_ns, int withhold_first_k) {
+    g_wait_limit_ns = limit_ns ? limit_ns : kWaitLimitNs;
+    g_withhold_first_k = withhold_first_k;
 }
 
 }  // namespace gsd

@@ -78,6 +78,7 @@ __global__ void __launch_bounds__(kThreads) commit_kernel(CommitArgs a) {
     const long total = (long)n * a.row16;
     for (long t = threadIdx.x; t < total; t += kThreads) {
         const int i = (int)(t / a.row16), ch = (int)(t % a.row16);
+        if (!GSD_IN_BOUNDS(s_src[i] >= 0 && s_src[i] < a.N && L + i < a.Lmax, a.status)) continue;
         const size_t src = ((size_t)b * a.N + s_src[i]) * a.row16 + ch;
         const size_t dst = ((size_t)b * a.Lmax + L + i) * a.row16 + ch;
         a.k_cache[dst] = a.draft_k[src];

@@ -2,10 +2,11 @@
 // k; Sec. 4.2: probability pruning and sibling pruning; Sec. 5.2: tau-redundant nodes; Sec. 5.3:
 // merge edges to the first occurrence).
 //
-// One launch.  Grid (F, B): the CTA of frontier row (b, fi) streams that row of draft logits
-// with 16-byte loads for the softmax statistics and a lower bound on the k-th best logit, reads
-// it once more (from L2) to collect the few entries above the bound, and leaves the row's k best
-// tokens and their probabilities in scratch.  The CTA that finishes last for a sequence appends the
+// Two launches.  Grid (F, B): the CTA of frontier row (b, fi) streams that row of draft logits
+// once with 16-byte loads - softmax statistics and every thread's two best (logit, token)
+// pairs - lets one warp pick the row's k best among the 512 pairs, and leaves tokens and
+// probabilities in scratch (a row where a thread's second pair is picked is redone exactly).
+// The second launch (one CTA per sequence, a programmatic dependent of the first) appends the
 // children (k per frontier node, in frontier order), applies the two pruning rules, looks for
 // an earlier node with the same tau-gram for every new node (first occurrence = lowest id),
 // and compacts the new frontier.
@@ -68,7 +69,6 @@ struct DraftArgs {
     int32_t* new_frontier_len;
     int32_t* wk_tok;     // [B,F,K]
     float* wk_q;         // [B,F,K]
-    unsigned* done;      // [B], zeroed before the launch
     int32_t* status;
     int B, F, V, Ncap, k, tau;
     float theta_prob, theta_sib;
@@ -117,6 +117,7 @@ __device__ void grow_sequence(const DraftArgs& a, int b) {
             flags |= GSD_DEV_BAD_FRONTIER;
             p = 0;
         }
+        if (!GSD_IN_BOUNDS(c < Ncap && fi < a.F && i < K, a.status)) continue;
         const float q = a.wk_q[w + i], qmax = a.wk_q[w];
         s_tok[c] = a.wk_tok[w + i];
         s_par[c] = p;
@@ -182,7 +183,8 @@ __device__ void grow_sequence(const DraftArgs& a, int b) {
         __syncthreads();
         int off = base;
         for (int w = 0; w < warp; ++w) off += s_cnt[w];
-        if (keep) nf[off + __popc(bal & ((1u << lane) - 1u))] = n0 + j;
+        if (keep && GSD_IN_BOUNDS(off + __popc(bal & ((1u << lane) - 1u)) < a.F * k, a.status))
+            nf[off + __popc(bal & ((1u << lane) - 1u))] = n0 + j;
         for (int w = 0; w < kWarps; ++w) base += s_cnt[w];
         __syncthreads();
     }
@@ -192,8 +194,6 @@ __device__ void grow_sequence(const DraftArgs& a, int b) {
     }
     if (flags && a.status) atomicOr((unsigned*)a.status, flags);
 }
-
-constexpr int kCand = 1024;   // candidates (logit >= bound) a row may have before the exact fallback takes over
 
 // Block-wide pick of the best remaining (value, index) pair, ranked by `before`; every thread
 // passes its own proposal and gets the winner (and the proposing thread) back.
@@ -213,177 +213,270 @@ __device__ __forceinline__ void block_best(float& v, int& i, int& owner, float* 
     __syncthreads();
 }
 
-// The k best tokens of one row of logits and their probabilities.
-// Pass 1 streams the row: running (maximum, sum of exponentials) per thread, and each thread's
-// own largest value.  The k-th largest of those 256 thread maxima is a lower bound on the row's
-// k-th best logit (they are k different entries).  Pass 2 reads the row again (it is still in
-// L2) and collects the entries >= that bound - a few dozen at most for any peaked or random row;
-// the k best of them, ties to the lower token id, are the answer.  A row with more than kCand
-// such entries (long runs of equal logits) takes the exact fallback: every thread keeps the K
-// best pairs it meets and the block merges the 256 lists.
+// The k best tokens of one row of logits and their probabilities, in one pass over the row.
+// Every thread streams its strided share (16-byte loads, eight in flight) and keeps the running
+// (maximum, sum of exponentials) pair and the two best (logit, token) pairs it has met.  The
+// 512 pairs go to shared memory and one warp picks the row's k best of them with shuffles
+// (ranked by logit, ties to the lower token id).  That is the exact answer unless a thread's
+// SECOND pair was picked - then a third entry of that thread could rank among the k best too
+// (for a random row: about one row in fifty).  Such a row is read once more (from L2): the k-th
+// pick bounds the k-th best entry from below, the entries at or before it form a short list,
+// and the pick is repeated over the list.  Only a list longer than 512 (long runs of equal
+// logits) takes the slow exact way: every thread keeps the K best pairs it meets and the block
+// merges the 256 lists.
+struct Two {
+    float v1, v2;
+    int i1, i2;
+};
+__device__ __forceinline__ void offer2(Two& t, float x, int idx) {
+    // a thread meets its entries in ascending token order: an equal logit never displaces an earlier one
+    if (x > t.v1) { t.v2 = t.v1; t.i2 = t.i1; t.v1 = x; t.i1 = idx; }
+    else if (x > t.v2) { t.v2 = x; t.i2 = idx; }
+}
+
+// One warp picks the k best of `count` <= 512 (logit, token) pairs in shared memory with
+// shuffles only and writes tokens and probabilities to the row's scratch entries.  Returns (to
+// every lane) bit 0: a pair in an odd slot was picked; bit 1: fewer than k pairs above -inf;
+// the k-th pick is left in (*last_v, *last_i).
+__device__ __forceinline__ int warp_pick_k(const float* s_cv, const int* s_ci, int count, int k, float rm, float rs,
+                                           int32_t* wk_tok, float* wk_q, float* last_v, int* last_i) {
+    const int lane = threadIdx.x & 31;
+    float cv[16];
+    int ci[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const bool in = lane + 32 * j < count;
+        cv[j] = in ? s_cv[lane + 32 * j] : -CUDART_INF_F;
+        ci[j] = in ? s_ci[lane + 32 * j] : 0x7FFFFFFF;
+    }
+    int result = 0;
+    float v = -CUDART_INF_F;
+    int i = 0x7FFFFFFF;
+    for (int r = 0; r < k; ++r) {
+        v = -CUDART_INF_F;
+        i = 0x7FFFFFFF;
+        int slot = -1;
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+            if (before(cv[j], ci[j], v, i)) { v = cv[j]; i = ci[j]; slot = lane + 32 * j; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float v2 = __shfl_xor_sync(0xFFFFFFFFu, v, o);
+            const int i2 = __shfl_xor_sync(0xFFFFFFFFu, i, o), t2 = __shfl_xor_sync(0xFFFFFFFFu, slot, o);
+            if (before(v2, i2, v, i)) { v = v2; i = i2; slot = t2; }
+        }
+        // pairs at -inf are never taken (slot stays -1 when nothing above -inf is left)
+        if (slot >= 0) {
+            if (slot & 1) result |= 1;
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (slot == lane + 32 * j) { cv[j] = -CUDART_INF_F; ci[j] = 0x7FFFFFFF; }
+        } else {
+            result |= 2;
+        }
+        if (lane == 0) {
+            wk_tok[r] = slot < 0 ? -1 : i;
+            wk_q[r] = slot < 0 ? 0.f : ex2((v - rm) * kLog2e) / rs;
+        }
+    }
+    *last_v = v;
+    *last_i = i;
+    return result;
+}
+
 template <bool kVec>
-__global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
-    __shared__ float s_cv[kCand];
-    __shared__ int s_ci[kCand];
+__global__ void __launch_bounds__(kThreads, 5) draft_expand_kernel(DraftArgs a) {
+    __shared__ float s_cv[2 * kThreads];
+    __shared__ int s_ci[2 * kThreads];
     __shared__ float s_rv[kWarps];
     __shared__ int s_ri[kWarps], s_rt[kWarps];
     __shared__ float s_m[kWarps], s_s[kWarps];
-    __shared__ int s_last, s_count;
+    __shared__ int s_redo, s_count, s_ti;
+    __shared__ float s_tv;
+    // the per-sequence pass (a programmatic dependent launch) may become resident as CTAs retire
+    if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int fi = blockIdx.x, b = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int V = a.V;
     const int fl = a.frontier_len[b];
-    if (fi < fl && fl <= a.F) {
-        const float* x = a.logits + ((size_t)b * a.F + fi) * V;
-        const float4* x4 = reinterpret_cast<const float4*>(x);
-        const int nvec = V >> 2;
-        float m = -CUDART_INF_F, s = 0.f;        // running maximum (= this thread's best) and sum
-        auto take = [&](float val) {
-            if (val > m) {
-                s = s * ex2((m - val) * kLog2e) + 1.f;
-                m = val;
-            } else if (val > -CUDART_INF_F) {
-                s += ex2((val - m) * kLog2e);
-            } else if (val != val) {
-                s = val;    // NaN poisons the sum and is reported below
-            }
-        };
-        if (kVec) {
-            int i = tid;
-            // four independent 16-byte loads in flight per thread; one rescale per sixteen values
-            for (; i + 3 * kThreads < nvec; i += 4 * kThreads) {
-                const float4 r0 = x4[i], r1 = x4[i + kThreads], r2 = x4[i + 2 * kThreads], r3 = x4[i + 3 * kThreads];
-                const float g01 = fmaxf(fmaxf(fmaxf(r0.x, r0.y), fmaxf(r0.z, r0.w)), fmaxf(fmaxf(r1.x, r1.y), fmaxf(r1.z, r1.w)));
-                const float g23 = fmaxf(fmaxf(fmaxf(r2.x, r2.y), fmaxf(r2.z, r2.w)), fmaxf(fmaxf(r3.x, r3.y), fmaxf(r3.z, r3.w)));
-                const float mn = fmaxf(m, fmaxf(g01, g23));
-                if (mn == -CUDART_INF_F) {
-                    // nothing finite yet; a NaN among the sixteen still has to poison the sum
-                    const float t16 = (r0.x + r0.y + r0.z + r0.w) + (r1.x + r1.y + r1.z + r1.w) + (r2.x + r2.y + r2.z + r2.w) + (r3.x + r3.y + r3.z + r3.w);
-                    if (t16 != t16) s = t16;
-                    continue;
-                }
-                const float kk = -mn * kLog2e;
-                float acc = s * ex2(fmaf(m, kLog2e, kk));
-                acc += ex2(fmaf(r0.x, kLog2e, kk)) + ex2(fmaf(r0.y, kLog2e, kk)) + ex2(fmaf(r0.z, kLog2e, kk)) + ex2(fmaf(r0.w, kLog2e, kk));
-                acc += ex2(fmaf(r1.x, kLog2e, kk)) + ex2(fmaf(r1.y, kLog2e, kk)) + ex2(fmaf(r1.z, kLog2e, kk)) + ex2(fmaf(r1.w, kLog2e, kk));
-                acc += ex2(fmaf(r2.x, kLog2e, kk)) + ex2(fmaf(r2.y, kLog2e, kk)) + ex2(fmaf(r2.z, kLog2e, kk)) + ex2(fmaf(r2.w, kLog2e, kk));
-                acc += ex2(fmaf(r3.x, kLog2e, kk)) + ex2(fmaf(r3.y, kLog2e, kk)) + ex2(fmaf(r3.z, kLog2e, kk)) + ex2(fmaf(r3.w, kLog2e, kk));
-                s = acc;
-                m = mn;
-            }
-            for (; i < nvec; i += kThreads) {
-                const float4 r = x4[i];
-                take(r.x); take(r.y); take(r.z); take(r.w);
-            }
-        } else {
-            for (int i = tid; i < V; i += kThreads) take(x[i]);
+    if (fi >= fl || fl > a.F) return;
+    const float* x = a.logits + ((size_t)b * a.F + fi) * V;
+    const float4* x4 = reinterpret_cast<const float4*>(x);
+    const int nvec = V >> 2;
+    float m = -CUDART_INF_F, s = 0.f;        // running maximum and sum
+    Two two{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF, 0x7FFFFFFF};
+    auto take = [&](float val, int idx) {
+        offer2(two, val, idx);
+        if (val > m) {
+            s = s * ex2((m - val) * kLog2e) + 1.f;
+            m = val;
+        } else if (val > -CUDART_INF_F) {
+            s += ex2((val - m) * kLog2e);
+        } else if (val != val) {
+            s = val;    // NaN poisons the sum and is reported below
         }
-        const float my_best = m;
-        // (maximum, sum) of the row
+    };
+    if (kVec) {
+        const float4 none = make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
+        for (int i = tid; i < nvec; i += 8 * kThreads) {
+            float4 r[8];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m, o), s2 = __shfl_xor_sync(0xFFFFFFFFu, s, o);
-            const float mm = fmaxf(m, m2);
-            s = (mm == -CUDART_INF_F) ? 0.f : s * ex2((m - mm) * kLog2e) + s2 * ex2((m2 - mm) * kLog2e);
-            m = mm;
+            for (int k = 0; k < 8; ++k) r[k] = i + k * kThreads < nvec ? __ldcs(x4 + i + k * kThreads) : none;
+            float g = m;
+            float nan_probe = 0.f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const float g4 = fmaxf(fmaxf(r[k].x, r[k].y), fmaxf(r[k].z, r[k].w));
+                g = fmaxf(g, g4);
+                nan_probe += (r[k].x + r[k].y) + (r[k].z + r[k].w);     // NaN if any entry is NaN (or +inf and -inf meet)
+                if (g4 > two.v2) {      // seldom true once the thread has seen a few entries
+                    const int e = (i + k * kThreads) * 4;
+                    offer2(two, r[k].x, e); offer2(two, r[k].y, e + 1); offer2(two, r[k].z, e + 2); offer2(two, r[k].w, e + 3);
+                }
+            }
+            if (nan_probe != nan_probe) {
+                // rare: find out entry by entry (a NaN poisons the sum; -inf next to +inf does not)
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const float q[4] = {r[k].x, r[k].y, r[k].z, r[k].w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (q[j] != q[j]) s = q[j];
+                }
+            }
+            if (g == -CUDART_INF_F) continue;      // nothing finite yet
+            // one rescale per thirty-two values
+            const float kk = -g * kLog2e;
+            float acc = s * ex2(fmaf(m, kLog2e, kk));
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                acc += (ex2(fmaf(r[k].x, kLog2e, kk)) + ex2(fmaf(r[k].y, kLog2e, kk))) + (ex2(fmaf(r[k].z, kLog2e, kk)) + ex2(fmaf(r[k].w, kLog2e, kk)));
+            s = acc;
+            m = g;
         }
-        if (lane == 0) { s_m[warp] = m; s_s[warp] = s; }
-        if (tid == 0) s_count = 0;
-        __syncthreads();
-        float rm = -CUDART_INF_F, rs = 0.f;
-        for (int w = 0; w < kWarps; ++w) {
-            const float mm = fmaxf(rm, s_m[w]);
-            rs = (mm == -CUDART_INF_F) ? 0.f : rs * ex2((rm - mm) * kLog2e) + s_s[w] * ex2((s_m[w] - mm) * kLog2e);
-            rm = mm;
+    } else {
+        for (int i = tid; i < V; i += kThreads) take(__ldcs(x + i), i);
+    }
+    s_cv[2 * tid] = two.v1; s_ci[2 * tid] = two.i1;
+    s_cv[2 * tid + 1] = two.v2; s_ci[2 * tid + 1] = two.i2;
+    // (maximum, sum) of the row
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m, o), s2 = __shfl_xor_sync(0xFFFFFFFFu, s, o);
+        const float mm = fmaxf(m, m2);
+        s = (mm == -CUDART_INF_F) ? ((s != s || s2 != s2) ? CUDART_NAN_F : 0.f)
+                                  : s * ex2((m - mm) * kLog2e) + s2 * ex2((m2 - mm) * kLog2e);
+        m = mm;
+    }
+    if (lane == 0) { s_m[warp] = m; s_s[warp] = s; }
+    if (tid == 0) s_redo = 0;
+    __syncthreads();
+    float rm = -CUDART_INF_F, rs = 0.f;
+    for (int w = 0; w < kWarps; ++w) {
+        const float mm = fmaxf(rm, s_m[w]);
+        rs = (mm == -CUDART_INF_F) ? ((rs != rs || s_s[w] != s_s[w]) ? CUDART_NAN_F : 0.f)
+                                   : rs * ex2((rm - mm) * kLog2e) + s_s[w] * ex2((s_m[w] - mm) * kLog2e);
+        rm = mm;
+    }
+    if (tid == 0 && (!(rs > 0.f) || rm == CUDART_INF_F) && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
+    const size_t w = ((size_t)b * a.F + fi) * K;
+    if (warp == 0) {
+        float tv;
+        int ti;
+        const int res = warp_pick_k(s_cv, s_ci, 2 * kThreads, a.k, rm, rs, a.wk_tok + w, a.wk_q + w, &tv, &ti);
+        if (lane == 0) {
+            // a thread's second pair among the picks: a third entry of that thread is unknown
+            s_redo = res & 1;
+            s_tv = tv;
+            s_ti = ti;
+            s_count = 0;
+            // (then the second pass below decides whether the row is short of k entries)
+            if ((res & 2) && !(res & 1) && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
         }
-        if (tid == 0 && (!(rs > 0.f) || rm == CUDART_INF_F) && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
-        // the k-th largest of the 256 thread maxima
-        float bound = -CUDART_INF_F;
-        {
-            bool taken = false;
-            for (int r = 0; r < a.k; ++r) {
-                float v = taken ? -CUDART_INF_F : my_best;
-                int i = tid, owner = tid;
-                block_best(v, i, owner, s_rv, s_ri, s_rt);
-                if (owner == tid) taken = true;
-                bound = v;
+    }
+    __syncthreads();
+    if (!s_redo) return;
+    // Second pass (about one random row in fifty): the k-th pick is a lower bound on the row's
+    // k-th best entry, so everything that ranks at or before it is collected from the row (now
+    // in L2) and the pick is repeated over that list.
+    const float tv = s_tv;
+    const int ti = s_ti;
+    __syncthreads();                        // the pairs have been read: the list takes their place
+    auto consider = [&](float val, int idx) {
+        if (val > tv || (val == tv && idx <= ti)) {
+            const int slot = atomicAdd(&s_count, 1);
+            if (slot < 2 * kThreads) { s_cv[slot] = val; s_ci[slot] = idx; }
+        }
+    };
+    if (kVec) {
+        const float4 none = make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
+        for (int i = tid; i < nvec; i += 8 * kThreads) {
+            float4 r[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) r[k] = i + k * kThreads < nvec ? x4[i + k * kThreads] : none;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int e = (i + k * kThreads) * 4;
+                if (fmaxf(fmaxf(r[k].x, r[k].y), fmaxf(r[k].z, r[k].w)) >= tv) {
+                    consider(r[k].x, e); consider(r[k].y, e + 1); consider(r[k].z, e + 2); consider(r[k].w, e + 3);
+                }
             }
         }
-        // pass 2: everything >= bound (and above -inf) is a candidate
-        auto consider = [&](float val, int idx) {
-            if (val >= bound && val > -CUDART_INF_F) {
-                const int slot = atomicAdd(&s_count, 1);
-                if (slot < kCand) { s_cv[slot] = val; s_ci[slot] = idx; }
-            }
-        };
+    } else {
+        for (int i = tid; i < V; i += kThreads) consider(x[i], i);
+    }
+    __syncthreads();
+    const int count = s_count;
+    if (count <= 2 * kThreads) {
+        if (warp == 0) {
+            float lv;
+            int li;
+            const int res = warp_pick_k(s_cv, s_ci, count, a.k, rm, rs, a.wk_tok + w, a.wk_q + w, &lv, &li);
+            if (lane == 0 && (res & 2) && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
+        }
+        return;
+    }
+    {
+        // more than 512 entries rank before the bound (long runs of equal logits in one thread's
+        // share): per-thread lists of the K best pairs, merged by the block
+        TopK t;
+#pragma unroll
+        for (int j = 0; j < K; ++j) {
+            t.v[j] = -CUDART_INF_F;
+            t.i[j] = 0x7FFFFFFF;
+        }
         if (kVec) {
             for (int i = tid; i < nvec; i += kThreads) {
                 const float4 r = x4[i];
-                const int e = i * 4;
-                if (fmaxf(fmaxf(r.x, r.y), fmaxf(r.z, r.w)) >= bound) {
-                    consider(r.x, e); consider(r.y, e + 1); consider(r.z, e + 2); consider(r.w, e + 3);
-                }
+                offer(t, r.x, 4 * i); offer(t, r.y, 4 * i + 1); offer(t, r.z, 4 * i + 2); offer(t, r.w, 4 * i + 3);
             }
         } else {
-            for (int i = tid; i < V; i += kThreads) consider(x[i], i);
-        }
-        __syncthreads();
-        const int count = s_count;
-        const size_t w = ((size_t)b * a.F + fi) * K;
-        if (count <= kCand) {
-            // k rounds over the candidate list: each thread proposes the best of its strided share
-            for (int r = 0; r < a.k; ++r) {
-                float v = -CUDART_INF_F;
-                int i = 0x7FFFFFFF, owner = -1;
-                for (int c = tid; c < count; c += kThreads)
-                    if (before(s_cv[c], s_ci[c], v, i)) { v = s_cv[c]; i = s_ci[c]; owner = c; }
-                block_best(v, i, owner, s_rv, s_ri, s_rt);
-                if (tid == 0) {
-                    if (i == 0x7FFFFFFF && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);   // fewer than k entries above -inf
-                    a.wk_tok[w + r] = i == 0x7FFFFFFF ? -1 : i;
-                    a.wk_q[w + r] = v == -CUDART_INF_F ? 0.f : ex2((v - rm) * kLog2e) / rs;
-                    if (owner >= 0) s_cv[owner] = -CUDART_INF_F;      // taken (an entry at -inf is never a candidate)
-                    if (owner >= 0) s_ci[owner] = 0x7FFFFFFF;
-                }
-                __syncthreads();
-            }
-        } else {
-            // exact fallback: per-thread lists of the K best pairs, merged by the block
-            TopK t;
-#pragma unroll
-            for (int j = 0; j < K; ++j) {
-                t.v[j] = -CUDART_INF_F;
-                t.i[j] = 0x7FFFFFFF;
-            }
             for (int i = tid; i < V; i += kThreads) offer(t, x[i], i);
-            int head = 0;
-            for (int r = 0; r < a.k; ++r) {
-                float v = -CUDART_INF_F;
-                int i = 0x7FFFFFFF;
+        }
+        int head = 0;
+        for (int r = 0; r < a.k; ++r) {
+            float v = -CUDART_INF_F;
+            int i = 0x7FFFFFFF;
 #pragma unroll
-                for (int j = 0; j < K; ++j)
-                    if (j == head) { v = t.v[j]; i = t.i[j]; }
-                int owner = tid;
-                block_best(v, i, owner, s_rv, s_ri, s_rt);
-                if (owner == tid) ++head;
-                if (tid == 0) {
-                    if (i == 0x7FFFFFFF && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
-                    a.wk_tok[w + r] = i == 0x7FFFFFFF ? -1 : i;
-                    a.wk_q[w + r] = v == -CUDART_INF_F ? 0.f : ex2((v - rm) * kLog2e) / rs;
-                }
+            for (int j = 0; j < K; ++j)
+                if (j == head) { v = t.v[j]; i = t.i[j]; }
+            int owner = tid;
+            block_best(v, i, owner, s_rv, s_ri, s_rt);
+            if (owner == tid && i != 0x7FFFFFFF) ++head;
+            if (tid == 0) {
+                if (i == 0x7FFFFFFF && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);   // fewer than k entries above -inf
+                a.wk_tok[w + r] = i == 0x7FFFFFFF ? -1 : i;
+                a.wk_q[w + r] = v == -CUDART_INF_F ? 0.f : ex2((v - rm) * kLog2e) / rs;
             }
         }
     }
-    if (tid == 0) {
-        __threadfence();
-        const unsigned prev = atomicAdd(a.done + b, 1u);
-        s_last = (prev == (unsigned)a.F - 1u);
-    }
-    __syncthreads();
-    if (s_last) {
-        __threadfence();
-        grow_sequence(a, b);
-    }
+}
+
+// Second launch: one CTA per sequence appends the children and updates the graph once every
+// row's result of the first launch is visible.
+__global__ void __launch_bounds__(kThreads) draft_grow_kernel(DraftArgs a) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    grow_sequence(a, blockIdx.x);
 }
 
 }  // namespace
@@ -391,7 +484,7 @@ __global__ void __launch_bounds__(kThreads) draft_expand_kernel(DraftArgs a) {
 
 extern "C" size_t gsd_draft_expand_workspace_bytes(const gsd_draft_params* p) {
     if (!p || p->B < 1 || p->F < 1) return 0;
-    return gsd::align_up((size_t)p->B * p->F * GSD_DRAFT_MAX_K * 8 + (size_t)p->B * 4, 256);
+    return gsd::align_up((size_t)p->B * p->F * GSD_DRAFT_MAX_K * 8, 256);
 }
 
 extern "C" int gsd_draft_expand(const float* logits, const int32_t* frontier, const int32_t* frontier_len,
@@ -418,16 +511,24 @@ extern "C" int gsd_draft_expand(const float* logits, const int32_t* frontier, co
     const size_t rows = (size_t)p->B * p->F * GSD_DRAFT_MAX_K;
     a.wk_tok = (int32_t*)workspace;
     a.wk_q = (float*)((char*)workspace + rows * 4);
-    a.done = (unsigned*)((char*)workspace + rows * 8);
     a.status = status;
     a.B = p->B; a.F = p->F; a.V = p->V; a.Ncap = p->Ncap; a.k = p->k; a.tau = p->tau;
     a.theta_prob = p->theta_prob; a.theta_sib = p->theta_sib;
-    // only the completion counters have to start at zero
-    GSD_CUDA_TRY(cudaMemsetAsync(a.done, 0, (size_t)p->B * 4, st));
+    // every scratch entry is written before it is read: nothing has to start at zero
     const bool vec = (p->V % 4 == 0) && (((uintptr_t)logits & 15u) == 0);
     dim3 grid((unsigned)p->F, (unsigned)p->B);
     if (vec) draft_expand_kernel<true><<<grid, kThreads, 0, st>>>(a);
     else draft_expand_kernel<false><<<grid, kThreads, 0, st>>>(a);
+    GSD_CUDA_TRY(cudaGetLastError());
+    cudaLaunchAttribute attr[1];
+    dependent_launch_attr(attr);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p->B);
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    GSD_CUDA_TRY(cudaLaunchKernelEx(&cfg, draft_grow_kernel, a));
     GSD_CUDA_TRY(cudaGetLastError());
     return GSD_OK;
 }

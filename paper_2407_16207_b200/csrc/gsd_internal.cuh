@@ -21,6 +21,21 @@ void set_error_text(const char* text);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Index checks of the checking build (compiled with -DGSD_BOUNDS_CHECK into libgsd_check.so; the
+// stand-in for a memory sanitizer): at the places where a kernel forms an index into global
+// memory from data or from its work plan, GSD_IN_BOUNDS(condition, status) is the condition
+// itself and, when it fails, ORs GSD_DEV_BOUNDS into the status word - the caller skips the
+// access, nothing traps.  In the ordinary build it is the constant true and costs nothing.
+#ifdef GSD_BOUNDS_CHECK
+__device__ __forceinline__ bool note_out_of_bounds(int32_t* status) {
+    if (status) atomicOr((unsigned*)status, GSD_DEV_BOUNDS);
+    return false;
+}
+#define GSD_IN_BOUNDS(cond, status) ((cond) ? true : ::gsd::note_out_of_bounds(status))
+#else
+#define GSD_IN_BOUNDS(cond, status) (true)
+#endif
+
 struct DeviceInfo {
     int sm_count;
     int max_smem_optin;
@@ -86,6 +101,8 @@ int launch_attn_mma(const AttnArgs& a);
 int launch_attn_tcgen05(const AttnArgs& a);
 bool attn_tcgen05_supports(int D, int G);
 int launch_attn_merge(const AttnArgs& a);
+// test hook behind gsd_debug_attn_wait (process-wide; 0 restores the default limit)
+void debug_attn_wait(unsigned long long limit_ns, int withhold_first_k);
 
 // ---- scratch words that must start at zero ----
 // Enqueues a small kernel that zeroes `n` 32-bit words and lets the next launch on the stream

@@ -196,6 +196,7 @@ __device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, St
     for (int i = tid; i <= io.Tcap; i += kPathThreads) {
         if (i <= m) {
             const int node = s_path[i];
+            if (!GSD_IN_BOUNDS(node >= 0 && node < N && i < GSD_MAX_NODES, io.status)) continue;
             if (io.out_nodes && i < io.Tcap) io.out_nodes[i] = node;
             if (i >= 1) io.out_tok[i - 1] = s_tok[node];    // i - 1 < Tcap
         } else if (i < io.Tcap) {

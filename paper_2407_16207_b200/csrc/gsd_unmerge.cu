@@ -157,6 +157,7 @@ unmerge_kernel(const int32_t* tok_all, const int32_t* pptr_all, const int32_t* p
                 const int idx = first + j;
                 if (idx >= Ucap) break;
                 const int child = s_child[s_cptr[src] + j];
+                if (!GSD_IN_BOUNDS(child > src && child < N && s_cptr[src] + j < kMaxEdges, status)) continue;
                 tt[idx] = s_tok[child];
                 tp[idx] = u;
                 ts[idx] = child;
