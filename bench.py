@@ -3,6 +3,7 @@
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
   python bench.py --sweep [--points B1_L512_N32,...]      one JSON line per point of the 70B-shaped sweep
+  python bench.py --ab-unmerge                             graph-direct vs unmerged-tree verification
 
 A step is one pass of the whole hot path over one batch of synthetic LLaMA-2-shaped input:
 DAG-masked attention of all draft nodes, then vocabulary argmax and longest accepted path.
@@ -358,6 +359,114 @@ def run_sweep(args):
         torch.cuda.empty_cache()
 
 
+def run_ab_unmerge(args):
+    """Verification of the token graph itself (a node merged from several branches attends to
+    the union of its ancestors) against verification of the paper's unmerged tree (Sec. 5.4): on
+    graphs grown on the device by gsd_draft_expand from seeded draft logits whose mass sits on a
+    small, context-dependent set of tokens (so that tau-grams re-occur as in the paper's Fig. 3),
+    with the paper's settings k = 4, tau = 2, theta_prob = 0.2, theta_sib = 0.3, six draft steps
+    (the paper allows ten; six keep the graph under this library's 512 nodes).
+    Prints one JSON line: node counts, attention time of both forms on the 70B layer shape, and
+    how far the attention rows of the two forms are apart."""
+    import paper_2407_16207_b200 as gsd
+    from gsd_inputs.torch_io import i32_tensor
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    B, V, Ncap, k, tau, steps = 8, 32000, 512, 4, 2, 6
+    Hq, Hkv, D, L = 64, 8, 128, 4096
+    hot = 48                                             # tokens that ever get mass
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(2407)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    tokens = torch.zeros((B, Ncap), dtype=torch.int32, device=dev)
+    tokens[:, 0] = torch.randint(0, hot, (B,), device=dev, generator=gen, dtype=torch.int32)
+    parent = torch.full((B, Ncap), -1, dtype=torch.int32, device=dev)
+    merge = torch.full((B, Ncap), -1, dtype=torch.int32, device=dev)
+    leaf = torch.zeros((B, Ncap), dtype=torch.uint8, device=dev)
+    prob = torch.zeros((B, Ncap), dtype=torch.float32, device=dev)
+    num = torch.ones((B,), dtype=torch.int32, device=dev)
+    frontier = torch.zeros((B, 1), dtype=torch.int32, device=dev)
+    flen = torch.ones((B,), dtype=torch.int32, device=dev)
+    # the draft distribution after a token t: mass on six tokens of the hot set chosen by t
+    table = torch.randint(0, hot, (hot, 6), device=dev, generator=gen)
+    lvl = torch.tensor([4.0, 3.9, 3.8, 3.0, 2.0, 1.0], device=dev)      # three children of a node pass theta_prob = 0.2
+    for _ in range(steps):
+        F = int(frontier.shape[1])
+        tok_f = torch.gather(tokens, 1, frontier.clamp(min=0).long())            # [B,F] token of each frontier node
+        lg = torch.full((B, F, V), -8.0, device=dev) + 0.3 * torch.randn((B, F, V), device=dev, generator=gen)
+        lg.scatter_(2, table[tok_f.long() % hot], (lvl + 0.2 * torch.randn((B, F, 6), device=dev, generator=gen)))
+        nf, nfl = gsd.gsd_draft_expand(lg, frontier, flen, tokens, parent, merge, leaf, prob, num, k=k, tau=tau,
+                                       theta_prob=0.2, theta_sib=0.3, status=status)
+        width = int(nfl.max().item())
+        if width == 0:
+            break
+        frontier, flen = nf[:, :width].contiguous().clamp(min=0), nfl
+    torch.cuda.synchronize()
+    graph_full = bool(int(status.item()) & 0x80)          # the node capacity ended the growth
+    status.zero_()
+    n = num.cpu().numpy()
+    par_h, mrg_h = parent.cpu().numpy(), merge.cpu().numpy()
+    N = int(n.max())
+    # parent lists of the verification DAG: a node also hangs under the nodes merged into its parent
+    parents = []
+    for b in range(B):
+        into = {}
+        for r in range(n[b]):
+            if mrg_h[b, r] >= 0:
+                into.setdefault(int(mrg_h[b, r]), []).append(r)
+        ps = [[]]
+        for x in range(1, n[b]):
+            p = int(par_h[b, x])
+            ps.append(sorted([p] + [r for r in into.get(p, []) if r < x]))
+        parents.append(ps + [[] for _ in range(N - n[b])])
+    ptr, idx = gi.parents_to_csr(parents)
+    d_ptr, d_idx = i32_tensor(ptr, dev), i32_tensor(idx, dev)
+    d_tok = tokens[:, :N].contiguous()
+    mask = gsd.gsd_build_mask(d_ptr, d_idx)
+    q = torch.randn((B, N, Hq, D), device=dev, generator=gen).to(torch.bfloat16)
+    dk = torch.randn((B, N, Hkv, D), device=dev, generator=gen).to(torch.bfloat16)
+    dv = torch.randn((B, N, Hkv, D), device=dev, generator=gen).to(torch.bfloat16)
+    kc = torch.randn((B, L, Hkv, D), device=dev, generator=gen).to(torch.bfloat16)
+    vc = torch.randn((B, L, Hkv, D), device=dev, generator=gen).to(torch.bfloat16)
+    sl = torch.full((B,), L, dtype=torch.int32, device=dev)
+    out_g = torch.empty_like(q)
+    t_graph = timed_calls(lambda i: gsd.gsd_verify_attn(q, kc, vc, dk, dv, mask, sl, out=out_g, status=status))
+    # the unmerged tree (at most Ncap nodes, at most `steps` edges deep), its single-parent lists and mask
+    _, _, _, cnt_all = gsd.gsd_unmerge_tree(d_tok, d_ptr, d_idx, Ucap=1 << 16, max_depth=steps, status=status)
+    tree_nodes_all = cnt_all.cpu().numpy()                 # the whole tree, for its size
+    status.zero_()
+    # the attention call takes at most 512 nodes: the first 512 of the level order are timed
+    tt, tp, ts, cnt = gsd.gsd_unmerge_tree(d_tok, d_ptr, d_idx, Ucap=Ncap, max_depth=steps, status=status)
+    torch.cuda.synchronize()
+    full = bool(int(status.item()) & 0x200)
+    status.zero_()
+    cnt_h, tp_h = cnt.cpu().numpy(), tp.cpu().numpy()
+    U = int(cnt_h.max())
+    tparents = [[[] if (u == 0 or u >= cnt_h[b]) else [int(tp_h[b, u])] for u in range(U)] for b in range(B)]
+    tptr, tidx = gi.parents_to_csr(tparents)
+    tmask = gsd.gsd_build_mask(i32_tensor(tptr, dev), i32_tensor(tidx, dev))
+    src = ts[:, :U].clamp(min=0).long()
+    take = lambda x: torch.gather(x, 1, src.view(B, U, 1, 1).expand(-1, -1, x.shape[2], x.shape[3])).contiguous()
+    q_t, dk_t, dv_t = take(q), take(dk), take(dv)
+    out_t = torch.empty_like(q_t)
+    t_tree = timed_calls(lambda i: gsd.gsd_verify_attn(q_t, kc, vc, dk_t, dv_t, tmask, sl, out=out_t, status=status))
+    # rows of the graph form against the rows of their tree copies
+    diff = (out_t.float() - take(out_g).float()).abs()
+    valid = (torch.arange(U, device=dev)[None, :] < cnt[:, None])
+    per_node = diff.amax(dim=(2, 3))[valid]
+    line = {"mode": "ab_unmerge", "sequences": B, "draft_steps": steps, "k": k, "tau": tau,
+            "graph_nodes_mean": float(n.mean()), "graph_nodes_max": N,
+            "merged_nodes_mean": float((mrg_h >= 0).sum() / B), "graph_capacity_reached": graph_full,
+            "tree_nodes_mean": float(tree_nodes_all.mean()), "tree_nodes_max": int(tree_nodes_all.max()),
+            "tree_nodes_timed_mean": float(cnt_h.mean()), "tree_truncated_to_512_for_timing": full,
+            "attn_us_graph": t_graph, "attn_us_tree": t_tree,
+            "rows_graph": int(n.sum()) * Hq, "rows_tree": int(cnt_h.sum()) * Hq,
+            "tree_copies_whose_row_differs": float((per_node > 1e-3).float().mean().item()),
+            "max_abs_difference": float(per_node.max().item()), "mean_abs_difference": float(diff[valid].mean().item()),
+            "shape": {"Hq": Hq, "Hkv": Hkv, "D": D, "L": L, "V": V}}
+    print(json.dumps(line), flush=True)
+
+
 def timed_calls(fn, before=None, n=20, warm=3):
     """Median CUDA-event time in microseconds of `fn(i)` over n calls after `warm` untimed ones;
     `before(i)` runs ahead of each call, outside its pair of events."""
@@ -388,12 +497,17 @@ def main():
                     help="auto: the whole step on the named configurations, a sample on sweep points")
     ap.add_argument("--sweep", action="store_true", help="one JSON line per point of the 70B-shaped sweep")
     ap.add_argument("--points", default="", help="with --sweep: comma-separated workload names")
+    ap.add_argument("--ab-unmerge", action="store_true",
+                    help="graph-direct against unmerged-tree verification on grown graphs; one JSON line")
     args = ap.parse_args()
     args.steps_given = args.steps is not None
     if args.steps is None:
         args.steps = 6000
     if args.sweep:
         run_sweep(args)
+        return
+    if args.ab_unmerge:
+        run_ab_unmerge(args)
         return
     cfg = config_by_name(args.workload)
     if args.impl == "reference":
@@ -476,8 +590,8 @@ def main():
     total_ms = ms_per_step * args.steps
 
     # ---- side timings on rank 0, each call between its own CUDA events; none is part of `value`
-    commit_us = sampled_us = draft_us = None
-    sampled_bytes = draft_bytes = 0.0
+    commit_us = sampled_us = draft_us = draft_us_big = None
+    sampled_bytes = draft_bytes = draft_bytes_big = 0.0
     if rank == 0:
         # the cache update that follows the step (gsd_commit_kv) on a cache with head room
         t0s = sets[0]
@@ -502,35 +616,42 @@ def main():
         usm = torch.rand((cfg.B,), device=dev, generator=gen)
         ws_s = torch.empty(gsd.gsd_accept_sampled_workspace_bytes(cfg.B, cfg.N), dtype=torch.uint8, device=dev)
 
+        acc_out_s = tuple(torch.empty_like(x) for x in acc_out)
+
         def sampled(i):
             ts, td = sets[i % NSETS], sets[(i + 1) % NSETS]
             gsd.gsd_accept_sampled(ts["logits"], ts["draft_tokens"], ts["parent_ptr"], ts["parent_idx"], dq, ua, usm,
-                                   draft_logits=td["logits"], workspace=ws_s, status=status)
+                                   draft_logits=td["logits"], workspace=ws_s, status=status, out=acc_out_s)
         sampled_us = timed_calls(sampled)
         sampled_bytes = 4.0 * cfg.V * (cfg.B * cfg.N + cfg.B)
 
         # one growth step of the draft token graph (gsd_draft_expand): 64 frontier rows per
-        # sequence of random draft logits over the same vocabulary, on a graph of 104 earlier nodes
-        gen.manual_seed(11)
-        Fr, Ncap, n_old = 64, 512, 104
-        dl = [torch.randn((cfg.B, Fr, cfg.V), device=dev, generator=gen) * 3 for _ in range(2)]
-        g_tok = torch.randint(0, cfg.V, (cfg.B, Ncap), device=dev, generator=gen, dtype=torch.int32)
-        g_par = (torch.arange(Ncap, device=dev, dtype=torch.int32) - 1).clamp(min=0).repeat(cfg.B, 1).contiguous()
-        g_par[:, 0] = -1
-        g_mrg = torch.full((cfg.B, Ncap), -1, dtype=torch.int32, device=dev)
-        g_leaf = torch.zeros((cfg.B, Ncap), dtype=torch.uint8, device=dev)
-        g_prob = torch.zeros((cfg.B, Ncap), dtype=torch.float32, device=dev)
-        n_ref = torch.full((cfg.B,), n_old, dtype=torch.int32, device=dev)
-        g_n = n_ref.clone()
-        fr = (torch.arange(Fr, device=dev, dtype=torch.int32) % n_old).repeat(cfg.B, 1).contiguous()
-        fl = torch.full((cfg.B,), Fr, dtype=torch.int32, device=dev)
+        # sequence of random draft logits over the same vocabulary, on a graph of 104 earlier nodes,
+        # k = 4; once with the workload's batch and once with 32 sequences (262 MB of draft logits)
+        def time_draft(Bd):
+            gen.manual_seed(11)
+            Fr, Ncap, n_old, k = 64, 512, 104, 4
+            dl = [torch.randn((Bd, Fr, cfg.V), device=dev, generator=gen) * 3 for _ in range(2)]
+            g_tok = torch.randint(0, cfg.V, (Bd, Ncap), device=dev, generator=gen, dtype=torch.int32)
+            g_par = (torch.arange(Ncap, device=dev, dtype=torch.int32) - 1).clamp(min=0).repeat(Bd, 1).contiguous()
+            g_par[:, 0] = -1
+            g_mrg = torch.full((Bd, Ncap), -1, dtype=torch.int32, device=dev)
+            g_leaf = torch.zeros((Bd, Ncap), dtype=torch.uint8, device=dev)
+            g_prob = torch.zeros((Bd, Ncap), dtype=torch.float32, device=dev)
+            n_ref = torch.full((Bd,), n_old, dtype=torch.int32, device=dev)
+            g_n = n_ref.clone()
+            fr = (torch.arange(Fr, device=dev, dtype=torch.int32) % n_old).repeat(Bd, 1).contiguous()
+            fl = torch.full((Bd,), Fr, dtype=torch.int32, device=dev)
+            nf = (torch.empty((Bd, Fr * k), dtype=torch.int32, device=dev), torch.empty((Bd,), dtype=torch.int32, device=dev))
+            ws_d = torch.empty(Bd * Fr * 8 * 8 + 256, dtype=torch.uint8, device=dev)
 
-        def draft(i):
-            gsd.gsd_draft_expand(dl[i % 2], fr, fl, g_tok, g_par, g_mrg, g_leaf, g_prob, g_n, k=4, tau=2,
-                                 theta_prob=0.01, theta_sib=0.1, status=status)
-        draft_us = timed_calls(draft, before=lambda i: g_n.copy_(n_ref))
-        draft_bytes = 4.0 * cfg.B * Fr * cfg.V
-        del dl
+            def draft(i):
+                gsd.gsd_draft_expand(dl[i % 2], fr, fl, g_tok, g_par, g_mrg, g_leaf, g_prob, g_n, k=k, tau=2,
+                                     theta_prob=0.01, theta_sib=0.1, status=status, workspace=ws_d, out=nf)
+            us = timed_calls(draft, before=lambda i: g_n.copy_(n_ref))
+            return us, 4.0 * Bd * Fr * cfg.V
+        draft_us, draft_bytes = time_draft(cfg.B)
+        draft_us_big, draft_bytes_big = time_draft(32)
 
     # ---- end to end through the host-buffer C-ABI call (pinned host tensors)
     e2e = None
@@ -614,6 +735,8 @@ def main():
         "accept_frac_of_hbm": accept_bytes / acc_mean / 1e9 / hbm,
         "accept_sampled_frac_of_hbm": (sampled_bytes / (sampled_us * 1e-6) / 1e9 / hbm) if sampled_us else None,
         "draft_expand_frac_of_hbm": (draft_bytes / (draft_us * 1e-6) / 1e9 / hbm) if draft_us else None,
+        "draft_expand_262mb_us": draft_us_big,
+        "draft_expand_262mb_frac_of_hbm": (draft_bytes_big / (draft_us_big * 1e-6) / 1e9 / hbm) if draft_us_big else None,
         "roofline": roof, "cpu_baseline": cpu, "e2e": e2e,
         # per step: the attention kernel (+ its merge pass when key ranges are cut), the scratch
         # clear of gsd_accept and the accept kernel
