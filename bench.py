@@ -161,7 +161,7 @@ class ClockSampler:
             except Exception as e:  # pragma: no cover
                 self.err = str(e)
                 return
-            self._stop.wait(0.01)
+            self._stop.wait(0.002)
 
     def stop(self):
         self._stop.set()

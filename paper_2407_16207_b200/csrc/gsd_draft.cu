@@ -80,6 +80,9 @@ __device__ void grow_sequence(const DraftArgs& a, int b) {
     __shared__ unsigned char s_leaf[GSD_MAX_NODES];
     __shared__ __align__(16) unsigned s_key[GSD_MAX_NODES];   // hash of the tau-gram that ends at a node (kNoGram: none)
     __shared__ int s_cnt[kWarps];
+    constexpr int kHashBits = 10, kHashSlots = 1 << kHashBits;     // twice the largest node count
+    __shared__ unsigned s_hkey[kHashSlots];
+    __shared__ int s_hmin[kHashSlots];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int Ncap = a.Ncap, k = a.k;
     int32_t* tok = a.tokens + (size_t)b * Ncap;
@@ -128,8 +131,7 @@ __device__ void grow_sequence(const DraftArgs& a, int b) {
     __syncthreads();
     // Sec. 5.2 / 5.3: a new node whose last tau tokens along its tree path equal those of an
     // earlier node is redundant; it becomes a leaf that points at the first such node.
-    // A 32-bit hash of every node's tau-gram makes the scan over the earlier nodes one
-    // comparison per node; equal hashes are confirmed token by token.
+    // Every node's tau-gram is reduced to a 32-bit hash; equal hashes are confirmed token by token.
     constexpr unsigned kNoGram = 0xFFFFFFFFu;
     for (int v = tid; v < n1; v += kThreads) {
         unsigned h = 2166136261u;
@@ -150,19 +152,51 @@ __device__ void grow_sequence(const DraftArgs& a, int b) {
         }
         return true;
     };
+    // first occurrences through a hash table in shared memory: every node with a tau-gram enters
+    // its id under its hash (open addressing; the slot keeps the lowest id), so a new node finds
+    // the lowest earlier node with its hash in one probe sequence instead of a scan over all
+    // earlier nodes.  Equal hashes are confirmed token by token; if the lowest id under the hash
+    // is a different gram (a collision of the 32-bit hash) the node falls back to the scan.
+    for (int t = tid; t < kHashSlots; t += kThreads) {
+        s_hkey[t] = kNoGram;
+        s_hmin[t] = 0x7FFFFFFF;
+    }
+    __syncthreads();
+    for (int v = tid; v < n1; v += kThreads) {
+        const unsigned kv = s_key[v];
+        if (kv == kNoGram) continue;
+        unsigned slot = (kv * 2654435761u) >> (32 - kHashBits);
+        for (int probe = 0; probe < kHashSlots; ++probe) {
+            const unsigned prev = atomicCAS(&s_hkey[slot], kNoGram, kv);
+            if (prev == kNoGram || prev == kv) {
+                atomicMin(&s_hmin[slot], v);
+                break;
+            }
+            slot = (slot + 1) & (kHashSlots - 1);
+        }
+    }
+    __syncthreads();
     for (int j = tid; j < want; j += kThreads) {
         const int c = n0 + j;
         const unsigned kc = s_key[c];
         int first = -1;
         if (kc != kNoGram) {
-            const uint4* k4 = reinterpret_cast<const uint4*>(s_key);
-            for (int e4 = 0; e4 * 4 < c && first < 0; ++e4) {
-                const uint4 q = k4[e4];
-                const int e = e4 * 4;
-                if (q.x == kc && e < c && same_gram(c, e)) first = e;
-                else if (q.y == kc && e + 1 < c && same_gram(c, e + 1)) first = e + 1;
-                else if (q.z == kc && e + 2 < c && same_gram(c, e + 2)) first = e + 2;
-                else if (q.w == kc && e + 3 < c && same_gram(c, e + 3)) first = e + 3;
+            unsigned slot = (kc * 2654435761u) >> (32 - kHashBits);
+            int lowest = c;
+            for (int probe = 0; probe < kHashSlots; ++probe) {
+                const unsigned k = s_hkey[slot];
+                if (k == kc) { lowest = s_hmin[slot]; break; }
+                if (k == kNoGram) break;                       // (cannot happen: c itself is in the table)
+                slot = (slot + 1) & (kHashSlots - 1);
+            }
+            if (lowest < c) {
+                if (same_gram(c, lowest)) {
+                    first = lowest;
+                } else {
+                    // another gram with the same hash sits below: look at every earlier node
+                    for (int e = 0; e < c && first < 0; ++e)
+                        if (s_key[e] == kc && same_gram(c, e)) first = e;
+                }
             }
         }
         if (first >= 0) s_leaf[c] = 1;
@@ -214,7 +248,7 @@ __device__ __forceinline__ void block_best(float& v, int& i, int& owner, float* 
 }
 
 // The k best tokens of one row of logits and their probabilities, in one pass over the row.
-// Every thread streams its strided share (16-byte loads, eight in flight) and keeps the running
+// Every thread streams its strided share (16-byte loads, kBatch in flight) and keeps the running
 // (maximum, sum of exponentials) pair and the two best (logit, token) pairs it has met.  The
 // 512 pairs go to shared memory and one warp picks the row's k best of them with shuffles
 // (ranked by logit, ties to the lower token id).  That is the exact answer unless a thread's
@@ -224,6 +258,7 @@ __device__ __forceinline__ void block_best(float& v, int& i, int& owner, float* 
 // and the pick is repeated over the list.  Only a list longer than 512 (long runs of equal
 // logits) takes the slow exact way: every thread keeps the K best pairs it meets and the block
 // merges the 256 lists.
+constexpr int kBatch = 8;     // 16-byte loads a thread keeps in flight while it streams a row
 struct Two {
     float v1, v2;
     int i1, i2;
@@ -318,14 +353,14 @@ __global__ void __launch_bounds__(kThreads, 5) draft_expand_kernel(DraftArgs a) 
     };
     if (kVec) {
         const float4 none = make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
-        for (int i = tid; i < nvec; i += 8 * kThreads) {
-            float4 r[8];
+        for (int i = tid; i < nvec; i += kBatch * kThreads) {
+            float4 r[kBatch];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) r[k] = i + k * kThreads < nvec ? __ldcs(x4 + i + k * kThreads) : none;
+            for (int k = 0; k < kBatch; ++k) r[k] = i + k * kThreads < nvec ? __ldcs(x4 + i + k * kThreads) : none;
             float g = m;
             float nan_probe = 0.f;
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
+            for (int k = 0; k < kBatch; ++k) {
                 const float g4 = fmaxf(fmaxf(r[k].x, r[k].y), fmaxf(r[k].z, r[k].w));
                 g = fmaxf(g, g4);
                 nan_probe += (r[k].x + r[k].y) + (r[k].z + r[k].w);     // NaN if any entry is NaN (or +inf and -inf meet)
@@ -337,7 +372,7 @@ __global__ void __launch_bounds__(kThreads, 5) draft_expand_kernel(DraftArgs a) 
             if (nan_probe != nan_probe) {
                 // rare: find out entry by entry (a NaN poisons the sum; -inf next to +inf does not)
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
+                for (int k = 0; k < kBatch; ++k) {
                     const float q[4] = {r[k].x, r[k].y, r[k].z, r[k].w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
@@ -345,11 +380,11 @@ __global__ void __launch_bounds__(kThreads, 5) draft_expand_kernel(DraftArgs a) 
                 }
             }
             if (g == -CUDART_INF_F) continue;      // nothing finite yet
-            // one rescale per thirty-two values
+            // one rescale per batch
             const float kk = -g * kLog2e;
             float acc = s * ex2(fmaf(m, kLog2e, kk));
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
+            for (int k = 0; k < kBatch; ++k)
                 acc += (ex2(fmaf(r[k].x, kLog2e, kk)) + ex2(fmaf(r[k].y, kLog2e, kk))) + (ex2(fmaf(r[k].z, kLog2e, kk)) + ex2(fmaf(r[k].w, kLog2e, kk)));
             s = acc;
             m = g;
