@@ -262,6 +262,9 @@ extern "C" int gsd_verify_step_host(const void* q, const void* k_cache, const vo
         return GSD_ERR_NULL_POINTER;
     const int ok = attn_params_ok(ap);
     if (ok != GSD_OK) return ok;
+    // everything gsd_accept would refuse is refused here, before a byte is copied
+    if (cp->B < 1 || cp->N < 1 || cp->N > GSD_MAX_NODES || cp->V < 1 || cp->Ecap < 1 || cp->Tcap < 1)
+        return GSD_ERR_BAD_SHAPE;
     ArenaLayout L;
     if (!arena_layout(ap, cp, &L)) return GSD_ERR_BAD_SHAPE;
     if (arena_bytes < L.total) return GSD_ERR_WORKSPACE;
@@ -274,6 +277,10 @@ extern "C" int gsd_verify_step_host(const void* q, const void* k_cache, const vo
     HostStepStreams* hs = host_step_streams();
     if (!hs) return GSD_ERR_CUDA;
     cudaStream_t cs = hs->copy;
+    int32_t dev_status = 0;
+    // From here on work is in flight on both streams: whatever goes wrong, both are drained before
+    // the call returns, so that the caller's host buffers and the arena are free again.
+    auto enqueue = [&]() -> int {
     GSD_CUDA_TRY(cudaEventRecord(hs->entered, st));           // the arena may still be in use by earlier work on `stream`
     GSD_CUDA_TRY(cudaStreamWaitEvent(cs, hs->entered, 0));
     auto h2d = [&](size_t off, const void* src, size_t bytes) {
@@ -311,9 +318,14 @@ extern "C" int gsd_verify_step_host(const void* q, const void* k_cache, const vo
     GSD_CUDA_TRY(cudaMemcpyAsync(accepted_len, base + L.alen, L.b_len, cudaMemcpyDeviceToHost, st));
     if (accepted_nodes)
         GSD_CUDA_TRY(cudaMemcpyAsync(accepted_nodes, base + L.anodes, L.b_acc, cudaMemcpyDeviceToHost, st));
-    int32_t dev_status = 0;
     GSD_CUDA_TRY(cudaMemcpyAsync(&dev_status, base + L.status, 4, cudaMemcpyDeviceToHost, st));
-    GSD_CUDA_TRY(cudaStreamSynchronize(st));
+    return GSD_OK;
+    };
+    const int rc_enqueue = enqueue();
+    const cudaError_t e_copy = cudaStreamSynchronize(cs), e_main = cudaStreamSynchronize(st);
+    if (rc_enqueue != GSD_OK) return rc_enqueue;
+    if (e_copy != cudaSuccess) { set_cuda_error(e_copy, "cudaStreamSynchronize(copy stream)"); return GSD_ERR_CUDA; }
+    if (e_main != cudaSuccess) { set_cuda_error(e_main, "cudaStreamSynchronize(stream)"); return GSD_ERR_CUDA; }
     if (device_status_out) *device_status_out = dev_status;
     return GSD_OK;
 }

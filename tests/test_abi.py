@@ -72,3 +72,11 @@ def test_host_side_validation_needs_no_gpu(library):
     ap = AcceptParams(1, 4, 10, 4, 4)
     assert library.gsd_accept(one, one, one, one, one, one, None, ctypes.byref(ap), None, 0,
                               None, None) == -4
+    # the host-buffer step refuses what its acceptance half would refuse before a byte is copied
+    # (V = 0 here): no device is needed to see that nothing was enqueued
+    good = AttnParams(1, 16, 4, 4, 64, 128, 0.0, 0, 0)
+    cp = AcceptParams(1, 16, 0, 8, 16)
+    args = [one] * 8 + [ctypes.byref(good)] + [one] * 6 + [None, ctypes.byref(cp), ctypes.c_void_p(256),
+                                                            ctypes.c_size_t(1 << 30), None, None]
+    library.gsd_verify_step_host.restype = ctypes.c_int
+    assert library.gsd_verify_step_host(*args) == -2
