@@ -67,9 +67,14 @@ typedef enum gsd_status {
 #define GSD_MAX_NODES 512          /* largest supported N (draft nodes per sequence) */
 
 /* kernel selection for gsd_verify_attn */
+/* GSD_ATTN_AUTO takes the tcgen05 kernel when it supports the shape and the stacked rows of one
+ * (sequence, kv head), N * Hq/Hkv, number at least 64; everything else runs on the mma.sync
+ * kernel, which reaches roughly a sixth of the tensor throughput (group sizes 3, 6, 12, ... and
+ * D == 64 therefore stay correct but slow).  Asking for GSD_ATTN_TCGEN05 on a shape it does
+ * not support returns GSD_ERR_UNSUPPORTED. */
 #define GSD_ATTN_AUTO 0
-#define GSD_ATTN_MMA  1            /* warp-level mma.sync kernel: D in {64,128}, any N */
-#define GSD_ATTN_TCGEN05 2         /* tcgen05/TMEM/TMA kernel: D == 128 */
+#define GSD_ATTN_MMA  1            /* warp-level mma.sync kernel: D in {64,128}, any N, any group size */
+#define GSD_ATTN_TCGEN05 2         /* tcgen05/TMEM/TMA kernel: D == 128 and Hq/Hkv a divisor of 128 */
 
 typedef struct gsd_attn_params {
     int32_t B;            /* sequences */
