@@ -12,7 +12,7 @@ CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libgsd.so")
 LIB_CHECK = os.path.join(PKG, "libgsd_check.so")
 OBJ_DIR = os.path.join(PKG, "_build")
-SOURCES = ["gsd_api.cu", "gsd_accept.cu", "gsd_accept_sampled.cu", "gsd_draft.cu", "gsd_attn_mma.cu", "gsd_attn_tc.cu", "gsd_commit.cu", "gsd_mask.cu", "gsd_unmerge.cu"]
+SOURCES = ["gsd_api.cu", "gsd_accept.cu", "gsd_accept_sampled.cu", "gsd_draft.cu", "gsd_attn_mma.cu", "gsd_attn_tc.cu", "gsd_attn_plan.cu", "gsd_commit.cu", "gsd_mask.cu", "gsd_unmerge.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -34,7 +34,7 @@ int device_info(DeviceInfo* out) {
 static int attn_params_ok(const gsd_attn_params* p) {
     if (!p) return GSD_ERR_NULL_POINTER;
     if (p->B < 1 || p->N < 1 || p->N > GSD_MAX_NODES || p->Hq < 1 || p->Hkv < 1 ||
-        p->Hq % p->Hkv != 0 || (p->D != 64 && p->D != 128) || p->Lmax < 1 || p->num_splits < 0 ||
+        p->Hq % p->Hkv != 0 || (p->D != 64 && p->D != 128) || p->Lmax < 1 || p->num_splits < GSD_ATTN_SPLIT_BALANCED ||
         p->num_splits > 64)
         return GSD_ERR_BAD_SHAPE;
     if ((long long)p->B * p->Hkv > 65535) return GSD_ERR_BAD_SHAPE;
@@ -71,6 +71,23 @@ AttnPlan attn_make_plan(const gsd_attn_params* p, int sm_count) {
     pl.dev.items_a = pl.items;
     pl.dev.splits_a = 1;
     pl.dev.splits_b = 1;
+    pl.dev.balanced = 0;
+    // Shares of key tiles dealt out on the device from the true sequence lengths: on request
+    // only.  Every cut costs a partial result (an fp32 accumulator tile written and read back,
+    // as much traffic as a key tile), so it pays when the lengths of a batch differ by far
+    // more than a share - one long context among short ones - and loses otherwise.
+    const int tpu = pl.dev.tiles_per_unit;
+    if (tc && p->num_splits == GSD_ATTN_SPLIT_BALANCED && resident <= 1024 && tpu <= resident &&
+        (long long)pl.items * tiles < (1ll << 30)) {
+        pl.dev.balanced = 1;
+        // one group of tpu CTAs (a CTA per row-tile item) per share of the line
+        const long long line = (long long)(pl.items / tpu) * tiles;   // tiles at full length
+        const int groups = (int)(line < resident / tpu ? line : resident / tpu);
+        pl.ctas = groups * tpu;
+        pl.slots = 2 * pl.ctas;                                        // a CTA's first and last unit
+        pl.ws_bytes = plan_part_o_bytes(pl, p->D) + plan_part_ml_bytes(pl) + plan_bal_bytes(pl, p->B);
+        return pl;
+    }
     if (p->num_splits > 0) {
         pl.dev.splits_a = p->num_splits;
     } else if (pl.items < resident) {
@@ -127,6 +144,7 @@ extern "C" int gsd_verify_attn_num_splits(const gsd_attn_params* p) {
     DeviceInfo di;
     if (device_info(&di) != 0) return 0;
     const AttnPlan pl = attn_make_plan(p, di.sm_count);
+    if (pl.dev.balanced) return GSD_ATTN_SPLIT_BALANCED;
     return pl.dev.splits_a > pl.dev.splits_b ? pl.dev.splits_a : pl.dev.splits_b;
 }
 
@@ -167,7 +185,9 @@ extern "C" int gsd_verify_attn(const void* q, const void* k_cache, const void* v
     a.scale_log2 = scale * 1.4426950408889634f;
     a.plan = plan; a.workspace = workspace; a.status = status;
     a.stream = (cudaStream_t)stream;
-    int rc = plan.kernel == GSD_ATTN_TCGEN05 ? launch_attn_tcgen05(a) : launch_attn_mma(a);
+    int rc = GSD_OK;
+    if (plan.dev.balanced && (rc = launch_attn_plan(a)) != GSD_OK) return rc;
+    rc = plan.kernel == GSD_ATTN_TCGEN05 ? launch_attn_tcgen05(a) : launch_attn_mma(a);
     if (rc != GSD_OK) return rc;
     if (plan.slots > 0) rc = launch_attn_merge(a);
     return rc;

@@ -350,18 +350,30 @@ struct MergeParams {
     __nv_bfloat16* out;
     PlanDev plan;
     int N, Hq, Hkv, G, R, D, rows_per_item, items;
-    long warps_total;  // split items * rows_per_item
+    int rows_used;     // min(rows_per_item, R): rows of an item that can exist
+    long warps_total;  // split items * rows_used
+    const int* bal_hdr;      // balanced plan: [0] = items to merge (known on the device only)
+    const int4* bal_merge;   // balanced plan: (pair, first slot, slots) per pair to merge, else nullptr
+    int bal_groups;          // balanced plan: groups of CTAs
 };
 
-__global__ void __launch_bounds__(256) attn_merge_kernel(MergeParams p) {
+__global__ void __launch_bounds__(256, 4) attn_merge_kernel(MergeParams p) {
     const long w = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (w >= p.warps_total) return;
     const int lane = threadIdx.x & 31;
-    const int k = (int)(w / p.rows_per_item), rloc = (int)(w % p.rows_per_item);
+    const int k = (int)(w / p.rows_used), rloc = (int)(w % p.rows_used);
     // the k-th item that owns slots: group a comes first when it is split at all
     int item, nsplit, slot0;
     const int split_a = p.plan.splits_a > 1 ? p.plan.items_a : 0;
-    if (k < split_a) {
+    if (p.bal_merge) {
+        // the list of cut items was made on the device; the grid covers the most there can be
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        const int tpu = p.plan.tiles_per_unit, rt = k % tpu;
+        const int listed = p.bal_hdr[0];
+        const int4 rec = p.bal_merge[k / tpu];       // a (sequence, kv head) pair that was cut (read beside the count)
+        if (k / tpu >= listed) return;
+        item = rec.x * tpu + rt; slot0 = rt * 2 * p.bal_groups + rec.y; nsplit = rec.z;
+    } else if (k < split_a) {
         item = k; nsplit = p.plan.splits_a; slot0 = k * p.plan.splits_a;
     } else {
         item = p.plan.items_a + (k - split_a); nsplit = p.plan.splits_b;
@@ -374,27 +386,14 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(MergeParams p) {
     // Launched as a programmatic dependent of the attention kernel: the blocks may become
     // resident while that kernel drains; its partial results are only visible after this wait.
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    // Loads are issued in groups of four before any of them is used, so that a row costs a few
-    // memory round trips instead of two per split.
+    // A row costs one trip to memory when it has up to four parts (maxima, sums and accumulators
+    // of all of them are fetched together), and two more per further group of four.
     const float* ml_base = p.part_ml + ((size_t)slot0 * p.rows_per_item + rloc) * 2;
     const size_t ml_stride = (size_t)p.rows_per_item * 2;
-    float m = -CUDART_INF_F;
-    for (int s0 = 0; s0 < nsplit; s0 += 4) {
-        float mv[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) mv[j] = s0 + j < nsplit ? ml_base[(size_t)(s0 + j) * ml_stride] : -CUDART_INF_F;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) m = fmaxf(m, mv[j]);
-    }
-    const float m_use = m == -CUDART_INF_F ? 0.f : m;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    float l = 0.f;
     const int per_lane = p.D / 32;  // 2 or 4 consecutive floats per lane
     const float* o_base = p.part_o + ((size_t)slot0 * p.rows_per_item + rloc) * p.D + lane * per_lane;
     const size_t o_stride = (size_t)p.rows_per_item * p.D;
-    for (int s0 = 0; s0 < nsplit; s0 += 4) {
-        float2 ml[4];
-        float4 v[4];
+    auto fetch = [&](int s0, float2 (&ml)[4], float4 (&v)[4]) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const bool in = s0 + j < nsplit;
@@ -405,6 +404,25 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(MergeParams p) {
             else if (per_lane == 4) v[j] = *reinterpret_cast<const float4*>(src);
             else { const float2 t = *reinterpret_cast<const float2*>(src); v[j] = make_float4(t.x, t.y, 0.f, 0.f); }
         }
+    };
+    float2 ml[4];
+    float4 v[4];
+    fetch(0, ml, v);
+    float m = fmaxf(fmaxf(ml[0].x, ml[1].x), fmaxf(ml[2].x, ml[3].x));
+#pragma unroll 1
+    for (int s0 = 4; s0 < nsplit; s0 += 4) {
+        float mv[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) mv[j] = s0 + j < nsplit ? ml_base[(size_t)(s0 + j) * ml_stride] : -CUDART_INF_F;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) m = fmaxf(m, mv[j]);
+    }
+    const float m_use = m == -CUDART_INF_F ? 0.f : m;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float l = 0.f;
+#pragma unroll 1
+    for (int s0 = 0; s0 < nsplit; s0 += 4) {
+        if (s0 > 0) fetch(s0, ml, v);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const float wgt = exp2f(ml[j].x - m_use);     // 0 for an absent or empty split
@@ -467,9 +485,21 @@ int launch_attn_merge(const AttnArgs& a) {
     p.plan = a.plan.dev;
     p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv; p.G = a.G; p.R = a.N * a.G; p.D = a.D;
     p.rows_per_item = a.plan.rows_per_item; p.items = a.plan.items;
-    const int split_items = (a.plan.dev.splits_a > 1 ? a.plan.dev.items_a : 0) +
-                            (a.plan.dev.splits_b > 1 ? a.plan.items - a.plan.dev.items_a : 0);
-    p.warps_total = (long)split_items * a.plan.rows_per_item;
+    int split_items = (a.plan.dev.splits_a > 1 ? a.plan.dev.items_a : 0) +
+                      (a.plan.dev.splits_b > 1 ? a.plan.items - a.plan.dev.items_a : 0);
+    p.bal_hdr = nullptr;
+    p.bal_merge = nullptr;
+    p.bal_groups = 0;
+    if (a.plan.dev.balanced) {
+        const BalTable t = plan_bal_table(a.plan, a.D, a.workspace);
+        p.bal_hdr = t.hdr;
+        p.bal_merge = t.merge;
+        const int tpu = a.plan.dev.tiles_per_unit, groups = a.plan.ctas / tpu, pairs = a.plan.items / tpu;
+        p.bal_groups = groups;
+        split_items = (pairs < groups - 1 ? pairs : groups - 1) * tpu;   // one pair per cut at most
+    }
+    p.rows_used = p.R < a.plan.rows_per_item ? p.R : a.plan.rows_per_item;
+    p.warps_total = (long)split_items * p.rows_used;
     if (p.warps_total == 0) return GSD_OK;
     const int warps = 8;
     const long blocks = (p.warps_total + warps - 1) / warps;

@@ -96,6 +96,8 @@ struct TcParams {
     PlanDev plan;
     int total_work;   // CTAs of the plan = units of work
     int slots;        // partial-result slots of the plan
+    const int2* bal_cta;     // balanced plan: (first unit, units) of every group of CTAs, else nullptr
+    const int4* bal_units;   // balanced plan: (pair, first tile, end tile, slot or -1)
     unsigned long long wait_limit_ns;
     int withhold_first_k;   // test hook: every CTA leaves out the K copy of its first key tile
 };
@@ -359,10 +361,22 @@ struct UnitInfo {
     bool two;        // the second row tile exists
 };
 
+// `w` is the work index of a fixed plan, or the index of the group's unit in the table of a balanced one.
 __device__ __forceinline__ UnitInfo unit_info(const TcParams& p, int w, int lane) {
     UnitInfo u;
-    int item;
-    plan_decode(p.plan, w, item, u.split, u.nsplit, u.slot);
+    int item, t0n = 0, t1n = 0;
+    const bool bal = p.bal_units != nullptr;
+    if (bal) {
+        // the unit of this CTA's group, for the row-tile item this CTA has in every pair
+        const int tpu = p.plan.tiles_per_unit, rt = (int)blockIdx.x % tpu;
+        const int4 rec = p.bal_units[w];
+        item = rec.x * tpu + rt; t0n = rec.y; t1n = rec.z;
+        u.slot = rec.w >= 0 ? rt * 2 * ((int)gridDim.x / tpu) + rec.w : -1;
+        u.split = 0;
+        u.nsplit = rec.w >= 0 ? 2 : 1;     // only "one piece or several" matters below
+    } else {
+        plan_decode(p.plan, w, item, u.split, u.nsplit, u.slot);
+    }
     const int unit = item / p.plan.tiles_per_unit;
     u.row0 = (item % p.plan.tiles_per_unit) * (2 * BM);
     u.b = unit / p.Hkv;
@@ -404,6 +418,13 @@ __device__ __forceinline__ UnitInfo unit_info(const TcParams& p, int w, int lane
     }
     u.live = __reduce_or_sync(0xFFFFFFFFu, live);
     u.nPT = (L + BN - 1) / BN;
+    if (bal) {
+        // the table counts every draft tile; here only those with a visible key are numbered
+        auto live_index = [&](int t) { return t <= u.nPT ? t : u.nPT + __popc(u.live & ((1u << (t - u.nPT)) - 1u)); };
+        u.t_begin = live_index(t0n);
+        u.ntiles = live_index(t1n) - u.t_begin;
+        return u;
+    }
     const int T = u.nPT + __popc(u.live);
     const int per = (T + u.nsplit - 1) / u.nsplit;
     u.t_begin = min(u.split * per, T);
@@ -465,14 +486,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&s_tmem_base)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    const int total_work = p.total_work;
+    // The CTA's units: work indices blockIdx.x, blockIdx.x + gridDim.x, ... of a fixed plan, or
+    // a run of the table that the planning kernel (this kernel is its programmatic dependent)
+    // has written.
+    int n_my;
+    if (p.bal_cta) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        n_my = p.bal_cta[blockIdx.x / p.plan.tiles_per_unit].y;
+    } else {
+        n_my = p.total_work > (int)blockIdx.x ? (p.total_work - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+    }
+    // (recomputed where it is needed rather than kept in a register through the key loops)
+    auto unit_index = [&](int it) -> int {
+        return p.bal_cta ? p.bal_cta[blockIdx.x / p.plan.tiles_per_unit].x + it : (int)blockIdx.x + it * (int)gridDim.x;
+    };
     // Decoding a unit costs two dependent trips to global memory (sequence length, mask rows).
     // Each warp decodes one of the CTA's first units here, all at once, so that no role pays
     // that latency between units.
     for (int k = warp; k < kUnitTable; k += kThreads / 32) {
-        const int w = blockIdx.x + k * gridDim.x;
-        if (w < total_work) {
-            const UnitInfo u = unit_info(p, w, lane);
+        if (k < n_my) {
+            const UnitInfo u = unit_info(p, unit_index(k), lane);
             if (lane == 0) s_units[k] = u;
         }
     }
@@ -480,7 +513,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem_base;
-    auto unit_of = [&](int w, int it) -> UnitInfo { return it < kUnitTable ? s_units[it] : unit_info(p, w, lane); };
+    auto unit_of = [&](int it) -> UnitInfo {
+        return it < kUnitTable ? s_units[it] : unit_info(p, unit_index(it), lane);
+    };
 
     if (warp >= 8) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 96;");
@@ -489,8 +524,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         int kvc = 0;          // key tiles loaded so far (ring position)
         int au = 0;           // non-empty units so far
         bool ok = true, q_pending = false;
-        for (int w = blockIdx.x, it = 0; w < total_work && ok; w += gridDim.x, ++it) {
-            const UnitInfo u = unit_of(w, it);
+        for (int it = 0; it < n_my && ok; ++it) {
+            const UnitInfo u = unit_of(it);
             if (u.ntiles == 0) continue;
             if (lane == 0) {
                 // Q of the previous unit is free once its last QK^T has completed
@@ -554,8 +589,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         static_assert(KST == 2, "two K stages are selected by a flag");
         const uint32_t qlo0 = desc_lo_kmajor(sQ), qlo1 = desc_lo_kmajor(sQ + TILE_BYTES);
         const uint32_t klo0 = desc_lo_kmajor(sK), klo1 = desc_lo_kmajor(sK + TILE_BYTES);
-        for (int w = blockIdx.x, it = 0; w < total_work && ok; w += gridDim.x, ++it) {
-            const UnitInfo u = unit_of(w, it);
+        for (int it = 0; it < n_my && ok; ++it) {
+            const UnitInfo u = unit_of(it);
             if (u.ntiles == 0) continue;
             const bool two = u.two;
             const int njobs = two ? 2 * u.ntiles : u.ntiles;
@@ -599,8 +634,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         auto wait = [&](int b, uint32_t par) -> bool { return mbar_wait_warp(bar(b), par, abort_flag, p.status); };
         static_assert(VST == 2, "two V stages are selected by a flag");
         const uint32_t vlo0 = desc_lo_mnmajor(sV), vlo1 = desc_lo_mnmajor(sV + TILE_BYTES);
-        for (int w = blockIdx.x, it = 0; w < total_work && ok; w += gridDim.x, ++it) {
-            const UnitInfo u = unit_of(w, it);
+        for (int it = 0; it < n_my && ok; ++it) {
+            const UnitInfo u = unit_of(it);
             if (u.ntiles == 0) continue;
             const bool two = u.two;
             const int njobs = two ? 2 * u.ntiles : u.ntiles;
@@ -654,8 +689,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         int auc1 = 0;     // units in which stream 1 had jobs (phase of its barriers as seen by warpgroup 0)
         int mlc = 0;      // single-row-tile units whose odd-tile stream had tiles
         bool ok = true;
-        for (int w = blockIdx.x, it = 0; w < total_work && ok; w += gridDim.x, ++it) {
-            const UnitInfo u = unit_of(w, it);
+        for (int it = 0; it < n_my && ok; ++it) {
+            const UnitInfo u = unit_of(it);
             const int ntiles = u.ntiles;
             // with one row tile only, the two warpgroups take the even / odd key tiles of the
             // same rows and warpgroup 0 merges the two partial results in the epilogue
@@ -1016,6 +1051,27 @@ int launch_attn_tcgen05(const AttnArgs& a) {
     p.withhold_first_k = g_withhold_first_k;
     DeviceInfo di;
     if (device_info(&di) != 0) return GSD_ERR_CUDA;
+    p.bal_cta = nullptr;
+    p.bal_units = nullptr;
+    if (a.plan.dev.balanced) {
+        // one CTA per share of the table; the table is being written by the planning kernel,
+        // beside which this kernel may start
+        const BalTable t = plan_bal_table(a.plan, a.D, a.workspace);
+        p.bal_cta = t.cta;
+        p.bal_units = t.units;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)a.plan.ctas);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = kSmemBytes;
+        cfg.stream = a.stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        GSD_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_tc_kernel, tq, tk, tv, tdk, tdv, tout, p));
+        return GSD_OK;
+    }
     dim3 grid(a.plan.ctas < di.sm_count ? a.plan.ctas : di.sm_count);
     attn_tc_kernel<<<grid, kThreads, kSmemBytes, a.stream>>>(tq, tk, tv, tdk, tdv, tout, p);
     GSD_CUDA_TRY(cudaGetLastError());

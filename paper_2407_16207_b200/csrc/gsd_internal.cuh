@@ -48,8 +48,20 @@ int device_info(DeviceInfo* out);
 // index = unit * tiles_per_unit + row tile.  The first items_a items are cut into splits_a
 // key ranges, the remaining ones into splits_b; CTAs are numbered group a first.  Only items
 // with more than one split own partial-result slots (one per split, numbered in CTA order).
+//
+// Balanced plan (tcgen05 back end only): the host cannot see the sequence lengths, so for
+// batches whose lengths differ a plan made from Lmax leaves CTAs idle.  Here the key tiles of
+// all (sequence, kv head) pairs are laid end to end - pair after pair, ceil(len/128) prefix
+// tiles plus the draft tiles each - and group g of `ctas / tiles_per_unit` groups takes the
+// g-th equal share of that line; CTA r of a group works on row-tile item r of every pair in
+// the share.  A small kernel builds the table from seq_lens on the device before the
+// attention kernel reads it: per group its units (pair, tile range, partial-result slot or -1
+// for a whole pair), and per pair that was cut the run of slots to merge.  Slots are numbered
+// along the line, so the pieces of one pair have consecutive slots; a group has at most two
+// partial units (its first and last).  CTA r adds r * 2 * groups to a slot of its group.
 struct PlanDev {
     int items_a, splits_a, splits_b, tiles_per_unit;
+    int balanced;       // 1: units come from the table built on the device
 };
 struct AttnPlan {
     int kernel;         // GSD_ATTN_MMA or GSD_ATTN_TCGEN05
@@ -59,6 +71,15 @@ struct AttnPlan {
     int slots;          // partial-result slots; 0 when nothing is split
     PlanDev dev;
     size_t ws_bytes;
+};
+// The table of a balanced plan, in the workspace behind the partial results.
+struct BalTable {
+    int* hdr;       // [0] pairs to merge, [1] tiles on the line, [2] tiles per group
+    int2* cta;      // [groups]  (index of the group's first unit, number of units)
+    int4* merge;    // [groups]  (pair, first slot, number of slots, -)
+    int4* units;    // [pairs + groups]  (pair, first tile, end tile, slot or -1); tiles count the
+                    //                   prefix tiles, then ALL draft tiles of the pair
+    int* off;       // [B + 1] start of each sequence on the line
 };
 __host__ __device__ inline void plan_decode(const PlanDev& pl, int cta, int& item, int& split, int& nsplit, int& slot) {
     const int ctas_a = pl.items_a * pl.splits_a;
@@ -97,6 +118,23 @@ int attn_pick_kernel(const gsd_attn_params* p);                 // GSD_ATTN_MMA 
 inline size_t plan_part_o_bytes(const AttnPlan& pl, int D) { return align_up((size_t)pl.slots * pl.rows_per_item * D * sizeof(float), 256); }
 inline size_t plan_part_ml_bytes(const AttnPlan& pl) { return align_up((size_t)pl.slots * pl.rows_per_item * 2 * sizeof(float), 256); }
 
+inline size_t plan_bal_bytes(const AttnPlan& pl, int B) {
+    if (!pl.dev.balanced) return 0;
+    return 256 + align_up((size_t)pl.ctas * sizeof(int2), 256) + align_up((size_t)pl.ctas * sizeof(int4), 256) +
+           align_up((size_t)(pl.items + pl.ctas) * sizeof(int4), 256) + align_up((size_t)(B + 1) * sizeof(int), 256);
+}
+inline BalTable plan_bal_table(const AttnPlan& pl, int D, void* workspace) {
+    char* at = (char*)workspace + plan_part_o_bytes(pl, D) + plan_part_ml_bytes(pl);
+    BalTable t;
+    t.hdr = (int*)at; at += 256;
+    t.cta = (int2*)at; at += align_up((size_t)pl.ctas * sizeof(int2), 256);
+    t.merge = (int4*)at; at += align_up((size_t)pl.ctas * sizeof(int4), 256);
+    t.units = (int4*)at; at += align_up((size_t)(pl.items + pl.ctas) * sizeof(int4), 256);
+    t.off = (int*)at;
+    return t;
+}
+
+int launch_attn_plan(const AttnArgs& a);      // balanced plans only: builds the table
 int launch_attn_mma(const AttnArgs& a);
 int launch_attn_tcgen05(const AttnArgs& a);
 bool attn_tcgen05_supports(int D, int G);
