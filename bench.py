@@ -366,6 +366,70 @@ def run_sweep(args):
         torch.cuda.empty_cache()
 
 
+def run_ab_balanced(args):
+    """gsd_verify_attn with its fixed plan (made on the host from Lmax) against the balanced plan
+    (key tiles shared out on the device from seq_lens) on the 70B layer shape, cold: a uniform
+    batch, a batch with lengths drawn uniformly from [256, 8192], and one 16384-token context
+    among 31 short ones.  One JSON line per batch."""
+    import paper_2407_16207_b200 as gsd
+    from gsd_inputs.torch_io import attn_tensors
+    gsd.lib()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peaks, peak_src = load_peaks()
+    base = gi.CONFIGS["llama70b"]
+    flush = torch.empty(4 * L2_BYTES, dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    reps = max(args.steps if args.steps_given else 20, 3)
+    cases = [("uniform_L4096", base.L, None), ("ragged_L256_8192", (256, 8192), None),
+             ("one_long_L16384", 16384, (256, 1024))]
+    for name, L, others in cases:
+        cfg = gi.VerifyConfig(**{**base.__dict__, "name": name, "L": L})
+        inp = gi.make_inputs(cfg, accept=False)
+        if others is not None:
+            # every sequence but the first is cut back to a short context
+            rng = np.random.default_rng(gi.seed_for(cfg, 1))
+            inp["seq_lens"][1:] = rng.integers(others[0], others[1] + 1, size=cfg.B - 1, dtype=np.int32)
+        t = attn_tensors(inp, dev)
+        out = torch.empty_like(t["q"])
+        Lmax = inp["Lmax"]
+        times, outs = {}, {}
+        for ns in (0, gsd.GSD_ATTN_SPLIT_BALANCED):
+            need = gsd.gsd_verify_attn_workspace_bytes(cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.D, Lmax, ns)
+            ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+
+            def attn():
+                gsd.gsd_verify_attn(t["q"], t["k_cache"], t["v_cache"], t["draft_k"], t["draft_v"],
+                                    t["ancestor_mask"], t["seq_lens"], out=out, workspace=ws, status=status,
+                                    num_splits=ns)
+            for _ in range(3):
+                attn()
+            torch.cuda.synchronize()
+            ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(reps)]
+            for i in range(reps):
+                flush.fill_(i & 0xFF)
+                ev[i][0].record(); attn(); ev[i][1].record()
+            torch.cuda.synchronize()
+            times[ns] = statistics.median(e[0].elapsed_time(e[1]) for e in ev) * 1e-3
+            outs[ns] = out.float().clone()
+        if int(status.item()) != 0:
+            raise RuntimeError(f"device status {int(status.item()):#x} on {name}")
+        flops, attn_bytes, _ = algorithmic_work(cfg, inp)
+        fixed, bal = times[0], times[gsd.GSD_ATTN_SPLIT_BALANCED]
+        lens = inp["seq_lens"]
+        line = {"mode": "ab_balanced", "n_gpus": 1, "steps": reps, "warmup": 3, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": name, "B": cfg.B, "N": cfg.N, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
+                           "seq_lens": {"min": int(lens.min()), "max": int(lens.max()), "mean": float(lens.mean())},
+                           "l2": "cold = a 504 MB buffer written between calls"},
+                "attn_us_fixed_plan": fixed * 1e6, "attn_us_balanced_plan": bal * 1e6, "fixed_over_balanced": fixed / bal,
+                "max_abs_difference_of_outputs": float((outs[0] - outs[gsd.GSD_ATTN_SPLIT_BALANCED]).abs().max().item()),
+                "roofline_fixed": roofline_of(flops, attn_bytes, fixed, peaks, peak_src),
+                "roofline_balanced": roofline_of(flops, attn_bytes, bal, peaks, peak_src)}
+        print(json.dumps(line), flush=True)
+        del t, out, outs
+        torch.cuda.empty_cache()
+
+
 def run_ab_unmerge(args):
     """Verification of the token graph itself (a node merged from several branches attends to
     the union of its ancestors) against verification of the paper's unmerged tree (Sec. 5.4): on
@@ -504,6 +568,8 @@ def main():
                     help="auto: the whole step on the named configurations, a sample on sweep points")
     ap.add_argument("--sweep", action="store_true", help="one JSON line per point of the 70B-shaped sweep")
     ap.add_argument("--points", default="", help="with --sweep: comma-separated workload names")
+    ap.add_argument("--ab-balanced", action="store_true",
+                    help="fixed plan against balanced plan of gsd_verify_attn on uniform and ragged batches")
     ap.add_argument("--ab-unmerge", action="store_true",
                     help="graph-direct against unmerged-tree verification on grown graphs; one JSON line")
     args = ap.parse_args()
@@ -512,6 +578,9 @@ def main():
         args.steps = 6000
     if args.sweep:
         run_sweep(args)
+        return
+    if args.ab_balanced:
+        run_ab_balanced(args)
         return
     if args.ab_unmerge:
         run_ab_unmerge(args)

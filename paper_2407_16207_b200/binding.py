@@ -13,6 +13,7 @@ from typing import Optional, Tuple
 import torch
 
 GSD_ATTN_AUTO, GSD_ATTN_MMA, GSD_ATTN_TCGEN05 = 0, 1, 2
+GSD_ATTN_SPLIT_BALANCED = -1      # num_splits: equal shares of key tiles per CTA, dealt out on the device
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libgsd.so")
