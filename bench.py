@@ -367,10 +367,11 @@ def run_sweep(args):
 
 
 def run_ab_balanced(args):
-    """gsd_verify_attn with its fixed plan (made on the host from Lmax) against the balanced plan
-    (key tiles shared out on the device from seq_lens) on the 70B layer shape, cold: a uniform
-    batch, a batch with lengths drawn uniformly from [256, 8192], and one 16384-token context
-    among 31 short ones.  One JSON line per batch."""
+    """gsd_verify_attn with its fixed plan (made on the host from Lmax) against the two plans made
+    on the device from seq_lens (equal shares of key tiles per group of CTAs; a split count per
+    sequence), cold.  70B layer shape: a uniform batch, lengths drawn uniformly from [256, 8192],
+    one 16384-token context among short ones; 13B layer shape (one kv head per query head): its
+    own lengths, and 16 sequences with one long context.  One JSON line per batch."""
     import paper_2407_16207_b200 as gsd
     from gsd_inputs.torch_io import attn_tensors
     gsd.lib()
@@ -381,10 +382,13 @@ def run_ab_balanced(args):
     flush = torch.empty(4 * L2_BYTES, dtype=torch.uint8, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     reps = max(args.steps if args.steps_given else 20, 3)
-    cases = [("uniform_L4096", base.L, None), ("ragged_L256_8192", (256, 8192), None),
-             ("one_long_L16384", 16384, (256, 1024))]
-    for name, L, others in cases:
-        cfg = gi.VerifyConfig(**{**base.__dict__, "name": name, "L": L})
+    mha = gi.CONFIGS["llama13b"]
+    cases = [(base, "uniform_L4096", base.L, None), (base, "ragged_L256_8192", (256, 8192), None),
+             (base, "one_long_L16384", 16384, (256, 1024)),
+             (mha, "llama13b", mha.L, None),
+             (gi.VerifyConfig(**{**mha.__dict__, "B": 16, "N": 64}), "mha_B16_one_long_L8192", 8192, (128, 1024))]
+    for shape, name, L, others in cases:
+        cfg = gi.VerifyConfig(**{**shape.__dict__, "name": name, "L": L})
         inp = gi.make_inputs(cfg, accept=False)
         if others is not None:
             # every sequence but the first is cut back to a short context
@@ -394,7 +398,7 @@ def run_ab_balanced(args):
         out = torch.empty_like(t["q"])
         Lmax = inp["Lmax"]
         times, outs = {}, {}
-        for ns in (0, gsd.GSD_ATTN_SPLIT_BALANCED):
+        for ns in (0, gsd.GSD_ATTN_SPLIT_BALANCED, gsd.GSD_ATTN_SPLIT_PER_SEQUENCE):
             need = gsd.gsd_verify_attn_workspace_bytes(cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.D, Lmax, ns)
             ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
 
@@ -415,16 +419,20 @@ def run_ab_balanced(args):
         if int(status.item()) != 0:
             raise RuntimeError(f"device status {int(status.item()):#x} on {name}")
         flops, attn_bytes, _ = algorithmic_work(cfg, inp)
-        fixed, bal = times[0], times[gsd.GSD_ATTN_SPLIT_BALANCED]
+        fixed, bal, seq = times[0], times[gsd.GSD_ATTN_SPLIT_BALANCED], times[gsd.GSD_ATTN_SPLIT_PER_SEQUENCE]
         lens = inp["seq_lens"]
         line = {"mode": "ab_balanced", "n_gpus": 1, "steps": reps, "warmup": 3, "dtype": "bf16", "data": "synthetic",
                 "config": {"workload": name, "B": cfg.B, "N": cfg.N, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
                            "seq_lens": {"min": int(lens.min()), "max": int(lens.max()), "mean": float(lens.mean())},
                            "l2": "cold = a 504 MB buffer written between calls"},
-                "attn_us_fixed_plan": fixed * 1e6, "attn_us_balanced_plan": bal * 1e6, "fixed_over_balanced": fixed / bal,
-                "max_abs_difference_of_outputs": float((outs[0] - outs[gsd.GSD_ATTN_SPLIT_BALANCED]).abs().max().item()),
+                "attn_us_fixed_plan": fixed * 1e6, "attn_us_balanced_plan": bal * 1e6,
+                "attn_us_per_sequence_plan": seq * 1e6, "fixed_over_balanced": fixed / bal,
+                "fixed_over_per_sequence": fixed / seq,
+                "max_abs_difference_of_outputs": max(float((outs[0] - outs[m]).abs().max().item())
+                                                     for m in (gsd.GSD_ATTN_SPLIT_BALANCED, gsd.GSD_ATTN_SPLIT_PER_SEQUENCE)),
                 "roofline_fixed": roofline_of(flops, attn_bytes, fixed, peaks, peak_src),
-                "roofline_balanced": roofline_of(flops, attn_bytes, bal, peaks, peak_src)}
+                "roofline_balanced": roofline_of(flops, attn_bytes, bal, peaks, peak_src),
+                "roofline_per_sequence": roofline_of(flops, attn_bytes, seq, peaks, peak_src)}
         print(json.dumps(line), flush=True)
         del t, out, outs
         torch.cuda.empty_cache()

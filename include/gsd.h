@@ -72,7 +72,8 @@ typedef enum gsd_status {
  * kernel, which reaches roughly a sixth of the tensor throughput (group sizes 3, 6, 12, ... and
  * D == 64 therefore stay correct but slow).  Asking for GSD_ATTN_TCGEN05 on a shape it does
  * not support returns GSD_ERR_UNSUPPORTED. */
-#define GSD_ATTN_SPLIT_BALANCED (-1)  /* value of gsd_attn_params.num_splits */
+#define GSD_ATTN_SPLIT_BALANCED (-1)      /* values of gsd_attn_params.num_splits */
+#define GSD_ATTN_SPLIT_PER_SEQUENCE (-2)
 
 #define GSD_ATTN_AUTO 0
 #define GSD_ATTN_MMA  1            /* warp-level mma.sync kernel: D in {64,128}, any N, any group size */
@@ -88,7 +89,9 @@ typedef struct gsd_attn_params {
     float softmax_scale;  /* <= 0 selects 1/sqrt(D) */
     int32_t num_splits;   /* key-range splits per (sequence, kv head, row tile); 0 = choose;
                              GSD_ATTN_SPLIT_BALANCED = equal shares of key tiles per CTA, dealt out on the
-                             device from seq_lens (tcgen05 kernel; the mma.sync kernel reads it as 0) */
+                             device from seq_lens; GSD_ATTN_SPLIT_PER_SEQUENCE = a split count per sequence,
+                             chosen on the device from seq_lens so that all units are about equally long
+                             (both: tcgen05 kernel; the mma.sync kernel reads them as 0) */
     int32_t kernel;       /* GSD_ATTN_AUTO / _MMA / _TCGEN05 */
 } gsd_attn_params;
 
@@ -160,8 +163,8 @@ void gsd_debug_attn_wait(uint64_t limit_ns, int32_t withhold_first_k);
 size_t gsd_verify_attn_workspace_bytes(const gsd_attn_params* p);
 
 /* The number of key-range splits gsd_verify_attn would use for *p on the current device
- * (p->num_splits if non-zero, else the automatic choice); GSD_ATTN_SPLIT_BALANCED when the
- * shares are dealt out on the device; 0 on invalid parameters. */
+ * (p->num_splits if positive, else the automatic choice); GSD_ATTN_SPLIT_BALANCED or
+ * GSD_ATTN_SPLIT_PER_SEQUENCE when the work is shared out on the device; 0 on invalid parameters. */
 int gsd_verify_attn_num_splits(const gsd_attn_params* p);
 
 /*

@@ -14,6 +14,7 @@ import torch
 
 GSD_ATTN_AUTO, GSD_ATTN_MMA, GSD_ATTN_TCGEN05 = 0, 1, 2
 GSD_ATTN_SPLIT_BALANCED = -1      # num_splits: equal shares of key tiles per CTA, dealt out on the device
+GSD_ATTN_SPLIT_PER_SEQUENCE = -2  # num_splits: a split count per sequence, chosen on the device
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libgsd.so")

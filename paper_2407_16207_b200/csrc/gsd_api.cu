@@ -34,7 +34,7 @@ int device_info(DeviceInfo* out) {
 static int attn_params_ok(const gsd_attn_params* p) {
     if (!p) return GSD_ERR_NULL_POINTER;
     if (p->B < 1 || p->N < 1 || p->N > GSD_MAX_NODES || p->Hq < 1 || p->Hkv < 1 ||
-        p->Hq % p->Hkv != 0 || (p->D != 64 && p->D != 128) || p->Lmax < 1 || p->num_splits < GSD_ATTN_SPLIT_BALANCED ||
+        p->Hq % p->Hkv != 0 || (p->D != 64 && p->D != 128) || p->Lmax < 1 || p->num_splits < GSD_ATTN_SPLIT_PER_SEQUENCE ||
         p->num_splits > 64)
         return GSD_ERR_BAD_SHAPE;
     if ((long long)p->B * p->Hkv > 65535) return GSD_ERR_BAD_SHAPE;
@@ -85,6 +85,19 @@ AttnPlan attn_make_plan(const gsd_attn_params* p, int sm_count) {
         const int groups = (int)(line < resident / tpu ? line : resident / tpu);
         pl.ctas = groups * tpu;
         pl.slots = 2 * pl.ctas;                                        // a CTA's first and last unit
+        pl.ws_bytes = plan_part_o_bytes(pl, p->D) + plan_part_ml_bytes(pl) + plan_bal_bytes(pl, p->B);
+        return pl;
+    }
+    if (tc && p->num_splits == GSD_ATTN_SPLIT_PER_SEQUENCE && resident <= 1024) {
+        // split counts per sequence, chosen on the device; persistent CTAs walk the units
+        pl.dev.balanced = 2;
+        pl.ctas = resident;
+        // slots: the sum over the cut sequences of items x splits is at most the units aimed at
+        // (tiles / target, and fewer where the four-tile floor of the target binds) plus half a
+        // slot per item from rounding
+        const long long bound = (long long)kSeqPlanWaves * resident + pl.items / 2 + 1;
+        const long long cap = (long long)pl.items * kSeqPlanMaxSplit;
+        pl.slots = (int)(bound < cap ? bound : cap);
         pl.ws_bytes = plan_part_o_bytes(pl, p->D) + plan_part_ml_bytes(pl) + plan_bal_bytes(pl, p->B);
         return pl;
     }
@@ -144,7 +157,7 @@ extern "C" int gsd_verify_attn_num_splits(const gsd_attn_params* p) {
     DeviceInfo di;
     if (device_info(&di) != 0) return 0;
     const AttnPlan pl = attn_make_plan(p, di.sm_count);
-    if (pl.dev.balanced) return GSD_ATTN_SPLIT_BALANCED;
+    if (pl.dev.balanced) return pl.dev.balanced == 2 ? GSD_ATTN_SPLIT_PER_SEQUENCE : GSD_ATTN_SPLIT_BALANCED;
     return pl.dev.splits_a > pl.dev.splits_b ? pl.dev.splits_a : pl.dev.splits_b;
 }
 

@@ -355,6 +355,7 @@ struct MergeParams {
     const int* bal_hdr;      // balanced plan: [0] = items to merge (known on the device only)
     const int4* bal_merge;   // balanced plan: (pair, first slot, slots) per pair to merge, else nullptr
     int bal_groups;          // balanced plan: groups of CTAs
+    SeqTable seq;            // per-sequence plan (hdr == nullptr otherwise); the grid then covers every item
 };
 
 __global__ void __launch_bounds__(256, 4) attn_merge_kernel(MergeParams p) {
@@ -373,6 +374,14 @@ __global__ void __launch_bounds__(256, 4) attn_merge_kernel(MergeParams p) {
         const int4 rec = p.bal_merge[k / tpu];       // a (sequence, kv head) pair that was cut (read beside the count)
         if (k / tpu >= listed) return;
         item = rec.x * tpu + rt; slot0 = rt * 2 * p.bal_groups + rec.y; nsplit = rec.z;
+    } else if (p.seq.hdr) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        const int per_seq = p.Hkv * p.plan.tiles_per_unit;
+        const int b = k / per_seq;
+        nsplit = p.seq.nsplit[b];
+        if (nsplit == 1) return;                       // the item was stored by its only unit
+        item = k;
+        slot0 = p.seq.slot_off[b] + (k - b * per_seq) * nsplit;
     } else if (k < split_a) {
         item = k; nsplit = p.plan.splits_a; slot0 = k * p.plan.splits_a;
     } else {
@@ -490,7 +499,11 @@ int launch_attn_merge(const AttnArgs& a) {
     p.bal_hdr = nullptr;
     p.bal_merge = nullptr;
     p.bal_groups = 0;
-    if (a.plan.dev.balanced) {
+    p.seq.hdr = nullptr; p.seq.nsplit = nullptr; p.seq.unit_off = nullptr; p.seq.slot_off = nullptr;
+    if (a.plan.dev.balanced == 2) {
+        p.seq = plan_seq_table(a.plan, a.D, a.B, a.workspace);
+        split_items = a.plan.items;
+    } else if (a.plan.dev.balanced) {
         const BalTable t = plan_bal_table(a.plan, a.D, a.workspace);
         p.bal_hdr = t.hdr;
         p.bal_merge = t.merge;

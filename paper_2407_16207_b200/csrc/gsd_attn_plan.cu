@@ -160,10 +160,87 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanParams p) {
     }
 }
 
+struct SeqPlanParams {
+    const int32_t* seq_lens;
+    int B, Lmax;
+    int per_seq;        // work items per sequence (kv heads x row-tile items)
+    int nd;             // draft tiles per item
+    int units_wanted;
+    int slots_cap;      // partial-result slots the workspace holds
+    SeqTable t;
+};
+
+// Per-sequence split counts: one block, sequences dealt out in contiguous chunks to its threads.
+__global__ void __launch_bounds__(kPlanThreads) attn_plan_seq_kernel(SeqPlanParams p) {
+    __shared__ unsigned long long s_warp[32];
+    const int tid = threadIdx.x;
+    if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    auto tiles_of = [&](int b) -> int {
+        int L = p.seq_lens[b];
+        L = L < 0 ? 0 : (L > p.Lmax ? p.Lmax : L);
+        return (L + 127) / 128 + p.nd;
+    };
+    const int chunk = (p.B + kPlanThreads - 1) / kPlanThreads;
+    const int b_lo = min(tid * chunk, p.B), b_hi = min(b_lo + chunk, p.B);
+    unsigned long long mine = 0;
+    for (int b = b_lo; b < b_hi; ++b) mine += (unsigned long long)p.per_seq * tiles_of(b);
+    unsigned long long total64;
+    block_scan(mine, s_warp, &total64);
+    // the common target length of a unit: at least four key tiles
+    const long long target64 = (long long)((total64 + p.units_wanted - 1) / p.units_wanted);
+    const int target = (int)(target64 < 4 ? 4 : (target64 > (1 << 30) ? (1 << 30) : target64));
+    auto splits_of = [&](int b) -> int {
+        const int n = (2 * tiles_of(b) + target) / (2 * target);      // tiles / target, rounded
+        return n < 1 ? 1 : (n > kSeqPlanMaxSplit ? kSeqPlanMaxSplit : n);
+    };
+    unsigned long long units = 0, slots = 0;
+    for (int b = b_lo; b < b_hi; ++b) {
+        const int n = splits_of(b);
+        units += (unsigned long long)n * p.per_seq;
+        if (n > 1) slots += (unsigned long long)n * p.per_seq;
+    }
+    // (both sums stay far below 2^31: at most 32 x items each)
+    unsigned long long tot;
+    const unsigned long long ex = block_scan(units | (slots << 32), s_warp, &tot);
+    // should the partial results not fit the workspace (the host's bound makes sure they do),
+    // nothing is cut at all
+    const bool fits = (tot >> 32) <= (unsigned long long)p.slots_cap;
+    unsigned long long u = ex & 0xFFFFFFFFull, sl = ex >> 32;
+    for (int b = b_lo; b < b_hi; ++b) {
+        const int n = fits ? splits_of(b) : 1;
+        p.t.nsplit[b] = n;
+        p.t.unit_off[b] = fits ? (int)u : b * p.per_seq;
+        p.t.slot_off[b] = fits ? (int)sl : 0;
+        u += (unsigned long long)n * p.per_seq;
+        if (n > 1) sl += (unsigned long long)n * p.per_seq;
+    }
+    if (tid == 0) {
+        const int total_units = fits ? (int)(tot & 0xFFFFFFFFull) : p.B * p.per_seq;
+        p.t.unit_off[p.B] = total_units;
+        p.t.slot_off[p.B] = fits ? (int)(tot >> 32) : 0;
+        p.t.hdr[0] = total_units;
+        p.t.hdr[1] = (int)(total64 > 0x7FFFFFFFull ? 0x7FFFFFFFull : total64);
+        p.t.hdr[2] = target;
+    }
+}
+
 }  // namespace
 
 int launch_attn_plan(const AttnArgs& a) {
     if (!a.plan.dev.balanced) return GSD_OK;
+    if (a.plan.dev.balanced == 2) {
+        SeqPlanParams p;
+        p.seq_lens = a.seq_lens;
+        p.B = a.B; p.Lmax = a.Lmax;
+        p.per_seq = a.Hkv * a.plan.dev.tiles_per_unit;
+        p.nd = (a.N + 127) / 128;
+        p.units_wanted = kSeqPlanWaves * a.plan.ctas;
+        p.slots_cap = a.plan.slots;
+        p.t = plan_seq_table(a.plan, a.D, a.B, a.workspace);
+        attn_plan_seq_kernel<<<1, kPlanThreads, 0, a.stream>>>(p);
+        GSD_CUDA_TRY(cudaGetLastError());
+        return GSD_OK;
+    }
     if (a.plan.ctas / a.plan.dev.tiles_per_unit > kPlanThreads) return GSD_ERR_BAD_SHAPE;
     PlanParams p;
     p.seq_lens = a.seq_lens;

@@ -98,6 +98,7 @@ struct TcParams {
     int slots;        // partial-result slots of the plan
     const int2* bal_cta;     // balanced plan: (first unit, units) of every group of CTAs, else nullptr
     const int4* bal_units;   // balanced plan: (pair, first tile, end tile, slot or -1)
+    SeqTable seq;            // per-sequence plan: split counts and unit / slot offsets (hdr == nullptr otherwise)
     unsigned long long wait_limit_ns;
     int withhold_first_k;   // test hook: every CTA leaves out the K copy of its first key tile
 };
@@ -374,6 +375,21 @@ __device__ __forceinline__ UnitInfo unit_info(const TcParams& p, int w, int lane
         u.slot = rec.w >= 0 ? rt * 2 * ((int)gridDim.x / tpu) + rec.w : -1;
         u.split = 0;
         u.nsplit = rec.w >= 0 ? 2 : 1;     // only "one piece or several" matters below
+    } else if (p.seq.hdr) {
+        // unit w of the per-sequence plan: the last sequence whose first unit is <= w, then
+        // (key range, item) inside it
+        int lo = 0, hi = p.B - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (p.seq.unit_off[mid] <= w) lo = mid; else hi = mid - 1;
+        }
+        const int per_seq = p.Hkv * p.plan.tiles_per_unit;
+        const int r = w - p.seq.unit_off[lo];
+        u.nsplit = p.seq.nsplit[lo];
+        u.split = r / per_seq;
+        const int i = r - u.split * per_seq;
+        item = lo * per_seq + i;
+        u.slot = u.nsplit > 1 ? p.seq.slot_off[lo] + i * u.nsplit + u.split : 0;
     } else {
         plan_decode(p.plan, w, item, u.split, u.nsplit, u.slot);
     }
@@ -493,6 +509,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     if (p.bal_cta) {
         asm volatile("griddepcontrol.wait;" ::: "memory");
         n_my = p.bal_cta[blockIdx.x / p.plan.tiles_per_unit].y;
+    } else if (p.seq.hdr) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        const int units = p.seq.hdr[0];
+        n_my = units > (int)blockIdx.x ? (units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
     } else {
         n_my = p.total_work > (int)blockIdx.x ? (p.total_work - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
     }
@@ -1053,12 +1073,17 @@ int launch_attn_tcgen05(const AttnArgs& a) {
     if (device_info(&di) != 0) return GSD_ERR_CUDA;
     p.bal_cta = nullptr;
     p.bal_units = nullptr;
+    p.seq.hdr = nullptr; p.seq.nsplit = nullptr; p.seq.unit_off = nullptr; p.seq.slot_off = nullptr;
     if (a.plan.dev.balanced) {
         // one CTA per share of the table; the table is being written by the planning kernel,
         // beside which this kernel may start
-        const BalTable t = plan_bal_table(a.plan, a.D, a.workspace);
-        p.bal_cta = t.cta;
-        p.bal_units = t.units;
+        if (a.plan.dev.balanced == 2) {
+            p.seq = plan_seq_table(a.plan, a.D, a.B, a.workspace);
+        } else {
+            const BalTable t = plan_bal_table(a.plan, a.D, a.workspace);
+            p.bal_cta = t.cta;
+            p.bal_units = t.units;
+        }
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)a.plan.ctas);
         cfg.blockDim = dim3(kThreads);

@@ -59,9 +59,17 @@ int device_info(DeviceInfo* out);
 // for a whole pair), and per pair that was cut the run of slots to merge.  Slots are numbered
 // along the line, so the pieces of one pair have consecutive slots; a group has at most two
 // partial units (its first and last).  CTA r adds r * 2 * groups to a slot of its group.
+//
+// Per-sequence plan (tcgen05 back end only): a lighter form of the same idea that keeps the
+// CTAs of one sequence in step.  Every item of sequence b is cut into nsplit[b] equal key
+// ranges, nsplit[b] = its tile count over a common target length (rounded), chosen on the
+// device so that the batch makes about `units_wanted` units; units are numbered sequence by
+// sequence, range by range, item by item, and CTA k walks units k, k + grid, ...  The heads of
+// a sequence then read the same cache rows at the same time, which the head-interleaved cache
+// layout rewards (a row of the cache holds all kv heads of a position).
 struct PlanDev {
     int items_a, splits_a, splits_b, tiles_per_unit;
-    int balanced;       // 1: units come from the table built on the device
+    int balanced;       // 1: units come from the table built on the device; 2: per-sequence split counts from the device
 };
 struct AttnPlan {
     int kernel;         // GSD_ATTN_MMA or GSD_ATTN_TCGEN05
@@ -118,8 +126,16 @@ int attn_pick_kernel(const gsd_attn_params* p);                 // GSD_ATTN_MMA 
 inline size_t plan_part_o_bytes(const AttnPlan& pl, int D) { return align_up((size_t)pl.slots * pl.rows_per_item * D * sizeof(float), 256); }
 inline size_t plan_part_ml_bytes(const AttnPlan& pl) { return align_up((size_t)pl.slots * pl.rows_per_item * 2 * sizeof(float), 256); }
 
+// The table of a per-sequence plan, in the workspace behind the partial results.
+struct SeqTable {
+    int* hdr;        // [0] units of work, [1] tiles of all items, [2] target tiles per unit
+    int* nsplit;     // [B]     key ranges per item of the sequence
+    int* unit_off;   // [B + 1] first unit of the sequence
+    int* slot_off;   // [B + 1] first partial-result slot of the sequence (sequences cut in two or more only)
+};
 inline size_t plan_bal_bytes(const AttnPlan& pl, int B) {
     if (!pl.dev.balanced) return 0;
+    if (pl.dev.balanced == 2) return 256 + 3 * align_up((size_t)(B + 1) * sizeof(int), 256);
     return 256 + align_up((size_t)pl.ctas * sizeof(int2), 256) + align_up((size_t)pl.ctas * sizeof(int4), 256) +
            align_up((size_t)(pl.items + pl.ctas) * sizeof(int4), 256) + align_up((size_t)(B + 1) * sizeof(int), 256);
 }
@@ -134,7 +150,20 @@ inline BalTable plan_bal_table(const AttnPlan& pl, int D, void* workspace) {
     return t;
 }
 
-int launch_attn_plan(const AttnArgs& a);      // balanced plans only: builds the table
+inline SeqTable plan_seq_table(const AttnPlan& pl, int D, int B, void* workspace) {
+    char* at = (char*)workspace + plan_part_o_bytes(pl, D) + plan_part_ml_bytes(pl);
+    const size_t row = align_up((size_t)(B + 1) * sizeof(int), 256);
+    SeqTable t;
+    t.hdr = (int*)at; at += 256;
+    t.nsplit = (int*)at; at += row;
+    t.unit_off = (int*)at; at += row;
+    t.slot_off = (int*)at;
+    return t;
+}
+constexpr int kSeqPlanWaves = 2;              // units a per-sequence plan aims at, per resident CTA
+constexpr int kSeqPlanMaxSplit = 32;
+
+int launch_attn_plan(const AttnArgs& a);      // plans made on the device only: builds the table
 int launch_attn_mma(const AttnArgs& a);
 int launch_attn_tcgen05(const AttnArgs& a);
 bool attn_tcgen05_supports(int D, int G);

@@ -1,5 +1,5 @@
 """gsd_verify_attn with the work shared out on the device from seq_lens (num_splits =
-GSD_ATTN_SPLIT_BALANCED): same results as the
+GSD_ATTN_SPLIT_BALANCED or GSD_ATTN_SPLIT_PER_SEQUENCE): same results as the
 fp64 oracle, and a table that covers every key tile of every (sequence, kv head) pair exactly once."""
 import numpy as np
 import pytest
@@ -13,6 +13,7 @@ pytestmark = pytest.mark.gpu
 
 MAX_ABS, MEAN_ABS = 1e-2, 1e-3
 BALANCED = -1
+PER_SEQUENCE = -2
 TCGEN05 = 2
 
 
@@ -65,12 +66,13 @@ def make(shape, seed=3):
     return cfg, inp
 
 
+@pytest.mark.parametrize("mode", [BALANCED, PER_SEQUENCE])
 @pytest.mark.parametrize("shape", sorted(SHAPES))
-def test_balanced_against_the_oracle(shape):
+def test_balanced_against_the_oracle(shape, mode):
     cfg, inp = make(shape)
-    got = run(inp, kernel=TCGEN05, num_splits=BALANCED)
+    got = run(inp, kernel=TCGEN05, num_splits=mode)
     assert_close(out_to_f64(got), want_of(inp))
-    again = run(inp, kernel=TCGEN05, num_splits=BALANCED)
+    again = run(inp, kernel=TCGEN05, num_splits=mode)
     assert torch.equal(got, again)                            # bit-identical run to run
     # and within one bf16 step (2^-8 relative, values below 0.5 counted as 0.5) of the fixed plan's result
     fixed = run(inp, kernel=TCGEN05, num_splits=1).float()
@@ -84,9 +86,12 @@ def test_balanced_is_chosen_on_request_only():
     dims = (cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.D, inp["Lmax"])
     assert gsd.gsd_verify_attn_num_splits(*dims) > 0
     assert gsd.gsd_verify_attn_num_splits(*dims, BALANCED) == BALANCED
+    assert gsd.gsd_verify_attn_num_splits(*dims, PER_SEQUENCE) == PER_SEQUENCE
     assert gsd.gsd_verify_attn_num_splits(*dims, BALANCED, 1) >= 1          # the mma.sync kernel has no such plan
-    assert_close(out_to_f64(run(inp, num_splits=BALANCED)), want_of(inp))
-    assert_close(out_to_f64(run(inp, num_splits=BALANCED, kernel=1)), want_of(inp))
+    assert gsd.gsd_verify_attn_num_splits(*dims, PER_SEQUENCE, 1) >= 1
+    for mode in (BALANCED, PER_SEQUENCE):
+        assert_close(out_to_f64(run(inp, num_splits=mode)), want_of(inp))
+        assert_close(out_to_f64(run(inp, num_splits=mode, kernel=1)), want_of(inp))
 
 
 def table_of(ws, ctas, items, B):
@@ -166,3 +171,46 @@ def test_the_table_covers_every_tile_once(shape):
         assert listed[pair] == (sl[0], len(sl))
         all_slots += sl
     assert len(set(all_slots)) == len(all_slots) and (not all_slots or max(all_slots) < 2 * groups)
+
+
+@pytest.mark.parametrize("shape", ["gqa_ragged", "one_long", "many_sequences", "no_prefix"])
+def test_the_split_counts_follow_the_lengths(shape):
+    """Per-sequence plan: the table behind the partial results holds, per sequence, a split
+    count = its tile count over the common target (rounded, 1..32), and running unit and slot
+    offsets that match those counts."""
+    import paper_2407_16207_b200 as gsd
+    cfg, inp = make(shape, seed=13)
+    t = attn_tensors(inp)
+    Lmax = max(inp["Lmax"], 1)          # (the cache tensor has at least one row)
+    need = gsd.gsd_verify_attn_workspace_bytes(cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.D, Lmax, PER_SEQUENCE, TCGEN05)
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    gsd.gsd_verify_attn(t["q"], t["k_cache"], t["v_cache"], t["draft_k"], t["draft_v"], t["ancestor_mask"],
+                        t["seq_lens"], kernel=TCGEN05, num_splits=PER_SEQUENCE, workspace=ws)
+    torch.cuda.synchronize()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    G = cfg.Hq // cfg.Hkv
+    tpu = (cfg.N * G + 255) // 256
+    per_seq = cfg.Hkv * tpu
+    items = cfg.B * per_seq
+    nd = (cfg.N + 127) // 128
+    slots = min(2 * sms + items // 2 + 1, items * 32)
+
+    def up(x):
+        return (x + 255) // 256 * 256
+    at = up(slots * 256 * 128 * 4) + up(slots * 256 * 2 * 4)
+    raw = ws.cpu().numpy()
+    row = up((cfg.B + 1) * 4)
+    hdr = raw[at:at + 12].view(np.int32)
+    nsplit = raw[at + 256:at + 256 + cfg.B * 4].view(np.int32)
+    unit_off = raw[at + 256 + row:at + 256 + row + (cfg.B + 1) * 4].view(np.int32)
+    slot_off = raw[at + 256 + 2 * row:at + 256 + 2 * row + (cfg.B + 1) * 4].view(np.int32)
+    T = np.array([(int(min(max(L, 0), Lmax)) + 127) // 128 + nd for L in inp["seq_lens"]])
+    total = per_seq * int(T.sum())
+    target = max(4, -(-total // (2 * sms)))
+    want_n = np.clip((2 * T + target) // (2 * target), 1, 32)
+    assert hdr[1] == total and hdr[2] == target
+    assert np.array_equal(nsplit, want_n)
+    assert np.array_equal(unit_off, np.concatenate([[0], np.cumsum(want_n * per_seq)]))
+    assert np.array_equal(slot_off, np.concatenate([[0], np.cumsum(np.where(want_n > 1, want_n * per_seq, 0))]))
+    assert hdr[0] == unit_off[-1] and slot_off[-1] <= slots
+

@@ -40,7 +40,7 @@ def test_every_call_keeps_its_indices_inside(checked_lib, name):
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     want_attn = oracle.attn(inp["q"], inp["k_cache"], inp["v_cache"], inp["draft_k"], inp["draft_v"],
                             inp["ancestor_mask"], inp["seq_lens"])
-    for kernel, splits in ((0, 0), (1, 0), (1, 3), (2, 0), (2, 3), (2, -1)):
+    for kernel, splits in ((0, 0), (1, 0), (1, 3), (2, 0), (2, 3), (2, -1), (2, -2)):
         if kernel == 2 and cfg.D != 128:
             continue
         out = gsd.gsd_verify_attn(t["q"], t["k_cache"], t["v_cache"], t["draft_k"], t["draft_v"], t["ancestor_mask"],

@@ -36,7 +36,7 @@ def all_intact(*guards):
     return all(g.intact() for g in guards)
 
 
-@pytest.mark.parametrize("kernel,splits", [(2, 0), (2, 3), (2, -1), (1, 0), (1, 3)])
+@pytest.mark.parametrize("kernel,splits", [(2, 0), (2, 3), (2, -1), (2, -2), (1, 0), (1, 3)])
 def test_attention_output_and_workspace(kernel, splits):
     import paper_2407_16207_b200 as gsd
     # R = N * G = 400 stacked rows: the last 128-row tile is partial, N is no multiple of 128 / G
