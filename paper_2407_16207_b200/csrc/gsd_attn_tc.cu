@@ -327,8 +327,8 @@ __device__ __forceinline__ void tc_pv4(uint32_t d_tmem, uint32_t a_tmem, uint32_
 
 struct TileInfo {
     int kind;     // 0 full prefix tile, 1 ragged prefix tile, 2 draft tile
-    int key0;     // first key (prefix position or draft node) of the tile
-    int nvalid;   // prefix: visible keys in the tile
+    int key0;     // first key (prefix position or draft node) of the tile; negative for a ragged tile of a prefix below 128
+    int nvalid;   // prefix: visible keys in the tile (the last nvalid of a ragged tile)
 };
 
 __device__ __forceinline__ TileInfo tile_info(int t, int nPT, int L, unsigned live) {
@@ -337,6 +337,11 @@ __device__ __forceinline__ TileInfo tile_info(int t, int nPT, int L, unsigned li
         ti.key0 = t * BN;
         ti.nvalid = min(BN, L - ti.key0);
         ti.kind = ti.nvalid == BN ? 0 : 1;
+        // The ragged last tile is loaded as the LAST 128 rows of the prefix (rows before position
+        // 0 are filled with zeros by the copy engine): it then holds no row past the sequence
+        // end, whose contents could be anything, and its first 128 - nvalid keys, which the tile
+        // before it has covered already, are masked like invisible draft keys.
+        if (ti.kind == 1) ti.key0 = L - BN;
     } else {
         int k = t - nPT, d = 0;
         for (;; ++d) {   // the k-th set bit of `live`
@@ -736,8 +741,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 } else if (ti.kind == 1) {
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
-                        const int rem = ti.nvalid - 32 * k;
-                        mw[k] = rem >= 32 ? 0xFFFFFFFFu : (rem <= 0 ? 0u : ((1u << rem) - 1u));
+                        const int from = (BN - ti.nvalid) - 32 * k;      // first visible key of the word
+                        mw[k] = from <= 0 ? 0xFFFFFFFFu : (from >= 32 ? 0u : ~((1u << from) - 1u));
                     }
                 } else {
 #pragma unroll
@@ -804,23 +809,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 m_ref = m_new;
                 const float m_use = m_ref == -CUDART_INF_F ? 0.f : m_ref;
 
-                if (ti.kind == 1 && (alt || i == 0)) {
-                    // cache rows past the sequence end may hold anything: clear them in the V tile
-                    // so that 0 * junk cannot reach the accumulator
-                    const int vs_stage = (kvc + idx) % VST;
-                    ok = mbar_wait(bar(BAR_V_FULL + vs_stage), (uint32_t)(((kvc + idx) / VST) & 1), abort_flag, p.status);
-                    ok = __all_sync(0xFFFFFFFFu, ok);
-                    if (!ok) break;
-                    if (rloc >= ti.nvalid) {
-                        unsigned char* vrow = smem_raw + (sV - smem_u32(smem_raw)) + vs_stage * TILE_BYTES + rloc * 128;
-#pragma unroll
-                        for (int h = 0; h < 2; ++h)
-#pragma unroll
-                            for (int k = 0; k < 8; ++k)
-                                *reinterpret_cast<uint4*>(vrow + h * HALF_BYTES + k * 16) = make_uint4(0, 0, 0, 0);
-                    }
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                }
                 // P = 2^(s*scale - m) as bf16 pairs into the 64 columns of P_i; a masked score is
                 // -inf and comes out as exactly 0
                 const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
