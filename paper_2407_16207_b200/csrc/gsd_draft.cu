@@ -249,24 +249,37 @@ __device__ __forceinline__ void block_best(float& v, int& i, int& owner, float* 
 
 // The k best tokens of one row of logits and their probabilities, in one pass over the row.
 // Every thread streams its strided share (16-byte loads, kBatch in flight) and keeps the running
-// (maximum, sum of exponentials) pair and the two best (logit, token) pairs it has met.  The
-// 512 pairs go to shared memory and one warp picks the row's k best of them with shuffles
-// (ranked by logit, ties to the lower token id).  That is the exact answer unless a thread's
-// SECOND pair was picked - then a third entry of that thread could rank among the k best too
-// (for a random row: about one row in fifty).  Such a row is read once more (from L2): the k-th
-// pick bounds the k-th best entry from below, the entries at or before it form a short list,
-// and the pick is repeated over the list.  Only a list longer than 512 (long runs of equal
-// logits) takes the slow exact way: every thread keeps the K best pairs it meets and the block
-// merges the 256 lists.
+// (maximum, sum of exponentials) pair, the best (logit, token) pair it has met and the VALUE of
+// its second best entry - all without a branch, so that no lane of a warp waits for another's
+// rare update.  The 256 best pairs are picked over in two stages, both with shuffles only (ranked
+// by logit, ties to the lower token id): every warp picks the k best of its 32 pairs, then one
+// warp picks the k best of those 8 k.  That is the exact answer unless some thread's second best
+// entry ranks at or before the k-th pick - then an entry that no thread offered could belong
+// to the k best (for a random row: about one row in fifty).  Such a row is read once more (from
+// L2): the k-th pick bounds the k-th best entry from below, the entries at or before it form a
+// short list, and the pick is repeated over the list.  Only a list longer than 512 (long runs
+// of equal logits) takes the slow exact way: every thread keeps the K best pairs it meets and
+// the block merges the 256 lists.
 constexpr int kBatch = 8;     // 16-byte loads a thread keeps in flight while it streams a row
-struct Two {
-    float v1, v2;
-    int i1, i2;
+struct Best {
+    float v1, v2;   // best and second best logit of the thread's share (v2: value only)
+    int i1;         // token of the best
 };
-__device__ __forceinline__ void offer2(Two& t, float x, int idx) {
+__device__ __forceinline__ void offer_best(Best& t, float x, int idx) {
     // a thread meets its entries in ascending token order: an equal logit never displaces an earlier one
-    if (x > t.v1) { t.v2 = t.v1; t.i2 = t.i1; t.v1 = x; t.i1 = idx; }
-    else if (x > t.v2) { t.v2 = x; t.i2 = idx; }
+    const bool up = x > t.v1;
+    t.v2 = fmaxf(t.v2, up ? t.v1 : x);
+    t.i1 = up ? idx : t.i1;
+    t.v1 = up ? x : t.v1;
+}
+// The best of the pairs the 32 lanes hold (ranked by `before`), and the lane that held it.
+__device__ __forceinline__ void warp_best(float& v, int& i, int& src) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float v2 = __shfl_xor_sync(0xFFFFFFFFu, v, o);
+        const int i2 = __shfl_xor_sync(0xFFFFFFFFu, i, o), s2 = __shfl_xor_sync(0xFFFFFFFFu, src, o);
+        if (before(v2, i2, v, i)) { v = v2; i = i2; src = s2; }
+    }
 }
 
 // One warp picks the k best of `count` <= 512 (logit, token) pairs in shared memory with
@@ -320,12 +333,12 @@ __device__ __forceinline__ int warp_pick_k(const float* s_cv, const int* s_ci, i
 }
 
 template <bool kVec>
-__global__ void __launch_bounds__(kThreads, 5) draft_expand_kernel(DraftArgs a) {
+__global__ void __launch_bounds__(kThreads, 4) draft_expand_kernel(DraftArgs a) {
     __shared__ float s_cv[2 * kThreads];
     __shared__ int s_ci[2 * kThreads];
     __shared__ float s_rv[kWarps];
     __shared__ int s_ri[kWarps], s_rt[kWarps];
-    __shared__ float s_m[kWarps], s_s[kWarps];
+    __shared__ float s_m[kWarps], s_s[kWarps], s_v2[kWarps];
     __shared__ int s_redo, s_count, s_ti;
     __shared__ float s_tv;
     // the per-sequence pass (a programmatic dependent launch) may become resident as CTAs retire
@@ -339,9 +352,9 @@ __global__ void __launch_bounds__(kThreads, 5) draft_expand_kernel(DraftArgs a) 
     const float4* x4 = reinterpret_cast<const float4*>(x);
     const int nvec = V >> 2;
     float m = -CUDART_INF_F, s = 0.f;        // running maximum and sum
-    Two two{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF, 0x7FFFFFFF};
+    Best best{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF};
     auto take = [&](float val, int idx) {
-        offer2(two, val, idx);
+        offer_best(best, val, idx);
         if (val > m) {
             s = s * ex2((m - val) * kLog2e) + 1.f;
             m = val;
@@ -364,10 +377,9 @@ __global__ void __launch_bounds__(kThreads, 5) draft_expand_kernel(DraftArgs a) 
                 const float g4 = fmaxf(fmaxf(r[k].x, r[k].y), fmaxf(r[k].z, r[k].w));
                 g = fmaxf(g, g4);
                 nan_probe += (r[k].x + r[k].y) + (r[k].z + r[k].w);     // NaN if any entry is NaN (or +inf and -inf meet)
-                if (g4 > two.v2) {      // seldom true once the thread has seen a few entries
-                    const int e = (i + k * kThreads) * 4;
-                    offer2(two, r[k].x, e); offer2(two, r[k].y, e + 1); offer2(two, r[k].z, e + 2); offer2(two, r[k].w, e + 3);
-                }
+                const int e = (i + k * kThreads) * 4;
+                offer_best(best, r[k].x, e); offer_best(best, r[k].y, e + 1);
+                offer_best(best, r[k].z, e + 2); offer_best(best, r[k].w, e + 3);
             }
             if (nan_probe != nan_probe) {
                 // rare: find out entry by entry (a NaN poisons the sum; -inf next to +inf does not)
@@ -392,8 +404,23 @@ __global__ void __launch_bounds__(kThreads, 5) draft_expand_kernel(DraftArgs a) 
     } else {
         for (int i = tid; i < V; i += kThreads) take(__ldcs(x + i), i);
     }
-    s_cv[2 * tid] = two.v1; s_ci[2 * tid] = two.i1;
-    s_cv[2 * tid + 1] = two.v2; s_ci[2 * tid + 1] = two.i2;
+    // stage 1: every warp picks the k best of its 32 pairs; lane r keeps the r-th pick
+    {
+        float cv = best.v1, pv = -CUDART_INF_F;
+        int ci = best.i1, pi = 0x7FFFFFFF;
+        for (int r = 0; r < a.k; ++r) {
+            float v = cv;
+            int i = ci, src = lane;
+            warp_best(v, i, src);
+            if (lane == r) { pv = v; pi = i; }
+            if (src == lane) { cv = -CUDART_INF_F; ci = 0x7FFFFFFF; }      // (a pair at -inf is never taken: its token is none)
+        }
+        if (lane < a.k) { s_cv[warp * K + lane] = pv; s_ci[warp * K + lane] = pi; }
+        float v2 = best.v2;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v2 = fmaxf(v2, __shfl_xor_sync(0xFFFFFFFFu, v2, o));
+        if (lane == 0) s_v2[warp] = v2;
+    }
     // (maximum, sum) of the row
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -407,26 +434,54 @@ __global__ void __launch_bounds__(kThreads, 5) draft_expand_kernel(DraftArgs a) 
     if (tid == 0) s_redo = 0;
     __syncthreads();
     float rm = -CUDART_INF_F, rs = 0.f;
-    for (int w = 0; w < kWarps; ++w) {
-        const float mm = fmaxf(rm, s_m[w]);
-        rs = (mm == -CUDART_INF_F) ? ((rs != rs || s_s[w] != s_s[w]) ? CUDART_NAN_F : 0.f)
-                                   : rs * ex2((rm - mm) * kLog2e) + s_s[w] * ex2((s_m[w] - mm) * kLog2e);
-        rm = mm;
-    }
-    if (tid == 0 && (!(rs > 0.f) || rm == CUDART_INF_F) && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
     const size_t w = ((size_t)b * a.F + fi) * K;
     if (warp == 0) {
-        float tv;
-        int ti;
-        const int res = warp_pick_k(s_cv, s_ci, 2 * kThreads, a.k, rm, rs, a.wk_tok + w, a.wk_q + w, &tv, &ti);
+        for (int q = 0; q < kWarps; ++q) {
+            const float mm = fmaxf(rm, s_m[q]);
+            rs = (mm == -CUDART_INF_F) ? ((rs != rs || s_s[q] != s_s[q]) ? CUDART_NAN_F : 0.f)
+                                       : rs * ex2((rm - mm) * kLog2e) + s_s[q] * ex2((s_m[q] - mm) * kLog2e);
+            rm = mm;
+        }
+        if (lane == 0 && (!(rs > 0.f) || rm == CUDART_INF_F) && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
+        // stage 2: the k best of the 8 k picks (two per lane at most)
+        const int n = kWarps * a.k;
+        float c0 = -CUDART_INF_F, c1 = -CUDART_INF_F;
+        int j0 = 0x7FFFFFFF, j1 = 0x7FFFFFFF;
+        if (lane < n) { c0 = s_cv[(lane / a.k) * K + lane % a.k]; j0 = s_ci[(lane / a.k) * K + lane % a.k]; }
+        if (lane + 32 < n) { c1 = s_cv[((lane + 32) / a.k) * K + (lane + 32) % a.k]; j1 = s_ci[((lane + 32) / a.k) * K + (lane + 32) % a.k]; }
+        float tv = -CUDART_INF_F;
+        int ti = 0x7FFFFFFF;
+        bool short_row = false;
+        for (int r = 0; r < a.k; ++r) {
+            const bool second = before(c1, j1, c0, j0);
+            float v = second ? c1 : c0;
+            int i = second ? j1 : j0, src = lane;
+            warp_best(v, i, src);
+            if (src == lane) {
+                if (second) { c1 = -CUDART_INF_F; j1 = 0x7FFFFFFF; } else { c0 = -CUDART_INF_F; j0 = 0x7FFFFFFF; }
+            }
+            const bool none = i == 0x7FFFFFFF;
+            short_row |= none;
+            if (lane == 0) {
+                a.wk_tok[w + r] = none ? -1 : i;
+                a.wk_q[w + r] = none ? 0.f : ex2((v - rm) * kLog2e) / rs;
+            }
+            tv = v;
+            ti = i;
+        }
+        // an entry that no thread offered can rank at or before the k-th pick only if some
+        // thread's second best does
+        float v2 = lane < kWarps ? s_v2[lane] : -CUDART_INF_F;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v2 = fmaxf(v2, __shfl_xor_sync(0xFFFFFFFFu, v2, o));
+        const bool redo = v2 > -CUDART_INF_F && v2 >= tv;
         if (lane == 0) {
-            // a thread's second pair among the picks: a third entry of that thread is unknown
-            s_redo = res & 1;
+            s_redo = redo ? 1 : 0;
             s_tv = tv;
             s_ti = ti;
             s_count = 0;
-            // (then the second pass below decides whether the row is short of k entries)
-            if ((res & 2) && !(res & 1) && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
+            // (a row that goes through the second pass finds out there whether it is short of k entries)
+            if (short_row && !redo && a.status) atomicOr((unsigned*)a.status, GSD_DEV_BAD_LOGITS);
         }
     }
     __syncthreads();
