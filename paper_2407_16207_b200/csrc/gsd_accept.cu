@@ -93,9 +93,10 @@ struct AcceptArgs {
 __device__ void path_pass(const AcceptArgs& a, int b) {
     __shared__ int s_amax[GSD_MAX_NODES];
     const int N = a.N, tid = threadIdx.x;
-    // the keys were written by other CTAs: read them past L1
+    // the keys were written by other CTAs: read them past L1.  (No barrier of its own: the path
+    // routine fetches the graph first and meets at a barrier before any step is tested, so the
+    // two trips to memory overlap.)
     for (int v = tid; v < N; v += kThreads) s_amax[v] = key_index(__ldcg(a.keys + (size_t)b * N + v));
-    __syncthreads();
     const int32_t* tok = a.tok + (size_t)b * N;
     PathIo io;
     io.tok = tok;

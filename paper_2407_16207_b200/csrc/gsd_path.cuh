@@ -20,6 +20,7 @@ constexpr int kPathThreads = 256;
 constexpr int kPathNone = 0x7FFFFFFF;
 constexpr int kPathNodeSlots = (GSD_MAX_NODES + kPathThreads - 1) / kPathThreads;
 constexpr int kPathEdgeCache = 3 * GSD_MAX_NODES;   // parent edges of one sequence kept in shared memory
+static_assert(kPathEdgeCache % kPathThreads == 0, "the edge prefetch is dealt out in whole rounds");
 
 struct PathIo {
     const int32_t* tok;     // [N] drafted tokens of the sequence
@@ -60,22 +61,41 @@ __device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, St
     if (tid == 0) s_flags = 0;
     // tokens, row pointers and (speculatively: the row holds Ecap entries whatever the pointers
     // say) the parent indices, all in one trip to memory
-    for (int v = tid; v < N; v += kPathThreads) {
-        const int t = io.tok[v];
-        s_tok[v] = t;
-        if (t < 0 || t >= io.V) flags |= GSD_DEV_BAD_TOKEN;
-        s_best[0][v] = v == 0 ? 0 : -1;
-    }
-    for (int v = tid; v <= N; v += kPathThreads) {
-        int e = io.pptr[v];
-        if (e < 0 || e > io.Ecap) {
-            flags |= GSD_DEV_BAD_CSR;
-            e = e < 0 ? 0 : io.Ecap;
-        }
-        s_ptr[v] = e;
-    }
+    // (every load is issued before the first of them is used: the loops below have constant
+    // trip counts and are unrolled, so the three arrays cost one round trip, not three)
     const int n_prefetch = min(io.Ecap, kPathEdgeCache);
-    for (int e = tid; e < n_prefetch; e += kPathThreads) s_edge[e] = io.pidx[e];
+    int r_tok[kPathNodeSlots], r_ptr[kPathNodeSlots + 1], r_edge[kPathEdgeCache / kPathThreads];
+#pragma unroll
+    for (int k = 0; k < kPathNodeSlots; ++k) r_tok[k] = tid + k * kPathThreads < N ? io.tok[tid + k * kPathThreads] : 0;
+#pragma unroll
+    for (int k = 0; k <= kPathNodeSlots; ++k) r_ptr[k] = tid + k * kPathThreads <= N ? io.pptr[tid + k * kPathThreads] : 0;
+#pragma unroll
+    for (int k = 0; k < kPathEdgeCache / kPathThreads; ++k)
+        r_edge[k] = tid + k * kPathThreads < n_prefetch ? io.pidx[tid + k * kPathThreads] : 0;
+#pragma unroll
+    for (int k = 0; k < kPathNodeSlots; ++k) {
+        const int v = tid + k * kPathThreads;
+        if (v < N) {
+            s_tok[v] = r_tok[k];
+            if (r_tok[k] < 0 || r_tok[k] >= io.V) flags |= GSD_DEV_BAD_TOKEN;
+            s_best[0][v] = v == 0 ? 0 : -1;
+        }
+    }
+#pragma unroll
+    for (int k = 0; k <= kPathNodeSlots; ++k) {
+        const int v = tid + k * kPathThreads;
+        if (v <= N) {
+            int e = r_ptr[k];
+            if (e < 0 || e > io.Ecap) {
+                flags |= GSD_DEV_BAD_CSR;
+                e = e < 0 ? 0 : io.Ecap;
+            }
+            s_ptr[v] = e;
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < kPathEdgeCache / kPathThreads; ++k)
+        if (tid + k * kPathThreads < n_prefetch) s_edge[tid + k * kPathThreads] = r_edge[k];
     __syncthreads();
     // Row pointers must start at zero and never decrease.  Otherwise they are replaced by their
     // running maximum (a row whose pointer goes backwards becomes empty, the rows stay disjoint
