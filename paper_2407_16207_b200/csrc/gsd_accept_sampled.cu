@@ -134,7 +134,8 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
         s_uq[v] = u[v] * q[v];       // the left side of the step test, fetched beside the pairs
         if (!(r.s > 0.f) || r.m == CUDART_INF_F) flags |= GSD_DEV_BAD_LOGITS;   // no finite entry, +inf or NaN
     }
-    __syncthreads();
+    // (no barrier here: the path routine fetches the graph first and meets at a barrier before
+    // any step is tested, so that trip to memory overlaps the one above)
     PathIo io;
     io.tok = tok;
     io.pptr = a.pptr + (size_t)b * (N + 1);
