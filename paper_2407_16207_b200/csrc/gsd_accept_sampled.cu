@@ -114,28 +114,34 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     const float* lg = a.logits + (size_t)b * N * V;
     const float* q = a.q + (size_t)b * N;
     const float* u = a.u + (size_t)b * N;
-    unsigned flags = 0;
-    for (int v = tid; v < N; v += kThreads) {
-        // the pairs were written by other CTAs: read them past L1
-        Ms r{-CUDART_INF_F, 0.f};
-        const float4* pp = reinterpret_cast<const float4*>(a.part + ((size_t)b * N + v) * a.slices * kWarps);
-        for (int k = 0; k < a.slices * (kWarps / 2); k += 4) {     // eight pairs (64 bytes) per round, loaded at once
-            float4 t[4];
+    // Softmax statistics of every node from the pairs of the first launch, and the left sides
+    // of the step tests.  This is the first thing that needs the first launch's results: the path
+    // routine calls it after the graph and one logit per step have been fetched, so those two
+    // trips to memory are over when the first launch ends.
+    auto combine_pairs = [&]() -> unsigned {
+        unsigned flags = 0;
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        for (int v = tid; v < N; v += kThreads) {
+            // the pairs were written by other CTAs: read them past L1
+            Ms r{-CUDART_INF_F, 0.f};
+            const float4* pp = reinterpret_cast<const float4*>(a.part + ((size_t)b * N + v) * a.slices * kWarps);
+            for (int k = 0; k < a.slices * (kWarps / 2); k += 4) {     // eight pairs (64 bytes) per round, loaded at once
+                float4 t[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) t[i] = __ldcg(pp + k + i);
+                for (int i = 0; i < 4; ++i) t[i] = __ldcg(pp + k + i);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                r = combine(r, Ms{t[i].x, t[i].y});
-                r = combine(r, Ms{t[i].z, t[i].w});
+                for (int i = 0; i < 4; ++i) {
+                    r = combine(r, Ms{t[i].x, t[i].y});
+                    r = combine(r, Ms{t[i].z, t[i].w});
+                }
             }
+            s_mx[v] = r.m;
+            s_sum[v] = r.s;
+            s_uq[v] = u[v] * q[v];       // the left side of the step test, fetched beside the pairs
+            if (!(r.s > 0.f) || r.m == CUDART_INF_F) flags |= GSD_DEV_BAD_LOGITS;   // no finite entry, +inf or NaN
         }
-        s_mx[v] = r.m;
-        s_sum[v] = r.s;
-        s_uq[v] = u[v] * q[v];       // the left side of the step test, fetched beside the pairs
-        if (!(r.s > 0.f) || r.m == CUDART_INF_F) flags |= GSD_DEV_BAD_LOGITS;   // no finite entry, +inf or NaN
-    }
-    // (no barrier here: the path routine fetches the graph first and meets at a barrier before
-    // any step is tested, so that trip to memory overlaps the one above)
+        return flags;
+    };
     PathIo io;
     io.tok = tok;
     io.pptr = a.pptr + (size_t)b * (N + 1);
@@ -147,11 +153,14 @@ __device__ void finish_sequence(const SampledArgs& a, int b) {
     io.N = N; io.V = V; io.Ecap = a.Ecap; io.Tcap = a.Tcap;
     // the test of one step: the target's probability of v's token under its parent p (one
     // logit gathered from global memory) against u q
-    const PathResult res = longest_accepted_path<true>(io, flags, [&](int p, int v) {
-        if (!GSD_IN_BOUNDS(p >= 0 && p < N && tok[v] >= 0 && tok[v] < V, a.status)) return false;
-        const float prob = ex2((lg[(size_t)p * V + tok[v]] - s_mx[p]) * kLog2e) / s_sum[p];
-        return s_uq[v] < prob;
-    });
+    const PathResult res = longest_accepted_path_ex<true>(
+        io, 0u,
+        [&](float logit, int p, int v) { return s_uq[v] < ex2((logit - s_mx[p]) * kLog2e) / s_sum[p]; },
+        [&](int p, int v) -> float {
+            if (!GSD_IN_BOUNDS(p >= 0 && p < N && tok[v] >= 0 && tok[v] < V, a.status)) return -CUDART_INF_F;
+            return lg[(size_t)p * V + tok[v]];
+        },
+        combine_pairs);
     const int s_m = res.edges, s_end = res.end;
     int32_t* out_tok = io.out_tok;
 
@@ -411,8 +420,7 @@ __global__ void __launch_bounds__(kThreads) accept_sampled_kernel(SampledArgs a)
 // Second launch: one CTA per sequence does the rest (statistics per node, step tests, longest
 // path, regenerated token) once every pair of the first launch is visible.
 __global__ void __launch_bounds__(kThreads, 1) accept_sampled_tail_kernel(SampledArgs a) {
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    finish_sequence(a, blockIdx.x);
+    finish_sequence(a, blockIdx.x);      // (waits for the first launch inside, as late as it can)
 }
 
 int pick_slices(long rows, int V, int sm_count) {

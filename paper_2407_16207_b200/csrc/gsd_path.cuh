@@ -39,19 +39,24 @@ struct PathResult {
     bool end_has_child;  // some node lists `end` as a parent (only filled in with kCacheOutcome)
 };
 
-// With kCacheOutcome, `step_ok(p, v)` is called once per step when the parent lists fit the
-// on-chip cache (one thread per step, all at once - for tests that touch global memory);
-// otherwise it is called again on every use (for tests that cost a comparison).  `flags` carries status bits the
-// caller has already found; the function adds its own and publishes them.  All threads of the
-// CTA must call it; all return the same result.  out_tok[edges] is left for the caller,
-// entries past it are set to -1.
-template <bool kCacheOutcome, class StepOk>
-__device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, StepOk step_ok) {
+// The test of a step p -> v comes in two halves: `edge_pre(p, v)` fetches what the test needs
+// from global memory (a float), `step_ok(pre, p, v)` decides.  With kCacheOutcome both are
+// called once per step when the parent lists fit the on-chip cache (one thread per step, all at
+// once - for tests that touch global memory); otherwise they are called again on every use (for
+// tests that cost a comparison).  Between the two halves the function calls `mid()` (all
+// threads; it returns status bits) and meets at a barrier: a caller whose decision needs results
+// of an earlier kernel waits for them there, AFTER the graph and the values of `edge_pre` have
+// been fetched.  `flags` carries status bits the caller has already found; the function adds its
+// own and publishes them.  All threads of the CTA must call it; all return the same result.
+// out_tok[edges] is left for the caller, entries past it are set to -1.
+template <bool kCacheOutcome, class StepOk, class EdgePre, class Mid>
+__device__ PathResult longest_accepted_path_ex(const PathIo& io, unsigned flags, StepOk step_ok, EdgePre edge_pre, Mid mid) {
     __shared__ int s_best[2][GSD_MAX_NODES];      // two copies: a round reads one and writes the other
     __shared__ int s_tok[GSD_MAX_NODES];
     __shared__ int s_ptr[GSD_MAX_NODES + 1];
     __shared__ int s_edge[kPathEdgeCache];
     __shared__ unsigned char s_eok[kPathEdgeCache];
+    __shared__ float s_eval[kCacheOutcome ? kPathEdgeCache : 1];   // what edge_pre fetched for each step
     __shared__ short s_enode[kPathEdgeCache];   // the node a step leads into
     __shared__ short s_path[GSD_MAX_NODES];     // the chosen path, root first
     __shared__ int s_red[kPathThreads / 32];
@@ -127,14 +132,22 @@ __device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, St
         __syncthreads();
         for (int e = tid; e < n_edges; e += kPathThreads) {
             const int p = s_edge[e], v = s_enode[e];
-            s_eok[e] = (p >= 0 && p < v && s_tok[v] >= 0 && s_tok[v] < io.V) ? (unsigned char)step_ok(p, v) : 0;
+            s_eval[e] = (p >= 0 && p < v && s_tok[v] >= 0 && s_tok[v] < io.V) ? edge_pre(p, v) : 0.f;
+        }
+    }
+    flags |= mid();
+    __syncthreads();
+    if (cached && kCacheOutcome) {
+        for (int e = tid; e < n_edges; e += kPathThreads) {
+            const int p = s_edge[e], v = s_enode[e];
+            s_eok[e] = (p >= 0 && p < v && s_tok[v] >= 0 && s_tok[v] < io.V) ? (unsigned char)step_ok(s_eval[e], p, v) : 0;
         }
         __syncthreads();
     }
     auto parent_at = [&](int e) -> int { return cached ? s_edge[e] : io.pidx[e]; };
     auto ok_at = [&](int e, int p, int v) -> bool {
         if (cached && kCacheOutcome) return s_eok[e] != 0;
-        return s_tok[v] >= 0 && s_tok[v] < io.V && step_ok(p, v);
+        return s_tok[v] >= 0 && s_tok[v] < io.V && step_ok(edge_pre(p, v), p, v);
     };
 
     // level-synchronous relaxation: after round r every node whose longest accepted root
@@ -233,6 +246,13 @@ __device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, St
         end_has_child = __syncthreads_or(has) != 0;
     }
     return PathResult{s_m, s_end, end_has_child};
+}
+
+// The plain form: a test `step_ok(p, v)` that needs nothing fetched and nothing waited for.
+template <bool kCacheOutcome, class StepOk>
+__device__ PathResult longest_accepted_path(const PathIo& io, unsigned flags, StepOk step_ok) {
+    return longest_accepted_path_ex<kCacheOutcome>(
+        io, flags, [&](float, int p, int v) { return step_ok(p, v); }, [](int, int) { return 0.f; }, []() { return 0u; });
 }
 
 }  // namespace gsd
