@@ -107,33 +107,39 @@ __device__ void grow_sequence(const DraftArgs& a, int b) {
         flags |= GSD_DEV_DRAFT_FULL;
     }
     const int n1 = n0 + want;
+    // Everything that does not need the row kernel's results comes first - this kernel is its
+    // programmatic dependent and is resident while it still runs: the graph as it stands, the
+    // parents of the children to come, the tau-gram hashes of the old nodes and their entries in
+    // the hash table.
+    constexpr int kChildSlots = (GSD_MAX_NODES + kThreads - 1) / kThreads;
+    int p_child[kChildSlots];
+#pragma unroll
+    for (int s = 0; s < kChildSlots; ++s) {
+        const int j = tid + s * kThreads;
+        int p = 0;
+        if (j < want) {
+            p = a.frontier[(size_t)b * a.F + j / k];
+            if (p < 0 || p >= n0) {
+                flags |= GSD_DEV_BAD_FRONTIER;
+                p = 0;
+            }
+        }
+        p_child[s] = p;
+    }
     for (int v = tid; v < n0; v += kThreads) {
         s_tok[v] = tok[v];
         s_par[v] = par[v];
     }
-    // the children: k per frontier node, in frontier order, best first
-    for (int j = tid; j < want; j += kThreads) {
-        const int fi = j / k, i = j % k, c = n0 + j;
-        const size_t w = ((size_t)b * a.F + fi) * K;
-        int p = a.frontier[(size_t)b * a.F + fi];
-        if (p < 0 || p >= n0) {
-            flags |= GSD_DEV_BAD_FRONTIER;
-            p = 0;
-        }
-        if (!GSD_IN_BOUNDS(c < Ncap && fi < a.F && i < K, a.status)) continue;
-        const float q = a.wk_q[w + i], qmax = a.wk_q[w];
-        s_tok[c] = a.wk_tok[w + i];
-        s_par[c] = p;
-        // Sec. 4.2: below the probability threshold, or too far below the best sibling
-        s_leaf[c] = (q < a.theta_prob) || (q < a.theta_sib * qmax);
-        prob[c] = q;
+    constexpr unsigned kNoGram = 0xFFFFFFFFu;
+    for (int t = tid; t < kHashSlots; t += kThreads) {
+        s_hkey[t] = kNoGram;
+        s_hmin[t] = 0x7FFFFFFF;
     }
     __syncthreads();
     // Sec. 5.2 / 5.3: a new node whose last tau tokens along its tree path equal those of an
     // earlier node is redundant; it becomes a leaf that points at the first such node.
     // Every node's tau-gram is reduced to a 32-bit hash; equal hashes are confirmed token by token.
-    constexpr unsigned kNoGram = 0xFFFFFFFFu;
-    for (int v = tid; v < n1; v += kThreads) {
+    auto gram_key = [&](int v) -> unsigned {
         unsigned h = 2166136261u;
         int x = v, t = 0;
         for (; t < a.tau && x >= 0; ++t) {
@@ -141,30 +147,17 @@ __device__ void grow_sequence(const DraftArgs& a, int b) {
             h ^= h >> 15;
             x = s_par[x];
         }
-        s_key[v] = (t == a.tau) ? (h == kNoGram ? 0u : h) : kNoGram;
-    }
-    __syncthreads();
-    auto same_gram = [&](int x, int y) -> bool {
-        for (int t = 0; t < a.tau; ++t) {
-            if (x < 0 || y < 0 || s_tok[x] != s_tok[y]) return false;
-            x = s_par[x];
-            y = s_par[y];
-        }
-        return true;
+        return (t == a.tau) ? (h == kNoGram ? 0u : h) : kNoGram;
     };
     // first occurrences through a hash table in shared memory: every node with a tau-gram enters
     // its id under its hash (open addressing; the slot keeps the lowest id), so a new node finds
     // the lowest earlier node with its hash in one probe sequence instead of a scan over all
     // earlier nodes.  Equal hashes are confirmed token by token; if the lowest id under the hash
     // is a different gram (a collision of the 32-bit hash) the node falls back to the scan.
-    for (int t = tid; t < kHashSlots; t += kThreads) {
-        s_hkey[t] = kNoGram;
-        s_hmin[t] = 0x7FFFFFFF;
-    }
-    __syncthreads();
-    for (int v = tid; v < n1; v += kThreads) {
-        const unsigned kv = s_key[v];
-        if (kv == kNoGram) continue;
+    auto enter = [&](int v) {
+        const unsigned kv = gram_key(v);
+        s_key[v] = kv;
+        if (kv == kNoGram) return;
         unsigned slot = (kv * 2654435761u) >> (32 - kHashBits);
         for (int probe = 0; probe < kHashSlots; ++probe) {
             const unsigned prev = atomicCAS(&s_hkey[slot], kNoGram, kv);
@@ -174,7 +167,35 @@ __device__ void grow_sequence(const DraftArgs& a, int b) {
             }
             slot = (slot + 1) & (kHashSlots - 1);
         }
+    };
+    for (int v = tid; v < n0; v += kThreads) enter(v);
+
+    // the children: k per frontier node, in frontier order, best first
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+#pragma unroll
+    for (int s = 0; s < kChildSlots; ++s) {
+        const int j = tid + s * kThreads;
+        if (j >= want) continue;
+        const int fi = j / k, i = j % k, c = n0 + j;
+        const size_t w = ((size_t)b * a.F + fi) * K;
+        if (!GSD_IN_BOUNDS(c < Ncap && fi < a.F && i < K, a.status)) continue;
+        const float q = a.wk_q[w + i], qmax = a.wk_q[w];
+        s_tok[c] = a.wk_tok[w + i];
+        s_par[c] = p_child[s];
+        // Sec. 4.2: below the probability threshold, or too far below the best sibling
+        s_leaf[c] = (q < a.theta_prob) || (q < a.theta_sib * qmax);
+        prob[c] = q;
     }
+    __syncthreads();
+    for (int v = n0 + tid; v < n1; v += kThreads) enter(v);
+    auto same_gram = [&](int x, int y) -> bool {
+        for (int t = 0; t < a.tau; ++t) {
+            if (x < 0 || y < 0 || s_tok[x] != s_tok[y]) return false;
+            x = s_par[x];
+            y = s_par[y];
+        }
+        return true;
+    };
     __syncthreads();
     for (int j = tid; j < want; j += kThreads) {
         const int c = n0 + j;
@@ -565,8 +586,7 @@ __global__ void __launch_bounds__(kThreads, 4) draft_expand_kernel(DraftArgs a) 
 // Second launch: one CTA per sequence appends the children and updates the graph once every
 // row's result of the first launch is visible.
 __global__ void __launch_bounds__(kThreads) draft_grow_kernel(DraftArgs a) {
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    grow_sequence(a, blockIdx.x);
+    grow_sequence(a, blockIdx.x);        // (waits for the first launch inside, as late as it can)
 }
 
 }  // namespace
