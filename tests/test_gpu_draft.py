@@ -129,6 +129,36 @@ def test_long_runs_of_equal_logits():
     assert list(got[0][0, 1:1 + k]) == list(range(k))
 
 
+def test_best_entries_in_one_threads_share():
+    # The row kernel offers one candidate per thread; a thread's share is every 256th group of
+    # four entries.  Here the k best entries of a row sit in one group, in groups 1024 entries
+    # apart, or tie with entries elsewhere - all cases in which an entry that no thread offered
+    # belongs to the k best and the row has to be read a second time.
+    rng = np.random.default_rng(21)
+    B, F, V, k = 2, 6, 32000, 4
+    lg = (rng.normal(size=(B, F, V)) * 2).astype(np.float32)
+    big = np.float32(30.0)
+    lg[0, 0, 4000:4004] = [big + 3, big + 2, big + 1, big]              # one group of four
+    lg[0, 1, [17, 17 + 1024, 17 + 2048, 17 + 3072]] = [big, big + 1, big + 2, big + 3]   # one thread, four groups
+    lg[0, 2, [5, 6]] = big                                              # two equal maxima side by side
+    lg[0, 2, [9000, 20000]] = big                                       # ... and two more elsewhere: ties by token id
+    lg[0, 3, 31996:32000] = [big, big, big, big]                        # the last group of the row
+    lg[0, 4, [100, 101]] = [big + 1, big - 1]                           # the second of a pair ranks third
+    lg[0, 4, [7000, 15000]] = [big, big - 2]
+    lg[0, 5, 0] = big                                                   # nothing special: one clear winner
+    lg[1] = lg[0][::-1]
+    fr = np.zeros((B, F), np.int32); fl = np.full((B,), F, np.int32)
+    state = fresh(B, 64)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got, nf_g, nfl_g = gpu_step(state, lg, fr, fl, k, 9, 0.0, 0.0, status=status)
+    out = oracle.draft_expand(lg, fr, fl, *state, k=k, tau=9, theta_prob=0.0, theta_sib=0.0)
+    compare(got, list(out[:6]), nf_g, nfl_g, out[6], out[7])
+    assert int(status.item()) == 0
+    assert list(got[0][0, 1:5]) == [4000, 4001, 4002, 4003]
+    assert list(got[0][0, 5:9]) == [17 + 3072, 17 + 2048, 17 + 1024, 17]
+    assert list(got[0][0, 9:13]) == [5, 6, 9000, 20000]
+
+
 def test_capacity_is_reported_and_respected():
     state, _ = grow_levels(B=2, V=64, k=4, tau=4, levels=8, Ncap=50, seed=5)
     assert (state[5] == 50).any()
