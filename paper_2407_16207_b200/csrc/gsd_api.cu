@@ -92,10 +92,10 @@ AttnPlan attn_make_plan(const gsd_attn_params* p, int sm_count) {
         // split counts per sequence, chosen on the device; persistent CTAs walk the units
         pl.dev.balanced = 2;
         pl.ctas = resident;
-        // slots: the sum over the cut sequences of items x splits is at most the units aimed at
-        // (tiles / target, and fewer where the four-tile floor of the target binds) plus half a
-        // slot per item from rounding
-        const long long bound = (long long)kSeqPlanWaves * resident + pl.items / 2 + 1;
+        // slots: a sequence is cut when its tiles / target rounds to two or more, i.e. is at least
+        // 1.5, and then gets at most tiles / target + 0.5 <= 4/3 tiles / target ranges per item;
+        // tiles / target summed over everything is at most the units aimed at
+        const long long bound = (4ll * kSeqPlanWaves * resident + 2) / 3 + 1;
         const long long cap = (long long)pl.items * kSeqPlanMaxSplit;
         pl.slots = (int)(bound < cap ? bound : cap);
         pl.ws_bytes = plan_part_o_bytes(pl, p->D) + plan_part_ml_bytes(pl) + plan_bal_bytes(pl, p->B);
