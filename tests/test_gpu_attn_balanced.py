@@ -8,6 +8,7 @@ import torch
 import gsd_inputs as gi
 import oracle
 from gpu_util import attn_tensors, out_to_f64
+from plan_model import balanced_table, per_sequence_table
 
 pytestmark = pytest.mark.gpu
 
@@ -163,6 +164,12 @@ def test_the_table_covers_every_tile_once(shape):
                 slots_of.setdefault(int(pair), []).append(int(slot))
         assert tiles <= share
     assert len(covered) == total
+    # entry by entry what the plain-Python model of the plan says
+    model = balanced_table(inp["seq_lens"], Lmax, per_seq, nd, groups)
+    assert (int(hdr[1]), share) == (model["total"], model["share"])
+    assert [tuple(int(x) for x in r) for r in cta[:groups]] == model["runs"]
+    assert [tuple(int(x) for x in u) for u in units[:n_units]] == model["units"]
+    assert [tuple(int(x) for x in r[:3]) for r in merge[:hdr[0]]] == model["merge"]
     # the cut pairs, each with a run of consecutive slots in tile order
     assert hdr[0] == len(slots_of)
     listed = {int(r[0]): (int(r[1]), int(r[2])) for r in merge[:hdr[0]]}
@@ -207,13 +214,10 @@ def test_the_split_counts_follow_the_lengths(shape):
     nsplit = raw[at + 256:at + 256 + cfg.B * 4].view(np.int32)
     unit_off = raw[at + 256 + row:at + 256 + row + (cfg.B + 1) * 4].view(np.int32)
     slot_off = raw[at + 256 + 2 * row:at + 256 + 2 * row + (cfg.B + 1) * 4].view(np.int32)
-    T = np.array([(int(min(max(L, 0), Lmax)) + 127) // 128 + nd for L in inp["seq_lens"]])
-    total = per_seq * int(T.sum())
-    target = max(4, -(-total // (2 * sms)))
-    want_n = np.clip((2 * T + target) // (2 * target), 1, 32)
-    assert hdr[1] == total and hdr[2] == target
-    assert np.array_equal(nsplit, want_n)
-    assert np.array_equal(unit_off, np.concatenate([[0], np.cumsum(want_n * per_seq)]))
-    assert np.array_equal(slot_off, np.concatenate([[0], np.cumsum(np.where(want_n > 1, want_n * per_seq, 0))]))
+    model = per_sequence_table(inp["seq_lens"], Lmax, per_seq, nd, 2 * sms)
+    assert (int(hdr[1]), int(hdr[2])) == (model["total"], model["target"])
+    assert nsplit.tolist() == model["nsplit"]
+    assert unit_off.tolist() == model["unit_off"]
+    assert slot_off.tolist() == model["slot_off"]
     assert hdr[0] == unit_off[-1] and slot_off[-1] <= slots
 
